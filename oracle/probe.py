@@ -1,0 +1,197 @@
+"""The quantized-matmul error probe, step by step, in the paper's order.
+
+TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).
+
+Operands are passed in "non-contracting x contracting" orientation: X[..., nc, c]
+(an optional leading matmul-batch axis).  For L of a product L.R this is L
+itself ([M, K]); for R ([K, N]) it is R transposed ([N, K]).  `probe` takes L
+and R in their natural orientation and does that transposition itself.
+
+Values are float32 arrays holding exactly the stored numbers (a bf16 value is
+exactly representable in float32).  Everything mathematical is float64; the
+two operations the paper writes as arithmetic on the stored tensors (the
+division that forms delta and the division x / delta of Eq. 1) are single IEEE
+float32 operations, which is the precision decision both sides of a parity
+test share.
+"""
+import numpy as np
+
+from .formats import decode_table, positive_grid, qmax
+
+
+def _as_f32(x):
+    x = np.asarray(x)
+    if x.dtype != np.float32:
+        raise TypeError("operands are float32 arrays of the stored values")
+    return x
+
+
+def scale(x, fmt, gran):
+    """Eq. 1, right half: delta = max|X| / qmax, one delta per scaling group.
+
+    gran == "tensor": one number for the whole (batched) tensor, shape [1].
+    gran == "channel": one number per index of the non-contracting dimension
+    (and per matmul-batch element), shape x.shape[:-1]  ("finer levels of
+    granularity on non-contracting dimensions", Methodology 4th bullet).
+    An all-zero group gets delta = 1.  Non-finite input is an error.
+    """
+    x = _as_f32(x)
+    if not np.all(np.isfinite(x)):
+        raise ValueError("non-finite input")
+    a = np.abs(x)
+    if gran == "tensor":
+        amax = np.array([a.max() if a.size else 0.0], dtype=np.float32)
+    elif gran == "channel":
+        amax = a.max(axis=-1).astype(np.float32) if a.shape[-1] else np.zeros(a.shape[:-1], np.float32)
+    else:
+        raise ValueError(gran)
+    delta = amax / np.float32(qmax(fmt))          # one float32 division
+    delta = np.where(amax == 0, np.float32(1.0), delta).astype(np.float32)
+    return delta
+
+
+def _expand(delta, x):
+    """Broadcast delta ([1] or x.shape[:-1]) against x."""
+    delta = np.asarray(delta, dtype=np.float32)
+    if delta.shape == (1,):
+        return delta.reshape((1,) * x.ndim)
+    if delta.shape != x.shape[:-1]:
+        raise ValueError("delta shape")
+    return delta[..., None]
+
+
+def quantize(x, fmt, delta):
+    """Eq. 1, left half, with the saturation rule of the Methodology section.
+
+    t = x / delta in float32; the code is the grid value nearest to t, a tie
+    going to the value whose code is even (round-to-nearest-even); |t| above the
+    largest expressible value saturates to it.  Magnitudes below half the
+    smallest positive grid value therefore become zero.  Returns uint8 bytes
+    (INT8: two's complement).
+    The nearest value is found by comparing t with the midpoints of adjacent
+    grid values, so no conversion instruction is involved.
+    """
+    x = _as_f32(x)
+    t = (x / _expand(delta, x)).astype(np.float32)      # IEEE float32 division
+    if not np.all(np.isfinite(t)):
+        raise ValueError("non-finite input")
+    g = positive_grid(fmt)                               # g[c] = value of code c
+    mid = (g[:-1] + g[1:]) / 2.0                         # exact in float64
+    a = np.abs(t.astype(np.float64))
+    idx = np.searchsorted(mid, a, side="left")           # number of midpoints < a
+    below_top = idx < len(g) - 1
+    tie = below_top & (a == mid[np.minimum(idx, len(mid) - 1)])
+    idx = idx + (tie & (idx % 2 == 1))                   # tie: take the even code
+    neg = np.signbit(t) & (idx > 0)
+    if fmt == "int8":
+        code = np.where(neg, 256 - idx, idx)
+    else:
+        code = np.where(neg, idx + 128, idx)
+    return code.astype(np.uint8)
+
+
+def dequantize(codes, fmt, delta=None):
+    """Code -> value (float64), times delta when given."""
+    v = decode_table(fmt)[np.asarray(codes, dtype=np.uint8)]
+    if delta is not None:
+        v = v * _expand(delta, v).astype(np.float64)
+    return v
+
+
+def gemm_lp(codes_l, fmt_l, codes_r, fmt_r):
+    """A = Lbar . Rbar on decoded code values, float64 accumulation (exact for
+    INT8 and E4M3: every partial sum is a multiple of the smallest product
+    below 2**53 of them).  codes_l [.., M, K], codes_r [.., N, K]."""
+    a = dequantize(codes_l, fmt_l)
+    b = dequantize(codes_r, fmt_r)
+    return np.matmul(a, np.swapaxes(b, -1, -2))
+
+
+def descale(acc, delta_l, delta_r):
+    """Q_ij = A_ij * delta_L[i] * delta_R[j] (descaling after the matmul)."""
+    dl = np.asarray(delta_l, dtype=np.float64)
+    dr = np.asarray(delta_r, dtype=np.float64)
+    dl = dl.reshape((1,) * acc.ndim) if dl.shape == (1,) else dl[..., :, None]
+    dr = dr.reshape((1,) * acc.ndim) if dr.shape == (1,) else dr[..., None, :]
+    return acc * dl * dr
+
+
+def gemm_ref(l, rt):
+    """C = L . R in float64 on the stored values (numerator of Eq. 3)."""
+    return np.matmul(_as_f32(l).astype(np.float64),
+                     np.swapaxes(_as_f32(rt).astype(np.float64), -1, -2))
+
+
+def gemm_den(l, rt):
+    """D = |L| . |R|: elementwise absolute values, then the matrix product
+    (denominator of Eq. 3, inner-product-level backward error)."""
+    return np.matmul(np.abs(_as_f32(l).astype(np.float64)),
+                     np.swapaxes(np.abs(_as_f32(rt).astype(np.float64)), -1, -2))
+
+
+def metric(c, q, d):
+    """Eq. 3 per inner product: BE_ij = |C_ij - Q_ij| / D_ij (0 where D_ij is
+    0), reduced to the statistics record."""
+    c = np.asarray(c, np.float64); q = np.asarray(q, np.float64); d = np.asarray(d, np.float64)
+    diff = c - q
+    be = np.zeros_like(diff)
+    nz = d != 0
+    be[nz] = np.abs(diff[nz]) / d[nz]
+    return {
+        "sum_be": float(be.sum()),
+        "max_be": float(be.max()) if be.size else 0.0,
+        "sum_diff2": float((diff * diff).sum()),
+        "sum_ref2": float((c * c).sum()),
+        "sum_den2": float((d * d).sum()),
+        "count": int(be.size),
+    }
+
+
+def derived(rec):
+    """Scalars derived from the record: mean BE (primary), norm-wise BE,
+    relative L2 error and SNR in dB."""
+    n = max(rec["count"], 1)
+    sd, sr, sden = rec["sum_diff2"], rec["sum_ref2"], rec["sum_den2"]
+    return {
+        "mean_be": rec["sum_be"] / n,
+        "max_be": rec["max_be"],
+        "normwise_be": (sd / sden) ** 0.5 if sden > 0 else 0.0,
+        "rel_l2": (sd / sr) ** 0.5 if sr > 0 else 0.0,
+        "snr_db": 10.0 * np.log10(sr / sd) if sd > 0 and sr > 0 else float("inf"),
+    }
+
+
+def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False):
+    """The whole probe for L [.., M, K] and R [.., K, N].
+
+    rows: optional index array of output rows to evaluate (row-sampled mode;
+    scales are still computed over the whole operands).  With full=True the
+    intermediate arrays are returned too.
+    """
+    l = _as_f32(l)
+    rt = np.swapaxes(_as_f32(r), -1, -2)
+    dl = scale(l, fmt_l, gran_l)
+    dr = scale(rt, fmt_r, gran_r)
+    if rows is not None:
+        l = l[..., rows, :]
+        dl_rows = dl if dl.shape == (1,) else dl[..., rows]
+    else:
+        dl_rows = dl
+    cl = quantize(l, fmt_l, dl_rows)
+    cr = quantize(rt, fmt_r, dr)
+    acc = gemm_lp(cl, fmt_l, cr, fmt_r)
+    q = descale(acc, dl_rows, dr)
+    c = gemm_ref(l, rt)
+    d = gemm_den(l, rt)
+    rec = metric(c, q, d)
+    if full:
+        return rec, {"delta_l": dl, "delta_r": dr, "codes_l": cl, "codes_r": cr,
+                     "acc": acc, "q": q, "c": c, "d": d}
+    return rec
+
+
+def relative_error(v, v_tilde):
+    """Eq. 2 with the denominator read as |v|; entries with v == 0 are NaN."""
+    v = np.asarray(v, np.float64); v_tilde = np.asarray(v_tilde, np.float64)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        return np.where(v != 0, np.abs(v - v_tilde) / np.abs(v), np.nan)
