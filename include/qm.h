@@ -1,0 +1,212 @@
+/*
+ * qm.h - C ABI of the quantized-matmul error probe for NVIDIA B200 (sm_100a).
+ *
+ * The probe measures, for one matrix product L.R of a network, how much error
+ * an 8-bit format would introduce.  Following the paper's Methodology section
+ * it (1) computes the dynamic symmetric absmax scale of each operand (Eq. 1),
+ * (2) quantizes each operand to INT8, FP8 E4M3 or FP8 E5M2 with
+ * round-to-nearest-even and saturation (Eq. 1 and the saturation rule),
+ * (3) multiplies the 8-bit operands on the tensor cores with a wide
+ * accumulator and descales the result, (4) multiplies the unquantized
+ * operands in high precision, and (5) reduces the two results into the
+ * inner-product-level backward error of Eq. 3,
+ *        BE_ij = |(L.R)_ij - Q(L,R)_ij| / (|L|.|R|)_ij ,
+ * together with the sums needed for relative L2 error and SNR.
+ *
+ * Conventions that hold for every entry point
+ *  - All data pointers are DEVICE memory owned by the caller unless a
+ *    parameter says "host".  The library allocates no device memory.
+ *  - `stream` is a cudaStream_t passed as void*.  Work is enqueued on it and
+ *    the call returns without waiting; results are valid once the caller has
+ *    synchronised the stream (the *_host entry point is the one exception).
+ *  - Argument errors are found on the host before anything is launched and
+ *    come back as a qm_status.  Nothing throws, prints, traps or exits.
+ *  - Conditions only the device can see (a NaN/Inf operand, a bounded wait
+ *    that ran out) set bits in qm_metric_result.device_error; the numbers in
+ *    that record are then meaningless.
+ *  - An operand is a (batched) 2-D view named by its NON-CONTRACTING and
+ *    CONTRACTING extents.  For L [M x K] of L.R these are M and K; for R
+ *    [K x N] they are N and K.  One of the two strides must be 1; the other
+ *    and the batch stride must be multiples of 8 elements.
+ *  - Codes are bytes: INT8 two's complement in -127..127, FP8 bit patterns.
+ *    A code tensor is [batch][noncontract][ldc] with the contracting index
+ *    contiguous and ldc = qm_code_ld(contract) (rows padded to 16 bytes,
+ *    padding bytes are zero).
+ */
+#ifndef QM_H_
+#define QM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QM_OK = 0,
+  QM_ERR_INVALID_ARG = 1,        /* null pointer, non-positive extent, bad enum           */
+  QM_ERR_UNSUPPORTED = 2,        /* valid request this build has no kernel for            */
+  QM_ERR_ALIGNMENT = 3,          /* pointer or stride breaks a stated alignment rule      */
+  QM_ERR_WORKSPACE_TOO_SMALL = 4,
+  QM_ERR_NONFINITE_INPUT = 5,    /* reported by the *_host entry point only               */
+  QM_ERR_CUDA = 6,               /* a CUDA runtime/driver call failed                     */
+  QM_ERR_TIMEOUT = 7             /* reported by the *_host entry point only               */
+} qm_status;
+
+typedef enum { QM_FMT_INT8 = 0, QM_FMT_E4M3 = 1, QM_FMT_E5M2 = 2 } qm_format;
+typedef enum { QM_DT_F32 = 0, QM_DT_BF16 = 1 } qm_dtype;
+/* Scale granularity (Methodology, 4th bullet): one number for the whole tensor,
+ * or one per index of the non-contracting dimension (and per batch element). */
+typedef enum { QM_GRAN_TENSOR = 0, QM_GRAN_CHANNEL = 1 } qm_gran;
+typedef enum { QM_ROUND_RTNE = 0 } qm_round;
+/* How the high-precision side of Eq. 3 is evaluated:
+ *  BF16_FP32ACC: bf16 operands on the tensor cores, fp32 accumulation (every
+ *                bf16 x bf16 product is exact in fp32);
+ *  FP32:         fp32 multiply-add on the CUDA cores (fp32 or bf16 operands). */
+typedef enum { QM_REF_BF16_FP32ACC = 0, QM_REF_FP32 = 1 } qm_ref;
+
+typedef struct {
+  const void* data;        /* device; 16-byte aligned                                     */
+  int32_t dtype;           /* qm_dtype                                                    */
+  int64_t noncontract;     /* extent of the non-contracting dimension (M for L, N for R)  */
+  int64_t contract;        /* extent of the contracting dimension (K)                     */
+  int64_t stride_nc;       /* element stride between non-contracting indices              */
+  int64_t stride_c;        /* element stride between contracting indices                  */
+  int64_t batch;           /* matmul batch count, 1 for a plain product                   */
+  int64_t stride_batch;    /* element stride between batch elements (ignored if batch==1) */
+} qm_operand;
+
+/* Bits of qm_metric_result.device_error */
+#define QM_DEVERR_NONFINITE 1u   /* an operand held NaN or Inf                            */
+#define QM_DEVERR_TIMEOUT   2u   /* a bounded device-side wait gave up                    */
+
+/* The statistics record of Eq. 3 over all count = batch*M*N inner products.
+ * mean BE = sum_be/count; norm-wise BE = sqrt(sum_diff2/sum_den2);
+ * relative L2 = sqrt(sum_diff2/sum_ref2); SNR = 10 log10(sum_ref2/sum_diff2). */
+typedef struct {
+  double sum_be;           /* sum of BE_ij (BE_ij = 0 where the denominator is 0)         */
+  double max_be;           /* max of BE_ij                                                */
+  double sum_diff2;        /* sum (C_ij - Q_ij)^2                                         */
+  double sum_ref2;         /* sum C_ij^2                                                  */
+  double sum_den2;         /* sum D_ij^2, D = |L|.|R|                                     */
+  uint64_t count;
+  uint32_t device_error;   /* QM_DEVERR_* bits, 0 when the record is valid                */
+  uint32_t reserved;
+} qm_metric_result;
+
+typedef struct {
+  int32_t fmt_l, fmt_r;    /* qm_format per operand                                       */
+  int32_t gran_l, gran_r;  /* qm_gran per operand                                         */
+  int32_t round;           /* qm_round                                                    */
+  int32_t ref;             /* qm_ref                                                      */
+} qm_probe_cfg;
+
+/* Row length in bytes of a code tensor whose contracting extent is `contract`. */
+int64_t qm_code_ld(int64_t contract);
+
+/*
+ * Eq. 1 (right half) with the "align absmax to the largest expressible value"
+ * rule: delta = max|X| / qmax, qmax = 127 / 448 / 57344, one IEEE fp32
+ * division.  `delta` (device, fp32) receives 1 value for QM_GRAN_TENSOR (the
+ * whole batched tensor shares it) or batch*noncontract values, batch-major,
+ * for QM_GRAN_CHANNEL.  An all-zero group gets delta = 1.  A NaN/Inf input
+ * makes the group's delta NaN/Inf.
+ */
+qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta, void* stream);
+
+/*
+ * Eq. 1 (left half) and the saturation rule: code = sat(RTNE(x / delta)), the
+ * division in IEEE fp32, ties to the even code, magnitudes above qmax clamp to
+ * +-qmax, magnitudes below half the smallest grid value become 0.
+ *  delta      device fp32 scales as produced by qm_scale, or NULL: the call
+ *             then computes them itself (scale and quantize fused) and stores
+ *             them in delta_out, which is then REQUIRED (it is the scratch the
+ *             scales live in).
+ *  codes      device bytes, [batch][noncontract][qm_code_ld(contract)].
+ *  abs_copy   optional (may be NULL) device bf16 [batch][noncontract][contract]:
+ *             |x| rounded to bf16, contracting index contiguous (operand of the
+ *             denominator product of Eq. 3).
+ *  kmaj_copy  optional (may be NULL) device bf16, same shape: x itself with the
+ *             contracting index contiguous (for operands stored the other way).
+ */
+qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t round,
+                      const float* delta, float* delta_out, uint8_t* codes,
+                      void* abs_copy, void* kmaj_copy, void* stream);
+
+/*
+ * The 8-bit product and its descaling (Methodology, 3rd bullet):
+ *   A = Lbar . Rbar^T accumulated in int32 (INT8, exact) or fp32 (FP8, any mix
+ *   of E4M3 and E5M2), Q_ij = A_ij * delta_l[i] * delta_r[j].
+ * codes_l [batch][M][qm_code_ld(K)], codes_r [batch][N][qm_code_ld(K)];
+ * delta_l has 1 value (gran_l TENSOR) or batch*M, delta_r 1 or batch*N.
+ * out_descaled (optional) fp32 [batch][M][N]; out_raw (optional) the raw
+ * accumulator [batch][M][N]: int32 for INT8 x INT8, fp32 bit patterns for FP8.
+ * Mixing INT8 with an FP8 format is QM_ERR_UNSUPPORTED.  use_simt != 0 selects
+ * the CUDA-core kernel (any K; test cross-check); the tensor-core kernel needs
+ * K to be a multiple of 16.
+ */
+qm_status qm_gemm(const uint8_t* codes_l, int32_t fmt_l, const float* delta_l, int32_t gran_l,
+                  const uint8_t* codes_r, int32_t fmt_r, const float* delta_r, int32_t gran_r,
+                  int64_t M, int64_t N, int64_t K, int64_t batch,
+                  float* out_descaled, void* out_raw, int32_t use_simt, void* stream);
+
+/*
+ * The high-precision side of Eq. 3 on its own: out = l . r^T with bf16 operands
+ * and fp32 accumulation on the tensor cores.  Passing L and R gives the
+ * numerator product C = L.R; passing the |x| copies that qm_quantize writes
+ * gives the denominator product D = |L|.|R|.  l [batch][M][K] and
+ * r [batch][N][K], contracting index contiguous, dense.  out fp32
+ * [batch][M][N].  K must be a multiple of 16.
+ */
+qm_status qm_gemm_ref(const void* l_bf16, const void* r_bf16, int64_t M, int64_t N, int64_t K,
+                      int64_t batch, float* out, void* stream);
+
+/*
+ * Eq. 3 on materialised arrays: ref = C, q = Q, den = D, each `count` fp32
+ * values.  `out` (device) receives the record.  `ws` is device scratch of at
+ * least qm_metric_workspace_bytes(count) bytes, 8-byte aligned.
+ */
+size_t qm_metric_workspace_bytes(int64_t count);
+qm_status qm_metric(const float* ref, const float* q, const float* den, int64_t count,
+                    qm_metric_result* out, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole probe for one product L.R: scale, quantize, the three products
+ * (8-bit, reference, denominator) and the Eq. 3 reduction fused so that no
+ * M x N matrix is written.  L: noncontract = M, contract = K.  R: noncontract
+ * = N, contract = K, same batch.  `out` (device) receives the record; `ws` is
+ * device scratch of at least qm_workspace_bytes(L, R, cfg) bytes, 256-byte
+ * aligned; its contents on entry do not matter and concurrent calls must not
+ * share it.
+ * QM_REF_BF16_FP32ACC needs bf16 operands and K a multiple of 16;
+ * QM_REF_FP32 takes fp32 or bf16 operands of any shape.
+ */
+size_t qm_workspace_bytes(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg);
+qm_status qm_probe_layer(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,
+                         qm_metric_result* out, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Same probe for operands that live in HOST memory (pinned memory makes the
+ * copies asynchronous).  L->data and R->data are host pointers; l_stage and
+ * r_stage are device buffers the caller owns, large enough for the operands'
+ * storage span (qm_operand_span_bytes), 16-byte aligned.  The call copies the
+ * operands to the device, runs the probe, copies the record back into
+ * *out_host and WAITS for the stream.  Device-detected conditions are returned
+ * as QM_ERR_NONFINITE_INPUT / QM_ERR_TIMEOUT.
+ */
+size_t qm_operand_span_bytes(const qm_operand* x);
+qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host,
+                              const qm_probe_cfg* cfg, void* l_stage, void* r_stage,
+                              qm_metric_result* out_host, qm_metric_result* out_dev,
+                              void* ws, size_t ws_bytes, void* stream);
+
+const char* qm_status_string(int32_t status);
+int32_t qm_version(void);
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* qm_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QM_H_ */

@@ -1,0 +1,115 @@
+// Eq. 3 on materialised arrays, and the deterministic final reduction shared with the fused
+// probe kernels.
+#include "qm_internal.h"
+
+namespace qm {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_maxd(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Each block owns a contiguous slice; the order of additions is fixed by the launch shape.
+__global__ void __launch_bounds__(kThreads)
+metric_partials_kernel(const float* __restrict__ ref, const float* __restrict__ q,
+                       const float* __restrict__ den, int64_t count, double* __restrict__ partials) {
+  __shared__ double s[5][kThreads / 32];
+  const int64_t per_block = (count + gridDim.x - 1) / gridDim.x;
+  const int64_t i0 = (int64_t)blockIdx.x * per_block;
+  const int64_t i1 = min(count, i0 + per_block);
+  double sbe = 0, mbe = 0, sd2 = 0, sr2 = 0, sn2 = 0;
+  for (int64_t base = i0; base < i1; base += kThreads * 8) {
+    // fp32 inside a short run, fp64 across runs
+    float fbe = 0, fmx = 0, fd2 = 0, fr2 = 0, fn2 = 0;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int64_t i = base + u * kThreads + threadIdx.x;
+      if (i < i1) {
+        const float c = __ldg(ref + i), qq = __ldg(q + i), d = __ldg(den + i);
+        const float diff = c - qq;
+        const float be = d != 0.f ? __fdiv_rn(fabsf(diff), d) : 0.f;
+        fbe += be; fmx = fmaxf(fmx, be);
+        fd2 = fmaf(diff, diff, fd2); fr2 = fmaf(c, c, fr2); fn2 = fmaf(d, d, fn2);
+      }
+    }
+    sbe += fbe; mbe = fmax(mbe, (double)fmx); sd2 += fd2; sr2 += fr2; sn2 += fn2;
+  }
+  sbe = warp_sum(sbe); sd2 = warp_sum(sd2); sr2 = warp_sum(sr2); sn2 = warp_sum(sn2);
+  mbe = warp_maxd(mbe);
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) { s[0][w] = sbe; s[1][w] = mbe; s[2][w] = sd2; s[3][w] = sr2; s[4][w] = sn2; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double a = 0, m = 0, b = 0, c = 0, d = 0;
+    for (int i = 0; i < kThreads / 32; ++i) {
+      a += s[0][i]; m = fmax(m, s[1][i]); b += s[2][i]; c += s[3][i]; d += s[4][i];
+    }
+    double* o = partials + (int64_t)blockIdx.x * kPartialDoubles;
+    o[0] = a; o[1] = m; o[2] = b; o[3] = c; o[4] = d;
+  }
+}
+
+// One block; thread t sums records t, t+256, ... in order, then a fixed tree.
+__global__ void __launch_bounds__(kThreads)
+metric_finalize_kernel(const double* __restrict__ partials, int n, uint64_t count,
+                       const uint32_t* __restrict__ err_word, qm_metric_result* __restrict__ out) {
+  __shared__ double s[5][kThreads];
+  double a = 0, m = 0, b = 0, c = 0, d = 0;
+  for (int i = threadIdx.x; i < n; i += kThreads) {
+    const double* p = partials + (int64_t)i * kPartialDoubles;
+    a += p[0]; m = fmax(m, p[1]); b += p[2]; c += p[3]; d += p[4];
+  }
+  s[0][threadIdx.x] = a; s[1][threadIdx.x] = m; s[2][threadIdx.x] = b;
+  s[3][threadIdx.x] = c; s[4][threadIdx.x] = d;
+  __syncthreads();
+  for (int o = kThreads / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      s[0][threadIdx.x] += s[0][threadIdx.x + o];
+      s[1][threadIdx.x] = fmax(s[1][threadIdx.x], s[1][threadIdx.x + o]);
+      s[2][threadIdx.x] += s[2][threadIdx.x + o];
+      s[3][threadIdx.x] += s[3][threadIdx.x + o];
+      s[4][threadIdx.x] += s[4][threadIdx.x + o];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    out->sum_be = s[0][0]; out->max_be = s[1][0]; out->sum_diff2 = s[2][0];
+    out->sum_ref2 = s[3][0]; out->sum_den2 = s[4][0];
+    out->count = count;
+    out->device_error = err_word ? *err_word : 0u;
+    out->reserved = 0;
+  }
+}
+
+}  // namespace
+
+int metric_blocks(int64_t count) {
+  int64_t want = (count + kThreads * 8 - 1) / (kThreads * 8);
+  int64_t cap = (int64_t)sm_count() * 8;
+  return (int)(want < 1 ? 1 : (want < cap ? want : cap));
+}
+
+qm_status launch_metric_partials(const float* ref, const float* q, const float* den, int64_t count,
+                                 double* partials, int nblocks, cudaStream_t s) {
+  metric_partials_kernel<<<nblocks, kThreads, 0, s>>>(ref, q, den, count, partials);
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+qm_status launch_metric_finalize(const double* partials, int n, uint64_t count,
+                                 const uint32_t* err_word, qm_metric_result* out, cudaStream_t s) {
+  metric_finalize_kernel<<<1, kThreads, 0, s>>>(partials, n, count, err_word, out);
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+}  // namespace qm

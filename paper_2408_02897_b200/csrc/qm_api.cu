@@ -1,0 +1,309 @@
+// The C ABI: argument checks, workspace layout and launch sequencing.  All arithmetic of the
+// probe runs in the kernels of the other translation units.
+#include <cstdio>
+#include <cstring>
+
+#include "qm_internal.h"
+
+namespace qm {
+
+static thread_local char g_last_error[256] = "";
+
+void note_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+  (void)cudaGetLastError();   // do not let a non-sticky error be blamed on a later call
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+namespace {
+
+bool valid_fmt(int f) { return f == QM_FMT_INT8 || f == QM_FMT_E4M3 || f == QM_FMT_E5M2; }
+bool valid_gran(int g) { return g == QM_GRAN_TENSOR || g == QM_GRAN_CHANNEL; }
+
+qm_status to_view(const qm_operand* x, View* v) {
+  if (!x || !x->data) return QM_ERR_INVALID_ARG;
+  if (x->dtype != QM_DT_F32 && x->dtype != QM_DT_BF16) return QM_ERR_INVALID_ARG;
+  if (x->noncontract <= 0 || x->contract <= 0 || x->batch <= 0) return QM_ERR_INVALID_ARG;
+  if (x->stride_nc <= 0 || x->stride_c <= 0) return QM_ERR_INVALID_ARG;
+  if (x->stride_nc != 1 && x->stride_c != 1) return QM_ERR_UNSUPPORTED;
+  if (x->batch > 1 && x->stride_batch <= 0) return QM_ERR_INVALID_ARG;
+  v->data = x->data; v->dtype = x->dtype;
+  v->nc = x->noncontract; v->c = x->contract;
+  v->s_nc = x->stride_nc; v->s_c = x->stride_c;
+  v->batch = x->batch;
+  // rows must not overlap
+  if (v->s_c == 1 && v->nc > 1 && v->s_nc < v->c) return QM_ERR_INVALID_ARG;
+  if (v->s_c != 1 && v->c > 1 && v->s_c < v->nc) return QM_ERR_INVALID_ARG;
+  const int64_t span = (v->nc - 1) * v->s_nc + (v->c - 1) * v->s_c + 1;
+  v->s_b = x->batch > 1 ? x->stride_batch : ((span + 7) & ~(int64_t)7);
+  if (v->batch > 1 && v->s_b < span) return QM_ERR_INVALID_ARG;
+  // 128-bit loads: base, the non-unit stride and the batch stride must keep 16-byte alignment
+  if (reinterpret_cast<uintptr_t>(x->data) & 15) return QM_ERR_ALIGNMENT;
+  const int64_t big = v->s_c == 1 ? v->s_nc : v->s_c;
+  if ((big & 7) || (v->batch > 1 && (v->s_b & 7))) return QM_ERR_ALIGNMENT;
+  return QM_OK;
+}
+
+int64_t delta_count(const View& v, int gran) { return gran == QM_GRAN_TENSOR ? 1 : v.nc * v.batch; }
+
+size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+struct Workspace {
+  size_t off_err, off_dl, off_dr, off_cl, off_cr, off_al, off_ar, off_kl, off_kr, off_part, total;
+  int n_part;
+  bool tc;
+};
+
+Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg) {
+  Workspace w{};
+  w.tc = cfg.ref == QM_REF_BF16_FP32ACC;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o += align256(bytes); return at; };
+  w.off_err = take(256);
+  w.off_dl = take(sizeof(float) * delta_count(L, cfg.gran_l));
+  w.off_dr = take(sizeof(float) * delta_count(R, cfg.gran_r));
+  const int64_t ldc = qm_code_ld(L.c);
+  w.off_cl = take((size_t)(L.batch * L.nc * ldc));
+  w.off_cr = take((size_t)(R.batch * R.nc * ldc));
+  if (w.tc) {
+    w.off_al = take((size_t)(L.batch * L.nc * L.c) * 2);
+    w.off_ar = take((size_t)(R.batch * R.nc * R.c) * 2);
+    w.off_kl = L.c_contig() ? 0 : take((size_t)(L.batch * L.nc * L.c) * 2);
+    w.off_kr = R.c_contig() ? 0 : take((size_t)(R.batch * R.nc * R.c) * 2);
+  }
+  GemmShape g{L.nc, R.nc, L.c, L.batch};
+  w.n_part = w.tc ? tc_probe_tiles(g) : simt_probe_blocks(g);
+  w.off_part = take(sizeof(double) * kPartialDoubles * (size_t)w.n_part);
+  w.total = o;
+  return w;
+}
+
+qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg, View* L, View* R) {
+  if (!cfg) return QM_ERR_INVALID_ARG;
+  qm_status st = to_view(Lo, L);
+  if (st != QM_OK) return st;
+  st = to_view(Ro, R);
+  if (st != QM_OK) return st;
+  if (!valid_fmt(cfg->fmt_l) || !valid_fmt(cfg->fmt_r) || !valid_gran(cfg->gran_l) || !valid_gran(cfg->gran_r))
+    return QM_ERR_INVALID_ARG;
+  if (cfg->round != QM_ROUND_RTNE) return QM_ERR_UNSUPPORTED;
+  if (cfg->ref != QM_REF_BF16_FP32ACC && cfg->ref != QM_REF_FP32) return QM_ERR_INVALID_ARG;
+  if (L->c != R->c || L->batch != R->batch) return QM_ERR_INVALID_ARG;
+  if ((cfg->fmt_l == QM_FMT_INT8) != (cfg->fmt_r == QM_FMT_INT8)) return QM_ERR_UNSUPPORTED;
+  if (cfg->ref == QM_REF_BF16_FP32ACC) {
+    if (L->dtype != QM_DT_BF16 || R->dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;
+    if (L->c % 16) return QM_ERR_UNSUPPORTED;
+  }
+  return QM_OK;
+}
+
+// scale + quantize of one operand inside the probe
+qm_status prepare_operand(const View& x, int fmt, int gran, float* delta, uint8_t* codes, void* abs_copy,
+                          void* kmaj_copy, uint32_t* err_word, cudaStream_t s) {
+  if (gran == QM_GRAN_CHANNEL && x.c_contig())
+    return launch_scale_quantize_rows(x, fmt, delta, codes, abs_copy, err_word, s);
+  qm_status st = launch_absmax(x, gran, reinterpret_cast<uint32_t*>(delta), s);
+  if (st != QM_OK) return st;
+  st = launch_finalize_delta(delta, delta_count(x, gran), fmt, err_word, s);
+  if (st != QM_OK) return st;
+  return launch_quantize(x, fmt, gran, delta, codes, abs_copy, kmaj_copy, s);
+}
+
+}  // namespace
+}  // namespace qm
+
+using namespace qm;
+
+extern "C" {
+
+int64_t qm_code_ld(int64_t contract) { return (contract + 15) & ~(int64_t)15; }
+
+qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta, void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (!valid_fmt(fmt) || !valid_gran(gran) || !delta) return QM_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t n = delta_count(v, gran);
+  QM_CUDA_OK(cudaMemsetAsync(delta, 0, sizeof(float) * n, s));
+  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta), s);
+  if (st != QM_OK) return st;
+  return launch_finalize_delta(delta, n, fmt, nullptr, s);
+}
+
+qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t round, const float* delta,
+                      float* delta_out, uint8_t* codes, void* abs_copy, void* kmaj_copy, void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (!valid_fmt(fmt) || !valid_gran(gran) || !codes) return QM_ERR_INVALID_ARG;
+  if (round != QM_ROUND_RTNE) return QM_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(codes) & 15) || (reinterpret_cast<uintptr_t>(abs_copy) & 15) ||
+      (reinterpret_cast<uintptr_t>(kmaj_copy) & 15))
+    return QM_ERR_ALIGNMENT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (delta) return launch_quantize(v, fmt, gran, delta, codes, abs_copy, kmaj_copy, s);
+  if (!delta_out) return QM_ERR_INVALID_ARG;
+  const int64_t n = delta_count(v, gran);
+  if (gran == QM_GRAN_CHANNEL && v.c_contig() && !kmaj_copy)
+    return launch_scale_quantize_rows(v, fmt, delta_out, codes, abs_copy, nullptr, s);
+  QM_CUDA_OK(cudaMemsetAsync(delta_out, 0, sizeof(float) * n, s));
+  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta_out), s);
+  if (st != QM_OK) return st;
+  st = launch_finalize_delta(delta_out, n, fmt, nullptr, s);
+  if (st != QM_OK) return st;
+  return launch_quantize(v, fmt, gran, delta_out, codes, abs_copy, kmaj_copy, s);
+}
+
+qm_status qm_gemm(const uint8_t* codes_l, int32_t fmt_l, const float* delta_l, int32_t gran_l,
+                  const uint8_t* codes_r, int32_t fmt_r, const float* delta_r, int32_t gran_r, int64_t M,
+                  int64_t N, int64_t K, int64_t batch, float* out_descaled, void* out_raw, int32_t use_simt,
+                  void* stream) {
+  if (!codes_l || !codes_r || !delta_l || !delta_r || (!out_descaled && !out_raw)) return QM_ERR_INVALID_ARG;
+  if (!valid_fmt(fmt_l) || !valid_fmt(fmt_r) || !valid_gran(gran_l) || !valid_gran(gran_r)) return QM_ERR_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return QM_ERR_INVALID_ARG;
+  if ((fmt_l == QM_FMT_INT8) != (fmt_r == QM_FMT_INT8)) return QM_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(codes_l) & 15) || (reinterpret_cast<uintptr_t>(codes_r) & 15)) return QM_ERR_ALIGNMENT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  GemmShape g{M, N, K, batch};
+  if (use_simt)
+    return launch_simt_gemm_lp(codes_l, fmt_l, delta_l, gran_l, codes_r, fmt_r, delta_r, gran_r, g,
+                               out_descaled, out_raw, s);
+  if (K % 16) return QM_ERR_UNSUPPORTED;
+  return launch_tc_gemm_lp(codes_l, fmt_l, delta_l, gran_l, codes_r, fmt_r, delta_r, gran_r, g, out_descaled,
+                           out_raw, nullptr, s);
+}
+
+qm_status qm_gemm_ref(const void* l_bf16, const void* r_bf16, int64_t M, int64_t N, int64_t K, int64_t batch,
+                      float* out, void* stream) {
+  if (!l_bf16 || !r_bf16 || !out) return QM_ERR_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return QM_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(l_bf16) & 15) || (reinterpret_cast<uintptr_t>(r_bf16) & 15)) return QM_ERR_ALIGNMENT;
+  if (K % 16) return QM_ERR_UNSUPPORTED;
+  GemmShape g{M, N, K, batch};
+  return launch_tc_gemm_ref(l_bf16, r_bf16, g, out, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+size_t qm_metric_workspace_bytes(int64_t count) {
+  if (count <= 0) return 0;
+  return align256(sizeof(double) * kPartialDoubles * (size_t)metric_blocks(count));
+}
+
+qm_status qm_metric(const float* ref, const float* q, const float* den, int64_t count, qm_metric_result* out,
+                    void* ws, size_t ws_bytes, void* stream) {
+  if (!ref || !q || !den || !out || !ws || count <= 0) return QM_ERR_INVALID_ARG;
+  if (ws_bytes < qm_metric_workspace_bytes(count)) return QM_ERR_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(ws) & 7) return QM_ERR_ALIGNMENT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int nb = metric_blocks(count);
+  qm_status st = launch_metric_partials(ref, q, den, count, static_cast<double*>(ws), nb, s);
+  if (st != QM_OK) return st;
+  return launch_metric_finalize(static_cast<double*>(ws), nb, (uint64_t)count, nullptr, out, s);
+}
+
+size_t qm_workspace_bytes(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg) {
+  View L, R;
+  if (check_probe(Lo, Ro, cfg, &L, &R) != QM_OK) return 0;
+  return plan(L, R, *cfg).total;
+}
+
+qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
+                         qm_metric_result* out, void* ws, size_t ws_bytes, void* stream) {
+  View L, R;
+  qm_status st = check_probe(Lo, Ro, cfg, &L, &R);
+  if (st != QM_OK) return st;
+  if (!out || !ws) return QM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255) return QM_ERR_ALIGNMENT;
+  const Workspace w = plan(L, R, *cfg);
+  if (ws_bytes < w.total) return QM_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  uint32_t* err = reinterpret_cast<uint32_t*>(base + w.off_err);
+  float* dl = reinterpret_cast<float*>(base + w.off_dl);
+  float* dr = reinterpret_cast<float*>(base + w.off_dr);
+  uint8_t* cl = base + w.off_cl;
+  uint8_t* cr = base + w.off_cr;
+  double* part = reinterpret_cast<double*>(base + w.off_part);
+  // the error word and both scale buffers are adjacent: one clear
+  QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_cl, s));
+  void* al = w.tc ? base + w.off_al : nullptr;
+  void* ar = w.tc ? base + w.off_ar : nullptr;
+  void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
+  void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
+  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, dl, cl, al, kl, err, s);
+  if (st != QM_OK) return st;
+  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, dr, cr, ar, kr, err, s);
+  if (st != QM_OK) return st;
+  GemmShape g{L.nc, R.nc, L.c, L.batch};
+  if (w.tc) {
+    TcProbeArgs p{};
+    p.l = kl ? kl : L.data; p.l_ld = kl ? L.c : L.s_nc; p.l_sb = kl ? L.nc * L.c : L.s_b;
+    p.r = kr ? kr : R.data; p.r_ld = kr ? R.c : R.s_nc; p.r_sb = kr ? R.nc * R.c : R.s_b;
+    p.l_abs = al; p.r_abs = ar; p.cl = cl; p.cr = cr;
+    p.fmt_l = cfg->fmt_l; p.fmt_r = cfg->fmt_r;
+    p.dl = dl; p.gran_l = cfg->gran_l; p.dr = dr; p.gran_r = cfg->gran_r;
+    p.g = g; p.partials = part; p.err_word = err;
+    st = launch_tc_probe(p, s);
+  } else {
+    st = launch_simt_probe(L, R, cl, cfg->fmt_l, dl, cfg->gran_l, cr, cfg->fmt_r, dr, cfg->gran_r, part, s);
+  }
+  if (st != QM_OK) return st;
+  return launch_metric_finalize(part, w.n_part, (uint64_t)(g.M * g.N * g.batch), err, out, s);
+}
+
+size_t qm_operand_span_bytes(const qm_operand* x) {
+  View v;
+  if (to_view(x, &v) != QM_OK) return 0;
+  const int64_t last = (v.batch - 1) * v.s_b + (v.nc - 1) * v.s_nc + (v.c - 1) * v.s_c;
+  return (size_t)(last + 1) * (v.dtype == QM_DT_BF16 ? 2 : 4);
+}
+
+qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host, const qm_probe_cfg* cfg,
+                              void* l_stage, void* r_stage, qm_metric_result* out_host,
+                              qm_metric_result* out_dev, void* ws, size_t ws_bytes, void* stream) {
+  if (!L_host || !R_host || !l_stage || !r_stage || !out_host || !out_dev) return QM_ERR_INVALID_ARG;
+  const size_t lb = qm_operand_span_bytes(L_host), rb = qm_operand_span_bytes(R_host);
+  if (lb == 0 || rb == 0) return QM_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  QM_CUDA_OK(cudaMemcpyAsync(l_stage, L_host->data, lb, cudaMemcpyHostToDevice, s));
+  QM_CUDA_OK(cudaMemcpyAsync(r_stage, R_host->data, rb, cudaMemcpyHostToDevice, s));
+  qm_operand L = *L_host, R = *R_host;
+  L.data = l_stage; R.data = r_stage;
+  qm_status st = qm_probe_layer(&L, &R, cfg, out_dev, ws, ws_bytes, stream);
+  if (st != QM_OK) return st;
+  QM_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, sizeof(qm_metric_result), cudaMemcpyDeviceToHost, s));
+  QM_CUDA_OK(cudaStreamSynchronize(s));
+  if (out_host->device_error & QM_DEVERR_TIMEOUT) return QM_ERR_TIMEOUT;
+  if (out_host->device_error & QM_DEVERR_NONFINITE) return QM_ERR_NONFINITE_INPUT;
+  return QM_OK;
+}
+
+const char* qm_status_string(int32_t st) {
+  switch (st) {
+    case QM_OK: return "ok";
+    case QM_ERR_INVALID_ARG: return "invalid argument";
+    case QM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case QM_ERR_ALIGNMENT: return "alignment";
+    case QM_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case QM_ERR_NONFINITE_INPUT: return "non-finite input";
+    case QM_ERR_CUDA: return "CUDA error";
+    case QM_ERR_TIMEOUT: return "device wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int32_t qm_version(void) { return 100; }
+
+const char* qm_last_cuda_error(void) { return qm::g_last_error; }
+
+}  // extern "C"

@@ -1,0 +1,96 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qm.h"
+
+namespace qm {
+
+// A validated operand view, extents as 64-bit, element strides.
+struct View {
+  const void* data;
+  int dtype;            // qm_dtype
+  int64_t nc, c;        // non-contracting / contracting extents
+  int64_t s_nc, s_c;    // element strides
+  int64_t batch, s_b;   // batch count / element stride
+  bool c_contig() const { return s_c == 1; }
+};
+
+// Largest expressible magnitude of a format (127, 448, 57344).
+__host__ __device__ inline float fmt_qmax(int fmt) {
+  return fmt == QM_FMT_INT8 ? 127.0f : (fmt == QM_FMT_E4M3 ? 448.0f : 57344.0f);
+}
+
+// Per-thread record of the last CUDA error text.
+void note_cuda_error(cudaError_t e, const char* where);
+#define QM_CUDA_OK(expr)                                   \
+  do {                                                     \
+    cudaError_t e__ = (expr);                              \
+    if (e__ != cudaSuccess) {                              \
+      ::qm::note_cuda_error(e__, #expr);                   \
+      return QM_ERR_CUDA;                                  \
+    }                                                      \
+  } while (0)
+
+int sm_count();
+
+// ---- scale / quantize (scale_quantize.cu) ---------------------------------
+// amax: uint32 buffer (1 or batch*nc entries) that must be zero on entry; on exit it holds
+// the bit pattern of max|x| per group.
+qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream_t s);
+// In place: bit pattern of max|x| -> delta = max|x| / qmax (1 where max|x| == 0).
+// err_word (optional): gets QM_DEVERR_NONFINITE or-ed in when a group max is NaN/Inf.
+qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s);
+// codes (+ optional |x| and x as bf16, contraction-major) from given deltas.
+qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, uint8_t* codes,
+                          void* abs_copy, void* kmaj_copy, cudaStream_t s);
+// Single pass per row: absmax, delta, codes (contiguous contraction, per-channel).
+qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
+                                     void* abs_copy, uint32_t* err_word, cudaStream_t s);
+
+// ---- metric (metric.cu) ----------------------------------------------------
+// One partial record per CTA: {sum_be, max_be, sum_diff2, sum_ref2, sum_den2} as doubles.
+constexpr int kPartialDoubles = 5;
+int metric_blocks(int64_t count);
+qm_status launch_metric_partials(const float* ref, const float* q, const float* den, int64_t count,
+                                 double* partials, int nblocks, cudaStream_t s);
+// Sums `n` partial records in a fixed order and writes the result record.
+qm_status launch_metric_finalize(const double* partials, int n, uint64_t count,
+                                 const uint32_t* err_word, qm_metric_result* out, cudaStream_t s);
+
+// ---- CUDA-core GEMMs (gemm_simt.cu) ---------------------------------------
+struct GemmShape { int64_t M, N, K, batch; };
+qm_status launch_simt_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
+                              const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
+                              GemmShape g, float* out_descaled, void* out_raw, cudaStream_t s);
+int simt_probe_blocks(GemmShape g);
+// Fused CUDA-core probe: three accumulators per output, Eq. 3 partials per CTA.
+qm_status launch_simt_probe(const View& L, const View& R, const uint8_t* cl, int fmt_l,
+                            const float* dl, int gran_l, const uint8_t* cr, int fmt_r,
+                            const float* dr, int gran_r, double* partials, cudaStream_t s);
+
+// ---- tensor-core GEMMs (gemm_tc.cu) ---------------------------------------
+struct TcProbeArgs {
+  // bf16, contraction contiguous; element strides between rows / batches
+  const void* l; int64_t l_ld, l_sb;
+  const void* r; int64_t r_ld, r_sb;
+  const void* l_abs; const void* r_abs;     // dense [batch][rows][K]
+  const uint8_t* cl; const uint8_t* cr;     // codes, rows of qm_code_ld(K) bytes
+  int fmt_l, fmt_r;
+  const float* dl; int gran_l;
+  const float* dr; int gran_r;
+  GemmShape g;
+  double* partials;                         // tc_probe_tiles(g) records
+  uint32_t* err_word;
+};
+int tc_probe_tiles(GemmShape g);
+qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
+qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
+                            const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
+                            GemmShape g, float* out_descaled, void* out_raw, uint32_t* err_word,
+                            cudaStream_t s);
+qm_status launch_tc_gemm_ref(const void* l, const void* r, GemmShape g, float* out,
+                             uint32_t* err_word, cudaStream_t s);
+
+}  // namespace qm

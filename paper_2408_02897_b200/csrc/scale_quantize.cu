@@ -1,0 +1,532 @@
+// Scale (Eq. 1, right half) and quantize (Eq. 1, left half + saturation rule) kernels.
+// All of them are HBM-bound streaming kernels: 128-bit coalesced loads, warp-shuffle and
+// shared-memory reductions, one atomicMax per block and group.
+#include <cuda_bf16.h>
+
+#include "qm_internal.h"
+
+namespace qm {
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------- element helpers
+// |x| as an order-preserving unsigned integer: for IEEE formats the bit pattern with the sign
+// cleared orders like the magnitude, and Inf / NaN patterns sort above every finite value, so
+// an integer max also carries "non-finite seen" to the end.  bf16 patterns are widened to the
+// fp32 pattern (shift by 16) so one code path serves both input types.
+__device__ __forceinline__ uint32_t absbits_f32(uint32_t w) { return w & 0x7fffffffu; }
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Two quantized bytes from t = x / delta: t0 in bits 0..7, t1 in bits 8..15.
+// RTNE, saturating at the largest finite magnitude.
+template <int FMT>
+__device__ __forceinline__ uint32_t quant2(float t0, float t1) {
+  if (FMT == QM_FMT_INT8) {
+    int a = __float2int_rn(t0), b = __float2int_rn(t1);      // round to nearest even
+    a = max(-127, min(127, a));
+    b = max(-127, min(127, b));
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8);
+  } else {
+    uint16_t r;
+    if (FMT == QM_FMT_E4M3)
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(t1), "f"(t0));
+    else
+      asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(t1), "f"(t0));
+    return r;
+  }
+}
+
+// 8 consecutive elements held as fp32.
+struct Vec8 { float v[8]; };
+
+template <typename T> struct Loader;
+template <> struct Loader<__nv_bfloat16> {
+  static __device__ __forceinline__ Vec8 load8(const void* p) {
+    uint4 w = __ldg(reinterpret_cast<const uint4*>(p));
+    Vec8 r;
+    r.v[0] = bf16_lo(w.x); r.v[1] = bf16_hi(w.x); r.v[2] = bf16_lo(w.y); r.v[3] = bf16_hi(w.y);
+    r.v[4] = bf16_lo(w.z); r.v[5] = bf16_hi(w.z); r.v[6] = bf16_lo(w.w); r.v[7] = bf16_hi(w.w);
+    return r;
+  }
+  static __device__ __forceinline__ float load1(const void* p, int64_t i) {
+    return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p) + i) << 16);
+  }
+};
+template <> struct Loader<float> {
+  static __device__ __forceinline__ Vec8 load8(const void* p) {
+    float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    Vec8 r;
+    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w;
+    r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+    return r;
+  }
+  static __device__ __forceinline__ float load1(const void* p, int64_t i) {
+    return __ldg(reinterpret_cast<const float*>(p) + i);
+  }
+};
+
+__device__ __forceinline__ uint32_t absmax8(const Vec8& x, uint32_t acc) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc = max(acc, absbits_f32(__float_as_uint(x.v[i])));
+  return acc;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // round to nearest even
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+template <int FMT>
+__device__ __forceinline__ uint2 quant8(const Vec8& x, float delta) {
+  float t[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) t[i] = __fdiv_rn(x.v[i], delta);   // IEEE division, as Eq. 1 writes it
+  uint2 r;
+  r.x = quant2<FMT>(t[0], t[1]) | (quant2<FMT>(t[2], t[3]) << 16);
+  r.y = quant2<FMT>(t[4], t[5]) | (quant2<FMT>(t[6], t[7]) << 16);
+  return r;
+}
+
+__device__ __forceinline__ uint4 abs_bf16x8(const Vec8& x) {
+  uint4 r;
+  r.x = pack_bf16x2(fabsf(x.v[0]), fabsf(x.v[1]));
+  r.y = pack_bf16x2(fabsf(x.v[2]), fabsf(x.v[3]));
+  r.z = pack_bf16x2(fabsf(x.v[4]), fabsf(x.v[5]));
+  r.w = pack_bf16x2(fabsf(x.v[6]), fabsf(x.v[7]));
+  return r;
+}
+__device__ __forceinline__ uint4 to_bf16x8(const Vec8& x) {
+  uint4 r;
+  r.x = pack_bf16x2(x.v[0], x.v[1]); r.y = pack_bf16x2(x.v[2], x.v[3]);
+  r.z = pack_bf16x2(x.v[4], x.v[5]); r.w = pack_bf16x2(x.v[6], x.v[7]);
+  return r;
+}
+
+__device__ __forceinline__ uint32_t warp_max(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t block_max(uint32_t v) {
+  __shared__ uint32_t s[32];
+  v = warp_max(v);
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) s[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    v = lane < (int)(blockDim.x >> 5) ? s[lane] : 0u;
+    v = warp_max(v);
+  }
+  return v;   // valid in warp 0
+}
+
+// ---------------------------------------------------------------- absmax, whole tensor
+// Rows of `c` contiguous elements (vector loads for the multiple-of-8 part, scalar loads for
+// the tail).  When the rows are dense the host flattens the tensor into a single row so that
+// every block gets an equal share.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+absmax_tensor_kernel(const T* __restrict__ x, int64_t rows, int64_t c, int64_t row_stride,
+                     uint32_t* __restrict__ amax) {
+  const int64_t vec_per_row = c >> 3;
+  const int64_t total_vec = rows * vec_per_row;
+  uint32_t acc = 0;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // four independent 128-bit loads in flight per thread
+  for (; i + 3 * stride < total_vec; i += 4 * stride) {
+    Vec8 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      int64_t j = i + u * stride;
+      int64_t r = j / vec_per_row, k = j - r * vec_per_row;
+      v[u] = Loader<T>::load8(x + r * row_stride + k * 8);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc = absmax8(v[u], acc);
+  }
+  for (; i < total_vec; i += stride) {
+    int64_t r = i / vec_per_row, k = i - r * vec_per_row;
+    acc = absmax8(Loader<T>::load8(x + r * row_stride + k * 8), acc);
+  }
+  const int64_t tail = c & 7;
+  if (tail) {
+    const int64_t total_tail = rows * tail;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < total_tail; j += stride) {
+      int64_t r = j / tail, k = j - r * tail;
+      acc = max(acc, absbits_f32(__float_as_uint(Loader<T>::load1(x, r * row_stride + (c - tail) + k))));
+    }
+  }
+  acc = block_max(acc);
+  if (threadIdx.x == 0 && acc) atomicMax(amax, acc);
+}
+
+// ---------------------------------------------------------------- absmax per row (contiguous rows)
+// G lanes share a row; rows are (batch, nc) pairs.
+template <typename T, int G>
+__global__ void __launch_bounds__(kThreads)
+absmax_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
+                   int64_t s_b, uint32_t* __restrict__ amax) {
+  const int64_t rows = nc * batch;
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int sub = threadIdx.x % G;
+  uint32_t acc = 0;
+  if (row < rows) {
+    const int64_t b = row / nc, r = row - b * nc;
+    const T* p = x + b * s_b + r * s_nc;
+    const int64_t nvec = c >> 3;
+    for (int64_t k = sub; k < nvec; k += G) acc = absmax8(Loader<T>::load8(p + k * 8), acc);
+    for (int64_t k = (nvec << 3) + sub; k < c; k += G)
+      acc = max(acc, absbits_f32(__float_as_uint(Loader<T>::load1(p, k))));
+  }
+#pragma unroll
+  for (int o = G / 2; o > 0; o >>= 1) acc = max(acc, __shfl_xor_sync(0xffffffffu, acc, o, G));
+  if (row < rows && sub == 0) amax[row] = acc;
+}
+
+// ---------------------------------------------------------------- absmax per column (strided contraction)
+// Storage is [c][nc] with nc contiguous; one value per column.  Each thread owns 8 adjacent
+// columns; blockDim = (32, 8): 256 columns wide, 8 row slices; grid.y splits the rows.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+absmax_cols_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
+                   int64_t rows_per_block, uint32_t* __restrict__ amax) {
+  __shared__ uint32_t s[8][256];
+  const int64_t b = blockIdx.z;
+  const int64_t col0 = ((int64_t)blockIdx.x * 32 + threadIdx.x) * 8;
+  const int64_t r0 = (int64_t)blockIdx.y * rows_per_block;
+  const int64_t r1 = min(c, r0 + rows_per_block);
+  uint32_t acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0;
+  const T* base = x + b * s_b;
+  if (col0 + 8 <= nc) {
+    for (int64_t r = r0 + threadIdx.y; r < r1; r += 8) {
+      Vec8 v = Loader<T>::load8(base + r * s_c + col0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = max(acc[i], absbits_f32(__float_as_uint(v.v[i])));
+    }
+  } else if (col0 < nc) {
+    for (int64_t r = r0 + threadIdx.y; r < r1; r += 8)
+      for (int i = 0; i < 8 && col0 + i < nc; ++i)
+        acc[i] = max(acc[i], absbits_f32(__float_as_uint(Loader<T>::load1(base, r * s_c + col0 + i))));
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s[threadIdx.y][threadIdx.x * 8 + i] = acc[i];
+  __syncthreads();
+  const int t = threadIdx.y * 32 + threadIdx.x;      // 0..255: one column each
+  uint32_t m = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) m = max(m, s[j][t]);
+  const int64_t col = (int64_t)blockIdx.x * 256 + t;
+  if (col < nc && m) atomicMax(amax + b * nc + col, m);
+}
+
+__global__ void finalize_delta_kernel(float* __restrict__ delta, int64_t n, float qmax,
+                                      uint32_t* __restrict__ err_word) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint32_t bits = __float_as_uint(delta[i]);
+  float amax = __uint_as_float(bits);
+  if (bits >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
+  delta[i] = bits == 0 ? 1.0f : __fdiv_rn(amax, qmax);
+}
+
+// ---------------------------------------------------------------- quantize, contiguous contraction
+// One thread handles 16 consecutive elements of a row: two 128-bit loads (bf16), one 128-bit
+// code store, optionally two 128-bit stores of |x| as bf16.
+template <typename T, int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
+                     int64_t s_b, const float* __restrict__ delta, int per_channel,
+                     uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy) {
+  const int64_t chunks_per_row = ldc >> 4;                  // 16 codes per chunk, padding included
+  const int64_t total = nc * batch * chunks_per_row;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const float d_tensor = per_channel ? 0.f : __ldg(delta);
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t row = i / chunks_per_row, ch = i - row * chunks_per_row;
+    const int64_t b = row / nc, r = row - b * nc;
+    const T* p = x + b * s_b + r * s_nc + ch * 16;
+    const float d = per_channel ? __ldg(delta + row) : d_tensor;
+    const int64_t k0 = ch * 16;
+    Vec8 v0, v1;
+    if (k0 + 16 <= c) {
+      v0 = Loader<T>::load8(p);
+      v1 = Loader<T>::load8(p + 8);
+    } else {                                                // ragged end of the row: zero fill
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        v0.v[j] = k0 + j < c ? Loader<T>::load1(p, j) : 0.f;
+        v1.v[j] = k0 + 8 + j < c ? Loader<T>::load1(p, 8 + j) : 0.f;
+      }
+    }
+    uint2 q0 = quant8<FMT>(v0, d), q1 = quant8<FMT>(v1, d);
+    *reinterpret_cast<uint4*>(codes + row * ldc + k0) = make_uint4(q0.x, q0.y, q1.x, q1.y);
+    if (abs_copy) {
+      __nv_bfloat16* a = abs_copy + row * c + k0;
+      if (k0 + 16 <= c && (c & 7) == 0) {
+        *reinterpret_cast<uint4*>(a) = abs_bf16x8(v0);
+        *reinterpret_cast<uint4*>(a + 8) = abs_bf16x8(v1);
+      } else {
+        for (int j = 0; j < 8; ++j) {
+          if (k0 + j < c) a[j] = __float2bfloat16_rn(fabsf(v0.v[j]));
+          if (k0 + 8 + j < c) a[8 + j] = __float2bfloat16_rn(fabsf(v1.v[j]));
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- fused per-row scale + quantize
+// G lanes own one row: pass 1 reduces max|x| over the row, pass 2 re-reads it (from L1/L2: the
+// same lanes touched it a moment ago) and writes codes.  HBM sees each element once.
+template <typename T, int FMT, int G>
+__global__ void __launch_bounds__(kThreads)
+scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc,
+                           int64_t batch, int64_t s_b, float qmax, float* __restrict__ delta_out,
+                           uint8_t* __restrict__ codes, int64_t ldc,
+                           __nv_bfloat16* __restrict__ abs_copy, uint32_t* __restrict__ err_word) {
+  const int64_t rows = nc * batch;
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+  const int sub = threadIdx.x % G;
+  const bool live = row < rows;
+  const int64_t b = live ? row / nc : 0, r = live ? row - b * nc : 0;
+  const T* p = x + b * s_b + r * s_nc;
+  const int64_t nvec = c >> 3;
+  uint32_t acc = 0;
+  if (live) {
+    for (int64_t k = sub; k < nvec; k += G) acc = absmax8(Loader<T>::load8(p + k * 8), acc);
+    for (int64_t k = (nvec << 3) + sub; k < c; k += G)
+      acc = max(acc, absbits_f32(__float_as_uint(Loader<T>::load1(p, k))));
+  }
+#pragma unroll
+  for (int o = G / 2; o > 0; o >>= 1) acc = max(acc, __shfl_xor_sync(0xffffffffu, acc, o, G));
+  if (!live) return;
+  const float d = acc == 0 ? 1.0f : __fdiv_rn(__uint_as_float(acc), qmax);
+  if (sub == 0) {
+    delta_out[row] = d;
+    if (acc >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
+  }
+  const int64_t nchunk = ldc >> 3;                          // 8 codes per step, padding included
+  for (int64_t k = sub; k < nchunk; k += G) {
+    const int64_t k0 = k * 8;
+    Vec8 v;
+    if (k0 + 8 <= c) v = Loader<T>::load8(p + k0);
+    else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v.v[j] = k0 + j < c ? Loader<T>::load1(p, k0 + j) : 0.f;
+    }
+    *reinterpret_cast<uint2*>(codes + row * ldc + k0) = quant8<FMT>(v, d);
+    if (abs_copy) {
+      __nv_bfloat16* a = abs_copy + row * c + k0;
+      if (k0 + 8 <= c && (c & 7) == 0) *reinterpret_cast<uint4*>(a) = abs_bf16x8(v);
+      else
+        for (int j = 0; j < 8 && k0 + j < c; ++j) a[j] = __float2bfloat16_rn(fabsf(v.v[j]));
+    }
+  }
+}
+
+// ---------------------------------------------------------------- quantize + transpose
+// Storage [c][nc] (nc contiguous) -> codes [nc][ldc] and optional bf16 copies [nc][c].
+// A 64(c) x 64(nc) tile goes through shared memory.
+template <typename T, int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
+                          const float* __restrict__ delta, int per_channel,
+                          uint8_t* __restrict__ codes, int64_t ldc,
+                          __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
+  __shared__ float tile[64][65];     // +1 column spreads the transposed accesses over the banks
+  const int64_t b = blockIdx.z;
+  const int64_t c0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
+  const T* base = x + b * s_b;
+  const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;    // 8 column-chunks x 32 rows
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int rr = ty + it * 32;
+    const int64_t cc = c0 + rr, nn = n0 + tx * 8;
+    Vec8 v;
+    if (cc < c && nn + 8 <= nc) v = Loader<T>::load8(base + cc * s_c + nn);
+    else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        v.v[j] = (cc < c && nn + j < nc) ? Loader<T>::load1(base, cc * s_c + nn + j) : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) tile[rr][tx * 8 + j] = v.v[j];
+  }
+  __syncthreads();
+  // output: row n (64 of them), 64 contraction entries = 8 chunks of 8
+  const float d_tensor = per_channel ? 0.f : __ldg(delta);
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int nrow = ty + it * 32;
+    const int64_t nn = n0 + nrow;
+    if (nn >= nc) continue;
+    const int64_t k0 = c0 + tx * 8;
+    if (k0 >= ldc) continue;
+    Vec8 v;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v.v[j] = tile[tx * 8 + j][nrow];
+    const float d = per_channel ? __ldg(delta + b * nc + nn) : d_tensor;
+    const int64_t orow = b * nc + nn;
+    *reinterpret_cast<uint2*>(codes + orow * ldc + k0) = quant8<FMT>(v, d);
+    if (abs_copy || kmaj_copy) {
+      if (k0 + 8 <= c && (c & 7) == 0) {
+        if (abs_copy) *reinterpret_cast<uint4*>(abs_copy + orow * c + k0) = abs_bf16x8(v);
+        if (kmaj_copy) *reinterpret_cast<uint4*>(kmaj_copy + orow * c + k0) = to_bf16x8(v);
+      } else {
+        for (int j = 0; j < 8 && k0 + j < c; ++j) {
+          if (abs_copy) abs_copy[orow * c + k0 + j] = __float2bfloat16_rn(fabsf(v.v[j]));
+          if (kmaj_copy) kmaj_copy[orow * c + k0 + j] = __float2bfloat16_rn(v.v[j]);
+        }
+      }
+    }
+  }
+}
+
+int grid_for(int64_t work_items, int per_sm) {
+  int64_t want = (work_items + kThreads - 1) / kThreads;
+  int64_t cap = (int64_t)sm_count() * per_sm;
+  return (int)(want < 1 ? 1 : (want < cap ? want : cap));
+}
+
+template <typename T>
+qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
+  const T* p = static_cast<const T*>(x.data);
+  if (x.c_contig()) {
+    if (gran == QM_GRAN_TENSOR) {
+      const bool dense = x.s_nc == x.c && (x.batch == 1 || x.s_b == x.nc * x.c);
+      const bool even = x.batch == 1 || x.s_b == x.nc * x.s_nc;
+      if (dense) {
+        const int64_t n = x.nc * x.batch * x.c;
+        absmax_tensor_kernel<T><<<grid_for(n / 8 + 1, 8), kThreads, 0, s>>>(p, 1, n, n, amax);
+      } else if (even) {
+        absmax_tensor_kernel<T><<<grid_for(x.nc * x.batch * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+            p, x.nc * x.batch, x.c, x.s_nc, amax);
+      } else {
+        for (int64_t b = 0; b < x.batch; ++b)
+          absmax_tensor_kernel<T><<<grid_for(x.nc * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+              p + b * x.s_b, x.nc, x.c, x.s_nc, amax);
+      }
+    } else {
+      const int64_t rows = x.nc * x.batch;
+      const int64_t nvec = x.c / 8;
+#define QM_ROWS(G)                                                                              \
+  absmax_rows_kernel<T, G><<<(unsigned)((rows * G + kThreads - 1) / kThreads), kThreads, 0, s>>>( \
+      p, x.nc, x.c, x.s_nc, x.batch, x.s_b, amax)
+      if (nvec <= 4) QM_ROWS(4);
+      else if (nvec <= 8) QM_ROWS(8);
+      else if (nvec <= 16) QM_ROWS(16);
+      else QM_ROWS(32);
+#undef QM_ROWS
+    }
+  } else {
+    if (gran == QM_GRAN_TENSOR) {
+      // storage rows are the contracting index: walk them as rows of nc contiguous elements
+      for (int64_t b = 0; b < x.batch; ++b)
+        absmax_tensor_kernel<T><<<grid_for(x.nc * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+            p + b * x.s_b, x.c, x.nc, x.s_c, amax);
+    } else {
+      const int64_t col_blocks = (x.nc + 255) / 256;
+      int64_t want_y = ((int64_t)sm_count() * 8 + col_blocks * x.batch - 1) / (col_blocks * x.batch);
+      int64_t rows_per_block = (x.c + want_y - 1) / want_y;
+      rows_per_block = (rows_per_block + 7) / 8 * 8;
+      if (rows_per_block < 64) rows_per_block = 64;
+      const int64_t gy = (x.c + rows_per_block - 1) / rows_per_block;
+      dim3 grid((unsigned)col_blocks, (unsigned)gy, (unsigned)x.batch), block(32, 8);
+      absmax_cols_kernel<T><<<grid, block, 0, s>>>(p, x.nc, x.c, x.s_c, x.s_b, rows_per_block, amax);
+    }
+  }
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+template <typename T, int FMT>
+qm_status quantize_t(const View& x, int gran, const float* delta, uint8_t* codes, void* abs_copy,
+                     void* kmaj_copy, cudaStream_t s) {
+  const T* p = static_cast<const T*>(x.data);
+  const int64_t ldc = qm_code_ld(x.c);
+  const int pc = gran == QM_GRAN_CHANNEL;
+  if (x.c_contig()) {
+    const int64_t total = x.nc * x.batch * (ldc >> 4);
+    quantize_rows_kernel<T, FMT><<<grid_for(total, 16), kThreads, 0, s>>>(
+        p, x.nc, x.c, x.s_nc, x.batch, x.s_b, delta, pc, codes, ldc,
+        static_cast<__nv_bfloat16*>(abs_copy));
+    if (kmaj_copy) {
+      // already contraction-major: a strided copy honours the parameter
+      if (x.dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;
+      for (int64_t b = 0; b < x.batch; ++b)
+        QM_CUDA_OK(cudaMemcpy2DAsync(static_cast<uint8_t*>(kmaj_copy) + b * x.nc * x.c * 2, x.c * 2,
+                                     static_cast<const uint8_t*>(x.data) + b * x.s_b * 2, x.s_nc * 2,
+                                     x.c * 2, x.nc, cudaMemcpyDeviceToDevice, s));
+    }
+  } else {
+    dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((ldc + 63) / 64), (unsigned)x.batch);
+    quantize_transpose_kernel<T, FMT><<<grid, kThreads, 0, s>>>(
+        p, x.nc, x.c, x.s_c, x.s_b, delta, pc, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
+        static_cast<__nv_bfloat16*>(kmaj_copy));
+  }
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+template <typename T, int FMT>
+qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes, void* abs_copy,
+                                uint32_t* err_word, cudaStream_t s) {
+  const T* p = static_cast<const T*>(x.data);
+  const int64_t rows = x.nc * x.batch, ldc = qm_code_ld(x.c), nvec = x.c / 8;
+  const float qmax = fmt_qmax(FMT);
+#define QM_SQ(G)                                                                                   \
+  scale_quantize_rows_kernel<T, FMT, G>                                                            \
+      <<<(unsigned)((rows * G + kThreads - 1) / kThreads), kThreads, 0, s>>>(                      \
+          p, x.nc, x.c, x.s_nc, x.batch, x.s_b, qmax, delta_out, codes, ldc,                       \
+          static_cast<__nv_bfloat16*>(abs_copy), err_word)
+  if (nvec <= 4) QM_SQ(4);
+  else if (nvec <= 8) QM_SQ(8);
+  else if (nvec <= 16) QM_SQ(16);
+  else QM_SQ(32);
+#undef QM_SQ
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+}  // namespace
+
+qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream_t s) {
+  return x.dtype == QM_DT_BF16 ? absmax_t<__nv_bfloat16>(x, gran, amax_bits, s)
+                               : absmax_t<float>(x, gran, amax_bits, s);
+}
+
+qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s) {
+  finalize_delta_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(delta, n, fmt_qmax(fmt), err_word);
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
+}
+
+qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, uint8_t* codes,
+                          void* abs_copy, void* kmaj_copy, cudaStream_t s) {
+#define QM_Q(T)                                                                                  \
+  (fmt == QM_FMT_INT8   ? quantize_t<T, QM_FMT_INT8>(x, gran, delta, codes, abs_copy, kmaj_copy, s) \
+   : fmt == QM_FMT_E4M3 ? quantize_t<T, QM_FMT_E4M3>(x, gran, delta, codes, abs_copy, kmaj_copy, s) \
+                        : quantize_t<T, QM_FMT_E5M2>(x, gran, delta, codes, abs_copy, kmaj_copy, s))
+  return x.dtype == QM_DT_BF16 ? QM_Q(__nv_bfloat16) : QM_Q(float);
+#undef QM_Q
+}
+
+qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
+                                     void* abs_copy, uint32_t* err_word, cudaStream_t s) {
+#define QM_Q(T)                                                                                       \
+  (fmt == QM_FMT_INT8   ? scale_quantize_rows_t<T, QM_FMT_INT8>(x, delta_out, codes, abs_copy, err_word, s) \
+   : fmt == QM_FMT_E4M3 ? scale_quantize_rows_t<T, QM_FMT_E4M3>(x, delta_out, codes, abs_copy, err_word, s) \
+                        : scale_quantize_rows_t<T, QM_FMT_E5M2>(x, delta_out, codes, abs_copy, err_word, s))
+  return x.dtype == QM_DT_BF16 ? QM_Q(__nv_bfloat16) : QM_Q(float);
+#undef QM_Q
+}
+
+}  // namespace qm
