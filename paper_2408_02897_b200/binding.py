@@ -1,0 +1,256 @@
+"""ctypes binding of include/qm.h.  Argument marshalling only.
+
+Tensors are torch CUDA tensors (torch is used for device memory and streams); an operand of a
+product L.R is described by `operand_of(tensor, contract_dim)`.
+"""
+import ctypes as C
+import math
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libqm.so")
+
+FMT = {"int8": 0, "e4m3": 1, "e5m2": 2}
+GRAN = {"tensor": 0, "channel": 1}
+REF = {"bf16": 0, "fp32": 1}
+_DT = {torch.float32: 0, torch.bfloat16: 1}
+
+
+class QmError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__(what)
+
+
+class Operand(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("dtype", C.c_int32), ("noncontract", C.c_int64),
+                ("contract", C.c_int64), ("stride_nc", C.c_int64), ("stride_c", C.c_int64),
+                ("batch", C.c_int64), ("stride_batch", C.c_int64)]
+
+
+class MetricResult(C.Structure):
+    _fields_ = [("sum_be", C.c_double), ("max_be", C.c_double), ("sum_diff2", C.c_double),
+                ("sum_ref2", C.c_double), ("sum_den2", C.c_double), ("count", C.c_uint64),
+                ("device_error", C.c_uint32), ("reserved", C.c_uint32)]
+
+    def record(self):
+        return {k: getattr(self, k) for k in ("sum_be", "max_be", "sum_diff2", "sum_ref2", "sum_den2", "count")}
+
+    def derived(self):
+        n = max(self.count, 1)
+        sd, sr, sn = self.sum_diff2, self.sum_ref2, self.sum_den2
+        return {"mean_be": self.sum_be / n, "max_be": self.max_be,
+                "normwise_be": math.sqrt(sd / sn) if sn > 0 else 0.0,
+                "rel_l2": math.sqrt(sd / sr) if sr > 0 else 0.0,
+                "snr_db": 10.0 * math.log10(sr / sd) if sd > 0 and sr > 0 else float("inf")}
+
+
+class ProbeCfg(C.Structure):
+    _fields_ = [("fmt_l", C.c_int32), ("fmt_r", C.c_int32), ("gran_l", C.c_int32), ("gran_r", C.c_int32),
+                ("round", C.c_int32), ("ref", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library.  Raises if it is missing: there is no fallback path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise QmError(-1, f"{_LIB_PATH} not built; run: python -m paper_2408_02897_b200.build")
+        L = C.CDLL(_LIB_PATH)
+        P, I32, I64, SZ = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        OP = C.POINTER(Operand)
+        sig = {
+            "qm_code_ld": (I64, [I64]),
+            "qm_scale": (I32, [OP, I32, I32, P, P]),
+            "qm_quantize": (I32, [OP, I32, I32, I32, P, P, P, P, P, P]),
+            "qm_gemm": (I32, [P, I32, P, I32, P, I32, P, I32, I64, I64, I64, I64, P, P, I32, P]),
+            "qm_gemm_ref": (I32, [P, P, I64, I64, I64, I64, P, P]),
+            "qm_metric_workspace_bytes": (SZ, [I64]),
+            "qm_metric": (I32, [P, P, P, I64, P, P, SZ, P]),
+            "qm_workspace_bytes": (SZ, [OP, OP, C.POINTER(ProbeCfg)]),
+            "qm_probe_layer": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, SZ, P]),
+            "qm_operand_span_bytes": (SZ, [OP]),
+            "qm_probe_layer_host": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, C.POINTER(MetricResult), P, P, SZ, P]),
+            "qm_status_string": (C.c_char_p, [I32]),
+            "qm_version": (I32, []),
+            "qm_last_cuda_error": (C.c_char_p, []),
+        }
+        for name, (res, args) in sig.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(st, what):
+    if st != 0:
+        L = lib()
+        msg = L.qm_status_string(st).decode()
+        if st == 6:
+            msg += " (" + L.qm_last_cuda_error().decode() + ")"
+        raise QmError(st, f"{what}: {msg}")
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def qm_code_ld(contract):
+    return (contract + 15) // 16 * 16
+
+
+def operand_of(t, contract_dim):
+    """Describes a 2-D [.., .] or batched 3-D [b, ., .] tensor as an operand whose contracting
+    dimension is `contract_dim` (-1 or -2).  No data is touched."""
+    if t.dim() not in (2, 3) or t.dtype not in _DT:
+        raise QmError(1, "operand must be a 2-D or 3-D float32/bfloat16 tensor")
+    cd = contract_dim % t.dim()
+    nd = t.dim() - 1 if cd == t.dim() - 2 else t.dim() - 2
+    if cd == nd or cd < t.dim() - 2:
+        raise QmError(1, "contract_dim must be one of the last two dimensions")
+    o = Operand()
+    o.data = t.data_ptr(); o.dtype = _DT[t.dtype]
+    o.noncontract = t.shape[nd]; o.contract = t.shape[cd]
+    o.stride_nc = t.stride(nd); o.stride_c = t.stride(cd)
+    o.batch = t.shape[0] if t.dim() == 3 else 1
+    o.stride_batch = t.stride(0) if t.dim() == 3 else 0
+    o._keep = t
+    return o
+
+
+def _n_delta(op, gran):
+    return 1 if GRAN[gran] == 0 else op.batch * op.noncontract
+
+
+def qm_scale(op, fmt, gran, stream=None):
+    """Eq. 1 scales of an operand -> float32 CUDA tensor (1 or batch*noncontract values)."""
+    delta = torch.empty(_n_delta(op, gran), dtype=torch.float32, device="cuda")
+    _check(lib().qm_scale(C.byref(op), FMT[fmt], GRAN[gran], _ptr(delta), _stream(stream)), "qm_scale")
+    return delta
+
+
+def qm_quantize(op, fmt, gran, delta=None, want_abs=False, want_kmaj=False, stream=None):
+    """Codes of an operand.  delta=None fuses the scale step.  Returns (codes, delta, abs, kmaj)."""
+    ldc = qm_code_ld(op.contract)
+    codes = torch.empty((op.batch, op.noncontract, ldc), dtype=torch.uint8, device="cuda")
+    shape = (op.batch, op.noncontract, op.contract)
+    ab = torch.empty(shape, dtype=torch.bfloat16, device="cuda") if want_abs else None
+    km = torch.empty(shape, dtype=torch.bfloat16, device="cuda") if want_kmaj else None
+    dout = None
+    if delta is None:
+        dout = torch.empty(_n_delta(op, gran), dtype=torch.float32, device="cuda")
+    _check(lib().qm_quantize(C.byref(op), FMT[fmt], GRAN[gran], 0, _ptr(delta), _ptr(dout), _ptr(codes),
+                             _ptr(ab), _ptr(km), _stream(stream)), "qm_quantize")
+    return codes, (delta if delta is not None else dout), ab, km
+
+
+def qm_gemm(codes_l, fmt_l, delta_l, gran_l, codes_r, fmt_r, delta_r, gran_r, K, want_raw=False,
+            use_simt=False, stream=None):
+    """Descaled 8-bit product from codes [b, M, ldc] x [b, N, ldc] -> (fp32 [b, M, N], raw or None)."""
+    b, M, _ = codes_l.shape
+    N = codes_r.shape[1]
+    out = torch.empty((b, M, N), dtype=torch.float32, device="cuda")
+    raw = None
+    if want_raw:
+        raw = torch.empty((b, M, N), dtype=torch.int32 if fmt_l == "int8" else torch.float32, device="cuda")
+    _check(lib().qm_gemm(_ptr(codes_l), FMT[fmt_l], _ptr(delta_l), GRAN[gran_l], _ptr(codes_r), FMT[fmt_r],
+                         _ptr(delta_r), GRAN[gran_r], M, N, K, b, _ptr(out), _ptr(raw), int(use_simt),
+                         _stream(stream)), "qm_gemm")
+    return out, raw
+
+
+def qm_gemm_ref(l, r, stream=None):
+    """out = l . r^T for dense bf16 [b, M, K] and [b, N, K] -> fp32 [b, M, N]."""
+    b, M, K = l.shape
+    N = r.shape[1]
+    assert l.is_contiguous() and r.is_contiguous() and l.dtype == torch.bfloat16 and r.dtype == torch.bfloat16
+    out = torch.empty((b, M, N), dtype=torch.float32, device="cuda")
+    _check(lib().qm_gemm_ref(_ptr(l), _ptr(r), M, N, K, b, _ptr(out), _stream(stream)), "qm_gemm_ref")
+    return out
+
+
+def _read_result(dev_buf):
+    host = dev_buf.cpu().numpy().tobytes()
+    return MetricResult.from_buffer_copy(host)
+
+
+def qm_metric(ref, q, den, stream=None):
+    """Eq. 3 record of three fp32 arrays of equal size."""
+    n = ref.numel()
+    L = lib()
+    ws_bytes = L.qm_metric_workspace_bytes(n)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    out = torch.empty(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+    _check(L.qm_metric(_ptr(ref), _ptr(q), _ptr(den), n, _ptr(out), _ptr(ws), ws_bytes, _stream(stream)), "qm_metric")
+    return _read_result(out)
+
+
+def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref):
+    c = ProbeCfg()
+    c.fmt_l, c.fmt_r, c.gran_l, c.gran_r, c.round, c.ref = FMT[fmt_l], FMT[fmt_r], GRAN[gran_l], GRAN[gran_r], 0, REF[ref]
+    return c
+
+
+def qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
+    c = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref)
+    n = lib().qm_workspace_bytes(C.byref(L_op), C.byref(R_op), C.byref(c))
+    if n == 0:
+        raise QmError(1, "qm_workspace_bytes: configuration rejected")
+    return n
+
+
+class ProbePlan:
+    """Pre-allocated workspace and result buffer for repeated probes of one shape."""
+
+    def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
+        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref)
+        self.ws_bytes = qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
+        self.out = torch.zeros(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+
+    def launch(self, L_op, R_op, stream=None):
+        _check(lib().qm_probe_layer(C.byref(L_op), C.byref(R_op), C.byref(self.cfg), _ptr(self.out),
+                                    _ptr(self.ws), self.ws_bytes, _stream(stream)), "qm_probe_layer")
+
+    def result(self):
+        return _read_result(self.out)
+
+
+def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None):
+    """The whole probe for one product; returns the MetricResult (synchronises to read it)."""
+    plan = ProbePlan(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
+    plan.launch(L_op, R_op, stream)
+    return plan.result()
+
+
+def qm_probe_layer_host(L_host, R_host, contract_l, contract_r, fmt_l, fmt_r, gran_l, gran_r, ref="bf16",
+                        stage=None, stream=None):
+    """Probe of operands held in (pinned) host tensors; copies are part of the call.
+    `stage` may carry (l_stage, r_stage, plan) from an earlier call to avoid re-allocation."""
+    Lh, Rh = operand_of(L_host, contract_l), operand_of(R_host, contract_r)
+    if stage is None:
+        l_stage = torch.empty(L_host.numel() if L_host.is_contiguous() else lib().qm_operand_span_bytes(C.byref(Lh)),
+                              dtype=L_host.dtype if L_host.is_contiguous() else torch.uint8, device="cuda")
+        r_stage = torch.empty(R_host.numel() if R_host.is_contiguous() else lib().qm_operand_span_bytes(C.byref(Rh)),
+                              dtype=R_host.dtype if R_host.is_contiguous() else torch.uint8, device="cuda")
+        Ld, Rd = Operand(), Operand()
+        C.memmove(C.byref(Ld), C.byref(Lh), C.sizeof(Operand)); C.memmove(C.byref(Rd), C.byref(Rh), C.sizeof(Operand))
+        Ld.data, Rd.data = l_stage.data_ptr(), r_stage.data_ptr()
+        plan = ProbePlan(Ld, Rd, fmt_l, fmt_r, gran_l, gran_r, ref)
+        stage = (l_stage, r_stage, plan)
+    l_stage, r_stage, plan = stage
+    res = MetricResult()
+    st = lib().qm_probe_layer_host(C.byref(Lh), C.byref(Rh), C.byref(plan.cfg), _ptr(l_stage), _ptr(r_stage),
+                                   C.byref(res), _ptr(plan.out), _ptr(plan.ws), plan.ws_bytes, _stream(stream))
+    _check(st, "qm_probe_layer_host")
+    return res, stage

@@ -1,0 +1,79 @@
+"""CPU-only checks of the C-ABI boundary: the library loads, exports every declared symbol,
+and rejects bad arguments on the host before anything is launched."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2408_02897_b200 as qm
+from paper_2408_02897_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "qm.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(qm_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = qm.lib()
+    names = declared_functions()
+    assert {"qm_scale", "qm_quantize", "qm_gemm", "qm_metric", "qm_probe_layer", "qm_workspace_bytes",
+            "qm_status_string", "qm_version"} <= set(names)
+    for n in names:
+        assert hasattr(L, n), n
+
+
+def test_struct_layouts_match_header():
+    assert C.sizeof(binding.MetricResult) == 56
+    assert C.sizeof(binding.Operand) == 64
+    assert C.sizeof(binding.ProbeCfg) == 24
+
+
+def test_host_side_argument_checks():
+    L = qm.lib()
+    assert L.qm_code_ld(1) == 16 and L.qm_code_ld(16) == 16 and L.qm_code_ld(17) == 32
+    assert L.qm_status_string(0) == b"ok"
+    op = binding.Operand()
+    assert L.qm_scale(C.byref(op), 1, 0, None, None) == 1           # null data
+    op.data = 0x1000; op.dtype = 1; op.noncontract = 8; op.contract = 32
+    op.stride_nc = 32; op.stride_c = 1; op.batch = 1
+    assert L.qm_scale(C.byref(op), 7, 0, C.c_void_p(0x2000), None) == 1    # bad format
+    assert L.qm_scale(C.byref(op), 1, 0, None, None) == 1                  # null output
+    op.stride_nc = 33
+    assert L.qm_scale(C.byref(op), 1, 0, C.c_void_p(0x2000), None) == 3    # stride alignment
+    op.stride_nc = 32; op.data = 0x1004
+    assert L.qm_scale(C.byref(op), 1, 0, C.c_void_p(0x2000), None) == 3    # pointer alignment
+    op.data = 0x1000; op.stride_c = 2
+    assert L.qm_scale(C.byref(op), 1, 0, C.c_void_p(0x2000), None) == 2    # no unit stride
+    op.stride_c = 1; op.stride_nc = 16
+    assert L.qm_scale(C.byref(op), 1, 0, C.c_void_p(0x2000), None) == 1    # overlapping rows
+    # probe configuration checks
+    a = binding.Operand(); b = binding.Operand()
+    for o, nc in ((a, 64), (b, 48)):
+        o.data = 0x1000; o.dtype = 1; o.noncontract = nc; o.contract = 32
+        o.stride_nc = 32; o.stride_c = 1; o.batch = 1
+    cfg = binding.ProbeCfg(1, 1, 0, 0, 0, 0)
+    assert L.qm_workspace_bytes(C.byref(a), C.byref(b), C.byref(cfg)) > 0
+    cfg.fmt_r = 0                                                          # INT8 mixed with FP8
+    assert L.qm_workspace_bytes(C.byref(a), C.byref(b), C.byref(cfg)) == 0
+    assert L.qm_probe_layer(C.byref(a), C.byref(b), C.byref(cfg), C.c_void_p(0x100), C.c_void_p(0x100), 1 << 30, None) == 2
+    cfg.fmt_r = 1; b.contract = 64; b.stride_nc = 64                       # K mismatch
+    assert L.qm_probe_layer(C.byref(a), C.byref(b), C.byref(cfg), C.c_void_p(0x100), C.c_void_p(0x100), 1 << 30, None) == 1
+    b.contract = 32; b.stride_nc = 32
+    assert L.qm_probe_layer(C.byref(a), C.byref(b), C.byref(cfg), C.c_void_p(0x100), C.c_void_p(0x100), 16, None) == 4
+    assert L.qm_probe_layer(C.byref(a), C.byref(b), C.byref(cfg), C.c_void_p(0x100), C.c_void_p(0x104), 1 << 30, None) == 3
+    a.dtype = 0                                                            # fp32 operand on the bf16 path
+    assert L.qm_probe_layer(C.byref(a), C.byref(b), C.byref(cfg), C.c_void_p(0x100), C.c_void_p(0x100), 1 << 30, None) == 2
+    assert L.qm_metric(None, None, None, 4, None, None, 0, None) == 1
+    assert L.qm_gemm(None, 0, None, 0, None, 0, None, 0, 1, 1, 16, 1, None, None, 0, None) == 1
+
+
+def test_missing_library_fails_loudly(monkeypatch):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/libqm.so")
+    with pytest.raises(qm.QmError):
+        binding.lib()

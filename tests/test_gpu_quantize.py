@@ -1,0 +1,145 @@
+"""GPU parity: scales and codes against the oracle, bit for bit (Eq. 1, saturation rule)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2408_02897_b200 as qm
+from helpers import oriented, as3
+
+pytestmark = pytest.mark.gpu
+FMTS = ["int8", "e4m3", "e5m2"]
+
+
+def make(shape, dtype, seed, dist="t"):
+    rng = np.random.default_rng(seed)
+    x = (rng.standard_t(3, shape) if dist == "t" else rng.standard_normal(shape)).astype(np.float32)
+    return torch.from_numpy(x).to(dtype)
+
+
+def check(t, contract_dim, fmt, gran, fused):
+    td = t.cuda()
+    op = qm.operand_of(td, contract_dim)
+    x = as3(oriented(t, contract_dim))                     # [b, nc, c]
+    want_d = oracle.scale(x, fmt, gran)
+    want_c = oracle.quantize(x, fmt, want_d)
+    d = qm.qm_scale(op, fmt, gran)
+    assert np.array_equal(d.cpu().numpy().view(np.uint32), want_d.ravel().view(np.uint32))
+    if fused:
+        codes, d2, ab, km = qm.qm_quantize(op, fmt, gran, None, want_abs=True, want_kmaj=(contract_dim == -2))
+        assert np.array_equal(d2.cpu().numpy().view(np.uint32), want_d.ravel().view(np.uint32))
+    else:
+        codes, _, ab, km = qm.qm_quantize(op, fmt, gran, d, want_abs=True, want_kmaj=True)
+    torch.cuda.synchronize()
+    c = codes.cpu().numpy()
+    K = x.shape[-1]
+    assert c.shape[-1] == (K + 15) // 16 * 16
+    assert np.array_equal(c[..., :K], want_c)
+    assert not c[..., K:].any()                            # padding bytes are zero
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    assert torch.equal(ab.cpu(), xb.abs())
+    if km is not None:
+        assert torch.equal(km.cpu(), xb)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("gran", ["tensor", "channel"])
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("layout", ["rows", "cols"])
+def test_codes_bf16(fmt, gran, fused, layout):
+    # several 64-wide tiles plus ragged tails in both directions
+    t = make((333, 200), torch.bfloat16, 1)
+    check(t, -1 if layout == "rows" else -2, fmt, gran, fused)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("gran", ["tensor", "channel"])
+@pytest.mark.parametrize("layout", ["rows", "cols"])
+def test_codes_fp32(fmt, gran, layout):
+    t = make((130, 264), torch.float32, 2, "n")
+    check(t, -1 if layout == "rows" else -2, fmt, gran, True)
+
+
+@pytest.mark.parametrize("gran", ["tensor", "channel"])
+@pytest.mark.parametrize("layout", ["rows", "cols"])
+def test_codes_batched(gran, layout):
+    t = make((5, 72, 64), torch.bfloat16, 3)
+    check(t, -1 if layout == "rows" else -2, "e4m3", gran, True)
+    check(t, -1 if layout == "rows" else -2, "int8", gran, False)
+
+
+def test_strided_view_and_long_rows():
+    big = make((64, 4104), torch.bfloat16, 4)
+    v = big[:, :4100]                                      # row stride 4104, ragged length
+    td = big.cuda()[:, :4100]
+    for gran in ("tensor", "channel"):
+        op = qm.operand_of(td, -1)
+        x = as3(v.float().numpy())
+        want_d = oracle.scale(x, "e5m2", gran)
+        codes, d, _, _ = qm.qm_quantize(op, "e5m2", gran, None)
+        assert np.array_equal(d.cpu().numpy().view(np.uint32), want_d.ravel().view(np.uint32))
+        assert np.array_equal(codes.cpu().numpy()[..., :4100], oracle.quantize(x, "e5m2", want_d))
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_exhaustive_bf16_inputs(fmt):
+    # every finite bf16 value, under several scales, including awkward non-power-of-two ones
+    bits = np.arange(65536, dtype=np.uint32)
+    vals = (bits << 16).view(np.float32)
+    vals = vals[np.isfinite(vals)]
+    for delta in (1.0, 0.75, 3.0, 1.0 / 3.0, 1e-3, 2.0 ** -20, 1.7e5, 7.3e-12):
+        lim = np.float32(delta) * np.float32(oracle.qmax(fmt)) * np.float32(4.0)
+        x = vals[np.abs(vals) <= lim]                      # include clear saturation cases
+        pad = (-len(x)) % 16
+        x = np.concatenate([x, np.zeros(pad, np.float32)])[None, None, :]
+        d = np.array([delta], np.float32)
+        want = oracle.quantize(x, fmt, d)
+        t = torch.from_numpy(x[0]).to(torch.bfloat16).cuda()
+        assert np.array_equal(t.float().cpu().numpy(), x[0])
+        codes, _, _, _ = qm.qm_quantize(qm.operand_of(t, -1), fmt, "tensor", torch.from_numpy(d).cuda())
+        got = codes.cpu().numpy()
+        bad = np.nonzero(got != want)
+        assert bad[0].size == 0, (fmt, delta, x[bad][:5], got[bad][:5], want[bad][:5])
+
+
+def test_zero_tensor_and_zero_rows():
+    t = torch.zeros((40, 64), dtype=torch.bfloat16)
+    t[3, 5] = -2.0
+    td = t.cuda()
+    op = qm.operand_of(td, -1)
+    d = qm.qm_scale(op, "e4m3", "channel").cpu().numpy()
+    want = oracle.scale(as3(t.float().numpy()), "e4m3", "channel").ravel()
+    assert np.array_equal(d, want) and d[0] == 1.0
+    codes, _, _, _ = qm.qm_quantize(op, "e4m3", "channel", None)
+    c = codes.cpu().numpy()[0]
+    assert c[3, 5] == 0xFE and c.sum() == 0xFE
+    z = torch.zeros((16, 32), dtype=torch.bfloat16).cuda()
+    assert qm.qm_scale(qm.operand_of(z, -1), "int8", "tensor").item() == 1.0
+
+
+def test_nonfinite_input_is_flagged_in_delta():
+    t = torch.ones((8, 64), dtype=torch.bfloat16)
+    t[2, 3] = float("inf")
+    d = qm.qm_scale(qm.operand_of(t.cuda(), -1), "int8", "channel").cpu().numpy()
+    assert not np.isfinite(d[2]) and np.isfinite(np.delete(d, 2)).all()
+    t[2, 3] = float("nan")
+    d = qm.qm_scale(qm.operand_of(t.cuda(), -1), "int8", "tensor").cpu().numpy()
+    assert not np.isfinite(d[0])
+
+
+def test_large_tensor_sampled():
+    # a size that spans every SM several times; scales exact, codes compared on sampled rows
+    t = make((4096, 3072), torch.bfloat16, 5, "n")
+    td = t.cuda()
+    x = as3(t.float().numpy())
+    for gran in ("tensor", "channel"):
+        for cd in (-1, -2):
+            op = qm.operand_of(td, cd)
+            xo = as3(oriented(t, cd))
+            want_d = oracle.scale(xo, "e4m3", gran)
+            codes, d, _, _ = qm.qm_quantize(op, "e4m3", gran, None)
+            assert np.array_equal(d.cpu().numpy(), want_d.ravel())
+            rows = np.random.default_rng(6).choice(xo.shape[1], 64, replace=False)
+            dsel = want_d if gran == "tensor" else want_d[:, rows]
+            want_c = oracle.quantize(xo[:, rows, :], "e4m3", dsel)
+            assert np.array_equal(codes.cpu().numpy()[:, rows, :xo.shape[2]], want_c)
