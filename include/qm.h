@@ -206,6 +206,20 @@ int32_t qm_version(void);
 /* Text of the last CUDA error seen by this thread inside the library ("" if none). */
 const char* qm_last_cuda_error(void);
 
+
+/*
+ * Measurement aids (no counterpart in the paper).
+ * qm_kernel_launches: how many kernels the library has launched in this
+ * process so far.  qm_profile_enable(1) makes every later qm_probe_layer record
+ * a CUDA event pair on the caller's stream around its fused tensor-core probe
+ * kernel; qm_profile_read waits for those events, returns the summed kernel
+ * time in milliseconds and the number of launches, and starts a new interval.
+ * Events are host objects; no device memory is involved.
+ */
+int64_t qm_kernel_launches(void);
+qm_status qm_profile_enable(int32_t on);
+qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -66,7 +66,8 @@ def quantize(x, fmt, delta):
     t = x / delta in float32; the code is the grid value nearest to t, a tie
     going to the value whose code is even (round-to-nearest-even); |t| above the
     largest expressible value saturates to it.  Magnitudes below half the
-    smallest positive grid value therefore become zero.  Returns uint8 bytes
+    smallest positive grid value therefore become zero (FP8: a zero that keeps
+    the sign bit of the input; INT8 has one zero).  Returns uint8 bytes
     (INT8: two's complement).
     The nearest value is found by comparing t with the midpoints of adjacent
     grid values, so no conversion instruction is involved.
@@ -82,11 +83,12 @@ def quantize(x, fmt, delta):
     below_top = idx < len(g) - 1
     tie = below_top & (a == mid[np.minimum(idx, len(mid) - 1)])
     idx = idx + (tie & (idx % 2 == 1))                   # tie: take the even code
-    neg = np.signbit(t) & (idx > 0)
     if fmt == "int8":
-        code = np.where(neg, 256 - idx, idx)
+        code = np.where(np.signbit(t) & (idx > 0), 256 - idx, idx)
     else:
-        code = np.where(neg, idx + 128, idx)
+        # FP8 is sign-magnitude with IEEE conventions (the FP8 rules the paper cites): the sign
+        # bit of the input survives rounding, so a negative value that rounds to zero is -0.
+        code = np.where(np.signbit(t), idx + 128, idx)
     return code.astype(np.uint8)
 
 

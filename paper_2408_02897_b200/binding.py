@@ -79,6 +79,9 @@ def lib():
             "qm_status_string": (C.c_char_p, [I32]),
             "qm_version": (I32, []),
             "qm_last_cuda_error": (C.c_char_p, []),
+            "qm_kernel_launches": (I64, []),
+            "qm_profile_enable": (I32, [I32]),
+            "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -254,3 +257,19 @@ def qm_probe_layer_host(L_host, R_host, contract_l, contract_r, fmt_l, fmt_r, gr
                                    C.byref(res), _ptr(plan.out), _ptr(plan.ws), plan.ws_bytes, _stream(stream))
     _check(st, "qm_probe_layer_host")
     return res, stage
+
+
+def kernel_launches():
+    """Kernels launched by the library in this process so far."""
+    return lib().qm_kernel_launches()
+
+
+def profile_enable(on=True):
+    _check(lib().qm_profile_enable(1 if on else 0), "qm_profile_enable")
+
+
+def profile_read():
+    """(summed milliseconds, launches) of the fused tensor-core probe kernel since the last read."""
+    ms, n = C.c_double(0), C.c_int32(0)
+    _check(lib().qm_profile_read(C.byref(ms), C.byref(n)), "qm_profile_read")
+    return ms.value, n.value

@@ -178,6 +178,7 @@ qm_status launch_simt_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int
   a.M = g.M; a.N = g.N; a.K = g.K; a.out_descaled = out_descaled; a.out_raw = out_raw;
   if (fmt_l == QM_FMT_INT8) simt_kernel<true, false><<<grid_of(g), kThreads, 0, s>>>(a);
   else simt_kernel<false, false><<<grid_of(g), kThreads, 0, s>>>(a);
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
@@ -195,6 +196,7 @@ qm_status launch_simt_probe(const View& L, const View& R, const uint8_t* cl, int
   a.M = L.nc; a.N = R.nc; a.K = L.c; a.partials = partials;
   if (fmt_l == QM_FMT_INT8) simt_kernel<true, true><<<grid_of(g), kThreads, 0, s>>>(a);
   else simt_kernel<false, true><<<grid_of(g), kThreads, 0, s>>>(a);
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }

@@ -448,7 +448,12 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   }
   dim3 grid((unsigned)((g.N + kBlockN - 1) / kBlockN), (unsigned)((g.M + kBlockM - 1) / kBlockM),
             (unsigned)g.batch);
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (MODE == kProbe) profile_events(&ev0, &ev1);
+  if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
   kern<<<grid, kThreads, smem_bytes<MODE>(), s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
+  if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }

@@ -101,6 +101,7 @@ int metric_blocks(int64_t count) {
 qm_status launch_metric_partials(const float* ref, const float* q, const float* den, int64_t count,
                                  double* partials, int nblocks, cudaStream_t s) {
   metric_partials_kernel<<<nblocks, kThreads, 0, s>>>(ref, q, den, count, partials);
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
@@ -108,6 +109,7 @@ qm_status launch_metric_partials(const float* ref, const float* q, const float* 
 qm_status launch_metric_finalize(const double* partials, int n, uint64_t count,
                                  const uint32_t* err_word, qm_metric_result* out, cudaStream_t s) {
   metric_finalize_kernel<<<1, kThreads, 0, s>>>(partials, n, count, err_word, out);
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }

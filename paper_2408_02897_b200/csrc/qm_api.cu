@@ -1,7 +1,10 @@
 // The C ABI: argument checks, workspace layout and launch sequencing.  All arithmetic of the
 // probe runs in the kernels of the other translation units.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "qm_internal.h"
 
@@ -25,6 +28,29 @@ int sm_count() {
   return n;
 }
 
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// profiling: a pool of event pairs recorded around the fused tensor-core probe kernel
+static std::mutex g_prof_mutex;
+static bool g_prof_on = false;
+static std::vector<cudaEvent_t> g_prof_events;   // start0, stop0, start1, stop1, ...
+static size_t g_prof_used = 0;
+
+void profile_events(cudaEvent_t* start, cudaEvent_t* stop) {
+  *start = *stop = nullptr;
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (!g_prof_on) return;
+  if (g_prof_used + 2 > g_prof_events.size()) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess) return;
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); return; }
+    g_prof_events.push_back(a); g_prof_events.push_back(b);
+  }
+  *start = g_prof_events[g_prof_used]; *stop = g_prof_events[g_prof_used + 1];
+  g_prof_used += 2;
+}
+
 namespace {
 
 bool valid_fmt(int f) { return f == QM_FMT_INT8 || f == QM_FMT_E4M3 || f == QM_FMT_E5M2; }
@@ -34,12 +60,17 @@ qm_status to_view(const qm_operand* x, View* v) {
   if (!x || !x->data) return QM_ERR_INVALID_ARG;
   if (x->dtype != QM_DT_F32 && x->dtype != QM_DT_BF16) return QM_ERR_INVALID_ARG;
   if (x->noncontract <= 0 || x->contract <= 0 || x->batch <= 0) return QM_ERR_INVALID_ARG;
-  if (x->stride_nc <= 0 || x->stride_c <= 0) return QM_ERR_INVALID_ARG;
-  if (x->stride_nc != 1 && x->stride_c != 1) return QM_ERR_UNSUPPORTED;
+  // the stride of an extent-1 dimension carries no information: give it the dense value
+  int64_t s_nc = x->stride_nc, s_c = x->stride_c;
+  if (x->noncontract == 1 && x->contract == 1) { s_nc = 8; s_c = 1; }
+  else if (x->noncontract == 1) s_nc = s_c == 1 ? ((x->contract + 7) & ~(int64_t)7) : 1;
+  else if (x->contract == 1) s_c = s_nc == 1 ? ((x->noncontract + 7) & ~(int64_t)7) : 1;
+  if (s_nc <= 0 || s_c <= 0) return QM_ERR_INVALID_ARG;
+  if (s_nc != 1 && s_c != 1) return QM_ERR_UNSUPPORTED;
   if (x->batch > 1 && x->stride_batch <= 0) return QM_ERR_INVALID_ARG;
   v->data = x->data; v->dtype = x->dtype;
   v->nc = x->noncontract; v->c = x->contract;
-  v->s_nc = x->stride_nc; v->s_c = x->stride_c;
+  v->s_nc = s_nc; v->s_c = s_c;
   v->batch = x->batch;
   // rows must not overlap
   if (v->s_c == 1 && v->nc > 1 && v->s_nc < v->c) return QM_ERR_INVALID_ARG;
@@ -305,5 +336,30 @@ const char* qm_status_string(int32_t st) {
 int32_t qm_version(void) { return 100; }
 
 const char* qm_last_cuda_error(void) { return qm::g_last_error; }
+
+int64_t qm_kernel_launches(void) { return (int64_t)qm::g_launches.load(); }
+
+qm_status qm_profile_enable(int32_t on) {
+  std::lock_guard<std::mutex> lock(qm::g_prof_mutex);
+  qm::g_prof_on = on != 0;
+  qm::g_prof_used = 0;
+  return QM_OK;
+}
+
+qm_status qm_profile_read(double* ms, int32_t* launches) {
+  if (!ms || !launches) return QM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(qm::g_prof_mutex);
+  double total = 0;
+  for (size_t i = 0; i + 1 < qm::g_prof_used; i += 2) {
+    QM_CUDA_OK(cudaEventSynchronize(qm::g_prof_events[i + 1]));
+    float t = 0;
+    QM_CUDA_OK(cudaEventElapsedTime(&t, qm::g_prof_events[i], qm::g_prof_events[i + 1]));
+    total += t;
+  }
+  *ms = total;
+  *launches = (int32_t)(qm::g_prof_used / 2);
+  qm::g_prof_used = 0;
+  return QM_OK;
+}
 
 }  // extern "C"

@@ -35,6 +35,12 @@ void note_cuda_error(cudaError_t e, const char* where);
 
 int sm_count();
 
+// Cumulative count of kernels this library has launched (profiling aid).
+void count_launch(int n = 1);
+// When profiling is on, returns an event pair to record around the fused tensor-core probe
+// kernel; nullptrs otherwise.
+void profile_events(cudaEvent_t* start, cudaEvent_t* stop);
+
 // ---- scale / quantize (scale_quantize.cu) ---------------------------------
 // amax: uint32 buffer (1 or batch*nc entries) that must be zero on entry; on exit it holds
 // the bit pattern of max|x| per group.

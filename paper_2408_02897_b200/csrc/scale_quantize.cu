@@ -443,6 +443,7 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
       absmax_cols_kernel<T><<<grid, block, 0, s>>>(p, x.nc, x.c, x.s_c, x.s_b, rows_per_block, amax);
     }
   }
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
@@ -472,6 +473,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, uint8_t* codes
         p, x.nc, x.c, x.s_c, x.s_b, delta, pc, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
         static_cast<__nv_bfloat16*>(kmaj_copy));
   }
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
@@ -492,6 +494,7 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
   else if (nvec <= 16) QM_SQ(16);
   else QM_SQ(32);
 #undef QM_SQ
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
@@ -505,6 +508,7 @@ qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream
 
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s) {
   finalize_delta_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(delta, n, fmt_qmax(fmt), err_word);
+  count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }

@@ -193,8 +193,16 @@ def test_rounding_against_outside_library(fmt, dt):
     t = t[np.abs(t) <= qmax(fmt)]
     lib = t.astype(dt).view(np.uint8)
     ours = oracle.quantize(t[None, :], fmt, np.array([1.0], np.float32))[0]
-    lib_v = oracle.dequantize(lib, fmt); our_v = oracle.dequantize(ours, fmt)
-    assert np.array_equal(lib_v, our_v)          # (-0 and +0 compare equal)
+    assert np.array_equal(lib, ours)             # byte for byte, signed zeros included
+    assert (ours == 0x80).any() and (ours == 0x00).any()
+
+
+def test_fp8_zero_keeps_sign_int8_does_not():
+    one = np.array([1.0], np.float32)
+    x = np.array([[-1e-30, 1e-30, -0.0, 0.0]], np.float32)
+    assert oracle.quantize(x, "e4m3", one)[0].tolist() == [0x80, 0, 0x80, 0]
+    assert oracle.quantize(x, "e5m2", one)[0].tolist() == [0x80, 0, 0x80, 0]
+    assert oracle.quantize(x, "int8", one)[0].tolist() == [0, 0, 0, 0]
 
 
 def test_int8_rounding_against_rint():
