@@ -1,0 +1,306 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized-matmul error probe on B200.
+
+A step is one pass of the whole probe path (scale, quantize, 8-bit product, reference and
+denominator products, Eq. 3 reduction) over every product of the workload.  The default
+workload is the BERT-base forward set (batch 8 x seq 512: QKV, attention output, FFN1, FFN2;
+E4M3 and INT8 with per-tensor scales): 8 probes per step.
+
+  python bench.py --gpus 1 --steps K --warmup W            -> one JSON line (this library)
+  python bench.py --impl reference ...                     -> one JSON line (CPU oracle)
+
+With N > 1 ranks (torchrun) every rank probes its own copy of the workload: the probes of a
+table are independent, there is no exchange step, so scaling is weak and no collective runs
+in the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2408_02897_b200 import workloads  # noqa: E402
+
+METRIC = "probe TFLOPS"
+UNIT = "TFLOP/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def build_workload(name):
+    if name == "bert_base_fwd":
+        return workloads.config2(), "BERT-base forward matmuls (batch 8 x seq 512), E4M3 + INT8, per-tensor scales"
+    if name == "bert_large_layer":
+        return workloads.config3(), "BERT-large layer fwd+dgrad+wgrad (batch 32 x seq 512), E4M3/E5M2, per-channel weights"
+    if name == "outlier":
+        return workloads.config4(), "FFN1 outlier stress [16384x1024]x[1024x4096], 3 formats x 2 granularities"
+    if name == "single":
+        return workloads.config1(), "single fp32 probe 128x256x256"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def probe_flops(ops):
+    """Flops of one step: the three products of Eq. 3 (8-bit, reference, denominator)."""
+    return sum(3.0 * workloads.op_flops(o)[1] for o in ops)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle_sample(ops, rows_per_op, seed=7):
+    """The CPU oracle, as it stands, on a bounded sample: `rows_per_op` output rows (all
+    columns) of every probe; scales and codes are still computed over the whole operands."""
+    import oracle
+    t0 = time.perf_counter()
+    flops = 0.0
+    for i, o in enumerate(ops):
+        (M, N, K, b), _ = workloads.op_flops(o)
+        rows = np.random.default_rng(seed + i).choice(M, min(rows_per_op, M), replace=False)
+        L, R = workloads.orient(o)
+        oracle.probe(L, R, o["fmt_l"], o["fmt_r"], o["gran_l"], o["gran_r"], rows=np.sort(rows))
+        flops += 3.0 * 2.0 * len(rows) * N * K * b
+    dt = time.perf_counter() - t0
+    return flops, dt
+
+
+def cpu_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count()
+
+
+def run_reference(args, ops, desc):
+    """--impl reference: the oracle on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = args.oracle_rows
+    for _ in range(min(args.warmup, 1)):
+        time_oracle_sample(ops, rows)
+    flops = secs = 0.0
+    for _ in range(args.steps):
+        f, t = time_oracle_sample(ops, rows)
+        flops += f; secs += t
+    val = flops / secs / 1e12
+    sample = f"{rows} of the output rows of each of the {len(ops)} probes per step (scales and codes over whole operands)"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "description": desc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bert_base_fwd")
+    ap.add_argument("--oracle-rows", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    ops, desc = build_workload(args.workload)
+    if args.impl == "reference":
+        if args.steps == 20 and args.warmup == 3:
+            args.steps, args.warmup = 3, 1
+        run_reference(args, ops, desc)
+        return
+
+    import paper_2408_02897_b200 as qm
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    qm.lib()   # fail now if the CUDA library is missing
+
+    # ---- inputs resident in HBM, one plan (workspace) per probe
+    dev_ops = []
+    for o in ops:
+        Ld, Rd = o["L"].cuda(), o["R"].cuda()
+        Lop, Rop = qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"])
+        plan = qm.ProbePlan(Lop, Rop, o["fmt_l"], o["fmt_r"], o["gran_l"], o["gran_r"], o["ref"])
+        dev_ops.append((Lop, Rop, plan))
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+
+    def step():
+        for Lop, Rop, plan in dev_ops:
+            plan.launch(Lop, Rop)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, each between its own event pair, L2 flushed in between
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = qm.kernel_launches()
+    qm.profile_enable(True)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for a, b in evs:
+        flush.zero_()
+        a.record()
+        step()
+        b.record()
+    barrier()
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    tc_ms, tc_launches = qm.profile_read()
+    qm.profile_enable(False)
+    launches = qm.kernel_launches() - launches0
+    clocks = sampler.stop()
+    total_ms = float(sum(step_ms))
+    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = t.item()
+    results = [plan.result() for _, _, plan in dev_ops]
+    if any(r.device_error for r in results):
+        raise SystemExit("device error flagged in a probe result")
+
+    flops_step = probe_flops(ops)
+    value = flops_step * args.steps * world / (total_ms * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point: H2D of every operand and D2H of the
+    # record inside the timed region
+    host_ops = [(o["L"].pin_memory(), o["R"].pin_memory(), o) for o in ops]
+    stages = [None] * len(ops)
+    h2d = sum(L.numel() * L.element_size() + R.numel() * R.element_size() for L, R, _ in host_ops)
+    d2h = 56 * len(ops)
+
+    def e2e_step():
+        for i, (Lh, Rh, o) in enumerate(host_ops):
+            _, stages[i] = qm.qm_probe_layer_host(Lh, Rh, o["cl"], o["cr"], o["fmt_l"], o["fmt_r"], o["gran_l"],
+                                                  o["gran_r"], o["ref"], stage=stages[i])
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()                      # each call synchronises the stream itself
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = flops_step * e2e_steps * world / (t.item() * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    # composite tensor bound of the fused kernel: per 2MNK, one product at the 8-bit rate
+    # (2 x bf16) and two at the bf16 rate  ->  3 / (1/(2P) + 2/P) = 1.2 P in summed flops
+    peak_tflops = 1.2 * peaks["bf16_tflops"]
+    achieved = flops_step * args.steps / (tc_ms * 1e-3) / 1e12 if tc_ms > 0 else None
+    roofline = {"bound": "tensor", "kernel": "tc_kernel<probe> (fused 8-bit + reference + denominator products, Eq. 3 epilogue)",
+                "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
+                "frac": achieved / peak_tflops if achieved else None, "traffic": None,
+                "peak_source": f"1.2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}",
+                "launches": tc_launches, "avg_launch_ms": tc_ms / max(tc_launches, 1)}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp8/int8 x bf16 (fp32/int32 accumulate)", "data": "synthetic",
+            "config": {"workload": args.workload, "description": desc, "probes_per_step": len(ops),
+                       "flops_counted": "3 x 2MNK per probe (8-bit, reference and denominator products)",
+                       "l2": "256 MiB buffer written between timed steps"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches), "roofline": roofline,
+            "pct_of_composite_tensor_peak": 100.0 * value / peak_tflops,
+            "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
+    if not args.no_cpu_baseline and world == 1:
+        f, s = time_oracle_sample(ops, args.oracle_rows)
+        line["cpu_baseline"] = {"value": f / s / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{args.oracle_rows} of the output rows of each of the {len(ops)} probes "
+                                          f"(scales and codes over whole operands), {s:.1f} s"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
