@@ -1,0 +1,48 @@
+"""Runs one probe (or only its scale/quantize stage) a few times on synthetic operands.
+
+Meant to be the command profiled by ncu on a small case, e.g.
+  python -m paper_2408_02897_b200.profile_case --M 4096 --N 3072 --K 768 --fmt e4m3 --iters 3
+"""
+import argparse
+
+import torch
+
+from . import binding as qm
+from . import workloads
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--M", type=int, default=4096)
+    ap.add_argument("--N", type=int, default=3072)
+    ap.add_argument("--K", type=int, default=768)
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--fmt", default="e4m3")
+    ap.add_argument("--gran", default="tensor")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--stage", default="probe", choices=["probe", "quantize"])
+    ap.add_argument("--r-layout", default="kn", choices=["kn", "nk"], help="R stored [K,N] or [N,K]")
+    a = ap.parse_args()
+    rng = workloads._rng(11)
+    lead = (a.batch,) if a.batch > 1 else ()
+    L = workloads.normal(rng, lead + (a.M, a.K)).cuda()
+    R = workloads.normal(rng, lead + ((a.K, a.N) if a.r_layout == "kn" else (a.N, a.K)), 0.02).cuda()
+    Lop = qm.operand_of(L, -1)
+    Rop = qm.operand_of(R, -2 if a.r_layout == "kn" else -1)
+    if a.stage == "probe":
+        plan = qm.ProbePlan(Lop, Rop, a.fmt, a.fmt, a.gran, a.gran)
+        for _ in range(a.iters):
+            plan.launch(Lop, Rop)
+        torch.cuda.synchronize()
+        r = plan.result()
+        print("mean_be", r.derived()["mean_be"], "device_error", r.device_error)
+    else:
+        for _ in range(a.iters):
+            qm.qm_quantize(Lop, a.fmt, a.gran, None, want_abs=True)
+            qm.qm_quantize(Rop, a.fmt, a.gran, None, want_abs=True, want_kmaj=(a.r_layout == "kn"))
+        torch.cuda.synchronize()
+        print("done")
+
+
+if __name__ == "__main__":
+    main()
