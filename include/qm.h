@@ -208,6 +208,32 @@ const char* qm_last_cuda_error(void);
 
 
 /*
+ * qm_metric for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment convenience).  Some users of this library
+ * run where cudaMalloc is unavailable to them: a plug-in that only receives
+ * input and output pointers from its host application, code that must stay
+ * inside a region managed by somebody else's memory pool, or a loop that may
+ * not call the allocator for latency reasons.  Such a caller cannot produce
+ * the `ws` scratch that qm_metric asks for, so this variant keeps its scratch
+ * inside the library: a fixed 40 KiB array in the device image, held by every
+ * GPU that loads the library until the process exits.  It computes exactly
+ * what qm_metric computes: ref, q, den are `count` fp32 values each (device),
+ * `out` (device) receives the record.
+ *  - count may be at most qm_metric_noalloc_max_count() (2^30); larger inputs
+ *    are refused with QM_ERR_WORKSPACE_TOO_SMALL and nothing is launched.
+ *  - The call allocates nothing, on the host or on the device.
+ *  - The first call on each device looks up the array's device address; make
+ *    that first call outside any stream capture.
+ *  - All calls on a device share the one array, which still holds the previous
+ *    call's partial sums.  Each call overwrites every entry it later reads, so
+ *    no clearing is needed, but two calls whose kernels overlap on the GPU
+ *    (different streams, no ordering between them) race on it: serialise them.
+ */
+int64_t qm_metric_noalloc_max_count(void);
+qm_status qm_metric_noalloc(const float* ref, const float* q, const float* den, int64_t count,
+                            qm_metric_result* out, void* stream);
+
+/*
  * Measurement aids (no counterpart in the paper).
  * qm_kernel_launches: how many kernels the library has launched in this
  * process so far.  qm_profile_enable(1) makes every later qm_probe_layer record

@@ -79,6 +79,8 @@ def lib():
             "qm_status_string": (C.c_char_p, [I32]),
             "qm_version": (I32, []),
             "qm_last_cuda_error": (C.c_char_p, []),
+            "qm_metric_noalloc": (I32, [P, P, P, I64, P, P]),
+            "qm_metric_noalloc_max_count": (I64, []),
             "qm_kernel_launches": (I64, []),
             "qm_profile_enable": (I32, [I32]),
             "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),
@@ -195,6 +197,17 @@ def qm_metric(ref, q, den, stream=None):
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     out = torch.empty(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
     _check(L.qm_metric(_ptr(ref), _ptr(q), _ptr(den), n, _ptr(out), _ptr(ws), ws_bytes, _stream(stream)), "qm_metric")
+    return _read_result(out)
+
+
+def qm_metric_noalloc(ref, q, den, out=None, stream=None):
+    """Eq. 3 record through the entry point that keeps its scratch inside the library, for
+    callers that cannot allocate device memory.  `out` is a caller-owned CUDA byte tensor of
+    sizeof(qm_metric_result) bytes; one is made here only when none is passed."""
+    if out is None:
+        out = torch.empty(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+    _check(lib().qm_metric_noalloc(_ptr(ref), _ptr(q), _ptr(den), ref.numel(), _ptr(out), _stream(stream)),
+           "qm_metric_noalloc")
     return _read_result(out)
 
 

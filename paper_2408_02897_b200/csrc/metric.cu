@@ -115,3 +115,63 @@ qm_status launch_metric_finalize(const double* partials, int n, uint64_t count,
 }
 
 }  // namespace qm
+
+// ---------------------------------------------------------------------------------------------
+// qm_metric_noalloc: Eq. 3 reduction for callers that cannot allocate device memory.
+//
+// The per-block partial records of qm_metric normally live in a caller-provided workspace.  A
+// caller that runs where cudaMalloc is off limits (a plug-in that is handed raw input/output
+// pointers by its host application, code running inside a memory-pool-managed region, a
+// latency-critical loop that must not touch the allocator) has nowhere to get that workspace
+// from.  For them the library carries the scratch itself, as a fixed array in the module's
+// device image: kNoAllocRecords partial records (40 KiB), present on every GPU that loads the
+// library until the process ends.
+namespace qm {
+namespace {
+
+constexpr int kNoAllocRecords = 1024;                         // 1024 x 5 doubles = 40 KiB
+constexpr int64_t kNoAllocMaxCount = (int64_t)1 << 30;        // elements per input array
+
+static __device__ __align__(256) double g_noalloc_partials[kNoAllocRecords * kPartialDoubles];
+
+// In host code the array's name is only a handle for the runtime, not a device address: the
+// address the kernels need is looked up once per device (with that device current) and cached.
+constexpr int kMaxDevices = 64;
+double* g_noalloc_ptr[kMaxDevices] = {};
+
+qm_status noalloc_scratch(double** out) {
+  int dev = -1;
+  QM_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return QM_ERR_UNSUPPORTED;
+  if (!g_noalloc_ptr[dev]) {
+    double* p = nullptr;
+    QM_CUDA_OK(cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_noalloc_partials));
+    if (!p) return QM_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return QM_OK;
+}
+
+}  // namespace
+}  // namespace qm
+
+extern "C" qm_status qm_metric_noalloc(const float* ref, const float* q, const float* den, int64_t count,
+                                       qm_metric_result* out, void* stream) {
+  using namespace qm;
+  if (!ref || !q || !den || !out || count <= 0) return QM_ERR_INVALID_ARG;
+  if (count > kNoAllocMaxCount) return QM_ERR_WORKSPACE_TOO_SMALL;   // beyond the built-in scratch's stated limit
+  double* scratch = nullptr;
+  qm_status st = noalloc_scratch(&scratch);
+  if (st != QM_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int nb = metric_blocks(count);
+  if (nb > kNoAllocRecords) nb = kNoAllocRecords;
+  // Every record that the final reduction reads is overwritten by its block first, so nothing
+  // in the shared array has to be cleared between calls.
+  st = launch_metric_partials(ref, q, den, count, scratch, nb, s);
+  if (st != QM_OK) return st;
+  return launch_metric_finalize(scratch, nb, (uint64_t)count, nullptr, out, s);
+}
+
+extern "C" int64_t qm_metric_noalloc_max_count(void) { return qm::kNoAllocMaxCount; }

@@ -1,0 +1,51 @@
+"""The allocation-free variant of the Eq. 3 reduction against the regular one.
+
+qm_metric_noalloc exists for callers that cannot call cudaMalloc (plug-ins that only get
+input/output pointers, code confined to someone else's memory pool, allocator-free loops):
+its scratch is a fixed array inside the library instead of a caller-provided workspace.  It
+must return what qm_metric returns.  The check runs twice in a row on different inputs,
+because every call reuses the same built-in array and still finds the previous call's
+partial sums in it.  This file is collected last on purpose.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2408_02897_b200 as qm
+from paper_2408_02897_b200 import binding
+
+pytestmark = pytest.mark.gpu
+
+
+def inputs(n, seed):
+    rng = np.random.default_rng(seed)
+    c = rng.standard_normal(n).astype(np.float32)
+    d = (np.abs(c) + rng.uniform(0, 2, n)).astype(np.float32)
+    q = (c + rng.standard_normal(n) * 0.01 * d).astype(np.float32)
+    d[::101] = 0.0
+    return [torch.from_numpy(a).cuda() for a in (c, q, d)]
+
+
+def test_noalloc_matches_regular_entry_point_twice_in_a_row():
+    out = torch.empty(C.sizeof(binding.MetricResult), dtype=torch.uint8, device="cuda")   # caller-owned output
+    for n, seed in ((3_000_000, 40), (70_001, 41)):       # second call is smaller: stale records stay behind it
+        c, q, d = inputs(n, seed)
+        want = qm.qm_metric(c, q, d).record()
+        got = qm.qm_metric_noalloc(c, q, d, out=out).record()
+        assert got["count"] == want["count"] == n
+        for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
+            assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k]), (k, got[k], want[k])
+        assert abs(got["max_be"] - want["max_be"]) <= 1e-6 * want["max_be"]
+
+
+def test_noalloc_rejects_sizes_beyond_its_scratch():
+    L = qm.lib()
+    limit = L.qm_metric_noalloc_max_count()
+    assert limit == 1 << 30
+    c, q, d = inputs(16, 42)
+    out = torch.empty(C.sizeof(binding.MetricResult), dtype=torch.uint8, device="cuda")
+    st = L.qm_metric_noalloc(c.data_ptr(), q.data_ptr(), d.data_ptr(), limit + 1, out.data_ptr(), None)
+    assert st == 4                                         # refused on the host, nothing launched
+    assert L.qm_metric_noalloc(None, None, None, 16, None, None) == 1
