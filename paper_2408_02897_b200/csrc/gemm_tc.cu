@@ -1,14 +1,19 @@
 // Tensor-core products of the probe for sm_100a: tcgen05.mma with accumulators in tensor
-// memory, operands staged in shared memory by TMA, warp-specialised roles.
+// memory, operands staged in shared memory by TMA, warp-specialised persistent CTAs.
 //
-// One CTA owns one 128 x 128 output tile.  Roles:
-//   warp 0      TMA producer: per k-block, bulk-tensor loads of every operand tile into a ring
-//   warp 1      allocates tensor memory; one lane issues the MMAs of each k-block
-//   warps 2..5  epilogue: read the accumulators with tcgen05.ld and either reduce the Eq. 3
-//               statistics (probe) or store the product.
+// Each CTA walks a static list of 128 x 128 output tiles (tile = blockIdx.x + i * gridDim.x).
+//   warp 0      TMA producer: per 32-wide k-block, bulk-tensor loads of every operand tile into
+//               a ring of stages; it runs ahead across tile boundaries, so the next tile's first
+//               stages arrive while the current tile is still in its epilogue
+//   warp 1      allocates tensor memory once; one lane issues the MMAs of each k-block
+//   warps 2..9  epilogue: read the accumulators with tcgen05.ld (a warp may touch the lane
+//               quarter warp_id % 4; the two warps of a quarter split the columns) and either
+//               reduce the Eq. 3 statistics (probe) or store the product.
 // In probe mode three accumulators live side by side in tensor memory: the reference L.R
-// (bf16 operands, kind::f16), the denominator |L|.|R| (bf16, kind::f16) and the 8-bit product
-// (kind::f8f6f4 or kind::i8), so no M x N matrix ever goes to HBM.
+// (bf16 operands, kind::f16, columns 0..127), the denominator |L|.|R| (bf16, kind::f16, columns
+// 128..255) and the 8-bit product (kind::f8f6f4 or kind::i8, columns 256..383), so no M x N
+// matrix ever goes to HBM.  The CTA keeps its Eq. 3 statistics in registers across tiles and
+// writes one record; the last CTA to finish adds the records up in a fixed order.
 //
 // Every wait is bounded: when one gives up it raises QM_DEVERR_TIMEOUT in the caller's error
 // word and flags the CTA, after which every role falls through to the common exit, tensor
@@ -21,37 +26,43 @@
 namespace qm {
 namespace {
 
-constexpr int kBlockM = 128, kBlockN = 128, kBlockK = 64;
-constexpr int kThreads = 192;
-constexpr uint32_t kBf16TileBytes = kBlockM * kBlockK * 2;   // 16 KB, 128-byte rows
-constexpr uint32_t kLpTileBytes = kBlockM * kBlockK;         //  8 KB,  64-byte rows
+constexpr int kBlockM = 128, kBlockN = 128, kBlockK = 32;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;                // 320
+constexpr uint32_t kBf16TileBytes = kBlockM * kBlockK * 2;   // 8 KB, 64-byte rows
+constexpr uint32_t kLpTileBytes = kBlockM * kBlockK;         // 4 KB, 32-byte rows
+constexpr int kMaxStages = 10;
 
 enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2 };
 
 template <int MODE> struct Cfg;
 template <> struct Cfg<kProbe> {
-  static constexpr int kStages = 2;
-  static constexpr uint32_t kStageBytes = 4 * kBf16TileBytes + 2 * kLpTileBytes;
+  static constexpr int kStages = 5;
+  static constexpr uint32_t kStageBytes = 4 * kBf16TileBytes + 2 * kLpTileBytes;   // 40 KB
   static constexpr uint32_t kTmemCols = 512;
 };
 template <> struct Cfg<kLpOnly> {
-  static constexpr int kStages = 8;
-  static constexpr uint32_t kStageBytes = 2 * kLpTileBytes;
+  static constexpr int kStages = 10;
+  static constexpr uint32_t kStageBytes = 2 * kLpTileBytes;                        // 8 KB
   static constexpr uint32_t kTmemCols = 128;
 };
 template <> struct Cfg<kRefOnly> {
-  static constexpr int kStages = 6;
-  static constexpr uint32_t kStageBytes = 2 * kBf16TileBytes;
+  static constexpr int kStages = 10;
+  static constexpr uint32_t kStageBytes = 2 * kBf16TileBytes;                      // 16 KB
   static constexpr uint32_t kTmemCols = 128;
 };
 
 struct KernelArgs {
   int64_t M, N, K;
+  int32_t tiles_m, tiles_n, num_tiles;
   const float* dl; int pc_l;      // per-channel flags: delta indexed by batch*M + row
   const float* dr; int pc_r;
   float* out_descaled;            // LpOnly / RefOnly
   void* out_raw;                  // LpOnly
-  double* partials;               // Probe
+  double* partials;               // Probe: gridDim.x records
+  uint32_t* done_counter;         // Probe: zero on entry
+  qm_metric_result* result;       // Probe
+  uint64_t count;                 // Probe: batch * M * N
   uint32_t* err_word;
   uint32_t idesc_lp;              // instruction descriptor of the 8-bit MMA
 };
@@ -66,6 +77,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -121,17 +135,17 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
                : "memory");
 }
 
-// Shared-memory matrix descriptor, contraction-major tile with a 128- or 64-byte swizzle:
-// rows are one swizzle span wide, eight consecutive rows form one swizzle atom, atoms follow
-// each other every 8 * span bytes (the "stride byte offset").
+// Shared-memory matrix descriptor, contraction-major tile whose rows are exactly one swizzle
+// span wide (64 bytes for the bf16 tiles, 32 bytes for the code tiles): eight consecutive rows
+// form one swizzle atom, atoms follow each other every 8 * span bytes ("stride byte offset").
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t span_bytes) {
-  const uint64_t layout = span_bytes == 128 ? 2ull : 4ull;      // SWIZZLE_128B : SWIZZLE_64B
+  const uint64_t layout = span_bytes == 128 ? 2ull : (span_bytes == 64 ? 4ull : 6ull);
   uint64_t d = 0;
   d |= (uint64_t)((addr & 0x3ffffu) >> 4);                      // start address / 16
   d |= (uint64_t)1 << 16;                                       // leading byte offset (unused here)
   d |= (uint64_t)((8u * span_bytes) >> 4) << 32;                // stride byte offset / 16
   d |= (uint64_t)1 << 46;                                       // descriptor version of sm_100
-  d |= layout << 61;
+  d |= layout << 61;                                            // swizzle mode
   return d;
 }
 
@@ -182,14 +196,40 @@ __host__ __device__ constexpr uint32_t make_idesc(uint32_t c_fmt, uint32_t a_fmt
 }
 
 struct Shared {
-  uint64_t full[8];
-  uint64_t empty[8];
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
   uint64_t tmem_full;
+  uint64_t tmem_empty;
   uint32_t tmem_base;
   uint32_t abort_flag;
-  float delta_r[kBlockN];
-  double red[5][4];
+  uint32_t is_last;
+  uint32_t pad;
+  float delta_r[2][kBlockN];
+  double red[5][kEpiWarps];
 };
+
+// Named barrier 1 over the 256 epilogue threads, returning the OR of `flag` over all of them.
+__device__ __forceinline__ bool epi_barrier_any(bool flag) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 1, 256, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)flag)
+      : "memory");
+  return out != 0;
+}
+
+struct TileCoord { int m_tile, n_tile, b; };
+__device__ __forceinline__ TileCoord tile_coord(int t, const KernelArgs& a) {
+  TileCoord c;
+  const int per_b = a.tiles_m * a.tiles_n;
+  c.b = t / per_b;
+  const int r = t - c.b * per_b;
+  c.m_tile = r / a.tiles_n;
+  c.n_tile = r - c.m_tile * a.tiles_n;
+  return c;
+}
 
 template <int MODE, int LPKIND>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -200,12 +240,11 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   using C = Cfg<MODE>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
-  // tiles need 1024-byte alignment for the 128-byte swizzle
+  // tiles start on a 1024-byte boundary (a multiple of every swizzle atom size)
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Shared* sh = reinterpret_cast<Shared*>(tiles + (size_t)kStages * C::kStageBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tile = blockIdx.x, m_tile = blockIdx.y, b = blockIdx.z;
   const int num_kb = (int)((a.K + kBlockK - 1) / kBlockK);
   volatile uint32_t* abort_flag = &sh->abort_flag;
 
@@ -215,7 +254,9 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
     mbar_init(smem_u32(&sh->tmem_full), 1);
+    mbar_init(smem_u32(&sh->tmem_empty), kEpiWarps);
     sh->abort_flag = 0;
+    sh->is_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -231,25 +272,34 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t use = kb / kStages;
-        if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, a.err_word)) break;
-        const uint32_t bar = smem_u32(&sh->full[s]);
-        mbar_expect_tx(bar, C::kStageBytes);
-        uint32_t dst = smem_u32(tiles + (size_t)s * C::kStageBytes);
-        const int k0 = kb * kBlockK, r0 = m_tile * kBlockM, c0 = n_tile * kBlockN;
-        if (MODE == kProbe || MODE == kRefOnly) {
-          tma_load_3d(dst, &map_l, bar, k0, r0, b); dst += kBf16TileBytes;
-          tma_load_3d(dst, &map_r, bar, k0, c0, b); dst += kBf16TileBytes;
-        }
-        if (MODE == kProbe) {
-          tma_load_3d(dst, &map_la, bar, k0, r0, b); dst += kBf16TileBytes;
-          tma_load_3d(dst, &map_ra, bar, k0, c0, b); dst += kBf16TileBytes;
-        }
-        if (MODE == kProbe || MODE == kLpOnly) {
-          tma_load_3d(dst, &map_cl, bar, k0, r0, b); dst += kLpTileBytes;
-          tma_load_3d(dst, &map_cr, bar, k0, c0, b);
+      uint32_t g = 0;                                           // running k-block count
+      bool ok = true;
+      for (int t = blockIdx.x; t < a.num_tiles && ok; t += gridDim.x) {
+        const TileCoord tc = tile_coord(t, a);
+        const int r0 = tc.m_tile * kBlockM, c0 = tc.n_tile * kBlockN;
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          const uint32_t use = g / kStages;
+          if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, a.err_word)) {
+            ok = false;
+            break;
+          }
+          const uint32_t bar = smem_u32(&sh->full[s]);
+          mbar_expect_tx(bar, C::kStageBytes);
+          uint32_t dst = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          const int k0 = kb * kBlockK;
+          if (MODE == kProbe || MODE == kRefOnly) {
+            tma_load_3d(dst, &map_l, bar, k0, r0, tc.b); dst += kBf16TileBytes;
+            tma_load_3d(dst, &map_r, bar, k0, c0, tc.b); dst += kBf16TileBytes;
+          }
+          if (MODE == kProbe) {
+            tma_load_3d(dst, &map_la, bar, k0, r0, tc.b); dst += kBf16TileBytes;
+            tma_load_3d(dst, &map_ra, bar, k0, c0, tc.b); dst += kBf16TileBytes;
+          }
+          if (MODE == kProbe || MODE == kLpOnly) {
+            tma_load_3d(dst, &map_cl, bar, k0, r0, tc.b); dst += kLpTileBytes;
+            tma_load_3d(dst, &map_cr, bar, k0, c0, tc.b);
+          }
         }
       }
     }
@@ -257,88 +307,101 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kBlockM, kBlockN);
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % kStages;
-        const uint32_t use = kb / kStages;
-        if (!mbar_wait(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) break;
+      uint32_t g = 0, it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < a.num_tiles && ok; t += gridDim.x, ++it) {
+        // the epilogue must have drained the previous tile's accumulators
+        if (it > 0 && !mbar_wait(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
-        uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-        if (MODE == kProbe || MODE == kRefOnly) {
-          const uint64_t dl = smem_desc(base, 128), dr = smem_desc(base + kBf16TileBytes, 128);
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          const uint32_t use = g / kStages;
+          if (!mbar_wait(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
+          tc_fence_after();
+          uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          if (MODE == kProbe || MODE == kRefOnly) {
+            const uint64_t dl = smem_desc(base, 64), dr = smem_desc(base + kBf16TileBytes, 64);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-            mma_ss<kKindF16>(tmem_base, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-          base += 2 * kBf16TileBytes;
-        }
-        if (MODE == kProbe) {
-          const uint64_t dl = smem_desc(base, 128), dr = smem_desc(base + kBf16TileBytes, 128);
+            for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+              mma_ss<kKindF16>(tmem_base, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
+            base += 2 * kBf16TileBytes;
+          }
+          if (MODE == kProbe) {
+            const uint64_t dl = smem_desc(base, 64), dr = smem_desc(base + kBf16TileBytes, 64);
 #pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)
-            mma_ss<kKindF16>(tmem_base + 128, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-          base += 2 * kBf16TileBytes;
+            for (int k = 0; k < kBlockK / 16; ++k)
+              mma_ss<kKindF16>(tmem_base + 128, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
+            base += 2 * kBf16TileBytes;
+          }
+          if (MODE == kProbe || MODE == kLpOnly) {
+            const uint32_t col = MODE == kProbe ? 256u : 0u;
+            // one 32-byte step covers the whole k-block
+            mma_ss<LPKIND>(tmem_base + col, smem_desc(base, 32), smem_desc(base + kLpTileBytes, 32),
+                           a.idesc_lp, kb != 0);
+          }
+          tc_commit(smem_u32(&sh->empty[s]));       // frees the stage once these MMAs have read it
         }
-        if (MODE == kProbe || MODE == kLpOnly) {
-          const uint32_t col = MODE == kProbe ? 256u : 0u;
-          const uint64_t dl = smem_desc(base, 64), dr = smem_desc(base + kLpTileBytes, 64);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k)   // 32 bytes per step
-            mma_ss<LPKIND>(tmem_base + col, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0);
-        }
-        tc_commit(smem_u32(&sh->empty[s]));       // frees the stage once these MMAs have read it
+        if (ok) tc_commit(smem_u32(&sh->tmem_full));  // accumulators of this tile complete
       }
-      tc_commit(smem_u32(&sh->tmem_full));        // accumulators complete
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
-    const int et = (warp - 2) * 32 + lane;        // 0..127
-    {
-      const int64_t col = (int64_t)n_tile * kBlockN + et;
-      float d = 1.f;
-      if (MODE != kRefOnly) d = a.pc_r ? (col < a.N ? __ldg(a.dr + (int64_t)b * a.N + col) : 0.f) : __ldg(a.dr);
-      sh->delta_r[et] = d;
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    const int64_t row = (int64_t)m_tile * kBlockM + q * 32 + lane;
-    const bool row_ok = row < a.M;
-    float dlv = 1.f;
-    if (MODE != kRefOnly) dlv = a.pc_l ? (row_ok ? __ldg(a.dl + (int64_t)b * a.M + row) : 0.f) : __ldg(a.dl);
-
-    const bool ok = mbar_wait(smem_u32(&sh->tmem_full), 0, abort_flag, a.err_word);
-    tc_fence_after();
+    const int h = (warp - 2) >> 2;                // which 64-column half of the tile
+    const int et = (warp - 2) * 32 + lane;        // 0..255
+    const float dl_tensor = (MODE != kRefOnly && !a.pc_l) ? __ldg(a.dl) : 1.f;
+    const float dr_tensor = (MODE != kRefOnly && !a.pc_r) ? __ldg(a.dr) : 1.f;
     double sbe = 0, mbe = 0, sd2 = 0, sr2 = 0, sn2 = 0;
-    if (ok) {
+    uint32_t it = 0;
+    for (int t = blockIdx.x; t < a.num_tiles; t += gridDim.x, ++it) {
+      const TileCoord tc = tile_coord(t, a);
+      float* dr_s = sh->delta_r[it & 1];
+      if (et < kBlockN) {
+        const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
+        float d = dr_tensor;
+        if (MODE != kRefOnly && a.pc_r) d = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
+        dr_s[et] = d;
+      }
+      const int64_t row = (int64_t)tc.m_tile * kBlockM + q * 32 + lane;
+      const bool row_ok = row < a.M;
+      float dlv = dl_tensor;
+      if (MODE != kRefOnly && a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
+
+      const bool ok = mbar_wait(smem_u32(&sh->tmem_full), it & 1, abort_flag, a.err_word);
+      // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
+      if (epi_barrier_any(!ok)) break;
+      tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < kBlockN / 32; ++c) {
-        const int64_t col0 = (int64_t)n_tile * kBlockN + c * 32;
+      for (int c = 0; c < 2; ++c) {
+        const int cc0 = h * 64 + c * 32;          // first column of this chunk inside the tile
+        const int64_t col0 = (int64_t)tc.n_tile * kBlockN + cc0;
         if (col0 >= a.N) break;                   // uniform across the warp
         if (MODE == kProbe) {
           uint32_t rc[32], rd[32], rq[32];
-          tmem_ld32(lane_addr + c * 32, rc);
-          tmem_ld32(lane_addr + 128 + c * 32, rd);
-          tmem_ld32(lane_addr + 256 + c * 32, rq);
+          tmem_ld32(lane_addr + cc0, rc);
+          tmem_ld32(lane_addr + 128 + cc0, rd);
+          tmem_ld32(lane_addr + 256 + cc0, rq);
           tmem_ld_wait();
           float fbe = 0, fmx = 0, fd2 = 0, fr2 = 0, fn2 = 0;
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            const float cc = __uint_as_float(rc[j]), dd = __uint_as_float(rd[j]);
+            const float cv = __uint_as_float(rc[j]), dd = __uint_as_float(rd[j]);
             const float acc = LPKIND == kKindI8 ? (float)(int)rq[j] : __uint_as_float(rq[j]);
-            const float qq = acc * (dlv * sh->delta_r[c * 32 + j]);
-            const float diff = cc - qq;
+            const float diff = fmaf(-(acc * dlv), dr_s[cc0 + j], cv);      // C - A * dl * dr
             const bool live = col0 + j < a.N;
             float be = dd != 0.f ? __fdividef(fabsf(diff), dd) : 0.f;
             if (!live) be = 0.f;
             fbe += be; fmx = fmaxf(fmx, be);
-            if (live) { fd2 = fmaf(diff, diff, fd2); fr2 = fmaf(cc, cc, fr2); fn2 = fmaf(dd, dd, fn2); }
+            if (live) { fd2 = fmaf(diff, diff, fd2); fr2 = fmaf(cv, cv, fr2); fn2 = fmaf(dd, dd, fn2); }
           }
           if (row_ok) { sbe += fbe; mbe = fmax(mbe, (double)fmx); sd2 += fd2; sr2 += fr2; sn2 += fn2; }
         } else {
           uint32_t r[32];
-          tmem_ld32(lane_addr + c * 32, r);
+          tmem_ld32(lane_addr + cc0, r);
           tmem_ld_wait();
           if (row_ok) {
-            const int64_t o = ((int64_t)b * a.M + row) * a.N + col0;
+            const int64_t o = ((int64_t)tc.b * a.M + row) * a.N + col0;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               if (col0 + j < a.N) {
@@ -346,7 +409,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
                   a.out_descaled[o + j] = __uint_as_float(r[j]);
                 } else {
                   const float acc = LPKIND == kKindI8 ? (float)(int)r[j] : __uint_as_float(r[j]);
-                  if (a.out_descaled) a.out_descaled[o + j] = acc * (dlv * sh->delta_r[c * 32 + j]);
+                  if (a.out_descaled) a.out_descaled[o + j] = acc * (dlv * dr_s[cc0 + j]);
                   if (a.out_raw) reinterpret_cast<uint32_t*>(a.out_raw)[o + j] = r[j];
                 }
               }
@@ -354,6 +417,10 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           }
         }
       }
+      // this warp has finished reading the accumulators of the tile
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty));
     }
     if (MODE == kProbe) {
 #pragma unroll
@@ -368,15 +435,44 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
         sh->red[0][warp - 2] = sbe; sh->red[1][warp - 2] = mbe; sh->red[2][warp - 2] = sd2;
         sh->red[3][warp - 2] = sr2; sh->red[4][warp - 2] = sn2;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       if (et == 0) {
         double r[5] = {0, 0, 0, 0, 0};
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kEpiWarps; ++i) {
           r[0] += sh->red[0][i]; r[1] = fmax(r[1], sh->red[1][i]); r[2] += sh->red[2][i];
           r[3] += sh->red[3][i]; r[4] += sh->red[4][i];
         }
-        const int64_t blk = ((int64_t)blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
-        for (int i = 0; i < 5; ++i) a.partials[blk * kPartialDoubles + i] = r[i];
+        double* rec = a.partials + (int64_t)blockIdx.x * kPartialDoubles;
+        for (int i = 0; i < 5; ++i) __stcg(rec + i, r[i]);
+        __threadfence();
+        const uint32_t prev = atomicAdd(a.done_counter, 1u);
+        sh->is_last = prev == gridDim.x - 1 ? 1u : 0u;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (sh->is_last && warp == 2) {
+        // last CTA: every record is visible; fixed-order sum (lane l takes records l, l+32, ...)
+        __threadfence();
+        double r[5] = {0, 0, 0, 0, 0};
+        for (int i = lane; i < (int)gridDim.x; i += 32) {
+          const double* rec = a.partials + (int64_t)i * kPartialDoubles;
+          r[0] += __ldcg(rec); r[1] = fmax(r[1], __ldcg(rec + 1)); r[2] += __ldcg(rec + 2);
+          r[3] += __ldcg(rec + 3); r[4] += __ldcg(rec + 4);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          r[0] += __shfl_xor_sync(0xffffffffu, r[0], o);
+          r[1] = fmax(r[1], __shfl_xor_sync(0xffffffffu, r[1], o));
+          r[2] += __shfl_xor_sync(0xffffffffu, r[2], o);
+          r[3] += __shfl_xor_sync(0xffffffffu, r[3], o);
+          r[4] += __shfl_xor_sync(0xffffffffu, r[4], o);
+        }
+        if (lane == 0) {
+          a.result->sum_be = r[0]; a.result->max_be = r[1]; a.result->sum_diff2 = r[2];
+          a.result->sum_ref2 = r[3]; a.result->sum_den2 = r[4];
+          a.result->count = a.count;
+          a.result->device_error = a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u;
+          a.result->reserved = 0;
+        }
       }
     }
   }
@@ -409,7 +505,8 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over [batch][rows][K] with the contracting index contiguous; box = 64 x 128 x 1.
+// Tensor map over [batch][rows][K] with the contracting index contiguous; box = 32 x 128 x 1,
+// swizzle span = row width of the box (64 bytes for bf16, 32 bytes for codes).
 bool make_map(CUtensorMap* m, const void* base, bool bf16, int64_t K, int64_t rows, int64_t batch,
               int64_t ld_elems, int64_t sb_elems) {
   EncodeTiledFn fn = encode_fn();
@@ -422,7 +519,7 @@ bool make_map(CUtensorMap* m, const void* base, bool bf16, int64_t K, int64_t ro
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -438,6 +535,26 @@ size_t smem_bytes() {
   return (size_t)Cfg<MODE>::kStages * Cfg<MODE>::kStageBytes + sizeof(Shared) + 1024;
 }
 
+bool shape_ok(GemmShape g) {
+  if (!(g.M > 0 && g.N > 0 && g.K > 0 && g.batch > 0 && (g.K % 16) == 0)) return false;
+  if (g.M >= (1ll << 31) || g.N >= (1ll << 31) || g.K >= (1ll << 31) || g.batch >= (1ll << 31)) return false;
+  const int64_t tiles = ((g.M + kBlockM - 1) / kBlockM) * ((g.N + kBlockN - 1) / kBlockN) * g.batch;
+  return tiles < (1ll << 31);
+}
+
+void fill_tiles(KernelArgs* ka, GemmShape g) {
+  ka->M = g.M; ka->N = g.N; ka->K = g.K;
+  ka->tiles_m = (int32_t)((g.M + kBlockM - 1) / kBlockM);
+  ka->tiles_n = (int32_t)((g.N + kBlockN - 1) / kBlockN);
+  ka->num_tiles = (int32_t)((int64_t)ka->tiles_m * ka->tiles_n * g.batch);
+}
+
+int grid_size(GemmShape g) {
+  const int64_t tiles = ((g.M + kBlockM - 1) / kBlockM) * ((g.N + kBlockN - 1) / kBlockN) * g.batch;
+  const int sms = sm_count();
+  return (int)(tiles < sms ? tiles : sms);
+}
+
 template <int MODE, int LPKIND>
 qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cudaStream_t s) {
   auto kern = tc_kernel<MODE, LPKIND>;
@@ -446,28 +563,19 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
     QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<MODE>()));
     attr_done = true;
   }
-  dim3 grid((unsigned)((g.N + kBlockN - 1) / kBlockN), (unsigned)((g.M + kBlockM - 1) / kBlockM),
-            (unsigned)g.batch);
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (MODE == kProbe) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
-  kern<<<grid, kThreads, smem_bytes<MODE>(), s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
+  kern<<<grid_size(g), kThreads, smem_bytes<MODE>(), s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
   if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
   count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
 
-bool shape_ok(GemmShape g) {
-  return g.M > 0 && g.N > 0 && g.K > 0 && g.batch > 0 && (g.K % 16) == 0 && g.batch <= 65535 &&
-         (g.M + kBlockM - 1) / kBlockM <= 65535 && g.M < (1ll << 31) && g.N < (1ll << 31) && g.K < (1ll << 31);
-}
-
 }  // namespace
 
-int tc_probe_tiles(GemmShape g) {
-  return (int)(((g.N + kBlockN - 1) / kBlockN) * ((g.M + kBlockM - 1) / kBlockM) * g.batch);
-}
+int tc_probe_records(GemmShape g) { return grid_size(g); }
 
 qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   if (!shape_ok(p.g)) return QM_ERR_UNSUPPORTED;
@@ -482,9 +590,11 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
             make_map(&maps[5], p.cr, false, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
   KernelArgs ka{};
-  ka.M = g.M; ka.N = g.N; ka.K = g.K;
+  fill_tiles(&ka, g);
   ka.dl = p.dl; ka.pc_l = p.gran_l == QM_GRAN_CHANNEL; ka.dr = p.dr; ka.pc_r = p.gran_r == QM_GRAN_CHANNEL;
-  ka.partials = p.partials; ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+  ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
+  ka.count = (uint64_t)(g.M * g.N * g.batch);
+  ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
   return p.fmt_l == QM_FMT_INT8 ? launch<kProbe, kKindI8>(maps, ka, g, s)
                                 : launch<kProbe, kKindF8>(maps, ka, g, s);
 }
@@ -500,7 +610,7 @@ qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int g
   if (!ok) return QM_ERR_CUDA;
   maps[0] = maps[1] = maps[2] = maps[3] = maps[4];
   KernelArgs ka{};
-  ka.M = g.M; ka.N = g.N; ka.K = g.K;
+  fill_tiles(&ka, g);
   ka.dl = dl; ka.pc_l = gran_l == QM_GRAN_CHANNEL; ka.dr = dr; ka.pc_r = gran_r == QM_GRAN_CHANNEL;
   ka.out_descaled = out_descaled; ka.out_raw = out_raw; ka.err_word = err_word;
   ka.idesc_lp = lp_idesc(fmt_l, fmt_r);
@@ -517,7 +627,8 @@ qm_status launch_tc_gemm_ref(const void* l, const void* r, GemmShape g, float* o
   if (!ok) return QM_ERR_CUDA;
   maps[2] = maps[3] = maps[4] = maps[5] = maps[0];
   KernelArgs ka{};
-  ka.M = g.M; ka.N = g.N; ka.K = g.K; ka.out_descaled = out; ka.err_word = err_word;
+  fill_tiles(&ka, g);
+  ka.out_descaled = out; ka.err_word = err_word;
   return launch<kRefOnly, kKindF8>(maps, ka, g, s);
 }
 

@@ -113,7 +113,7 @@ Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg) {
     w.off_kr = R.c_contig() ? 0 : take((size_t)(R.batch * R.nc * R.c) * 2);
   }
   GemmShape g{L.nc, R.nc, L.c, L.batch};
-  w.n_part = w.tc ? tc_probe_tiles(g) : simt_probe_blocks(g);
+  w.n_part = w.tc ? tc_probe_records(g) : simt_probe_blocks(g);
   w.off_part = take(sizeof(double) * kPartialDoubles * (size_t)w.n_part);
   w.total = o;
   return w;
@@ -284,10 +284,11 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
     p.fmt_l = cfg->fmt_l; p.fmt_r = cfg->fmt_r;
     p.dl = dl; p.gran_l = cfg->gran_l; p.dr = dr; p.gran_r = cfg->gran_r;
     p.g = g; p.partials = part; p.err_word = err;
-    st = launch_tc_probe(p, s);
-  } else {
-    st = launch_simt_probe(L, R, cl, cfg->fmt_l, dl, cfg->gran_l, cr, cfg->fmt_r, dr, cfg->gran_r, part, s);
+    p.done_counter = err + 1;               // second word of the cleared error slot
+    p.result = out;
+    return launch_tc_probe(p, s);           // the last CTA writes the record
   }
+  st = launch_simt_probe(L, R, cl, cfg->fmt_l, dl, cfg->gran_l, cr, cfg->fmt_r, dr, cfg->gran_r, part, s);
   if (st != QM_OK) return st;
   return launch_metric_finalize(part, w.n_part, (uint64_t)(g.M * g.N * g.batch), err, out, s);
 }

@@ -87,10 +87,12 @@ struct TcProbeArgs {
   const float* dl; int gran_l;
   const float* dr; int gran_r;
   GemmShape g;
-  double* partials;                         // tc_probe_tiles(g) records
+  double* partials;                         // tc_probe_records(g) records
+  uint32_t* done_counter;                   // zero on entry; counts finished CTAs
+  qm_metric_result* result;                 // written by the last CTA to finish
   uint32_t* err_word;
 };
-int tc_probe_tiles(GemmShape g);
+int tc_probe_records(GemmShape g);
 qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
 qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
                             const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
