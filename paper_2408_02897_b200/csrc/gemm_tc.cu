@@ -1,23 +1,29 @@
 // Tensor-core products of the probe for sm_100a: tcgen05.mma with accumulators in tensor
-// memory, operands staged in shared memory by TMA, warp-specialised persistent CTAs.
+// memory, operands staged in shared memory by TMA, warp-specialised persistent CTA pairs.
 //
-// Each CTA walks a static list of 128 x 128 output tiles (tile = blockIdx.x + i * gridDim.x).
-//   warp 0      TMA producer: per 32-wide k-block, bulk-tensor loads of every operand tile into
-//               a ring of stages; it runs ahead across tile boundaries, so the next tile's first
-//               stages arrive while the current tile is still in its epilogue
-//   warp 1      allocates tensor memory once; one lane issues the MMAs of each k-block
-//   warps 2..9  epilogue: read the accumulators with tcgen05.ld (a warp may touch the lane
-//               quarter warp_id % 4; the two warps of a quarter split the columns) and either
-//               reduce the Eq. 3 statistics (probe) or store the product.
+// Two CTAs on the two SMs of a TPC form a cluster and work on one 256 x 128 output tile with
+// cta_group::2 MMAs: each CTA stages its own 128 rows of the left operand and HALF (64 rows) of
+// the right operand's tile, so every byte of the right operand enters and leaves shared memory
+// once per pair instead of once per SM.  The kernel is bound by shared-memory traffic (TMA
+// writes plus MMA operand reads), so this is what sets its speed.
+//
+// Roles in each CTA (320 threads):
+//   warp 0      TMA producer: per 64-wide k-block, bulk-tensor loads of its operand tiles into a
+//               ring of stages; completion is signalled on the LEADER CTA's barrier.  It runs
+//               ahead across tile boundaries, so loads overlap the epilogue.
+//   warp 1      allocates tensor memory; in the leader CTA one lane issues the pair's MMAs
+//   warps 2..9  epilogue: read the CTA's 128 x 128 accumulators with tcgen05.ld (a warp may touch
+//               the lane quarter warp_id % 4; the two warps of a quarter split the columns) and
+//               either reduce the Eq. 3 statistics (probe) or store the product.
 // In probe mode three accumulators live side by side in tensor memory: the reference L.R
 // (bf16 operands, kind::f16, columns 0..127), the denominator |L|.|R| (bf16, kind::f16, columns
 // 128..255) and the 8-bit product (kind::f8f6f4 or kind::i8, columns 256..383), so no M x N
-// matrix ever goes to HBM.  The CTA keeps its Eq. 3 statistics in registers across tiles and
+// matrix ever goes to HBM.  A CTA keeps its Eq. 3 statistics in registers across tiles and
 // writes one record; the last CTA to finish adds the records up in a fixed order.
 //
-// Every wait is bounded: when one gives up it raises QM_DEVERR_TIMEOUT in the caller's error
-// word and flags the CTA, after which every role falls through to the common exit, tensor
-// memory is freed and the kernel returns.
+// Every mbarrier wait is bounded: when one gives up it raises QM_DEVERR_TIMEOUT in the caller's
+// error word and flags the CTA, after which every role falls through to the common exit, tensor
+// memory is freed and the kernel returns.  No load uses cluster multicast.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -26,50 +32,75 @@
 namespace qm {
 namespace {
 
-constexpr int kBlockM = 128, kBlockN = 128, kBlockK = 32;
+constexpr int kBlockM = 128;             // rows per CTA
+constexpr int kPairM = 256;              // rows per CTA pair
+constexpr int kBlockN = 128;             // columns per tile
+constexpr int kHalfN = 64;               // right-operand rows staged by each CTA
+constexpr int kBlockK = 64;
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = 64 + 32 * kEpiWarps;                // 320
-constexpr uint32_t kBf16TileBytes = kBlockM * kBlockK * 2;   // 8 KB, 64-byte rows
-constexpr uint32_t kLpTileBytes = kBlockM * kBlockK;         // 4 KB, 32-byte rows
-constexpr int kMaxStages = 10;
+constexpr int kThreads = 64 + 32 * kEpiWarps;                     // 320
+constexpr uint32_t kABf16 = kBlockM * kBlockK * 2;                // 16 KB, 128-byte rows
+constexpr uint32_t kALp = kBlockM * kBlockK;                      //  8 KB,  64-byte rows
+constexpr uint32_t kBBf16 = kHalfN * kBlockK * 2;                 //  8 KB
+constexpr uint32_t kBLp = kHalfN * kBlockK;                       //  4 KB
+constexpr int kMaxStages = 8;
 
 enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2 };
 
+// Stage layout: left-operand tiles first (L, |L|, codes), then the right-operand halves.
 template <int MODE> struct Cfg;
 template <> struct Cfg<kProbe> {
-  static constexpr int kStages = 5;
-  static constexpr uint32_t kStageBytes = 4 * kBf16TileBytes + 2 * kLpTileBytes;   // 40 KB
+  static constexpr int kStages = 3;
+  static constexpr uint32_t kOffL = 0, kOffLa = kABf16, kOffCl = 2 * kABf16;
+  static constexpr uint32_t kOffR = 2 * kABf16 + kALp, kOffRa = kOffR + kBBf16, kOffCr = kOffRa + kBBf16;
+  static constexpr uint32_t kStageBytes = kOffCr + kBLp;          // 60 KB
   static constexpr uint32_t kTmemCols = 512;
 };
 template <> struct Cfg<kLpOnly> {
-  static constexpr int kStages = 10;
-  static constexpr uint32_t kStageBytes = 2 * kLpTileBytes;                        // 8 KB
+  static constexpr int kStages = 8;
+  static constexpr uint32_t kOffL = 0, kOffLa = 0, kOffCl = 0, kOffR = 0, kOffRa = 0, kOffCr = kALp;
+  static constexpr uint32_t kStageBytes = kALp + kBLp;            // 12 KB
   static constexpr uint32_t kTmemCols = 128;
 };
 template <> struct Cfg<kRefOnly> {
-  static constexpr int kStages = 10;
-  static constexpr uint32_t kStageBytes = 2 * kBf16TileBytes;                      // 16 KB
+  static constexpr int kStages = 6;
+  static constexpr uint32_t kOffL = 0, kOffLa = 0, kOffCl = 0, kOffR = kABf16, kOffRa = 0, kOffCr = 0;
+  static constexpr uint32_t kStageBytes = kABf16 + kBBf16;        // 24 KB
   static constexpr uint32_t kTmemCols = 128;
 };
 
 struct KernelArgs {
   int64_t M, N, K;
-  int32_t tiles_m, tiles_n, num_tiles;
-  const float* dl; int pc_l;      // per-channel flags: delta indexed by batch*M + row
+  int32_t tiles_m, tiles_n, num_tiles;   // tiles of 256 x 128
+  const float* dl; int pc_l;             // per-channel flags: delta indexed by batch*M + row
   const float* dr; int pc_r;
-  float* out_descaled;            // LpOnly / RefOnly
-  void* out_raw;                  // LpOnly
-  double* partials;               // Probe: gridDim.x records
-  uint32_t* done_counter;         // Probe: zero on entry
-  qm_metric_result* result;       // Probe
-  uint64_t count;                 // Probe: batch * M * N
+  float* out_descaled;                   // LpOnly / RefOnly
+  void* out_raw;                         // LpOnly
+  double* partials;                      // Probe: gridDim.x records
+  uint32_t* done_counter;                // Probe: zero on entry
+  qm_metric_result* result;              // Probe
+  uint64_t count;                        // Probe: batch * M * N
   uint32_t* err_word;
-  uint32_t idesc_lp;              // instruction descriptor of the 8-bit MMA
+  uint32_t idesc_lp;                     // instruction descriptor of the 8-bit MMA
 };
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -78,14 +109,15 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// arrive on a barrier given by its shared::cluster address (own CTA or the peer)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -118,25 +150,31 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+// Tile load into this CTA's shared memory; the byte count is credited to the barrier at
+// `bar_cluster_addr`, which may live in the peer CTA (cta_group::2 form).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
                                             int c0, int c1, int c2) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
       " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      ::"r"(dst), "l"(map), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-               : "memory");
+// Arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once all MMAs
+// issued so far have completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(mask) : "memory");
 }
 
 // Shared-memory matrix descriptor, contraction-major tile whose rows are exactly one swizzle
-// span wide (64 bytes for the bf16 tiles, 32 bytes for the code tiles): eight consecutive rows
+// span wide (128 bytes for the bf16 tiles, 64 bytes for the code tiles): eight consecutive rows
 // form one swizzle atom, atoms follow each other every 8 * span bytes ("stride byte offset").
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t span_bytes) {
   const uint64_t layout = span_bytes == 128 ? 2ull : (span_bytes == 64 ? 4ull : 6ull);
@@ -151,23 +189,24 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t span_bytes
 
 enum MmaKind { kKindF16 = 0, kKindF8 = 1, kKindI8 = 2 };
 
+// D[256 x N] (+)= A[256 x k] . B[N x k]^T across the CTA pair; issued by one thread of the leader.
 template <int KIND>
-__device__ __forceinline__ void mma_ss(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
-                                       uint32_t accumulate) {
+__device__ __forceinline__ void mma_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
+                                         uint32_t accumulate) {
   if (KIND == kKindF16) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
   } else if (KIND == kKindF8) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
   } else {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
   }
 }
@@ -196,10 +235,10 @@ __host__ __device__ constexpr uint32_t make_idesc(uint32_t c_fmt, uint32_t a_fmt
 }
 
 struct Shared {
-  uint64_t full[kMaxStages];
-  uint64_t empty[kMaxStages];
-  uint64_t tmem_full;
-  uint64_t tmem_empty;
+  uint64_t full[kMaxStages];     // used in the leader CTA: both CTAs' loads of a stage have landed
+  uint64_t empty[kMaxStages];    // per CTA: the pair's MMAs have finished reading the stage
+  uint64_t tmem_full;            // per CTA: the tile's accumulators are complete
+  uint64_t tmem_empty;           // leader: both CTAs' epilogues have drained the accumulators
   uint32_t tmem_base;
   uint32_t abort_flag;
   uint32_t is_last;
@@ -231,6 +270,29 @@ __device__ __forceinline__ TileCoord tile_coord(int t, const KernelArgs& a) {
   return c;
 }
 
+// Eq. 3 statistics of 32 consecutive columns of one row.
+struct Stats { float be, mx, d2, r2, n2; };
+
+template <int LPKIND, bool RAGGED>
+__device__ __forceinline__ void stats32(const uint32_t (&rc)[32], const uint32_t (&rd)[32], const uint32_t (&rq)[32],
+                                        float dlv, const float* dr_s, bool per_col, float dr_tensor, int n_live,
+                                        Stats& s) {
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const float cv = __uint_as_float(rc[j]), dd = __uint_as_float(rd[j]);
+    const float acc = LPKIND == kKindI8 ? (float)(int)rq[j] : __uint_as_float(rq[j]);
+    const float drj = per_col ? dr_s[j] : dr_tensor;
+    const float diff = fmaf(-(acc * dlv), drj, cv);                 // C - A * delta_l * delta_r
+    // D == 0 implies C == Q == 0, so clamping the divisor keeps BE = 0 there without a branch
+    float be = __fdividef(fabsf(diff), fmaxf(dd, 1e-37f));
+    if (RAGGED) {
+      if (j >= n_live) continue;
+    }
+    s.be += be; s.mx = fmaxf(s.mx, be);
+    s.d2 = fmaf(diff, diff, s.d2); s.r2 = fmaf(cv, cv, s.r2); s.n2 = fmaf(dd, dd, s.n2);
+  }
+}
+
 template <int MODE, int LPKIND>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r,
@@ -240,11 +302,14 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   using C = Cfg<MODE>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
-  // tiles start on a 1024-byte boundary (a multiple of every swizzle atom size)
+  // tiles start on a 1024-byte boundary (the 128-byte swizzle atom); the offset is the same in
+  // both CTAs of the pair because their dynamic shared memory starts at the same address
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Shared* sh = reinterpret_cast<Shared*>(tiles + (size_t)kStages * C::kStageBytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();                   // 0 = leader
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_kb = (int)((a.K + kBlockK - 1) / kBlockK);
   volatile uint32_t* abort_flag = &sh->abort_flag;
 
@@ -254,29 +319,32 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
     mbar_init(smem_u32(&sh->tmem_full), 1);
-    mbar_init(smem_u32(&sh->tmem_empty), kEpiWarps);
+    mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
     sh->abort_flag = 0;
     sh->is_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                      smem_u32(&sh->tmem_base)), "r"(C::kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  __syncwarp();
+  cluster_sync();          // the peer's barriers and tensor memory exist before anyone uses them
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
       uint32_t g = 0;                                           // running k-block count
       bool ok = true;
-      for (int t = blockIdx.x; t < a.num_tiles && ok; t += gridDim.x) {
+      for (int t = pair; t < a.num_tiles && ok; t += num_pairs) {
         const TileCoord tc = tile_coord(t, a);
-        const int r0 = tc.m_tile * kBlockM, c0 = tc.n_tile * kBlockN;
+        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
+        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;     // this CTA's half of the right operand
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t use = g / kStages;
@@ -284,33 +352,34 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             ok = false;
             break;
           }
-          const uint32_t bar = smem_u32(&sh->full[s]);
-          mbar_expect_tx(bar, C::kStageBytes);
-          uint32_t dst = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          // one barrier (the leader's) collects the bytes of both CTAs
+          if (rank == 0) mbar_expect_tx(smem_u32(&sh->full[s]), 2 * C::kStageBytes);
+          const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
+          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
           const int k0 = kb * kBlockK;
           if (MODE == kProbe || MODE == kRefOnly) {
-            tma_load_3d(dst, &map_l, bar, k0, r0, tc.b); dst += kBf16TileBytes;
-            tma_load_3d(dst, &map_r, bar, k0, c0, tc.b); dst += kBf16TileBytes;
+            tma_load_3d(base + C::kOffL, &map_l, bar, k0, r0, tc.b);
+            tma_load_3d(base + C::kOffR, &map_r, bar, k0, c0, tc.b);
           }
           if (MODE == kProbe) {
-            tma_load_3d(dst, &map_la, bar, k0, r0, tc.b); dst += kBf16TileBytes;
-            tma_load_3d(dst, &map_ra, bar, k0, c0, tc.b); dst += kBf16TileBytes;
+            tma_load_3d(base + C::kOffLa, &map_la, bar, k0, r0, tc.b);
+            tma_load_3d(base + C::kOffRa, &map_ra, bar, k0, c0, tc.b);
           }
           if (MODE == kProbe || MODE == kLpOnly) {
-            tma_load_3d(dst, &map_cl, bar, k0, r0, tc.b); dst += kLpTileBytes;
-            tma_load_3d(dst, &map_cr, bar, k0, c0, tc.b);
+            tma_load_3d(base + C::kOffCl, &map_cl, bar, k0, r0, tc.b);
+            tma_load_3d(base + C::kOffCr, &map_cr, bar, k0, c0, tc.b);
           }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kBlockM, kBlockN);
+    // ------------------------------------------------------------ MMA issuer (leader CTA only)
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
       uint32_t g = 0, it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < a.num_tiles && ok; t += gridDim.x, ++it) {
-        // the epilogue must have drained the previous tile's accumulators
+      for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
+        // both epilogues must have drained the previous tile's accumulators
         if (it > 0 && !mbar_wait(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
@@ -318,51 +387,50 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           const uint32_t use = g / kStages;
           if (!mbar_wait(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
           tc_fence_after();
-          uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
           if (MODE == kProbe || MODE == kRefOnly) {
-            const uint64_t dl = smem_desc(base, 64), dr = smem_desc(base + kBf16TileBytes, 64);
+            const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-              mma_ss<kKindF16>(tmem_base, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-            base += 2 * kBf16TileBytes;
+              mma_pair<kKindF16>(tmem_base, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
           }
           if (MODE == kProbe) {
-            const uint64_t dl = smem_desc(base, 64), dr = smem_desc(base + kBf16TileBytes, 64);
+            const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)
-              mma_ss<kKindF16>(tmem_base + 128, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-            base += 2 * kBf16TileBytes;
+              mma_pair<kKindF16>(tmem_base + 128, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
           }
           if (MODE == kProbe || MODE == kLpOnly) {
             const uint32_t col = MODE == kProbe ? 256u : 0u;
-            // one 32-byte step covers the whole k-block
-            mma_ss<LPKIND>(tmem_base + col, smem_desc(base, 32), smem_desc(base + kLpTileBytes, 32),
-                           a.idesc_lp, kb != 0);
+            const uint64_t dl = smem_desc(base + C::kOffCl, 64), dr = smem_desc(base + C::kOffCr, 64);
+#pragma unroll
+            for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
+              mma_pair<LPKIND>(tmem_base + col, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0);
           }
-          tc_commit(smem_u32(&sh->empty[s]));       // frees the stage once these MMAs have read it
+          tc_commit_pair(smem_u32(&sh->empty[s]));        // frees the stage in both CTAs
         }
-        if (ok) tc_commit(smem_u32(&sh->tmem_full));  // accumulators of this tile complete
+        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full)); // this tile's accumulators are complete
       }
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..9)
+    // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
     const int h = (warp - 2) >> 2;                // which 64-column half of the tile
     const int et = (warp - 2) * 32 + lane;        // 0..255
     const float dl_tensor = (MODE != kRefOnly && !a.pc_l) ? __ldg(a.dl) : 1.f;
     const float dr_tensor = (MODE != kRefOnly && !a.pc_r) ? __ldg(a.dr) : 1.f;
+    const bool per_col = MODE != kRefOnly && a.pc_r;
+    const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
     double sbe = 0, mbe = 0, sd2 = 0, sr2 = 0, sn2 = 0;
     uint32_t it = 0;
-    for (int t = blockIdx.x; t < a.num_tiles; t += gridDim.x, ++it) {
+    for (int t = pair; t < a.num_tiles; t += num_pairs, ++it) {
       const TileCoord tc = tile_coord(t, a);
       float* dr_s = sh->delta_r[it & 1];
-      if (et < kBlockN) {
+      if (per_col && et < kBlockN) {
         const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
-        float d = dr_tensor;
-        if (MODE != kRefOnly && a.pc_r) d = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
-        dr_s[et] = d;
+        dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
       }
-      const int64_t row = (int64_t)tc.m_tile * kBlockM + q * 32 + lane;
+      const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
       const bool row_ok = row < a.M;
       float dlv = dl_tensor;
       if (MODE != kRefOnly && a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
@@ -377,25 +445,17 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
         const int cc0 = h * 64 + c * 32;          // first column of this chunk inside the tile
         const int64_t col0 = (int64_t)tc.n_tile * kBlockN + cc0;
         if (col0 >= a.N) break;                   // uniform across the warp
+        const int n_live = (int)(a.N - col0 < 32 ? a.N - col0 : 32);
         if (MODE == kProbe) {
           uint32_t rc[32], rd[32], rq[32];
           tmem_ld32(lane_addr + cc0, rc);
           tmem_ld32(lane_addr + 128 + cc0, rd);
           tmem_ld32(lane_addr + 256 + cc0, rq);
           tmem_ld_wait();
-          float fbe = 0, fmx = 0, fd2 = 0, fr2 = 0, fn2 = 0;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float cv = __uint_as_float(rc[j]), dd = __uint_as_float(rd[j]);
-            const float acc = LPKIND == kKindI8 ? (float)(int)rq[j] : __uint_as_float(rq[j]);
-            const float diff = fmaf(-(acc * dlv), dr_s[cc0 + j], cv);      // C - A * dl * dr
-            const bool live = col0 + j < a.N;
-            float be = dd != 0.f ? __fdividef(fabsf(diff), dd) : 0.f;
-            if (!live) be = 0.f;
-            fbe += be; fmx = fmaxf(fmx, be);
-            if (live) { fd2 = fmaf(diff, diff, fd2); fr2 = fmaf(cv, cv, fr2); fn2 = fmaf(dd, dd, fn2); }
-          }
-          if (row_ok) { sbe += fbe; mbe = fmax(mbe, (double)fmx); sd2 += fd2; sr2 += fr2; sn2 += fn2; }
+          Stats st{0.f, 0.f, 0.f, 0.f, 0.f};
+          if (n_live == 32) stats32<LPKIND, false>(rc, rd, rq, dlv, dr_s + cc0, per_col, dr_tensor, 32, st);
+          else stats32<LPKIND, true>(rc, rd, rq, dlv, dr_s + cc0, per_col, dr_tensor, n_live, st);
+          if (row_ok) { sbe += st.be; mbe = fmax(mbe, (double)st.mx); sd2 += st.d2; sr2 += st.r2; sn2 += st.n2; }
         } else {
           uint32_t r[32];
           tmem_ld32(lane_addr + cc0, r);
@@ -404,12 +464,13 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             const int64_t o = ((int64_t)tc.b * a.M + row) * a.N + col0;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              if (col0 + j < a.N) {
+              if (j < n_live) {
                 if (MODE == kRefOnly) {
                   a.out_descaled[o + j] = __uint_as_float(r[j]);
                 } else {
                   const float acc = LPKIND == kKindI8 ? (float)(int)r[j] : __uint_as_float(r[j]);
-                  if (a.out_descaled) a.out_descaled[o + j] = acc * (dlv * dr_s[cc0 + j]);
+                  const float drj = per_col ? dr_s[cc0 + j] : dr_tensor;
+                  if (a.out_descaled) a.out_descaled[o + j] = acc * (dlv * drj);
                   if (a.out_raw) reinterpret_cast<uint32_t*>(a.out_raw)[o + j] = r[j];
                 }
               }
@@ -417,10 +478,10 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           }
         }
       }
-      // this warp has finished reading the accumulators of the tile
+      // this warp has finished reading the accumulators of the tile: tell the leader's MMA lane
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty));
+      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
     }
     if (MODE == kProbe) {
 #pragma unroll
@@ -478,11 +539,16 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   }
 
   // ---------------------------------------------------------------- common exit
+  // Neither CTA may leave while the other can still read its shared memory, signal its
+  // barriers or write its tensor memory.
   tc_fence_before();
   __syncthreads();
+  __syncwarp();
+  cluster_sync();
   if (warp == 1) {
+    __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols)
                  : "memory");
   }
 }
@@ -505,9 +571,9 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// Tensor map over [batch][rows][K] with the contracting index contiguous; box = 32 x 128 x 1,
-// swizzle span = row width of the box (64 bytes for bf16, 32 bytes for codes).
-bool make_map(CUtensorMap* m, const void* base, bool bf16, int64_t K, int64_t rows, int64_t batch,
+// Tensor map over [batch][rows][K] with the contracting index contiguous; box = 64 x box_rows x 1,
+// swizzle span = row width of the box (128 bytes for bf16, 64 bytes for codes).
+bool make_map(CUtensorMap* m, const void* base, bool bf16, int box_rows, int64_t K, int64_t rows, int64_t batch,
               int64_t ld_elems, int64_t sb_elems) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -515,19 +581,19 @@ bool make_map(CUtensorMap* m, const void* base, bool bf16, int64_t K, int64_t ro
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
   cuuint64_t sb = batch > 1 ? (cuuint64_t)sb_elems * es : (cuuint64_t)rows * ld_elems * es;
   cuuint64_t strides[2] = {(cuuint64_t)ld_elems * es, sb};
-  cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)kBlockM, 1};
+  cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
+                  bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
 uint32_t lp_idesc(int fmt_l, int fmt_r) {
-  if (fmt_l == QM_FMT_INT8) return make_idesc(2, 1, 1, kBlockM, kBlockN);          // s8 x s8 -> s32
+  if (fmt_l == QM_FMT_INT8) return make_idesc(2, 1, 1, kPairM, kBlockN);           // s8 x s8 -> s32
   const uint32_t fa = fmt_l == QM_FMT_E4M3 ? 0u : 1u, fb = fmt_r == QM_FMT_E4M3 ? 0u : 1u;
-  return make_idesc(1, fa, fb, kBlockM, kBlockN);                                  // fp8 x fp8 -> f32
+  return make_idesc(1, fa, fb, kPairM, kBlockN);                                   // fp8 x fp8 -> f32
 }
 
 template <int MODE>
@@ -535,24 +601,32 @@ size_t smem_bytes() {
   return (size_t)Cfg<MODE>::kStages * Cfg<MODE>::kStageBytes + sizeof(Shared) + 1024;
 }
 
+int64_t tile_count(GemmShape g) {
+  return ((g.M + kPairM - 1) / kPairM) * ((g.N + kBlockN - 1) / kBlockN) * g.batch;
+}
+
 bool shape_ok(GemmShape g) {
   if (!(g.M > 0 && g.N > 0 && g.K > 0 && g.batch > 0 && (g.K % 16) == 0)) return false;
   if (g.M >= (1ll << 31) || g.N >= (1ll << 31) || g.K >= (1ll << 31) || g.batch >= (1ll << 31)) return false;
-  const int64_t tiles = ((g.M + kBlockM - 1) / kBlockM) * ((g.N + kBlockN - 1) / kBlockN) * g.batch;
-  return tiles < (1ll << 31);
+  return tile_count(g) < (1ll << 31);
 }
 
 void fill_tiles(KernelArgs* ka, GemmShape g) {
   ka->M = g.M; ka->N = g.N; ka->K = g.K;
-  ka->tiles_m = (int32_t)((g.M + kBlockM - 1) / kBlockM);
+  ka->tiles_m = (int32_t)((g.M + kPairM - 1) / kPairM);
   ka->tiles_n = (int32_t)((g.N + kBlockN - 1) / kBlockN);
-  ka->num_tiles = (int32_t)((int64_t)ka->tiles_m * ka->tiles_n * g.batch);
+  ka->num_tiles = (int32_t)tile_count(g);
 }
 
+// CTA pairs that can be resident at once (one per TPC unless the device says fewer).
+int g_max_pairs = 0;
+int max_pairs() { return g_max_pairs > 0 ? g_max_pairs : sm_count() / 2; }
+
+// CTAs to launch: two per tile, at most the resident number of pairs.
 int grid_size(GemmShape g) {
-  const int64_t tiles = ((g.M + kBlockM - 1) / kBlockM) * ((g.N + kBlockN - 1) / kBlockN) * g.batch;
-  const int sms = sm_count();
-  return (int)(tiles < sms ? tiles : sms);
+  const int64_t tiles = tile_count(g);
+  const int pairs = max_pairs();
+  return 2 * (int)(tiles < pairs ? tiles : pairs);
 }
 
 template <int MODE, int LPKIND>
@@ -563,13 +637,38 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
     QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<MODE>()));
     attr_done = true;
   }
+  if (MODE == kProbe && g_max_pairs == 0) {
+    // the probe configuration has the largest footprint: its residency bounds the grid of all modes
+    cudaLaunchConfig_t q{};
+    q.gridDim = dim3((unsigned)(2 * (sm_count() / 2))); q.blockDim = dim3(kThreads);
+    q.dynamicSmemBytes = smem_bytes<MODE>();
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa; q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &q) == cudaSuccess && n > 0)
+      g_max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+    else
+      g_max_pairs = sm_count() / 2;
+    (void)cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid_size(g));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes<MODE>();
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (MODE == kProbe) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
-  kern<<<grid_size(g), kThreads, smem_bytes<MODE>(), s>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
+  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka));
   if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
   count_launch();
-  QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
 }
 
@@ -582,12 +681,12 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   const GemmShape g = p.g;
   const int64_t ldc = qm_code_ld(g.K);
   CUtensorMap maps[6];
-  bool ok = make_map(&maps[0], p.l, true, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
-            make_map(&maps[1], p.r, true, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
-            make_map(&maps[2], p.l_abs, true, g.K, g.M, g.batch, g.K, g.M * g.K) &&
-            make_map(&maps[3], p.r_abs, true, g.K, g.N, g.batch, g.K, g.N * g.K) &&
-            make_map(&maps[4], p.cl, false, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-            make_map(&maps[5], p.cr, false, g.K, g.N, g.batch, ldc, g.N * ldc);
+  bool ok = make_map(&maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
+            make_map(&maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
+            make_map(&maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
+            make_map(&maps[3], p.r_abs, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K) &&
+            make_map(&maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+            make_map(&maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
   KernelArgs ka{};
   fill_tiles(&ka, g);
@@ -605,8 +704,8 @@ qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int g
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
   const int64_t ldc = qm_code_ld(g.K);
   CUtensorMap maps[6];
-  bool ok = make_map(&maps[4], cl, false, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-            make_map(&maps[5], cr, false, g.K, g.N, g.batch, ldc, g.N * ldc);
+  bool ok = make_map(&maps[4], cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+            make_map(&maps[5], cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
   maps[0] = maps[1] = maps[2] = maps[3] = maps[4];
   KernelArgs ka{};
@@ -622,8 +721,8 @@ qm_status launch_tc_gemm_ref(const void* l, const void* r, GemmShape g, float* o
                              cudaStream_t s) {
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
   CUtensorMap maps[6];
-  bool ok = make_map(&maps[0], l, true, g.K, g.M, g.batch, g.K, g.M * g.K) &&
-            make_map(&maps[1], r, true, g.K, g.N, g.batch, g.K, g.N * g.K);
+  bool ok = make_map(&maps[0], l, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
+            make_map(&maps[1], r, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K);
   if (!ok) return QM_ERR_CUDA;
   maps[2] = maps[3] = maps[4] = maps[5] = maps[0];
   KernelArgs ka{};
