@@ -124,6 +124,55 @@ def time_oracle_sample(ops, rows_per_op, seed=7):
     return flops, dt
 
 
+def scale_quantize_rates(qm, hbm_gbs, rows=16384, cols=4096, iters=10):
+    """Algorithmic GB/s of the scale / quantize kernels on one FFN-activation-sized bf16 tensor
+    (rows x cols, 134 MB: larger than L2), each timed with CUDA events after a warm-up."""
+    x = torch.randn(rows, cols, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    n = x.numel()
+    op_rows, op_cols = qm.operand_of(x, -1), qm.operand_of(x, -2)
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e-3
+
+    delta = qm.qm_scale(op_rows, "e4m3", "tensor")
+    ldc = qm.qm_code_ld(cols)
+    codes = torch.empty((1, rows, ldc), dtype=torch.uint8, device="cuda")
+    codes_t = torch.empty((1, cols, qm.qm_code_ld(rows)), dtype=torch.uint8, device="cuda")
+    dch = torch.empty(rows, dtype=torch.float32, device="cuda")
+    d1 = torch.empty(1, dtype=torch.float32, device="cuda")
+    import ctypes as C
+    L = qm.lib()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def raw_quant(op, gran, dl, dout, cod):
+        rc = L.qm_quantize(C.byref(op), 1, gran, 0, C.c_void_p(dl.data_ptr()) if dl is not None else None,
+                           C.c_void_p(dout.data_ptr()) if dout is not None else None, C.c_void_p(cod.data_ptr()),
+                           None, None, st)
+        assert rc == 0, rc
+
+    t_scale = timed(lambda: L.qm_scale(C.byref(op_rows), 1, 0, C.c_void_p(d1.data_ptr()), st))
+    t_quant = timed(lambda: raw_quant(op_rows, 0, delta, None, codes))
+    t_fused = timed(lambda: raw_quant(op_rows, 1, None, dch, codes))
+    t_trans = timed(lambda: raw_quant(op_cols, 0, delta, None, codes_t))
+    out = {"tensor": f"bf16 [{rows} x {cols}] ({n * 2 / 1e6:.0f} MB)", "hbm_peak_gbs": hbm_gbs,
+           "scale_tensor_gbs": 2 * n / t_scale / 1e9,                 # 2 B/elem read
+           "quantize_gbs": 3 * n / t_quant / 1e9,                     # 2 B read + 1 B code
+           "scale_quantize_rows_gbs": 3 * n / t_fused / 1e9,          # fused per-row scale + codes, input read once
+           "quantize_transpose_gbs": 3 * n / t_trans / 1e9}
+    for k in ("scale_tensor", "quantize", "scale_quantize_rows", "quantize_transpose"):
+        out[k + "_frac_of_hbm"] = out[k + "_gbs"] / hbm_gbs
+    return out
+
+
 def cpu_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -272,6 +321,7 @@ def main():
         return
 
     peaks = load_peaks()
+    sq = scale_quantize_rates(qm, peaks["hbm_gbs"])
     # composite tensor bound of the fused kernel: per 2MNK, one product at the 8-bit rate
     # (2 x bf16) and two at the bf16 rate  ->  3 / (1/(2P) + 2/P) = 1.2 P in summed flops
     peak_tflops = 1.2 * peaks["bf16_tflops"]
@@ -291,6 +341,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "roofline": roofline,
             "pct_of_composite_tensor_peak": 100.0 * value / peak_tflops,
+            "scale_quantize": sq,
             "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
     if not args.no_cpu_baseline and world == 1:
         f, s = time_oracle_sample(ops, args.oracle_rows)

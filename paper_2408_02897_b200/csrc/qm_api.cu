@@ -90,7 +90,7 @@ int64_t delta_count(const View& v, int gran) { return gran == QM_GRAN_TENSOR ? 1
 size_t align256(size_t n) { return (n + 255) & ~(size_t)255; }
 
 struct Workspace {
-  size_t off_err, off_dl, off_dr, off_cl, off_cr, off_al, off_ar, off_kl, off_kr, off_part, total;
+  size_t off_err, off_ml, off_mr, off_dl, off_dr, off_cl, off_cr, off_al, off_ar, off_kl, off_kr, off_part, total;
   int n_part;
   bool tc;
 };
@@ -101,6 +101,8 @@ Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg) {
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += align256(bytes); return at; };
   w.off_err = take(256);
+  w.off_ml = take(sizeof(float) * delta_count(L, cfg.gran_l));      // max|x| bit patterns (cleared)
+  w.off_mr = take(sizeof(float) * delta_count(R, cfg.gran_r));
   w.off_dl = take(sizeof(float) * delta_count(L, cfg.gran_l));
   w.off_dr = take(sizeof(float) * delta_count(R, cfg.gran_r));
   const int64_t ldc = qm_code_ld(L.c);
@@ -139,15 +141,15 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
 }
 
 // scale + quantize of one operand inside the probe
-qm_status prepare_operand(const View& x, int fmt, int gran, float* delta, uint8_t* codes, void* abs_copy,
-                          void* kmaj_copy, uint32_t* err_word, cudaStream_t s) {
+qm_status prepare_operand(const View& x, int fmt, int gran, uint32_t* amax, float* delta, uint8_t* codes,
+                          void* abs_copy, void* kmaj_copy, uint32_t* err_word, cudaStream_t s) {
   if (gran == QM_GRAN_CHANNEL && x.c_contig())
     return launch_scale_quantize_rows(x, fmt, delta, codes, abs_copy, err_word, s);
-  qm_status st = launch_absmax(x, gran, reinterpret_cast<uint32_t*>(delta), s);
+  qm_status st = launch_absmax(x, gran, amax, s);
   if (st != QM_OK) return st;
-  st = launch_finalize_delta(delta, delta_count(x, gran), fmt, err_word, s);
-  if (st != QM_OK) return st;
-  return launch_quantize(x, fmt, gran, delta, codes, abs_copy, kmaj_copy, s);
+  // the quantize kernel turns max|x| into delta itself
+  return launch_quantize(x, fmt, gran, reinterpret_cast<const float*>(amax), true, delta, err_word, codes,
+                         abs_copy, kmaj_copy, s);
 }
 
 }  // namespace
@@ -183,7 +185,7 @@ qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t ro
       (reinterpret_cast<uintptr_t>(kmaj_copy) & 15))
     return QM_ERR_ALIGNMENT;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (delta) return launch_quantize(v, fmt, gran, delta, codes, abs_copy, kmaj_copy, s);
+  if (delta) return launch_quantize(v, fmt, gran, delta, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s);
   if (!delta_out) return QM_ERR_INVALID_ARG;
   const int64_t n = delta_count(v, gran);
   if (gran == QM_GRAN_CHANNEL && v.c_contig() && !kmaj_copy)
@@ -193,7 +195,7 @@ qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t ro
   if (st != QM_OK) return st;
   st = launch_finalize_delta(delta_out, n, fmt, nullptr, s);
   if (st != QM_OK) return st;
-  return launch_quantize(v, fmt, gran, delta_out, codes, abs_copy, kmaj_copy, s);
+  return launch_quantize(v, fmt, gran, delta_out, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s);
 }
 
 qm_status qm_gemm(const uint8_t* codes_l, int32_t fmt_l, const float* delta_l, int32_t gran_l,
@@ -265,15 +267,17 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   uint8_t* cl = base + w.off_cl;
   uint8_t* cr = base + w.off_cr;
   double* part = reinterpret_cast<double*>(base + w.off_part);
-  // the error word and both scale buffers are adjacent: one clear
-  QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_cl, s));
+  // the error word, the finished-CTA counter and both max|x| buffers are adjacent: one clear
+  QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
+  uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.off_ml);
+  uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.off_mr);
   void* al = w.tc ? base + w.off_al : nullptr;
   void* ar = w.tc ? base + w.off_ar : nullptr;
   void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
-  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, dl, cl, al, kl, err, s);
+  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err, s);
   if (st != QM_OK) return st;
-  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, dr, cr, ar, kr, err, s);
+  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err, s);
   if (st != QM_OK) return st;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {

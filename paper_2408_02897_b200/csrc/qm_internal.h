@@ -48,9 +48,12 @@ qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream
 // In place: bit pattern of max|x| -> delta = max|x| / qmax (1 where max|x| == 0).
 // err_word (optional): gets QM_DEVERR_NONFINITE or-ed in when a group max is NaN/Inf.
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s);
-// codes (+ optional |x| and x as bf16, contraction-major) from given deltas.
-qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, uint8_t* codes,
-                          void* abs_copy, void* kmaj_copy, cudaStream_t s);
+// codes (+ optional |x| and x as bf16, contraction-major).  `delta` holds finished deltas, or,
+// with from_amax, the max|x| bit patterns of launch_absmax: the kernel then does the division
+// itself, writes the deltas to delta_out and raises QM_DEVERR_NONFINITE in err_word (optional).
+qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, bool from_amax,
+                          float* delta_out, uint32_t* err_word, uint8_t* codes, void* abs_copy,
+                          void* kmaj_copy, cudaStream_t s);
 // Single pass per row: absmax, delta, codes (contiguous contraction, per-channel).
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
                                      void* abs_copy, uint32_t* err_word, cudaStream_t s);

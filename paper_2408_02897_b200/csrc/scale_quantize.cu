@@ -237,23 +237,46 @@ __global__ void finalize_delta_kernel(float* __restrict__ delta, int64_t n, floa
   delta[i] = bits == 0 ? 1.0f : __fdiv_rn(amax, qmax);
 }
 
+// Where a quantize kernel gets its scales from.  Either finished deltas, or (from_amax) the bit
+// patterns of max|x| left by an absmax kernel: the division of Eq. 1 is then done here, which
+// saves a launch; the thread named `writer` stores the delta for later consumers and raises
+// the non-finite flag.
+struct DeltaSrc {
+  const float* p;
+  int per_channel;
+  int from_amax;
+  float qmax;
+  float* out;           // from_amax only: where the finished deltas go
+  uint32_t* err_word;   // from_amax only, optional
+  __device__ __forceinline__ float get(int64_t i, bool writer) const {
+    if (!from_amax) return __ldg(p + i);
+    const uint32_t bits = __ldg(reinterpret_cast<const uint32_t*>(p) + i);
+    const float d = bits == 0 ? 1.0f : __fdiv_rn(__uint_as_float(bits), qmax);
+    if (writer) {
+      out[i] = d;
+      if (bits >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
+    }
+    return d;
+  }
+};
+
 // ---------------------------------------------------------------- quantize, contiguous contraction
 // One thread handles 16 consecutive elements of a row: two 128-bit loads (bf16), one 128-bit
 // code store, optionally two 128-bit stores of |x| as bf16.
 template <typename T, int FMT>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
-                     int64_t s_b, const float* __restrict__ delta, int per_channel,
+                     int64_t s_b, const DeltaSrc ds,
                      uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy) {
   const int64_t chunks_per_row = ldc >> 4;                  // 16 codes per chunk, padding included
   const int64_t total = nc * batch * chunks_per_row;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  const float d_tensor = per_channel ? 0.f : __ldg(delta);
+  const float d_tensor = ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && threadIdx.x == 0);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
     const int64_t row = i / chunks_per_row, ch = i - row * chunks_per_row;
     const int64_t b = row / nc, r = row - b * nc;
     const T* p = x + b * s_b + r * s_nc + ch * 16;
-    const float d = per_channel ? __ldg(delta + row) : d_tensor;
+    const float d = ds.per_channel ? ds.get(row, ch == 0) : d_tensor;
     const int64_t k0 = ch * 16;
     Vec8 v0, v1;
     if (k0 + 16 <= c) {
@@ -338,7 +361,7 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
 template <typename T, int FMT>
 __global__ void __launch_bounds__(kThreads)
 quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
-                          const float* __restrict__ delta, int per_channel,
+                          const DeltaSrc ds,
                           uint8_t* __restrict__ codes, int64_t ldc,
                           __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
   __shared__ float tile[64][65];     // +1 column spreads the transposed accesses over the banks
@@ -362,7 +385,9 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
   }
   __syncthreads();
   // output: row n (64 of them), 64 contraction entries = 8 chunks of 8
-  const float d_tensor = per_channel ? 0.f : __ldg(delta);
+  const float d_tensor = ds.per_channel
+                             ? 0.f
+                             : ds.get(0, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0);
 #pragma unroll
   for (int it = 0; it < 2; ++it) {
     const int nrow = ty + it * 32;
@@ -373,7 +398,7 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
     Vec8 v;
 #pragma unroll
     for (int j = 0; j < 8; ++j) v.v[j] = tile[tx * 8 + j][nrow];
-    const float d = per_channel ? __ldg(delta + b * nc + nn) : d_tensor;
+    const float d = ds.per_channel ? ds.get(b * nc + nn, blockIdx.y == 0 && tx == 0) : d_tensor;
     const int64_t orow = b * nc + nn;
     *reinterpret_cast<uint2*>(codes + orow * ldc + k0) = quant8<FMT>(v, d);
     if (abs_copy || kmaj_copy) {
@@ -449,15 +474,17 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
 }
 
 template <typename T, int FMT>
-qm_status quantize_t(const View& x, int gran, const float* delta, uint8_t* codes, void* abs_copy,
-                     void* kmaj_copy, cudaStream_t s) {
+qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax, float* delta_out,
+                     uint32_t* err_word, uint8_t* codes, void* abs_copy, void* kmaj_copy, cudaStream_t s) {
   const T* p = static_cast<const T*>(x.data);
   const int64_t ldc = qm_code_ld(x.c);
-  const int pc = gran == QM_GRAN_CHANNEL;
+  DeltaSrc ds;
+  ds.p = delta; ds.per_channel = gran == QM_GRAN_CHANNEL; ds.from_amax = from_amax ? 1 : 0;
+  ds.qmax = fmt_qmax(FMT); ds.out = delta_out; ds.err_word = err_word;
   if (x.c_contig()) {
     const int64_t total = x.nc * x.batch * (ldc >> 4);
     quantize_rows_kernel<T, FMT><<<grid_for(total, 16), kThreads, 0, s>>>(
-        p, x.nc, x.c, x.s_nc, x.batch, x.s_b, delta, pc, codes, ldc,
+        p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, codes, ldc,
         static_cast<__nv_bfloat16*>(abs_copy));
     if (kmaj_copy) {
       // already contraction-major: a strided copy honours the parameter
@@ -470,7 +497,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, uint8_t* codes
   } else {
     dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((ldc + 63) / 64), (unsigned)x.batch);
     quantize_transpose_kernel<T, FMT><<<grid, kThreads, 0, s>>>(
-        p, x.nc, x.c, x.s_c, x.s_b, delta, pc, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
+        p, x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
         static_cast<__nv_bfloat16*>(kmaj_copy));
   }
   count_launch();
@@ -513,14 +540,17 @@ qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_
   return QM_OK;
 }
 
-qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, uint8_t* codes,
-                          void* abs_copy, void* kmaj_copy, cudaStream_t s) {
-#define QM_Q(T)                                                                                  \
-  (fmt == QM_FMT_INT8   ? quantize_t<T, QM_FMT_INT8>(x, gran, delta, codes, abs_copy, kmaj_copy, s) \
-   : fmt == QM_FMT_E4M3 ? quantize_t<T, QM_FMT_E4M3>(x, gran, delta, codes, abs_copy, kmaj_copy, s) \
-                        : quantize_t<T, QM_FMT_E5M2>(x, gran, delta, codes, abs_copy, kmaj_copy, s))
+qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, bool from_amax,
+                          float* delta_out, uint32_t* err_word, uint8_t* codes, void* abs_copy,
+                          void* kmaj_copy, cudaStream_t s) {
+#define QM_ARGS x, gran, delta, from_amax, delta_out, err_word, codes, abs_copy, kmaj_copy, s
+#define QM_Q(T)                                                    \
+  (fmt == QM_FMT_INT8   ? quantize_t<T, QM_FMT_INT8>(QM_ARGS)      \
+   : fmt == QM_FMT_E4M3 ? quantize_t<T, QM_FMT_E4M3>(QM_ARGS)      \
+                        : quantize_t<T, QM_FMT_E5M2>(QM_ARGS))
   return x.dtype == QM_DT_BF16 ? QM_Q(__nv_bfloat16) : QM_Q(float);
 #undef QM_Q
+#undef QM_ARGS
 }
 
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
