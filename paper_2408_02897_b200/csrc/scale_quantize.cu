@@ -80,11 +80,35 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// x / delta, correctly rounded (the IEEE quotient Eq. 1 asks for), for many x under one delta.
+// With r = RN(1/delta) computed once per scaling group, a product and two residual corrections
+//   q0 = x r;  q1 = q0 + (x - q0 delta) r;  q = q1 + (x - q1 delta) r      (residuals exact by FMA)
+// give RN(x / delta): q1 is within one ulp of the quotient, and one more correction of a
+// faithful quotient with the correctly rounded reciprocal rounds correctly (Markstein's
+// theorem).  This needs the intermediate values inside the normal range, so it is used only for
+// 2^-60 <= delta <= 2^60, where any |x| small enough to leave that range quantizes to zero in
+// every format; other deltas take the division instruction sequence.
+struct Quotient {
+  float delta, recip;
+  bool fast;
+  __device__ __forceinline__ explicit Quotient(float d) : delta(d) {
+    fast = d >= 8.6736174e-19f && d <= 1.1529215e18f;        // 2^-60 .. 2^60
+    recip = fast ? __frcp_rn(d) : 0.f;
+  }
+  __device__ __forceinline__ float operator()(float x) const {
+    if (!fast) return __fdiv_rn(x, delta);
+    const float q0 = x * recip;
+    const float q1 = fmaf(fmaf(-q0, delta, x), recip, q0);
+    const float q = fmaf(fmaf(-q1, delta, x), recip, q1);
+    return copysignf(q, x);                                   // keeps the sign of a zero input
+  }
+};
+
 template <int FMT>
-__device__ __forceinline__ uint2 quant8(const Vec8& x, float delta) {
+__device__ __forceinline__ uint2 quant8(const Vec8& x, const Quotient& quot) {
   float t[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) t[i] = __fdiv_rn(x.v[i], delta);   // IEEE division, as Eq. 1 writes it
+  for (int i = 0; i < 8; ++i) t[i] = quot(x.v[i]);
   uint2 r;
   r.x = quant2<FMT>(t[0], t[1]) | (quant2<FMT>(t[2], t[3]) << 16);
   r.y = quant2<FMT>(t[4], t[5]) | (quant2<FMT>(t[6], t[7]) << 16);
@@ -125,6 +149,23 @@ __device__ __forceinline__ uint32_t block_max(uint32_t v) {
   return v;   // valid in warp 0
 }
 
+// Division of a 32-bit index by a launch-time constant without a divide instruction
+// (multiply-high and shift; the magic numbers come from the host).
+struct FastDiv {
+  uint32_t d, m, s;
+  __host__ explicit FastDiv(uint32_t div = 1) : d(div), m(0), s(0) {
+    if (d > 1) {
+      while ((1ull << s) < d) ++s;                          // s = ceil(log2 d)
+      m = (uint32_t)((((1ull << s) - d) << 32) / d + 1);
+    }
+  }
+  __device__ __forceinline__ uint32_t div(uint32_t n) const {
+    if (d == 1) return n;
+    const uint32_t t = __umulhi(m, n);
+    return (t + ((n - t) >> 1)) >> (s - 1);
+  }
+};
+
 // ---------------------------------------------------------------- absmax, whole tensor
 // Rows of `c` contiguous elements (vector loads for the multiple-of-8 part, scalar loads for
 // the tail).  When the rows are dense the host flattens the tensor into a single row so that
@@ -138,21 +179,34 @@ absmax_tensor_kernel(const T* __restrict__ x, int64_t rows, int64_t c, int64_t r
   uint32_t acc = 0;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  // four independent 128-bit loads in flight per thread
-  for (; i + 3 * stride < total_vec; i += 4 * stride) {
-    Vec8 v[4];
+  if (rows == 1) {
+    // dense tensor walked as one row: no index arithmetic beyond the stride;
+    // eight independent 128-bit loads in flight per thread
+    for (; i + 7 * stride < total_vec; i += 8 * stride) {
+      Vec8 v[8];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      int64_t j = i + u * stride;
-      int64_t r = j / vec_per_row, k = j - r * vec_per_row;
-      v[u] = Loader<T>::load8(x + r * row_stride + k * 8);
+      for (int u = 0; u < 8; ++u) v[u] = Loader<T>::load8(x + (i + u * stride) * 8);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc = absmax8(v[u], acc);
     }
+    for (; i < total_vec; i += stride) acc = absmax8(Loader<T>::load8(x + i * 8), acc);
+  } else {
+    // four independent 128-bit loads in flight per thread
+    for (; i + 3 * stride < total_vec; i += 4 * stride) {
+      Vec8 v[4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) acc = absmax8(v[u], acc);
-  }
-  for (; i < total_vec; i += stride) {
-    int64_t r = i / vec_per_row, k = i - r * vec_per_row;
-    acc = absmax8(Loader<T>::load8(x + r * row_stride + k * 8), acc);
+      for (int u = 0; u < 4; ++u) {
+        int64_t j = i + u * stride;
+        int64_t r = j / vec_per_row, k = j - r * vec_per_row;
+        v[u] = Loader<T>::load8(x + r * row_stride + k * 8);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc = absmax8(v[u], acc);
+    }
+    for (; i < total_vec; i += stride) {
+      int64_t r = i / vec_per_row, k = i - r * vec_per_row;
+      acc = absmax8(Loader<T>::load8(x + r * row_stride + k * 8), acc);
+    }
   }
   const int64_t tail = c & 7;
   if (tail) {
@@ -266,17 +320,18 @@ struct DeltaSrc {
 template <typename T, int FMT>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
-                     int64_t s_b, const DeltaSrc ds,
+                     int64_t s_b, const DeltaSrc ds, const FastDiv by_chunks, const FastDiv by_nc,
                      uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy) {
-  const int64_t chunks_per_row = ldc >> 4;                  // 16 codes per chunk, padding included
-  const int64_t total = nc * batch * chunks_per_row;
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const uint32_t chunks_per_row = (uint32_t)(ldc >> 4);     // 16 codes per chunk, padding included
+  const uint32_t total = (uint32_t)(nc * batch) * chunks_per_row;   // < 2^32, checked by the host
+  const uint32_t stride = gridDim.x * blockDim.x;
   const float d_tensor = ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && threadIdx.x == 0);
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
-    const int64_t row = i / chunks_per_row, ch = i - row * chunks_per_row;
-    const int64_t b = row / nc, r = row - b * nc;
-    const T* p = x + b * s_b + r * s_nc + ch * 16;
-    const float d = ds.per_channel ? ds.get(row, ch == 0) : d_tensor;
+  const Quotient quot_tensor(d_tensor);
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const uint32_t row = by_chunks.div(i), ch = i - row * chunks_per_row;
+    const uint32_t b = by_nc.div(row), r = row - b * (uint32_t)nc;
+    const T* p = x + (int64_t)b * s_b + (int64_t)r * s_nc + ch * 16;
+    const Quotient quot = ds.per_channel ? Quotient(ds.get(row, ch == 0)) : quot_tensor;
     const int64_t k0 = ch * 16;
     Vec8 v0, v1;
     if (k0 + 16 <= c) {
@@ -289,7 +344,7 @@ quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_n
         v1.v[j] = k0 + 8 + j < c ? Loader<T>::load1(p, 8 + j) : 0.f;
       }
     }
-    uint2 q0 = quant8<FMT>(v0, d), q1 = quant8<FMT>(v1, d);
+    uint2 q0 = quant8<FMT>(v0, quot), q1 = quant8<FMT>(v1, quot);
     *reinterpret_cast<uint4*>(codes + row * ldc + k0) = make_uint4(q0.x, q0.y, q1.x, q1.y);
     if (abs_copy) {
       __nv_bfloat16* a = abs_copy + row * c + k0;
@@ -336,6 +391,7 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
     delta_out[row] = d;
     if (acc >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
   }
+  const Quotient quot(d);
   const int64_t nchunk = ldc >> 3;                          // 8 codes per step, padding included
   for (int64_t k = sub; k < nchunk; k += G) {
     const int64_t k0 = k * 8;
@@ -345,7 +401,7 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
 #pragma unroll
       for (int j = 0; j < 8; ++j) v.v[j] = k0 + j < c ? Loader<T>::load1(p, k0 + j) : 0.f;
     }
-    *reinterpret_cast<uint2*>(codes + row * ldc + k0) = quant8<FMT>(v, d);
+    *reinterpret_cast<uint2*>(codes + row * ldc + k0) = quant8<FMT>(v, quot);
     if (abs_copy) {
       __nv_bfloat16* a = abs_copy + row * c + k0;
       if (k0 + 8 <= c && (c & 7) == 0) *reinterpret_cast<uint4*>(a) = abs_bf16x8(v);
@@ -398,9 +454,9 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
     Vec8 v;
 #pragma unroll
     for (int j = 0; j < 8; ++j) v.v[j] = tile[tx * 8 + j][nrow];
-    const float d = ds.per_channel ? ds.get(b * nc + nn, blockIdx.y == 0 && tx == 0) : d_tensor;
+    const Quotient quot(ds.per_channel ? ds.get(b * nc + nn, blockIdx.y == 0 && tx == 0) : d_tensor);
     const int64_t orow = b * nc + nn;
-    *reinterpret_cast<uint2*>(codes + orow * ldc + k0) = quant8<FMT>(v, d);
+    *reinterpret_cast<uint2*>(codes + orow * ldc + k0) = quant8<FMT>(v, quot);
     if (abs_copy || kmaj_copy) {
       if (k0 + 8 <= c && (c & 7) == 0) {
         if (abs_copy) *reinterpret_cast<uint4*>(abs_copy + orow * c + k0) = abs_bf16x8(v);
@@ -483,9 +539,10 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
   ds.qmax = fmt_qmax(FMT); ds.out = delta_out; ds.err_word = err_word;
   if (x.c_contig()) {
     const int64_t total = x.nc * x.batch * (ldc >> 4);
+    if (total >= (1ll << 32) || x.nc >= (1ll << 32)) return QM_ERR_UNSUPPORTED;   // 32-bit chunk index
     quantize_rows_kernel<T, FMT><<<grid_for(total, 16), kThreads, 0, s>>>(
-        p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, codes, ldc,
-        static_cast<__nv_bfloat16*>(abs_copy));
+        p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
+        codes, ldc, static_cast<__nv_bfloat16*>(abs_copy));
     if (kmaj_copy) {
       // already contraction-major: a strided copy honours the parameter
       if (x.dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;

@@ -143,3 +143,74 @@ def test_large_tensor_sampled():
             dsel = want_d if gran == "tensor" else want_d[:, rows]
             want_c = oracle.quantize(xo[:, rows, :], "e4m3", dsel)
             assert np.array_equal(codes.cpu().numpy()[:, rows, :xo.shape[2]], want_c)
+
+
+def adversarial_deltas(rng, n_random):
+    """Scales whose reciprocal or quotients are awkward: significands of all ones, one ulp above a
+    power of two, thirds and sevenths, plus log-uniform random ones."""
+    bits = []
+    for e in (100, 117, 127, 130, 150):                     # biased exponents well inside the range
+        for m in (0x7FFFFF, 0x7FFFFE, 0x000001, 0x000000, 0x2AAAAB, 0x555555, 0x124925, 0x400000, 0x7FF000):
+            bits.append((e << 23) | m)
+    d = np.array(bits, dtype=np.uint32).view(np.float32)
+    r = np.exp(rng.uniform(np.log(1e-6), np.log(1e6), n_random)).astype(np.float32)
+    return np.concatenate([d, r])
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_quotient_is_exact_for_many_scales_bf16(fmt):
+    # all finite bf16 inputs against ~250 scales in one call (one scale per row)
+    rng = np.random.default_rng(50)
+    deltas = adversarial_deltas(rng, 203)          # 248 rows: a multiple of 8 for the transposed view
+    bits = np.arange(65536, dtype=np.uint32)
+    vals = (bits << 16).view(np.float32)
+    vals = np.where(np.isfinite(vals), vals, 0.0).astype(np.float32)
+    x = np.tile(vals, (len(deltas), 1))
+    lim = (deltas * np.float32(oracle.qmax(fmt)) * np.float32(4.0))[:, None]
+    x = np.where(np.abs(x) <= lim, x, 0.0).astype(np.float32)[None]       # [1, rows, 65536]
+    want = oracle.quantize(x, fmt, deltas[None, :])
+    t = torch.from_numpy(x[0]).to(torch.bfloat16).cuda()
+    codes, _, _, _ = qm.qm_quantize(qm.operand_of(t, -1), fmt, "channel", torch.from_numpy(deltas).cuda())
+    got = codes.cpu().numpy()
+    bad = np.nonzero(got != want)
+    assert bad[0].size == 0, (fmt, bad[0].size, deltas[bad[1][:5]], x[bad][:5], got[bad][:5], want[bad][:5])
+    # the same scales through the transposing kernel (one scale per column)
+    tt = t.t().contiguous()                                               # [65536, rows]
+    codes_t, _, _, _ = qm.qm_quantize(qm.operand_of(tt, -2), fmt, "channel", torch.from_numpy(deltas).cuda())
+    assert np.array_equal(codes_t.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_quotient_is_exact_for_fp32_inputs(fmt):
+    # fp32 operands have full 24-bit significands: random values near the rounding boundaries
+    rng = np.random.default_rng(51)
+    deltas = adversarial_deltas(rng, 150)
+    g = oracle.positive_grid(fmt)
+    mid = ((g[:-1] + g[1:]) / 2).astype(np.float32)
+    base = rng.choice(np.concatenate([mid, g[1:].astype(np.float32)]), (len(deltas), 2048)).astype(np.float32)
+    x = base * deltas[:, None]                                            # lands near ties and grid points
+    jitter = rng.integers(-3, 4, x.shape)
+    x = (x.view(np.int32) + jitter).view(np.float32)                      # a few ulps either side
+    x = (x * rng.choice([-1.0, 1.0], x.shape)).astype(np.float32)[None]
+    want = oracle.quantize(x, fmt, deltas[None, :])
+    t = torch.from_numpy(x[0]).cuda()
+    codes, _, _, _ = qm.qm_quantize(qm.operand_of(t, -1), fmt, "channel", torch.from_numpy(deltas).cuda())
+    got = codes.cpu().numpy()
+    bad = np.nonzero(got != want)
+    assert bad[0].size == 0, (fmt, bad[0].size, deltas[bad[1][:5]], x[bad][:5], got[bad][:5], want[bad][:5])
+
+
+def test_extreme_scales_take_the_division_path():
+    # deltas outside 2^-60 .. 2^60, including subnormal ones
+    for d in (1e-30, 3e-39, 1e-44, 2.5e25, 1e32):
+        d32 = np.float32(d)
+        vals = (np.arange(1, 20000, dtype=np.float32) * d32 * np.float32(0.013)).astype(np.float32)
+        vals = vals[np.isfinite(vals)]
+        vals = np.concatenate([vals, -vals])
+        pad = (-len(vals)) % 16
+        x = np.concatenate([vals, np.zeros(pad, np.float32)])[None, None, :]
+        dd = np.array([d32], np.float32)
+        want = oracle.quantize(x, "e4m3", dd)
+        t = torch.from_numpy(x[0]).cuda()
+        codes, _, _, _ = qm.qm_quantize(qm.operand_of(t, -1), "e4m3", "tensor", torch.from_numpy(dd).cuda())
+        assert np.array_equal(codes.cpu().numpy(), want), d
