@@ -111,13 +111,15 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 // arrive on a barrier given by its shared::cluster address (own CTA or the peer)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  // default semantics (release at CTA scope): the data this barrier orders lives in tensor
+  // memory and is fenced by tcgen05.fence; a cluster-scope release costs a long memory fence
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -270,26 +272,90 @@ __device__ __forceinline__ TileCoord tile_coord(int t, const KernelArgs& a) {
   return c;
 }
 
-// Eq. 3 statistics of 32 consecutive columns of one row.
-struct Stats { float be, mx, d2, r2, n2; };
+// 32 lanes x 16 consecutive 32-bit columns.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 
+// Two-wide fp32 arithmetic (one instruction for a pair of values).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t x, uint64_t y, uint64_t z) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(x), "l"(y), "l"(z));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t x, uint64_t y) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(x), "l"(y));
+  return r;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float max3(float x, float y, float z) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(x), "f"(y), "f"(z));
+  return r;
+}
+
+// Eq. 3 statistics of one row, kept two-wide across the columns of a tile.
+struct Stats2 {
+  uint64_t be, d2, r2, n2;
+  float mx;
+};
+
+// 16 consecutive columns of one row: reference rc, denominator rd, raw 8-bit accumulator rq.
+// ndl2 holds (-delta_l, -delta_l); dr_s points at the 16 column scales (per_col) or is unused.
+// n_live < 16 only in the last, ragged column chunk of a matrix.
 template <int LPKIND, bool RAGGED>
-__device__ __forceinline__ void stats32(const uint32_t (&rc)[32], const uint32_t (&rd)[32], const uint32_t (&rq)[32],
-                                        float dlv, const float* dr_s, bool per_col, float dr_tensor, int n_live,
-                                        Stats& s) {
+__device__ __forceinline__ void stats16(const uint32_t* rc, const uint32_t* rd, const uint32_t* rq,
+                                        uint64_t ndl2, const float* dr_s, bool per_col, uint64_t dr_tensor2,
+                                        int n_live, Stats2& s) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j) {
-    const float cv = __uint_as_float(rc[j]), dd = __uint_as_float(rd[j]);
-    const float acc = LPKIND == kKindI8 ? (float)(int)rq[j] : __uint_as_float(rq[j]);
-    const float drj = per_col ? dr_s[j] : dr_tensor;
-    const float diff = fmaf(-(acc * dlv), drj, cv);                 // C - A * delta_l * delta_r
+  for (int j = 0; j < 16; j += 2) {
+    const bool live0 = !RAGGED || j < n_live, live1 = !RAGGED || j + 1 < n_live;
+    const float a0 = LPKIND == kKindI8 ? (float)(int)rq[j] : __uint_as_float(rq[j]);
+    const float a1 = LPKIND == kKindI8 ? (float)(int)rq[j + 1] : __uint_as_float(rq[j + 1]);
+    const uint64_t dr2 = per_col ? *reinterpret_cast<const uint64_t*>(dr_s + j) : dr_tensor2;
+    float c0 = __uint_as_float(rc[j]), c1 = __uint_as_float(rc[j + 1]);
+    float d0 = __uint_as_float(rd[j]), d1 = __uint_as_float(rd[j + 1]);
+    if (!live0) { c0 = 0.f; d0 = 0.f; }
+    if (!live1) { c1 = 0.f; d1 = 0.f; }
+    const uint64_t cv2 = pack2(c0, c1), dd2 = pack2(d0, d1);
+    uint64_t diff2 = fma2(mul2(pack2(live0 ? a0 : 0.f, live1 ? a1 : 0.f), ndl2), dr2, cv2);   // C - A dl dr
+    float e0, e1;
+    unpack2(diff2, e0, e1);
     // D == 0 implies C == Q == 0, so clamping the divisor keeps BE = 0 there without a branch
-    float be = __fdividef(fabsf(diff), fmaxf(dd, 1e-37f));
-    if (RAGGED) {
-      if (j >= n_live) continue;
-    }
-    s.be += be; s.mx = fmaxf(s.mx, be);
-    s.d2 = fmaf(diff, diff, s.d2); s.r2 = fmaf(cv, cv, s.r2); s.n2 = fmaf(dd, dd, s.n2);
+    const float r0 = rcp_approx(fmaxf(d0, 1e-37f)), r1 = rcp_approx(fmaxf(d1, 1e-37f));
+    const uint64_t be2 = mul2(pack2(fabsf(e0), fabsf(e1)), pack2(r0, r1));
+    float b0, b1;
+    unpack2(be2, b0, b1);
+    s.be = add2(s.be, be2);
+    s.mx = max3(s.mx, b0, b1);
+    s.d2 = fma2(diff2, diff2, s.d2);
+    s.r2 = fma2(cv2, cv2, s.r2);
+    s.n2 = fma2(dd2, dd2, s.n2);
   }
 }
 
@@ -379,7 +445,13 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       uint32_t g = 0, it = 0;
       bool ok = true;
       for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
-        // both epilogues must have drained the previous tile's accumulators
+        // Probe: the three accumulators rotate through the four 128-column blocks of tensor
+        // memory (see the epilogue).  This tile may start once both epilogues have copied the
+        // previous tile's reference and denominator blocks out; that signal also implies that
+        // the epilogue of the tile before it is finished, which frees this tile's third block.
+        const uint32_t col_ref = MODE == kProbe ? ((3 * it) & 3) * 128u : 0u;
+        const uint32_t col_den = ((3 * it + 1) & 3) * 128u;
+        const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : 0u;
         if (it > 0 && !mbar_wait(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
@@ -392,20 +464,19 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-              mma_pair<kKindF16>(tmem_base, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
+              mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
           }
           if (MODE == kProbe) {
             const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
 #pragma unroll
             for (int k = 0; k < kBlockK / 16; ++k)
-              mma_pair<kKindF16>(tmem_base + 128, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
+              mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
           }
           if (MODE == kProbe || MODE == kLpOnly) {
-            const uint32_t col = MODE == kProbe ? 256u : 0u;
             const uint64_t dl = smem_desc(base + C::kOffCl, 64), dr = smem_desc(base + C::kOffCr, 64);
 #pragma unroll
             for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
-              mma_pair<LPKIND>(tmem_base + col, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0);
+              mma_pair<LPKIND>(tmem_base + col_lp, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0);
           }
           tc_commit_pair(smem_u32(&sh->empty[s]));        // frees the stage in both CTAs
         }
@@ -440,23 +511,53 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       if (epi_barrier_any(!ok)) break;
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+      if (MODE == kProbe) {
+        // Accumulator blocks of this tile (they rotate so that the next tile's MMAs never wait
+        // for this arithmetic): copy this warp's 64 columns of the reference and denominator
+        // blocks into registers, hand those two blocks back to the MMA lane, then walk the
+        // 8-bit block in chunks of 16 columns.
+        const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
+        const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
+        const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;      // first column of this warp
+        uint32_t rc[64], rd[64], rq[16];
+        tmem_ld32(lane_addr + col_ref + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
+        tmem_ld32(lane_addr + col_ref + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
+        tmem_ld32(lane_addr + col_den + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
+        tmem_ld32(lane_addr + col_den + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+        Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f};
+        const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int cc0 = h * 64 + c * 16;
+          const int64_t col0 = colw + c * 16;
+          if (col0 < a.N) {                       // uniform across the warp
+            tmem_ld16(lane_addr + col_lp + cc0, rq);
+            tmem_ld_wait();
+            const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
+            if (n_live == 16) stats16<LPKIND, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
+            else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
+          }
+        }
+        if (row_ok) {
+          float x0, x1;
+          unpack2(st.be, x0, x1); sbe += (double)x0 + (double)x1;
+          unpack2(st.d2, x0, x1); sd2 += (double)x0 + (double)x1;
+          unpack2(st.r2, x0, x1); sr2 += (double)x0 + (double)x1;
+          unpack2(st.n2, x0, x1); sn2 += (double)x0 + (double)x1;
+          mbe = fmax(mbe, (double)st.mx);
+        }
+        tc_fence_before();                        // the 8-bit block's loads are complete as well
+      } else {
 #pragma unroll 1
-      for (int c = 0; c < 2; ++c) {
-        const int cc0 = h * 64 + c * 32;          // first column of this chunk inside the tile
-        const int64_t col0 = (int64_t)tc.n_tile * kBlockN + cc0;
-        if (col0 >= a.N) break;                   // uniform across the warp
-        const int n_live = (int)(a.N - col0 < 32 ? a.N - col0 : 32);
-        if (MODE == kProbe) {
-          uint32_t rc[32], rd[32], rq[32];
-          tmem_ld32(lane_addr + cc0, rc);
-          tmem_ld32(lane_addr + 128 + cc0, rd);
-          tmem_ld32(lane_addr + 256 + cc0, rq);
-          tmem_ld_wait();
-          Stats st{0.f, 0.f, 0.f, 0.f, 0.f};
-          if (n_live == 32) stats32<LPKIND, false>(rc, rd, rq, dlv, dr_s + cc0, per_col, dr_tensor, 32, st);
-          else stats32<LPKIND, true>(rc, rd, rq, dlv, dr_s + cc0, per_col, dr_tensor, n_live, st);
-          if (row_ok) { sbe += st.be; mbe = fmax(mbe, (double)st.mx); sd2 += st.d2; sr2 += st.r2; sn2 += st.n2; }
-        } else {
+        for (int c = 0; c < 2; ++c) {
+          const int cc0 = h * 64 + c * 32;          // first column of this chunk inside the tile
+          const int64_t col0 = (int64_t)tc.n_tile * kBlockN + cc0;
+          if (col0 >= a.N) break;                   // uniform across the warp
+          const int n_live = (int)(a.N - col0 < 32 ? a.N - col0 : 32);
           uint32_t r[32];
           tmem_ld32(lane_addr + cc0, r);
           tmem_ld_wait();
@@ -478,10 +579,12 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           }
         }
       }
-      // this warp has finished reading the accumulators of the tile: tell the leader's MMA lane
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+      if (MODE != kProbe) {
+        // this warp has finished reading the accumulator of the tile: tell the leader's MMA lane
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+      }
     }
     if (MODE == kProbe) {
 #pragma unroll
