@@ -30,9 +30,25 @@ def gpu_probe(o):
     return res
 
 
-def assert_record_close(got, want, rtol=1e-4, rtol_max=1e-3, what=""):
-    """Scalar-metric tolerance: sums within rtol relative, max BE within rtol_max."""
+def _derived(rec):
+    n = max(rec["count"], 1)
+    sd, sr, sn = rec["sum_diff2"], rec["sum_ref2"], rec["sum_den2"]
+    return {"mean_be": rec["sum_be"] / n, "normwise_be": (sd / sn) ** 0.5 if sn > 0 else 0.0,
+            "rel_l2": (sd / sr) ** 0.5 if sr > 0 else 0.0}
+
+
+def assert_record_close(got, want, rtol=1e-4, rtol_max=1e-3, what="", K=None):
+    """Scalar-metric tolerance.  The metrics (mean BE, norm-wise BE, relative L2) must agree within
+    rtol = 1e-4 and max BE within 1e-3, at every size.  The raw sums behind them get the same 1e-4
+    up to K = 8192; beyond that the bound grows in proportion to K, because the tensor cores
+    truncate when they add each 16-deep partial product to the fp32 accumulator: the all-positive
+    denominator loses about 6e-8 per step relative, so its sum of squares is low by about
+    1.6e-4 at K = 16384 (1024 steps) while the ratios that form the metrics stay inside 1e-4."""
     assert got["count"] == want["count"], what
+    raw_tol = rtol if (K is None or K <= 8192) else rtol * K / 8192.0
     for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
-        assert abs(got[k] - want[k]) <= rtol * abs(want[k]) + 1e-300, (what, k, got[k], want[k])
+        assert abs(got[k] - want[k]) <= raw_tol * abs(want[k]) + 1e-300, (what, k, got[k], want[k])
+    dg, dw = _derived(got), _derived(want)
+    for k in dg:
+        assert abs(dg[k] - dw[k]) <= rtol * abs(dw[k]) + 1e-300, (what, k, dg[k], dw[k])
     assert abs(got["max_be"] - want["max_be"]) <= rtol_max * abs(want["max_be"]) + 1e-300, (what, got, want)
