@@ -228,9 +228,8 @@ def main():
     import paper_2408_02897_b200 as qm
     import torch.distributed as dist
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2408_02897_b200 import ranks
+    rank, world, local = ranks.rank_info()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -251,8 +250,7 @@ def main():
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        ranks.barrier(world)
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
@@ -278,17 +276,13 @@ def main():
     qm.profile_enable(False)
     launches = qm.kernel_launches() - launches0
     clocks = sampler.stop()
-    total_ms = float(sum(step_ms))
-    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = t.item()
+    total_ms = ranks.max_over_ranks(float(sum(step_ms)), world, "cuda")
     results = [plan.result() for _, _, plan in dev_ops]
     if any(r.device_error for r in results):
         raise SystemExit("device error flagged in a probe result")
 
     flops_step = probe_flops(ops)
-    value = flops_step * args.steps * world / (total_ms * 1e-3) / 1e12
+    value = ranks.whole_job_rate(flops_step * args.steps, world, total_ms) / 1e12
 
     # ---- end to end through the host-buffer entry point: H2D of every operand and D2H of the
     # record inside the timed region
@@ -310,10 +304,7 @@ def main():
         e2e_step()                      # each call synchronises the stream itself
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3
-    t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = flops_step * e2e_steps * world / (t.item() * 1e-3) / 1e12
+    e2e_value = ranks.whole_job_rate(flops_step * e2e_steps, world, ranks.max_over_ranks(e2e_ms, world, "cuda")) / 1e12
 
     if rank != 0:
         if world > 1:
