@@ -189,7 +189,18 @@ absmax_tensor_kernel(const T* __restrict__ x, int64_t rows, int64_t c, int64_t r
 #pragma unroll
       for (int u = 0; u < 8; ++u) acc = absmax8(v[u], acc);
     }
-    for (; i < total_vec; i += stride) acc = absmax8(Loader<T>::load8(x + i * 8), acc);
+    if (i < total_vec) {
+      // remainder (fewer than eight per thread): still issued together, not one after another;
+      // lanes past the end re-read the last vector, which cannot change a maximum
+      Vec8 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int64_t j = i + u * stride;
+        v[u] = Loader<T>::load8(x + (j < total_vec ? j : total_vec - 1) * 8);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc = absmax8(v[u], acc);
+    }
   } else {
     // four independent 128-bit loads in flight per thread
     for (; i + 3 * stride < total_vec; i += 4 * stride) {
@@ -361,6 +372,57 @@ quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_n
   }
 }
 
+// ---------------------------------------------------------------- quantize, dense bf16 fast path
+// The common case of the probe: a dense bf16 tensor whose rows are a multiple of 16 long, so the
+// whole tensor is one flat run of 16-element chunks and codes have no padding.  Each thread
+// takes kDenseChunks chunks a block-width apart and issues all of their 128-bit loads before
+// touching any of them (2 x kDenseChunks loads in flight per thread); |x| copies are the raw
+// bit patterns with the sign bits cleared.
+constexpr int kDenseChunks = 4;
+
+template <int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const DeltaSrc ds,
+                      const FastDiv by_chunks, uint32_t chunks_per_row, uint4* __restrict__ codes,
+                      uint4* __restrict__ abs_copy) {
+  const uint32_t base = blockIdx.x * (kThreads * kDenseChunks) + threadIdx.x;
+  uint4 w[kDenseChunks][2];
+#pragma unroll
+  for (int u = 0; u < kDenseChunks; ++u) {
+    const uint32_t i = base + u * kThreads;
+    const uint32_t j = i < total_chunks ? i : total_chunks - 1;     // clamp: results of dead lanes are dropped
+    w[u][0] = __ldg(x + 2 * (size_t)j);
+    w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+  }
+  const float d_tensor = ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && threadIdx.x == 0);
+  const Quotient quot_tensor(d_tensor);
+#pragma unroll
+  for (int u = 0; u < kDenseChunks; ++u) {
+    const uint32_t i = base + u * kThreads;
+    if (i >= total_chunks) break;
+    Quotient quot = quot_tensor;
+    if (ds.per_channel) {
+      const uint32_t row = by_chunks.div(i);
+      quot = Quotient(ds.get(row, i == row * chunks_per_row));
+    }
+    uint4 out;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint4 v = w[u][h];
+      Vec8 f;
+      f.v[0] = bf16_lo(v.x); f.v[1] = bf16_hi(v.x); f.v[2] = bf16_lo(v.y); f.v[3] = bf16_hi(v.y);
+      f.v[4] = bf16_lo(v.z); f.v[5] = bf16_hi(v.z); f.v[6] = bf16_lo(v.w); f.v[7] = bf16_hi(v.w);
+      const uint2 q = quant8<FMT>(f, quot);
+      if (h == 0) { out.x = q.x; out.y = q.y; } else { out.z = q.x; out.w = q.y; }
+      if (abs_copy) {
+        const uint32_t m = 0x7fff7fffu;
+        abs_copy[2 * (size_t)i + h] = make_uint4(v.x & m, v.y & m, v.z & m, v.w & m);
+      }
+    }
+    codes[i] = out;
+  }
+}
+
 // ---------------------------------------------------------------- fused per-row scale + quantize
 // G lanes own one row: pass 1 reduces max|x| over the row, pass 2 re-reads it (from L1/L2: the
 // same lanes touched it a moment ago) and writes codes.  HBM sees each element once.
@@ -407,6 +469,59 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
       if (k0 + 8 <= c && (c & 7) == 0) *reinterpret_cast<uint4*>(a) = abs_bf16x8(v);
       else
         for (int j = 0; j < 8 && k0 + j < c; ++j) a[j] = __float2bfloat16_rn(fabsf(v.v[j]));
+    }
+  }
+}
+
+// ---------------------------------------------------------------- fused per-row, row held in registers
+// bf16 rows of at most VPL * 256 elements (a multiple of 16): one warp per row loads the whole row
+// with VPL independent 128-bit loads per lane, reduces max|x| with shuffles, and quantizes from
+// the registers.  Every element crosses the memory system once.
+template <int FMT, int VPL>
+__global__ void __launch_bounds__(kThreads)
+scale_quantize_rows_reg_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int nvec, int64_t s_nc,
+                               int64_t batch, int64_t s_b, float qmax, float* __restrict__ delta_out,
+                               uint2* __restrict__ codes, uint4* __restrict__ abs_copy,
+                               uint32_t* __restrict__ err_word) {
+  const int64_t rows = nc * batch;
+  const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;                                  // whole warps leave together
+  const int64_t b = row / nc, r = row - b * nc;
+  const uint4* p = reinterpret_cast<const uint4*>(x + b * s_b + r * s_nc);
+  uint4 w[VPL];
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    const int k = lane + 32 * u;
+    w[u] = k < nvec ? __ldg(p + k) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  // max over sign-cleared 16-bit patterns, two per word
+  uint32_t m2 = 0;
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    const uint32_t k = 0x7fff7fffu;
+    m2 = __vmaxu2(m2, __vmaxu2(__vmaxu2(w[u].x & k, w[u].y & k), __vmaxu2(w[u].z & k, w[u].w & k)));
+  }
+  uint32_t acc = max(m2 & 0xffffu, m2 >> 16) << 16;         // as an fp32 bit pattern
+  acc = warp_max(acc);
+  const float d = acc == 0 ? 1.0f : __fdiv_rn(__uint_as_float(acc), qmax);
+  if (lane == 0) {
+    delta_out[row] = d;
+    if (acc >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
+  }
+  const Quotient quot(d);
+#pragma unroll
+  for (int u = 0; u < VPL; ++u) {
+    const int k = lane + 32 * u;
+    if (k >= nvec) break;
+    const uint4 v = w[u];
+    Vec8 f;
+    f.v[0] = bf16_lo(v.x); f.v[1] = bf16_hi(v.x); f.v[2] = bf16_lo(v.y); f.v[3] = bf16_hi(v.y);
+    f.v[4] = bf16_lo(v.z); f.v[5] = bf16_hi(v.z); f.v[6] = bf16_lo(v.w); f.v[7] = bf16_hi(v.w);
+    codes[row * nvec + k] = quant8<FMT>(f, quot);
+    if (abs_copy) {
+      const uint32_t m = 0x7fff7fffu;
+      abs_copy[row * nvec + k] = make_uint4(v.x & m, v.y & m, v.z & m, v.w & m);
     }
   }
 }
@@ -540,6 +655,14 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
   if (x.c_contig()) {
     const int64_t total = x.nc * x.batch * (ldc >> 4);
     if (total >= (1ll << 32) || x.nc >= (1ll << 32)) return QM_ERR_UNSUPPORTED;   // 32-bit chunk index
+    const bool dense = x.dtype == QM_DT_BF16 && x.s_nc == x.c && (x.c & 15) == 0 &&
+                       (x.batch == 1 || x.s_b == x.nc * x.c);
+    if (dense) {
+      const int64_t per_block = (int64_t)kThreads * kDenseChunks;
+      quantize_dense_kernel<FMT><<<(unsigned)((total + per_block - 1) / per_block), kThreads, 0, s>>>(
+          reinterpret_cast<const uint4*>(x.data), (uint32_t)total, ds, FastDiv((uint32_t)(ldc >> 4)),
+          (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes), reinterpret_cast<uint4*>(abs_copy));
+    } else
     quantize_rows_kernel<T, FMT><<<grid_for(total, 16), kThreads, 0, s>>>(
         p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
         codes, ldc, static_cast<__nv_bfloat16*>(abs_copy));
@@ -568,6 +691,24 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
   const T* p = static_cast<const T*>(x.data);
   const int64_t rows = x.nc * x.batch, ldc = qm_code_ld(x.c), nvec = x.c / 8;
   const float qmax = fmt_qmax(FMT);
+  if (x.dtype == QM_DT_BF16 && (x.c & 15) == 0 && x.c <= 16 * 256) {
+    // the row fits in one warp's registers
+    const unsigned blocks = (unsigned)((rows * 32 + kThreads - 1) / kThreads);
+    const __nv_bfloat16* pb = static_cast<const __nv_bfloat16*>(x.data);
+#define QM_SQR(V)                                                                                 \
+  scale_quantize_rows_reg_kernel<FMT, V><<<blocks, kThreads, 0, s>>>(                             \
+      pb, x.nc, (int)nvec, x.s_nc, x.batch, x.s_b, qmax, delta_out, reinterpret_cast<uint2*>(codes), \
+      reinterpret_cast<uint4*>(abs_copy), err_word)
+    if (nvec <= 32) QM_SQR(1);
+    else if (nvec <= 64) QM_SQR(2);
+    else if (nvec <= 128) QM_SQR(4);
+    else if (nvec <= 256) QM_SQR(8);
+    else QM_SQR(16);
+#undef QM_SQR
+    count_launch();
+    QM_CUDA_OK(cudaGetLastError());
+    return QM_OK;
+  }
 #define QM_SQ(G)                                                                                   \
   scale_quantize_rows_kernel<T, FMT, G>                                                            \
       <<<(unsigned)((rows * G + kThreads - 1) / kThreads), kThreads, 0, s>>>(                      \
