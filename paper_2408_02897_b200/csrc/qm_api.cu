@@ -145,7 +145,7 @@ qm_status prepare_operand(const View& x, int fmt, int gran, uint32_t* amax, floa
                           void* abs_copy, void* kmaj_copy, uint32_t* err_word, cudaStream_t s) {
   if (gran == QM_GRAN_CHANNEL && x.c_contig())
     return launch_scale_quantize_rows(x, fmt, delta, codes, abs_copy, err_word, s);
-  qm_status st = launch_absmax(x, gran, amax, err_word, s);
+  qm_status st = launch_absmax(x, gran, amax, s);
   if (st != QM_OK) return st;
   // the quantize kernel turns max|x| into delta itself
   return launch_quantize(x, fmt, gran, reinterpret_cast<const float*>(amax), true, delta, err_word, codes,
@@ -169,7 +169,7 @@ qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n = delta_count(v, gran);
   QM_CUDA_OK(cudaMemsetAsync(delta, 0, sizeof(float) * n, s));
-  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta), nullptr, s);
+  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta), s);
   if (st != QM_OK) return st;
   return launch_finalize_delta(delta, n, fmt, nullptr, s);
 }
@@ -191,7 +191,7 @@ qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t ro
   if (gran == QM_GRAN_CHANNEL && v.c_contig() && !kmaj_copy)
     return launch_scale_quantize_rows(v, fmt, delta_out, codes, abs_copy, nullptr, s);
   QM_CUDA_OK(cudaMemsetAsync(delta_out, 0, sizeof(float) * n, s));
-  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta_out), nullptr, s);
+  st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta_out), s);
   if (st != QM_OK) return st;
   st = launch_finalize_delta(delta_out, n, fmt, nullptr, s);
   if (st != QM_OK) return st;

@@ -292,92 +292,6 @@ absmax_cols_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, 
   if (col < nc && m) atomicMax(amax + b * nc + col, m);
 }
 
-// ---------------------------------------------------------------- absmax, dense tensor, bulk-copy staged
-// Large dense tensors are streamed through shared memory with the bulk-copy engine
-// (cp.async.bulk + mbarrier): a CTA keeps kBulkStages chunks of kBulkBytes in flight, far more
-// than its threads could keep outstanding with ordinary loads.  `bytes` is a multiple of 16.
-constexpr int kBulkThreads = 128;
-constexpr uint32_t kBulkBytes = 16384;
-constexpr int kBulkStages = 4;
-
-__device__ __forceinline__ uint32_t sq_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-// Bounded wait on an mbarrier phase; false when it gave up (about a second).
-__device__ __forceinline__ bool sq_mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t polls = 0; polls < (1u << 26); ++polls) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    if (ok) return true;
-  }
-  return false;
-}
-
-__global__ void __launch_bounds__(kBulkThreads)
-absmax_bulk_kernel(const uint8_t* __restrict__ x, int64_t bytes, int is_bf16, uint32_t* __restrict__ amax,
-                   uint32_t* __restrict__ err_word) {
-  extern __shared__ __align__(128) uint8_t sq_smem[];
-  __shared__ uint64_t full[kBulkStages];
-  __shared__ uint32_t give_up;
-  const int64_t chunks = (bytes + kBulkBytes - 1) / kBulkBytes;
-  // this CTA's chunks: blockIdx.x, blockIdx.x + gridDim.x, ...
-  const int64_t mine = blockIdx.x < chunks ? (chunks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kBulkStages; ++s)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sq_smem_u32(&full[s])));
-    give_up = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  auto issue = [&](int64_t j) {            // j-th chunk of this CTA into stage j % kBulkStages
-    const int64_t c = blockIdx.x + j * gridDim.x;
-    const int64_t off = c * kBulkBytes;
-    const uint32_t n = (uint32_t)(bytes - off < kBulkBytes ? bytes - off : kBulkBytes);
-    const uint32_t bar = sq_smem_u32(&full[j % kBulkStages]);
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(sq_smem_u32(sq_smem + (j % kBulkStages) * kBulkBytes)), "l"(x + off), "r"(n), "r"(bar)
-        : "memory");
-  };
-  if (threadIdx.x == 0)
-    for (int64_t j = 0; j < mine && j < kBulkStages; ++j) issue(j);
-  uint32_t acc = 0, acc2 = 0;
-  for (int64_t j = 0; j < mine; ++j) {
-    const int s = (int)(j % kBulkStages);
-    if (!sq_mbar_wait(sq_smem_u32(&full[s]), (uint32_t)((j / kBulkStages) & 1))) give_up = 1;
-    const int64_t off = (blockIdx.x + j * gridDim.x) * (int64_t)kBulkBytes;
-    const uint32_t n = (uint32_t)(bytes - off < kBulkBytes ? bytes - off : kBulkBytes);
-    const uint4* src = reinterpret_cast<const uint4*>(sq_smem + s * kBulkBytes);
-    if (!give_up) {
-#pragma unroll
-      for (int u = 0; u < (int)(kBulkBytes / 16 / kBulkThreads); ++u) {
-        const uint32_t idx = threadIdx.x + u * kBulkThreads;
-        if (idx * 16 < n) {
-          const uint4 w = src[idx];
-          if (is_bf16) {
-            const uint32_t k = 0x7fff7fffu;
-            acc2 = __vmaxu2(acc2, __vmaxu2(__vmaxu2(w.x & k, w.y & k), __vmaxu2(w.z & k, w.w & k)));
-          } else {
-            const uint32_t k = 0x7fffffffu;
-            acc = max(acc, max(max(w.x & k, w.y & k), max(w.z & k, w.w & k)));
-          }
-        }
-      }
-    }
-    __syncthreads();                        // everyone is done with stage s
-    if (threadIdx.x == 0 && j + kBulkStages < mine && !give_up) issue(j + kBulkStages);
-  }
-  if (is_bf16) acc = max(acc2 & 0xffffu, acc2 >> 16) << 16;
-  acc = block_max(acc);
-  if (threadIdx.x == 0) {
-    if (acc) atomicMax(amax, acc);
-    if (give_up && err_word) atomicOr(err_word, QM_DEVERR_TIMEOUT);
-  }
-}
-
 __global__ void finalize_delta_kernel(float* __restrict__ delta, int64_t n, float qmax,
                                       uint32_t* __restrict__ err_word) {
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -679,25 +593,13 @@ int grid_for(int64_t work_items, int per_sm) {
 }
 
 template <typename T>
-qm_status absmax_t(const View& x, int gran, uint32_t* amax, uint32_t* err_word, cudaStream_t s) {
+qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
   const T* p = static_cast<const T*>(x.data);
   if (x.c_contig()) {
     if (gran == QM_GRAN_TENSOR) {
       const bool dense = x.s_nc == x.c && (x.batch == 1 || x.s_b == x.nc * x.c);
       const bool even = x.batch == 1 || x.s_b == x.nc * x.s_nc;
-      const int64_t nbytes = x.nc * x.batch * x.c * (int64_t)sizeof(T);
-      if (dense && nbytes >= (8ll << 20) && (nbytes & 15) == 0) {
-        static bool attr_done = false;
-        const int smem = kBulkStages * kBulkBytes;
-        if (!attr_done) {
-          QM_CUDA_OK(cudaFuncSetAttribute(absmax_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-          attr_done = true;
-        }
-        const int64_t chunks = (nbytes + kBulkBytes - 1) / kBulkBytes;
-        const int64_t cap = (int64_t)sm_count() * 3;
-        absmax_bulk_kernel<<<(unsigned)(chunks < cap ? chunks : cap), kBulkThreads, smem, s>>>(
-            static_cast<const uint8_t*>(x.data), nbytes, x.dtype == QM_DT_BF16, amax, err_word);
-      } else if (dense) {
+      if (dense) {
         const int64_t n = x.nc * x.batch * x.c;
         absmax_tensor_kernel<T><<<grid_for(n / 8 + 1, 8), kThreads, 0, s>>>(p, 1, n, n, amax);
       } else if (even) {
@@ -824,9 +726,9 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
 
 }  // namespace
 
-qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, uint32_t* err_word, cudaStream_t s) {
-  return x.dtype == QM_DT_BF16 ? absmax_t<__nv_bfloat16>(x, gran, amax_bits, err_word, s)
-                               : absmax_t<float>(x, gran, amax_bits, err_word, s);
+qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream_t s) {
+  return x.dtype == QM_DT_BF16 ? absmax_t<__nv_bfloat16>(x, gran, amax_bits, s)
+                               : absmax_t<float>(x, gran, amax_bits, s);
 }
 
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s) {
