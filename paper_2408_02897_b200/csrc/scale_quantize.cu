@@ -586,6 +586,67 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
   }
 }
 
+// ---------------------------------------------------------------- quantize + transpose, bf16 fast path
+// Storage [c][nc] (nc contiguous, bf16) with c a multiple of 32 and nc even.  A thread owns two
+// adjacent columns and 32 consecutive contraction rows: it issues its 32 four-byte loads (each
+// warp-wide load is one 128-byte row segment) before using any, then writes 32 bytes of codes
+// and 64 bytes of each bf16 copy per column - whole sectors, no shared memory, no barrier.
+// Block = 8 warps = 64 columns x 256 rows.
+template <int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
+                               int64_t s_b, const DeltaSrc ds, uint8_t* __restrict__ codes, int64_t ldc,
+                               __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t b = blockIdx.z;
+  const int64_t n = ((int64_t)blockIdx.x * 32 + lane) * 2;                 // first of this thread's two columns
+  const int64_t k0 = ((int64_t)blockIdx.y * 8 + warp) * 32;                // first contraction row
+  const float d_tensor =
+      ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0);
+  if (n >= nc || k0 >= c) return;
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(x + b * s_b + k0 * s_c + n);
+  const int64_t step = s_c >> 1;                                           // row stride in 32-bit words
+  uint32_t w[32];
+#pragma unroll
+  for (int r = 0; r < 32; ++r) w[r] = __ldg(src + r * step);
+#pragma unroll
+  for (int col = 0; col < 2; ++col) {
+    const int64_t orow = b * nc + n + col;
+    const Quotient quot(ds.per_channel ? ds.get(orow, k0 == 0) : d_tensor);
+    uint32_t cw[8];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      Vec8 f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) f.v[j] = col == 0 ? bf16_lo(w[g * 8 + j]) : bf16_hi(w[g * 8 + j]);
+      const uint2 q = quant8<FMT>(f, quot);
+      cw[2 * g] = q.x; cw[2 * g + 1] = q.y;
+    }
+    uint4* cdst = reinterpret_cast<uint4*>(codes + orow * ldc + k0);
+    cdst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+    cdst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+    if (abs_copy || kmaj_copy) {
+      // gather this column's 32 values as 16 words of two bf16 each
+      uint32_t pw[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        pw[j] = col == 0 ? __byte_perm(w[2 * j], w[2 * j + 1], 0x5410) : __byte_perm(w[2 * j], w[2 * j + 1], 0x7632);
+      if (kmaj_copy) {
+        uint4* d = reinterpret_cast<uint4*>(kmaj_copy + orow * c + k0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) d[j] = make_uint4(pw[4 * j], pw[4 * j + 1], pw[4 * j + 2], pw[4 * j + 3]);
+      }
+      if (abs_copy) {
+        const uint32_t m = 0x7fff7fffu;
+        uint4* d = reinterpret_cast<uint4*>(abs_copy + orow * c + k0);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          d[j] = make_uint4(pw[4 * j] & m, pw[4 * j + 1] & m, pw[4 * j + 2] & m, pw[4 * j + 3] & m);
+      }
+    }
+  }
+}
+
 int grid_for(int64_t work_items, int per_sm) {
   int64_t want = (work_items + kThreads - 1) / kThreads;
   int64_t cap = (int64_t)sm_count() * per_sm;
@@ -675,6 +736,15 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
                                      x.c * 2, x.nc, cudaMemcpyDeviceToDevice, s));
     }
   } else {
+    if (x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535) {
+      dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
+      quantize_transpose_bf16_kernel<FMT><<<grid, kThreads, 0, s>>>(
+          static_cast<const __nv_bfloat16*>(x.data), x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc,
+          static_cast<__nv_bfloat16*>(abs_copy), static_cast<__nv_bfloat16*>(kmaj_copy));
+      count_launch();
+      QM_CUDA_OK(cudaGetLastError());
+      return QM_OK;
+    }
     dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((ldc + 63) / 64), (unsigned)x.batch);
     quantize_transpose_kernel<T, FMT><<<grid, kThreads, 0, s>>>(
         p, x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
