@@ -399,6 +399,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   __syncthreads();
   __syncwarp();
   cluster_sync();          // the peer's barriers and tensor memory exist before anyone uses them
+  pdl_prologue();          // everything above overlapped the tail of the previous kernel
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
@@ -761,11 +762,13 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem_bytes<MODE>();
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see pdl_prologue()
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (MODE == kProbe) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));

@@ -35,6 +35,28 @@ void note_cuda_error(cudaError_t e, const char* where);
 
 int sm_count();
 
+// Programmatic dependent launch.  Every kernel of the probe's chain is launched with the
+// attribute that lets its CTAs be scheduled while the kernel before it in the stream is still
+// draining, and starts with pdl_prologue(): wait until that kernel's results are visible, then
+// allow the next kernel in the stream to be scheduled early in the same way.  This removes the
+// launch gap between the short dependent kernels of a probe.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+template <typename... P, typename... A>
+inline cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, A... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+#endif
+
 // Cumulative count of kernels this library has launched (profiling aid).
 void count_launch(int n = 1);
 // When profiling is on, returns an event pair to record around the fused tensor-core probe

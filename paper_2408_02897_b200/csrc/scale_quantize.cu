@@ -174,6 +174,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 absmax_tensor_kernel(const T* __restrict__ x, int64_t rows, int64_t c, int64_t row_stride,
                      uint32_t* __restrict__ amax) {
+  pdl_prologue();
   const int64_t vec_per_row = c >> 3;
   const int64_t total_vec = rows * vec_per_row;
   uint32_t acc = 0;
@@ -237,6 +238,7 @@ template <typename T, int G>
 __global__ void __launch_bounds__(kThreads)
 absmax_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
                    int64_t s_b, uint32_t* __restrict__ amax) {
+  pdl_prologue();
   const int64_t rows = nc * batch;
   const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
   const int sub = threadIdx.x % G;
@@ -261,6 +263,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 absmax_cols_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
                    int64_t rows_per_block, uint32_t* __restrict__ amax) {
+  pdl_prologue();
   __shared__ uint32_t s[8][256];
   const int64_t b = blockIdx.z;
   const int64_t col0 = ((int64_t)blockIdx.x * 32 + threadIdx.x) * 8;
@@ -294,6 +297,7 @@ absmax_cols_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, 
 
 __global__ void finalize_delta_kernel(float* __restrict__ delta, int64_t n, float qmax,
                                       uint32_t* __restrict__ err_word) {
+  pdl_prologue();
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   uint32_t bits = __float_as_uint(delta[i]);
@@ -333,6 +337,7 @@ __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
                      int64_t s_b, const DeltaSrc ds, const FastDiv by_chunks, const FastDiv by_nc,
                      uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy) {
+  pdl_prologue();
   const uint32_t chunks_per_row = (uint32_t)(ldc >> 4);     // 16 codes per chunk, padding included
   const uint32_t total = (uint32_t)(nc * batch) * chunks_per_row;   // < 2^32, checked by the host
   const uint32_t stride = gridDim.x * blockDim.x;
@@ -385,6 +390,7 @@ __global__ void __launch_bounds__(kThreads)
 quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const DeltaSrc ds,
                       const FastDiv by_chunks, uint32_t chunks_per_row, uint4* __restrict__ codes,
                       uint4* __restrict__ abs_copy) {
+  pdl_prologue();
   const uint32_t base = blockIdx.x * (kThreads * kDenseChunks) + threadIdx.x;
   uint4 w[kDenseChunks][2];
 #pragma unroll
@@ -432,6 +438,7 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
                            int64_t batch, int64_t s_b, float qmax, float* __restrict__ delta_out,
                            uint8_t* __restrict__ codes, int64_t ldc,
                            __nv_bfloat16* __restrict__ abs_copy, uint32_t* __restrict__ err_word) {
+  pdl_prologue();
   const int64_t rows = nc * batch;
   const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
   const int sub = threadIdx.x % G;
@@ -483,6 +490,7 @@ scale_quantize_rows_reg_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, 
                                int64_t batch, int64_t s_b, float qmax, float* __restrict__ delta_out,
                                uint2* __restrict__ codes, uint4* __restrict__ abs_copy,
                                uint32_t* __restrict__ err_word) {
+  pdl_prologue();
   const int64_t rows = nc * batch;
   const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
@@ -535,6 +543,7 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
                           const DeltaSrc ds,
                           uint8_t* __restrict__ codes, int64_t ldc,
                           __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
+  pdl_prologue();
   __shared__ float tile[64][65];     // +1 column spreads the transposed accesses over the banks
   const int64_t b = blockIdx.z;
   const int64_t c0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
@@ -597,6 +606,7 @@ __global__ void __launch_bounds__(kThreads)
 quantize_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
                                int64_t s_b, const DeltaSrc ds, uint8_t* __restrict__ codes, int64_t ldc,
                                __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
+  pdl_prologue();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t b = blockIdx.z;
   const int64_t n = ((int64_t)blockIdx.x * 32 + lane) * 2;                 // first of this thread's two columns
@@ -662,20 +672,20 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
       const bool even = x.batch == 1 || x.s_b == x.nc * x.s_nc;
       if (dense) {
         const int64_t n = x.nc * x.batch * x.c;
-        absmax_tensor_kernel<T><<<grid_for(n / 8 + 1, 8), kThreads, 0, s>>>(p, 1, n, n, amax);
+        launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s, p, 1, n, n, amax);
       } else if (even) {
-        absmax_tensor_kernel<T><<<grid_for(x.nc * x.batch * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+        launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.batch * x.c / 8 + 1, 8)), dim3(kThreads), 0, s, 
             p, x.nc * x.batch, x.c, x.s_nc, amax);
       } else {
         for (int64_t b = 0; b < x.batch; ++b)
-          absmax_tensor_kernel<T><<<grid_for(x.nc * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+          launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.c / 8 + 1, 8)), dim3(kThreads), 0, s, 
               p + b * x.s_b, x.nc, x.c, x.s_nc, amax);
       }
     } else {
       const int64_t rows = x.nc * x.batch;
       const int64_t nvec = x.c / 8;
 #define QM_ROWS(G)                                                                              \
-  absmax_rows_kernel<T, G><<<(unsigned)((rows * G + kThreads - 1) / kThreads), kThreads, 0, s>>>( \
+  launch_pdl(absmax_rows_kernel<T, G>, dim3((unsigned)((rows * G + kThreads - 1) / kThreads)), dim3(kThreads), 0, s,  \
       p, x.nc, x.c, x.s_nc, x.batch, x.s_b, amax)
       if (nvec <= 4) QM_ROWS(4);
       else if (nvec <= 8) QM_ROWS(8);
@@ -687,7 +697,7 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
     if (gran == QM_GRAN_TENSOR) {
       // storage rows are the contracting index: walk them as rows of nc contiguous elements
       for (int64_t b = 0; b < x.batch; ++b)
-        absmax_tensor_kernel<T><<<grid_for(x.nc * x.c / 8 + 1, 8), kThreads, 0, s>>>(
+        launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.c / 8 + 1, 8)), dim3(kThreads), 0, s, 
             p + b * x.s_b, x.c, x.nc, x.s_c, amax);
     } else {
       const int64_t col_blocks = (x.nc + 255) / 256;
@@ -697,7 +707,7 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
       if (rows_per_block < 64) rows_per_block = 64;
       const int64_t gy = (x.c + rows_per_block - 1) / rows_per_block;
       dim3 grid((unsigned)col_blocks, (unsigned)gy, (unsigned)x.batch), block(32, 8);
-      absmax_cols_kernel<T><<<grid, block, 0, s>>>(p, x.nc, x.c, x.s_c, x.s_b, rows_per_block, amax);
+      launch_pdl(absmax_cols_kernel<T>, dim3(grid), dim3(block), 0, s, p, x.nc, x.c, x.s_c, x.s_b, rows_per_block, amax);
     }
   }
   count_launch();
@@ -720,11 +730,11 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
                        (x.batch == 1 || x.s_b == x.nc * x.c);
     if (dense) {
       const int64_t per_block = (int64_t)kThreads * kDenseChunks;
-      quantize_dense_kernel<FMT><<<(unsigned)((total + per_block - 1) / per_block), kThreads, 0, s>>>(
+      launch_pdl(quantize_dense_kernel<FMT>, dim3((unsigned)((total + per_block - 1) / per_block)), dim3(kThreads), 0, s, 
           reinterpret_cast<const uint4*>(x.data), (uint32_t)total, ds, FastDiv((uint32_t)(ldc >> 4)),
           (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes), reinterpret_cast<uint4*>(abs_copy));
     } else
-    quantize_rows_kernel<T, FMT><<<grid_for(total, 16), kThreads, 0, s>>>(
+    launch_pdl(quantize_rows_kernel<T, FMT>, dim3(grid_for(total, 16)), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
         codes, ldc, static_cast<__nv_bfloat16*>(abs_copy));
     if (kmaj_copy) {
@@ -738,7 +748,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
   } else {
     if (x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535) {
       dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
-      quantize_transpose_bf16_kernel<FMT><<<grid, kThreads, 0, s>>>(
+      launch_pdl(quantize_transpose_bf16_kernel<FMT>, dim3(grid), dim3(kThreads), 0, s, 
           static_cast<const __nv_bfloat16*>(x.data), x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc,
           static_cast<__nv_bfloat16*>(abs_copy), static_cast<__nv_bfloat16*>(kmaj_copy));
       count_launch();
@@ -746,7 +756,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
       return QM_OK;
     }
     dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((ldc + 63) / 64), (unsigned)x.batch);
-    quantize_transpose_kernel<T, FMT><<<grid, kThreads, 0, s>>>(
+    launch_pdl(quantize_transpose_kernel<T, FMT>, dim3(grid), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
         static_cast<__nv_bfloat16*>(kmaj_copy));
   }
@@ -766,7 +776,7 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
     const unsigned blocks = (unsigned)((rows * 32 + kThreads - 1) / kThreads);
     const __nv_bfloat16* pb = static_cast<const __nv_bfloat16*>(x.data);
 #define QM_SQR(V)                                                                                 \
-  scale_quantize_rows_reg_kernel<FMT, V><<<blocks, kThreads, 0, s>>>(                             \
+  launch_pdl(scale_quantize_rows_reg_kernel<FMT, V>, dim3(blocks), dim3(kThreads), 0, s,                              \
       pb, x.nc, (int)nvec, x.s_nc, x.batch, x.s_b, qmax, delta_out, reinterpret_cast<uint2*>(codes), \
       reinterpret_cast<uint4*>(abs_copy), err_word)
     if (nvec <= 32) QM_SQR(1);
@@ -780,10 +790,10 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
     return QM_OK;
   }
 #define QM_SQ(G)                                                                                   \
-  scale_quantize_rows_kernel<T, FMT, G>                                                            \
-      <<<(unsigned)((rows * G + kThreads - 1) / kThreads), kThreads, 0, s>>>(                      \
-          p, x.nc, x.c, x.s_nc, x.batch, x.s_b, qmax, delta_out, codes, ldc,                       \
-          static_cast<__nv_bfloat16*>(abs_copy), err_word)
+  launch_pdl(scale_quantize_rows_kernel<T, FMT, G>,                                                \
+             dim3((unsigned)((rows * G + kThreads - 1) / kThreads)), dim3(kThreads), 0, s,         \
+             p, x.nc, x.c, x.s_nc, x.batch, x.s_b, qmax, delta_out, codes, ldc,                    \
+             static_cast<__nv_bfloat16*>(abs_copy), err_word)
   if (nvec <= 4) QM_SQ(4);
   else if (nvec <= 8) QM_SQ(8);
   else if (nvec <= 16) QM_SQ(16);
@@ -802,7 +812,7 @@ qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream
 }
 
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s) {
-  finalize_delta_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(delta, n, fmt_qmax(fmt), err_word);
+  launch_pdl(finalize_delta_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, s, delta, n, fmt_qmax(fmt), err_word);
   count_launch();
   QM_CUDA_OK(cudaGetLastError());
   return QM_OK;
