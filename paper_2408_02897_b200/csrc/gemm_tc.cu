@@ -768,7 +768,7 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see pdl_prologue()
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 2;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (MODE == kProbe) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));

@@ -2,6 +2,7 @@
 // probe runs in the kernels of the other translation units.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <vector>
@@ -26,6 +27,14 @@ int sm_count() {
       n = 148;
   }
   return n;
+}
+
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("QM_PDL");
+    return !(e && e[0] == '0');
+  }();
+  return on;
 }
 
 static std::atomic<long long> g_launches{0};

@@ -40,6 +40,7 @@ int sm_count();
 // draining, and starts with pdl_prologue(): wait until that kernel's results are visible, then
 // allow the next kernel in the stream to be scheduled early in the same way.  This removes the
 // launch gap between the short dependent kernels of a probe.
+bool pdl_enabled();   // on unless the environment has QM_PDL=0
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_prologue() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -52,7 +53,7 @@ inline cudaError_t launch_pdl(void (*kernel)(P...), dim3 grid, dim3 block, size_
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
+  cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
 }
 #endif
