@@ -380,21 +380,20 @@ quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_n
 // ---------------------------------------------------------------- quantize, dense bf16 fast path
 // The common case of the probe: a dense bf16 tensor whose rows are a multiple of 16 long, so the
 // whole tensor is one flat run of 16-element chunks and codes have no padding.  Each thread
-// takes kDenseChunks chunks a block-width apart and issues all of their 128-bit loads before
-// touching any of them (2 x kDenseChunks loads in flight per thread); |x| copies are the raw
+// takes CHUNKS chunks a block-width apart and issues all of their 128-bit loads before touching
+// any of them (2 x CHUNKS loads in flight per thread; 4 for tensors that fill the GPU several
+// times over, 1 for small ones, which need the parallelism more); |x| copies are the raw
 // bit patterns with the sign bits cleared.
-constexpr int kDenseChunks = 4;
-
-template <int FMT>
+template <int FMT, int CHUNKS>
 __global__ void __launch_bounds__(kThreads)
 quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const DeltaSrc ds,
                       const FastDiv by_chunks, uint32_t chunks_per_row, uint4* __restrict__ codes,
                       uint4* __restrict__ abs_copy) {
   pdl_prologue();
-  const uint32_t base = blockIdx.x * (kThreads * kDenseChunks) + threadIdx.x;
-  uint4 w[kDenseChunks][2];
+  const uint32_t base = blockIdx.x * (kThreads * CHUNKS) + threadIdx.x;
+  uint4 w[CHUNKS][2];
 #pragma unroll
-  for (int u = 0; u < kDenseChunks; ++u) {
+  for (int u = 0; u < CHUNKS; ++u) {
     const uint32_t i = base + u * kThreads;
     const uint32_t j = i < total_chunks ? i : total_chunks - 1;     // clamp: results of dead lanes are dropped
     w[u][0] = __ldg(x + 2 * (size_t)j);
@@ -403,7 +402,7 @@ quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const 
   const float d_tensor = ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && threadIdx.x == 0);
   const Quotient quot_tensor(d_tensor);
 #pragma unroll
-  for (int u = 0; u < kDenseChunks; ++u) {
+  for (int u = 0; u < CHUNKS; ++u) {
     const uint32_t i = base + u * kThreads;
     if (i >= total_chunks) break;
     Quotient quot = quot_tensor;
@@ -729,10 +728,18 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
     const bool dense = x.dtype == QM_DT_BF16 && x.s_nc == x.c && (x.c & 15) == 0 &&
                        (x.batch == 1 || x.s_b == x.nc * x.c);
     if (dense) {
-      const int64_t per_block = (int64_t)kThreads * kDenseChunks;
-      launch_pdl(quantize_dense_kernel<FMT>, dim3((unsigned)((total + per_block - 1) / per_block)), dim3(kThreads), 0, s, 
-          reinterpret_cast<const uint4*>(x.data), (uint32_t)total, ds, FastDiv((uint32_t)(ldc >> 4)),
-          (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes), reinterpret_cast<uint4*>(abs_copy));
+      const uint4* src = reinterpret_cast<const uint4*>(x.data);
+      const FastDiv by_chunks((uint32_t)(ldc >> 4));
+      if (total >= (int64_t)sm_count() * 8 * kThreads * 4) {
+        const int64_t per_block = (int64_t)kThreads * 4;
+        launch_pdl(quantize_dense_kernel<FMT, 4>, dim3((unsigned)((total + per_block - 1) / per_block)), dim3(kThreads),
+                   0, s, src, (uint32_t)total, ds, by_chunks, (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes),
+                   reinterpret_cast<uint4*>(abs_copy));
+      } else {
+        launch_pdl(quantize_dense_kernel<FMT, 1>, dim3((unsigned)((total + kThreads - 1) / kThreads)), dim3(kThreads),
+                   0, s, src, (uint32_t)total, ds, by_chunks, (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes),
+                   reinterpret_cast<uint4*>(abs_copy));
+      }
     } else
     launch_pdl(quantize_rows_kernel<T, FMT>, dim3(grid_for(total, 16)), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
@@ -746,7 +753,8 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
                                      x.c * 2, x.nc, cudaMemcpyDeviceToDevice, s));
     }
   } else {
-    if (x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535) {
+    if (x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
+        ((x.nc + 63) / 64) * ((x.c + 255) / 256) * x.batch >= 4 * (int64_t)sm_count()) {
       dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
       launch_pdl(quantize_transpose_bf16_kernel<FMT>, dim3(grid), dim3(kThreads), 0, s, 
           static_cast<const __nv_bfloat16*>(x.data), x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc,
