@@ -29,6 +29,18 @@ sys.path.insert(0, ROOT)
 
 from paper_2408_02897_b200 import workloads  # noqa: E402
 
+# DRAM traffic of the fused probe kernel from one ncu capture (profiles/tc_kernel_probe_*.md):
+# dram__bytes_read + dram__bytes_write for M=4096 N=2304 K=768 E4M3, and the library's kernel
+# revision the counters were taken at.  Traffic grows with the operand bytes (every operand is
+# read from DRAM once), so a launch of another shape is scaled by its operand bytes.
+NCU_TC = {"revision": "tc-pair-rot4", "dram_bytes": 24.646e6, "shape": (4096, 2304, 768)}
+
+
+def tc_operand_bytes(M, N, K, b=1):
+    """Bytes the fused kernel reads per launch: L, |L| (bf16), R, |R| (bf16) and both code tensors."""
+    return b * ((M + N) * K * 2 * 2 + (M + N) * K)
+
+
 METRIC = "probe TFLOPS"
 UNIT = "TFLOP/s"
 
@@ -214,7 +226,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="bert_base_fwd")
-    ap.add_argument("--oracle-rows", type=int, default=2048)
+    ap.add_argument("--oracle-rows", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
 
@@ -317,9 +329,15 @@ def main():
     # (2 x bf16) and two at the bf16 rate  ->  3 / (1/(2P) + 2/P) = 1.2 P in summed flops
     peak_tflops = 1.2 * peaks["bf16_tflops"]
     achieved = flops_step * args.steps / (tc_ms * 1e-3) / 1e12 if tc_ms > 0 else None
+    traffic = None
+    if qm.lib().qm_kernel_revision().decode() == NCU_TC["revision"]:
+        per_byte = NCU_TC["dram_bytes"] / tc_operand_bytes(*NCU_TC["shape"])
+        shapes = [workloads.op_flops(o)[0] for o in ops]
+        traffic = per_byte * sum(tc_operand_bytes(*sh) for sh in shapes) / len(shapes)
     roofline = {"bound": "tensor", "kernel": "tc_kernel<probe> (fused 8-bit + reference + denominator products, Eq. 3 epilogue)",
                 "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
-                "frac": achieved / peak_tflops if achieved else None, "traffic": None,
+                "frac": achieved / peak_tflops if achieved else None, "traffic": traffic,
+                "traffic_note": "bytes per launch (mean over the step's launches), scaled from the ncu capture by operand bytes",
                 "peak_source": f"1.2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}",
                 "launches": tc_launches, "avg_launch_ms": tc_ms / max(tc_launches, 1)}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),

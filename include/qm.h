@@ -243,6 +243,9 @@ qm_status qm_metric_noalloc(const float* ref, const float* q, const float* den, 
  * Events are host objects; no device memory is involved.
  */
 int64_t qm_kernel_launches(void);
+/* Tag of the fused tensor-core kernel's current design; changes whenever that kernel changes,
+ * so that stored profiler counters can be recognised as stale. */
+const char* qm_kernel_revision(void);
 qm_status qm_profile_enable(int32_t on);
 qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
 

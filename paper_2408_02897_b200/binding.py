@@ -81,6 +81,7 @@ def lib():
             "qm_last_cuda_error": (C.c_char_p, []),
             "qm_metric_noalloc": (I32, [P, P, P, I64, P, P]),
             "qm_metric_noalloc_max_count": (I64, []),
+            "qm_kernel_revision": (C.c_char_p, []),
             "qm_kernel_launches": (I64, []),
             "qm_profile_enable": (I32, [I32]),
             "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),
