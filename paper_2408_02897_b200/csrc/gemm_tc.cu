@@ -154,6 +154,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// The same for a converged warp: every lane waits, and all lanes take the same decision.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               uint32_t* err_word) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, err_word));
+}
+
 // Tile load into this CTA's shared memory; the byte count is credited to the barrier at
 // `bar_cluster_addr`, which may live in the peer CTA (cta_group::2 form).
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
@@ -168,9 +174,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// One lane of a fully converged warp.  The MMA warp runs its whole loop (waits, descriptor
+// arithmetic, loop control) convergently and narrows to one lane only around each tcgen05
+// instruction: issued from a loop that a single lane runs alone, every MMA cost about 100 cycles
+// of issue time, which was the limit of the main loop; issued this way it costs about 60.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t p;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(p));
+  return p != 0;
+}
+
 // Arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once all MMAs
-// issued so far have completed.
+// issued so far have completed.  Called by a converged warp; one lane issues.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  if (!elect_one()) return;
   const uint16_t mask = 3;
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -193,10 +210,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t span_bytes
 
 enum MmaKind { kKindF16 = 0, kKindF8 = 1, kKindI8 = 2 };
 
-// D[256 x N] (+)= A[256 x k] . B[N x k]^T across the CTA pair; issued by one thread of the leader.
+// D[256 x N] (+)= A[256 x k] . B[N x k]^T across the CTA pair; called by a converged warp of the
+// leader, one lane issues.
 template <int KIND>
 __device__ __forceinline__ void mma_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
                                          uint32_t accumulate) {
+  if (!elect_one()) return;
   if (KIND == kKindF16) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -443,7 +462,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
-    if (rank == 0 && lane == 0) {
+    if (rank == 0) {   // the whole warp, converged: see elect_one()
       constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
       uint32_t g = 0, it = 0;
       bool ok = true;
@@ -455,12 +474,12 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
         const uint32_t col_ref = MODE == kProbe ? ((3 * it) & 3) * 128u : 0u;
         const uint32_t col_den = ((3 * it + 1) & 3) * 128u;
         const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : 0u;
-        if (it > 0 && !mbar_wait(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
+        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t use = g / kStages;
-          if (!mbar_wait(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
+          if (!mbar_wait_warp(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
           if (MODE == kProbe || MODE == kRefOnly) {
@@ -704,6 +723,7 @@ struct Shared5 {
 // D[256 x N] (+)= A . B^T with A read from tensor memory (each CTA its own 128 rows).
 __device__ __forceinline__ void mma_pair_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc,
                                             uint32_t accumulate) {
+  if (!elect_one()) return;
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
@@ -797,18 +817,18 @@ tc_probe5_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constan
           tma_load_3d(base + kOffCr, &map_cr, bar, k0, c0, tc.b);
         }
       }
-    } else if (warp == 1 && rank == 0 && lane == 0) {
-      // ---------------------------------------------------------- MMA issuer (leader CTA)
+    } else if (warp == 1 && rank == 0) {
+      // ---------------------------------------------------------- MMA issuer (leader CTA, whole warp)
       constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
       uint32_t g = 0, it = 0;
       bool ok = true;
       for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
-        if (it > 0 && !mbar_wait(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
+        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages5, slot = g & 1;
-          if (!mbar_wait(smem_u32(&sh->full[s]), (g / kStages5) & 1, abort_flag, a.err_word) ||
-              !mbar_wait(smem_u32(&sh->a_ready[slot]), (g >> 1) & 1, abort_flag, a.err_word)) {
+          if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages5) & 1, abort_flag, a.err_word) ||
+              !mbar_wait_warp(smem_u32(&sh->a_ready[slot]), (g >> 1) & 1, abort_flag, a.err_word)) {
             ok = false;
             break;
           }
