@@ -46,6 +46,7 @@ constexpr uint32_t kALp = kBlockM * kBlockK;                      //  8 KB,  64-
 constexpr uint32_t kBBf16 = kHalfN * kBlockK * 2;                 //  8 KB
 constexpr uint32_t kBLp = kHalfN * kBlockK;                       //  4 KB
 constexpr int kMaxStages = 8;
+constexpr int kRefAhead = 2;               // k-blocks of reference MMAs issued before the hand-back wait
 
 enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2 };
 
@@ -186,8 +187,8 @@ __device__ __forceinline__ bool elect_one() {
 
 // Arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once all MMAs
 // issued so far have completed.  Called by a converged warp; one lane issues.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  if (!elect_one()) return;
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, bool lead) {
+  if (!lead) return;
   const uint16_t mask = 3;
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -214,8 +215,8 @@ enum MmaKind { kKindF16 = 0, kKindF8 = 1, kKindI8 = 2 };
 // leader, one lane issues.
 template <int KIND>
 __device__ __forceinline__ void mma_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc,
-                                         uint32_t accumulate) {
-  if (!elect_one()) return;
+                                         uint32_t accumulate, bool lead) {
+  if (!lead) return;
   if (KIND == kKindF16) {
     asm volatile(
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -262,6 +263,7 @@ struct Shared {
   uint64_t empty[kMaxStages];    // per CTA: the pair's MMAs have finished reading the stage
   uint64_t tmem_full;            // per CTA: the tile's accumulators are complete
   uint64_t tmem_empty;           // leader: both CTAs' epilogues have drained the accumulators
+  uint64_t lp_done;              // leader (probe): both CTAs' epilogues have finished a tile
   uint32_t tmem_base;
   uint32_t abort_flag;
   uint32_t is_last;
@@ -407,6 +409,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
     }
     mbar_init(smem_u32(&sh->tmem_full), 1);
     mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
+    mbar_init(smem_u32(&sh->lp_done), 2 * kEpiWarps);
     sh->abort_flag = 0;
     sh->is_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -463,46 +466,80 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader CTA only)
     if (rank == 0) {   // the whole warp, converged: see elect_one()
+      const bool lead = elect_one();
       constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
       uint32_t g = 0, it = 0;
       bool ok = true;
       for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
         // Probe: the three accumulators rotate through the four 128-column blocks of tensor
-        // memory (see the epilogue).  This tile may start once both epilogues have copied the
-        // previous tile's reference and denominator blocks out; that signal also implies that
-        // the epilogue of the tile before it is finished, which frees this tile's third block.
+        // memory (see the epilogue).  The reference block of this tile has been free since the
+        // epilogue of tile it-2 ended (awaited before tile it-1 was committed, below), so the
+        // reference MMAs of the first k-blocks are issued at once and keep the tensor pipe busy
+        // while both epilogues copy the previous tile's reference and denominator blocks out
+        // and hand them back; the denominator and 8-bit MMAs of those k-blocks follow that
+        // signal.
         const uint32_t col_ref = MODE == kProbe ? ((3 * it) & 3) * 128u : 0u;
         const uint32_t col_den = ((3 * it + 1) & 3) * 128u;
         const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : 0u;
+        auto issue_ref = [&](uint32_t base, int kb) {
+          const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+            mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+        };
+        auto issue_den = [&](uint32_t base, int kb) {
+          const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)
+            mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+        };
+        auto issue_lp = [&](uint32_t base, int kb) {
+          const uint64_t dl = smem_desc(base + C::kOffCl, 64), dr = smem_desc(base + C::kOffCr, 64);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
+            mma_pair<LPKIND>(tmem_base + col_lp, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0, lead);
+        };
+        int kb = 0;
+        if (MODE == kProbe) {
+          const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
+          for (int j = 0; j < n_ahead && ok; ++j) {
+            const int s = (g + j) % kStages;
+            if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, a.err_word)) ok = false;
+            tc_fence_after();
+            if (ok) issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
+          }
+          if (!ok) break;
+        }
         if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
         tc_fence_after();
-        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+        if (MODE == kProbe) {
+          const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
+          for (; kb < n_ahead; ++kb, ++g) {
+            const int s = g % kStages;
+            const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+            issue_den(base, kb);
+            issue_lp(base, kb);
+            tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+          }
+        }
+        for (; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t use = g / kStages;
           if (!mbar_wait_warp(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-          if (MODE == kProbe || MODE == kRefOnly) {
-            const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
-#pragma unroll
-            for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-              mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-          }
-          if (MODE == kProbe) {
-            const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
-#pragma unroll
-            for (int k = 0; k < kBlockK / 16; ++k)
-              mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-          }
-          if (MODE == kProbe || MODE == kLpOnly) {
-            const uint64_t dl = smem_desc(base + C::kOffCl, 64), dr = smem_desc(base + C::kOffCr, 64);
-#pragma unroll
-            for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
-              mma_pair<LPKIND>(tmem_base + col_lp, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0);
-          }
-          tc_commit_pair(smem_u32(&sh->empty[s]));        // frees the stage in both CTAs
+          if (MODE == kProbe || MODE == kRefOnly) issue_ref(base, kb);
+          if (MODE == kProbe) issue_den(base, kb);
+          if (MODE == kProbe || MODE == kLpOnly) issue_lp(base, kb);
+          tc_commit_pair(smem_u32(&sh->empty[s]), lead);        // frees the stage in both CTAs
         }
-        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full)); // this tile's accumulators are complete
+        // The next tile's reference block is this tile's free one, last read by the epilogue of
+        // tile it-1: wait for that epilogue here, where the barrier cannot yet have moved on to
+        // this tile's phase.
+        if (MODE == kProbe && ok && it > 0 &&
+            !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, a.err_word))
+          ok = false;
+        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full), lead); // this tile's accumulators are complete
       }
     }
   } else {
@@ -573,6 +610,8 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           mbe = fmax(mbe, (double)st.mx);
         }
         tc_fence_before();                        // the 8-bit block's loads are complete as well
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
       } else {
 #pragma unroll 1
         for (int c = 0; c < 2; ++c) {
@@ -677,358 +716,6 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
                  : "memory");
   }
 }
-
-// ------------------------------------------------------------------ probe kernel, left operand through tensor memory
-// Same CTA-pair tiling, but the reference and denominator MMAs take their left operand from
-// TENSOR MEMORY: four converter warps read each landed L tile from shared memory once and
-// write it, and its sign-cleared copy, into a two-slot ring of 64 tensor-memory columns
-// (tcgen05.st).  |L| is therefore neither loaded by TMA nor read from shared memory, and L is read
-// once instead of by four MMAs: 88 KB of shared-memory traffic per 64-deep k-block instead of
-// 120 KB.  The ring takes the 128 columns the accumulator rotation would need, so the epilogue
-// instead empties tensor memory quickly: reference and denominator columns into registers, the
-// 8-bit columns into a shared-memory staging area private to each thread, hand-back, then the
-// arithmetic under the next tile's main loop.
-//
-// 512 threads = four warpgroups with re-balanced registers (setmaxnreg):
-//   warps 0..3   warp 0 lane 0: TMA producer; warp 1: tensor-memory allocation, lane 0 of the
-//                leader CTA issues the MMAs; warps 2, 3 idle
-//   warps 4..7   converters (warp w owns tensor-memory lanes 32 (w % 4) ..)
-//   warps 8..15  epilogue
-namespace v5 {
-
-constexpr int kThreads5 = 512;
-constexpr int kStages5 = 3;
-constexpr uint32_t kOffL = 0, kOffCl = kABf16, kOffR = kABf16 + kALp, kOffRa = kOffR + kBBf16, kOffCr = kOffRa + kBBf16;
-constexpr uint32_t kStageBytes5 = kOffCr + kBLp;                 // 44 KB
-constexpr uint32_t kLeaderBytes = kStageBytes5 - kABf16;         // per CTA, credited to the leader's barrier
-constexpr uint32_t kStagingBytes = kBlockM * kBlockN * 4;        // 64 KB, [column][row] fp32
-constexpr uint32_t kColRef = 0, kColDen = 128, kColLp = 256, kColA = 384;
-
-struct Shared5 {
-  uint64_t full_a[kStages5];     // local: this CTA's L tile has landed
-  uint64_t full[kStages5];       // leader: the other tiles of both CTAs have landed
-  uint64_t empty[kStages5];      // local: MMAs (1) and converter warps (4) are done with the stage
-  uint64_t a_ready[2];           // leader: both CTAs' converters have filled the slot (8 warps)
-  uint64_t a_empty[2];           // local: the MMAs that read the slot have completed
-  uint64_t tmem_full;            // local
-  uint64_t tmem_empty;           // leader: 16 epilogue warps
-  uint32_t tmem_base;
-  uint32_t abort_flag;
-  uint32_t is_last;
-  uint32_t pad;
-  float delta_r[2][kBlockN];
-  double red[5][kEpiWarps];
-};
-
-// D[256 x N] (+)= A . B^T with A read from tensor memory (each CTA its own 128 rows).
-__device__ __forceinline__ void mma_pair_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc,
-                                            uint32_t accumulate) {
-  if (!elect_one()) return;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-
-template <int LPKIND>
-__global__ void __launch_bounds__(kThreads5, 1)
-tc_probe5_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r,
-                 const __grid_constant__ CUtensorMap map_ra, const __grid_constant__ CUtensorMap map_cl,
-                 const __grid_constant__ CUtensorMap map_cr, const KernelArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  float* staging = reinterpret_cast<float*>(tiles + (size_t)kStages5 * kStageBytes5);
-  Shared5* sh = reinterpret_cast<Shared5*>(tiles + (size_t)kStages5 * kStageBytes5 + kStagingBytes);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();
-  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const int num_kb = (int)((a.K + kBlockK - 1) / kBlockK);
-  volatile uint32_t* abort_flag = &sh->abort_flag;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages5; ++s) {
-      mbar_init(smem_u32(&sh->full_a[s]), 1);
-      mbar_init(smem_u32(&sh->full[s]), 1);
-      mbar_init(smem_u32(&sh->empty[s]), 5);
-    }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&sh->a_ready[s]), 8);
-      mbar_init(smem_u32(&sh->a_empty[s]), 1);
-    }
-    mbar_init(smem_u32(&sh->tmem_full), 1);
-    mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
-    sh->abort_flag = 0;
-    sh->is_last = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&sh->tmem_base)), "r"(512u) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  __syncwarp();
-  cluster_sync();
-  pdl_prologue();
-  tc_fence_after();
-  const uint32_t tmem_base = sh->tmem_base;
-
-  if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
-    if (warp == 0 && lane == 0) {
-      // ---------------------------------------------------------- TMA producer (both CTAs)
-      uint32_t g = 0;
-      bool ok = true;
-      for (int t = pair; t < a.num_tiles && ok; t += num_pairs) {
-        const TileCoord tc = tile_coord(t, a);
-        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;
-        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;
-        for (int kb = 0; kb < num_kb; ++kb, ++g) {
-          const int s = g % kStages5;
-          const uint32_t use = g / kStages5;
-          if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, a.err_word)) {
-            ok = false;
-            break;
-          }
-          if (rank == 0) mbar_expect_tx(smem_u32(&sh->full[s]), 2 * kLeaderBytes);
-          mbar_expect_tx(smem_u32(&sh->full_a[s]), kABf16);
-          const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
-          const uint32_t bar_a = map_to_cta(smem_u32(&sh->full_a[s]), rank);
-          const uint32_t base = smem_u32(tiles + (size_t)s * kStageBytes5);
-          const int k0 = kb * kBlockK;
-          tma_load_3d(base + kOffL, &map_l, bar_a, k0, r0, tc.b);
-          tma_load_3d(base + kOffR, &map_r, bar, k0, c0, tc.b);
-          tma_load_3d(base + kOffRa, &map_ra, bar, k0, c0, tc.b);
-          tma_load_3d(base + kOffCl, &map_cl, bar, k0, r0, tc.b);
-          tma_load_3d(base + kOffCr, &map_cr, bar, k0, c0, tc.b);
-        }
-      }
-    } else if (warp == 1 && rank == 0) {
-      // ---------------------------------------------------------- MMA issuer (leader CTA, whole warp)
-      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
-      uint32_t g = 0, it = 0;
-      bool ok = true;
-      for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
-        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
-        tc_fence_after();
-        for (int kb = 0; kb < num_kb; ++kb, ++g) {
-          const int s = g % kStages5, slot = g & 1;
-          if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages5) & 1, abort_flag, a.err_word) ||
-              !mbar_wait_warp(smem_u32(&sh->a_ready[slot]), (g >> 1) & 1, abort_flag, a.err_word)) {
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t base = smem_u32(tiles + (size_t)s * kStageBytes5);
-          const uint32_t a_l = tmem_base + kColA + slot * 64, a_la = a_l + 32;
-          const uint64_t dr = smem_desc(base + kOffR, 128), dra = smem_desc(base + kOffRa, 128);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 8 tensor-memory columns of A, 32 bytes of B
-            mma_pair_ts(tmem_base + kColRef, a_l + 8 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)
-            mma_pair_ts(tmem_base + kColDen, a_la + 8 * k, dra + 2 * k, idesc_bf16, (kb | k) != 0);
-          const uint64_t dcl = smem_desc(base + kOffCl, 64), dcr = smem_desc(base + kOffCr, 64);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k)
-            mma_pair<LPKIND>(tmem_base + kColLp, dcl + 2 * k, dcr + 2 * k, a.idesc_lp, (kb | k) != 0);
-          tc_commit_pair(smem_u32(&sh->empty[s]));
-          tc_commit_pair(smem_u32(&sh->a_empty[slot]));
-        }
-        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full));
-      }
-    }
-  } else if (warp < 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    // ------------------------------------------------------------ converters (both CTAs)
-    const int q = warp & 3;
-    const int r = q * 32 + lane;                                 // row of the CTA's L tile = tensor-memory lane
-    const uint32_t a_ready_leader0 = map_to_cta(smem_u32(&sh->a_ready[0]), 0);
-    const uint32_t a_ready_leader1 = map_to_cta(smem_u32(&sh->a_ready[1]), 0);
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kColA;
-    uint32_t g = 0;
-    bool ok = true;
-    for (int t = pair; t < a.num_tiles && ok; t += num_pairs) {
-      for (int kb = 0; kb < num_kb; ++kb, ++g) {
-        const int s = g % kStages5, slot = g & 1;
-        bool w = mbar_wait(smem_u32(&sh->full_a[s]), (g / kStages5) & 1, abort_flag, a.err_word);
-        if (w && g >= 2) w = mbar_wait(smem_u32(&sh->a_empty[slot]), ((g >> 1) - 1) & 1, abort_flag, a.err_word);
-        if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-        tc_fence_after();
-        // the row's eight 16-byte chunks sit at chunk index c ^ (r % 8) (128-byte swizzle)
-        const uint8_t* row = tiles + (size_t)s * kStageBytes5 + kOffL + r * 128;
-        uint32_t v[32], va[32];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 x = *reinterpret_cast<const uint4*>(row + ((c ^ (r & 7)) << 4));
-          v[4 * c] = x.x; v[4 * c + 1] = x.y; v[4 * c + 2] = x.z; v[4 * c + 3] = x.w;
-        }
-#pragma unroll
-        for (int i = 0; i < 32; ++i) va[i] = v[i] & 0x7fff7fffu;
-        tmem_st32(lane_addr + slot * 64, v);
-        tmem_st32(lane_addr + slot * 64 + 32, va);
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive_cluster(slot ? a_ready_leader1 : a_ready_leader0);
-          mbar_arrive_cluster(map_to_cta(smem_u32(&sh->empty[s]), rank));
-        }
-      }
-    }
-  } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
-    // ------------------------------------------------------------ epilogue (warps 8..15, both CTAs)
-    const int q = warp & 3;
-    const int h = (warp - 8) >> 2;
-    const int et = (warp - 8) * 32 + lane;
-    const float dl_tensor = !a.pc_l ? __ldg(a.dl) : 1.f;
-    const float dr_tensor = !a.pc_r ? __ldg(a.dr) : 1.f;
-    const bool per_col = a.pc_r;
-    const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
-    float* stg = staging + (h * 64) * kBlockM + q * 32 + lane;   // [column][row], this thread's row
-    double sbe = 0, mbe = 0, sd2 = 0, sr2 = 0, sn2 = 0;
-    uint32_t it = 0;
-    for (int t = pair; t < a.num_tiles; t += num_pairs, ++it) {
-      const TileCoord tc = tile_coord(t, a);
-      float* dr_s = sh->delta_r[it & 1];
-      if (per_col && et < kBlockN) {
-        const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
-        dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
-      }
-      const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
-      const bool row_ok = row < a.M;
-      float dlv = dl_tensor;
-      if (a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
-
-      const bool ok = mbar_wait(smem_u32(&sh->tmem_full), it & 1, abort_flag, a.err_word);
-      if (epi_barrier_any(!ok)) break;
-      tc_fence_after();
-      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;
-      // empty tensor memory: reference and denominator columns into registers, 8-bit columns
-      // into this thread's staging cells
-      uint32_t rc[64], rd[64];
-      tmem_ld32(lane_addr + kColRef + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
-      tmem_ld32(lane_addr + kColRef + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
-      tmem_ld32(lane_addr + kColDen + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
-      tmem_ld32(lane_addr + kColDen + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t rq[32];
-        tmem_ld32(lane_addr + kColLp + h * 64 + c * 32, rq);
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) stg[(c * 32 + j) * kBlockM] = __uint_as_float(rq[j]);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
-      Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f};
-      const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int cc0 = h * 64 + c * 16;
-        const int64_t col0 = colw + c * 16;
-        if (col0 < a.N) {
-          uint32_t rq[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) rq[j] = __float_as_uint(stg[(c * 16 + j) * kBlockM]);
-          const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
-          if (n_live == 16) stats16<LPKIND, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
-          else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
-        }
-      }
-      if (row_ok) {
-        float x0, x1;
-        unpack2(st.be, x0, x1); sbe += (double)x0 + (double)x1;
-        unpack2(st.d2, x0, x1); sd2 += (double)x0 + (double)x1;
-        unpack2(st.r2, x0, x1); sr2 += (double)x0 + (double)x1;
-        unpack2(st.n2, x0, x1); sn2 += (double)x0 + (double)x1;
-        mbe = fmax(mbe, (double)st.mx);
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      sbe += __shfl_xor_sync(0xffffffffu, sbe, o);
-      mbe = fmax(mbe, __shfl_xor_sync(0xffffffffu, mbe, o));
-      sd2 += __shfl_xor_sync(0xffffffffu, sd2, o);
-      sr2 += __shfl_xor_sync(0xffffffffu, sr2, o);
-      sn2 += __shfl_xor_sync(0xffffffffu, sn2, o);
-    }
-    if (lane == 0) {
-      sh->red[0][warp - 8] = sbe; sh->red[1][warp - 8] = mbe; sh->red[2][warp - 8] = sd2;
-      sh->red[3][warp - 8] = sr2; sh->red[4][warp - 8] = sn2;
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (et == 0) {
-      double r[5] = {0, 0, 0, 0, 0};
-      for (int i = 0; i < kEpiWarps; ++i) {
-        r[0] += sh->red[0][i]; r[1] = fmax(r[1], sh->red[1][i]); r[2] += sh->red[2][i];
-        r[3] += sh->red[3][i]; r[4] += sh->red[4][i];
-      }
-      double* rec = a.partials + (int64_t)blockIdx.x * kPartialDoubles;
-      for (int i = 0; i < 5; ++i) __stcg(rec + i, r[i]);
-      __threadfence();
-      const uint32_t prev = atomicAdd(a.done_counter, 1u);
-      sh->is_last = prev == gridDim.x - 1 ? 1u : 0u;
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (sh->is_last && warp == 8) {
-      __threadfence();
-      double r[5] = {0, 0, 0, 0, 0};
-      for (int i = lane; i < (int)gridDim.x; i += 32) {
-        const double* rec = a.partials + (int64_t)i * kPartialDoubles;
-        r[0] += __ldcg(rec); r[1] = fmax(r[1], __ldcg(rec + 1)); r[2] += __ldcg(rec + 2);
-        r[3] += __ldcg(rec + 3); r[4] += __ldcg(rec + 4);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        r[0] += __shfl_xor_sync(0xffffffffu, r[0], o);
-        r[1] = fmax(r[1], __shfl_xor_sync(0xffffffffu, r[1], o));
-        r[2] += __shfl_xor_sync(0xffffffffu, r[2], o);
-        r[3] += __shfl_xor_sync(0xffffffffu, r[3], o);
-        r[4] += __shfl_xor_sync(0xffffffffu, r[4], o);
-      }
-      if (lane == 0) {
-        a.result->sum_be = r[0]; a.result->max_be = r[1]; a.result->sum_diff2 = r[2];
-        a.result->sum_ref2 = r[3]; a.result->sum_den2 = r[4];
-        a.result->count = a.count;
-        a.result->device_error = a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u;
-        a.result->reserved = 0;
-      }
-    }
-  }
-
-  // ---------------------------------------------------------------- common exit
-  tc_fence_before();
-  __syncthreads();
-  __syncwarp();
-  cluster_sync();
-  if (warp == 1) {
-    __syncwarp();
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
-  }
-}
-
-constexpr size_t kSmem5 = (size_t)kStages5 * kStageBytes5 + kStagingBytes + sizeof(Shared5) + 1024;
-
-}  // namespace v5
 
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1151,48 +838,9 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   return QM_OK;
 }
 
-template <int LPKIND>
-qm_status launch5(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cudaStream_t s) {
-  auto kern = v5::tc_probe5_kernel<LPKIND>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)v5::kSmem5));
-    attr_done = true;
-  }
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)grid_size(g));
-  cfg.blockDim = dim3(v5::kThreads5);
-  cfg.dynamicSmemBytes = v5::kSmem5;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[1].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = pdl_enabled() ? 2 : 1;
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  profile_events(&ev0, &ev1);
-  if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
-  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[3], maps[4], maps[5], ka));
-  if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
-  count_launch();
-  return QM_OK;
-}
-
-// Which probe kernel runs: the tensor-memory-fed one unless QM_TC_KERNEL=rot4 is in the environment.
-bool use_v5() {
-  static const bool on = [] {
-    const char* e = getenv("QM_TC_KERNEL");
-    return e && e[0] == 'v';     // "v5"
-  }();
-  return on;
-}
-
 }  // namespace
 
 int tc_probe_records(GemmShape g) { return grid_size(g); }
-bool tc_probe_needs_left_abs() { return !use_v5(); }
 
 qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   if (!shape_ok(p.g)) return QM_ERR_UNSUPPORTED;
@@ -1201,8 +849,7 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   CUtensorMap maps[6];
   bool ok = make_map(&maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
             make_map(&maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
-            (use_v5() ? ((maps[2] = maps[0]), true)
-                      : make_map(&maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K)) &&
+            make_map(&maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
             make_map(&maps[3], p.r_abs, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K) &&
             make_map(&maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
             make_map(&maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
@@ -1213,8 +860,6 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
   ka.count = (uint64_t)(g.M * g.N * g.batch);
   ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
-  if (use_v5())
-    return p.fmt_l == QM_FMT_INT8 ? launch5<kKindI8>(maps, ka, g, s) : launch5<kKindF8>(maps, ka, g, s);
   return p.fmt_l == QM_FMT_INT8 ? launch<kProbe, kKindI8>(maps, ka, g, s)
                                 : launch<kProbe, kKindF8>(maps, ka, g, s);
 }

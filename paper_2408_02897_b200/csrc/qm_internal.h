@@ -119,8 +119,6 @@ struct TcProbeArgs {
   uint32_t* err_word;
 };
 int tc_probe_records(GemmShape g);
-// false when the fused kernel derives |L| itself and the quantize step need not write it
-bool tc_probe_needs_left_abs();
 qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
 qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
                             const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
