@@ -402,6 +402,11 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   const int num_kb = (int)((a.K + kBlockK - 1) / kBlockK);
   volatile uint32_t* abort_flag = &sh->abort_flag;
 
+  if (warp == 0 && lane < 6) {
+    // fetch the tensor maps into the descriptor cache while the CTA sets itself up
+    const CUtensorMap* maps[6] = {&map_l, &map_r, &map_la, &map_ra, &map_cl, &map_cr};
+    asm volatile("prefetch.tensormap [%0];" ::"l"(maps[lane]) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
