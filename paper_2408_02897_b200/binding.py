@@ -76,6 +76,9 @@ def lib():
             "qm_probe_layer": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, SZ, P]),
             "qm_operand_span_bytes": (SZ, [OP]),
             "qm_probe_layer_host": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, C.POINTER(MetricResult), P, P, SZ, P]),
+            "qm_probe_batch": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), P, C.POINTER(P), C.POINTER(SZ), P]),
+            "qm_probe_batch_host": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), C.POINTER(P), C.POINTER(P),
+                                          C.POINTER(MetricResult), P, C.POINTER(P), C.POINTER(SZ), P]),
             "qm_status_string": (C.c_char_p, [I32]),
             "qm_version": (I32, []),
             "qm_last_cuda_error": (C.c_char_p, []),
@@ -271,6 +274,91 @@ def qm_probe_layer_host(L_host, R_host, contract_l, contract_r, fmt_l, fmt_r, gr
                                    C.byref(res), _ptr(plan.out), _ptr(plan.ws), plan.ws_bytes, _stream(stream))
     _check(st, "qm_probe_layer_host")
     return res, stage
+
+
+def _copy_operand(op, data_ptr=None):
+    o = Operand()
+    C.memmove(C.byref(o), C.byref(op), C.sizeof(Operand))
+    if data_ptr is not None:
+        o.data = data_ptr
+    return o
+
+
+def _records(raw, n):
+    sz = C.sizeof(MetricResult)
+    return [MetricResult.from_buffer_copy(raw[i * sz:(i + 1) * sz]) for i in range(n)]
+
+
+class ProbeBatch:
+    """Workspaces and result records of a fixed list of probes that are issued together
+    (qm_probe_batch).  `probes` is a list of (L_op, R_op, fmt_l, fmt_r, gran_l, gran_r[, ref])."""
+
+    def __init__(self, probes):
+        n = self.n = len(probes)
+        self._keep = [(p[0], p[1]) for p in probes]
+        self.L = (Operand * n)(*[_copy_operand(p[0]) for p in probes])
+        self.R = (Operand * n)(*[_copy_operand(p[1]) for p in probes])
+        refs = [p[6] if len(p) > 6 else "bf16" for p in probes]
+        self.cfg = (ProbeCfg * n)(*[_cfg(p[2], p[3], p[4], p[5], r) for p, r in zip(probes, refs)])
+        sizes = [qm_workspace_bytes(p[0], p[1], p[2], p[3], p[4], p[5], r) for p, r in zip(probes, refs)]
+        self._ws = [torch.empty(b, dtype=torch.uint8, device="cuda") for b in sizes]
+        self.ws = (C.c_void_p * n)(*[t.data_ptr() for t in self._ws])
+        self.ws_bytes = (C.c_size_t * n)(*sizes)
+        self.out = torch.zeros(n * C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+
+    def launch(self, stream=None):
+        _check(lib().qm_probe_batch(self.n, self.L, self.R, self.cfg, _ptr(self.out), self.ws, self.ws_bytes,
+                                    _stream(stream)), "qm_probe_batch")
+
+    def launch_serial(self, stream=None):
+        """The same probes one after the other on one stream (qm_probe_layer per probe)."""
+        sz = C.sizeof(MetricResult)
+        for i in range(self.n):
+            _check(lib().qm_probe_layer(C.byref(self.L[i]), C.byref(self.R[i]), C.byref(self.cfg[i]),
+                                        C.c_void_p(self.out.data_ptr() + i * sz), self.ws[i], self.ws_bytes[i],
+                                        _stream(stream)), "qm_probe_layer")
+
+    def results(self):
+        return _records(self.out.cpu().numpy().tobytes(), self.n)
+
+
+class HostProbeBatch:
+    """The same for operands in (pinned) host tensors (qm_probe_batch_host): device staging
+    buffers, workspaces and records are made once; run() copies, probes and returns the records.
+    `probes` is a list of (L_host, contract_l, R_host, contract_r, fmt_l, fmt_r, gran_l, gran_r[, ref])."""
+
+    def __init__(self, probes):
+        n = self.n = len(probes)
+        Lh = [operand_of(p[0], p[1]) for p in probes]
+        Rh = [operand_of(p[2], p[3]) for p in probes]
+        self._keep = (Lh, Rh)
+        span = lib().qm_operand_span_bytes
+        self._ls = [torch.empty(span(C.byref(o)), dtype=torch.uint8, device="cuda") for o in Lh]
+        self._rs = [torch.empty(span(C.byref(o)), dtype=torch.uint8, device="cuda") for o in Rh]
+        self.L = (Operand * n)(*[_copy_operand(o) for o in Lh])
+        self.R = (Operand * n)(*[_copy_operand(o) for o in Rh])
+        self.l_stage = (C.c_void_p * n)(*[t.data_ptr() for t in self._ls])
+        self.r_stage = (C.c_void_p * n)(*[t.data_ptr() for t in self._rs])
+        refs = [p[8] if len(p) > 8 else "bf16" for p in probes]
+        self.cfg = (ProbeCfg * n)(*[_cfg(p[4], p[5], p[6], p[7], r) for p, r in zip(probes, refs)])
+        sizes = []
+        for i, (p, r) in enumerate(zip(probes, refs)):
+            Ld, Rd = _copy_operand(Lh[i], self._ls[i].data_ptr()), _copy_operand(Rh[i], self._rs[i].data_ptr())
+            sizes.append(qm_workspace_bytes(Ld, Rd, p[4], p[5], p[6], p[7], r))
+        self._ws = [torch.empty(b, dtype=torch.uint8, device="cuda") for b in sizes]
+        self.ws = (C.c_void_p * n)(*[t.data_ptr() for t in self._ws])
+        self.ws_bytes = (C.c_size_t * n)(*sizes)
+        self.out_dev = torch.zeros(n * C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+        self._out_host = torch.zeros(n * C.sizeof(MetricResult), dtype=torch.uint8).pin_memory()
+        self.h2d_bytes = sum(t.numel() for t in self._ls) + sum(t.numel() for t in self._rs)
+        self.d2h_bytes = n * C.sizeof(MetricResult)
+
+    def run(self, stream=None):
+        out = C.cast(C.c_void_p(self._out_host.data_ptr()), C.POINTER(MetricResult))
+        _check(lib().qm_probe_batch_host(self.n, self.L, self.R, self.cfg, self.l_stage, self.r_stage, out,
+                                         _ptr(self.out_dev), self.ws, self.ws_bytes, _stream(stream)),
+               "qm_probe_batch_host")
+        return _records(self._out_host.numpy().tobytes(), self.n)
 
 
 def kernel_launches():

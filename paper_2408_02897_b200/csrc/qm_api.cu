@@ -313,23 +313,121 @@ size_t qm_operand_span_bytes(const qm_operand* x) {
   return (size_t)(last + 1) * (v.dtype == QM_DT_BF16 ? 2 : 4);
 }
 
-qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host, const qm_probe_cfg* cfg,
-                              void* l_stage, void* r_stage, qm_metric_result* out_host,
-                              qm_metric_result* out_dev, void* ws, size_t ws_bytes, void* stream) {
+// copies in, probe, record out: everything qm_probe_layer_host puts into the stream
+static qm_status enqueue_host_probe(const qm_operand* L_host, const qm_operand* R_host, const qm_probe_cfg* cfg,
+                                    void* l_stage, void* r_stage, qm_metric_result* out_host,
+                                    qm_metric_result* out_dev, void* ws, size_t ws_bytes, cudaStream_t s) {
   if (!L_host || !R_host || !l_stage || !r_stage || !out_host || !out_dev) return QM_ERR_INVALID_ARG;
   const size_t lb = qm_operand_span_bytes(L_host), rb = qm_operand_span_bytes(R_host);
   if (lb == 0 || rb == 0) return QM_ERR_INVALID_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   QM_CUDA_OK(cudaMemcpyAsync(l_stage, L_host->data, lb, cudaMemcpyHostToDevice, s));
   QM_CUDA_OK(cudaMemcpyAsync(r_stage, R_host->data, rb, cudaMemcpyHostToDevice, s));
   qm_operand L = *L_host, R = *R_host;
   L.data = l_stage; R.data = r_stage;
-  qm_status st = qm_probe_layer(&L, &R, cfg, out_dev, ws, ws_bytes, stream);
+  qm_status st = qm_probe_layer(&L, &R, cfg, out_dev, ws, ws_bytes, s);
   if (st != QM_OK) return st;
   QM_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, sizeof(qm_metric_result), cudaMemcpyDeviceToHost, s));
+  return QM_OK;
+}
+
+static qm_status host_record_status(const qm_metric_result* r) {
+  if (r->device_error & QM_DEVERR_TIMEOUT) return QM_ERR_TIMEOUT;
+  if (r->device_error & QM_DEVERR_NONFINITE) return QM_ERR_NONFINITE_INPUT;
+  return QM_OK;
+}
+
+qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host, const qm_probe_cfg* cfg,
+                              void* l_stage, void* r_stage, qm_metric_result* out_host,
+                              qm_metric_result* out_dev, void* ws, size_t ws_bytes, void* stream) {
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  qm_status st = enqueue_host_probe(L_host, R_host, cfg, l_stage, r_stage, out_host, out_dev, ws, ws_bytes, s);
+  if (st != QM_OK) return st;
   QM_CUDA_OK(cudaStreamSynchronize(s));
-  if (out_host->device_error & QM_DEVERR_TIMEOUT) return QM_ERR_TIMEOUT;
-  if (out_host->device_error & QM_DEVERR_NONFINITE) return QM_ERR_NONFINITE_INPUT;
+  return host_record_status(out_host);
+}
+
+}  // extern "C"
+
+// ---- batches of probes over the library's own streams ------------------------------------------
+namespace {
+constexpr int kBatchStreams = 3;
+struct BatchStreams {
+  bool ready = false;
+  cudaStream_t s[kBatchStreams];
+  cudaEvent_t fork, join[kBatchStreams];
+};
+// One set per device, created on first use (never inside a stream capture) and kept.
+qm_status batch_streams(BatchStreams** out) {
+  static BatchStreams pool[64];
+  static std::mutex mu;
+  int dev = 0;
+  QM_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QM_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(mu);
+  BatchStreams& b = pool[dev];
+  if (!b.ready) {
+    for (int i = 0; i < kBatchStreams; ++i) {
+      QM_CUDA_OK(cudaStreamCreateWithFlags(&b.s[i], cudaStreamNonBlocking));
+      QM_CUDA_OK(cudaEventCreateWithFlags(&b.join[i], cudaEventDisableTiming));
+    }
+    QM_CUDA_OK(cudaEventCreateWithFlags(&b.fork, cudaEventDisableTiming));
+    b.ready = true;
+  }
+  *out = &b;
+  return QM_OK;
+}
+
+// Runs issue(i, stream_i) for i < n round-robin over the library's streams, between a fork from
+// and a join back into the caller's stream.  The join happens even when a probe was refused.
+template <typename F>
+qm_status run_batch(int32_t n, cudaStream_t user, F issue) {
+  if (n < 0) return QM_ERR_INVALID_ARG;
+  if (n == 0) return QM_OK;
+  BatchStreams* b = nullptr;
+  qm_status st = batch_streams(&b);
+  if (st != QM_OK) return st;
+  const int used = n < kBatchStreams ? n : kBatchStreams;
+  QM_CUDA_OK(cudaEventRecord(b->fork, user));
+  for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
+  for (int32_t i = 0; i < n && st == QM_OK; ++i) st = issue(i, b->s[i % kBatchStreams]);
+  for (int j = 0; j < used; ++j) {
+    QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
+    QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
+  }
+  return st;
+}
+}  // namespace
+
+extern "C" {
+
+qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,
+                         qm_metric_result* out, void* const* ws, const size_t* ws_bytes, void* stream) {
+  if (n > 0 && (!L || !R || !cfg || !out || !ws || !ws_bytes)) return QM_ERR_INVALID_ARG;
+  return run_batch(n, static_cast<cudaStream_t>(stream), [&](int32_t i, cudaStream_t s) {
+    return qm_probe_layer(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], s);
+  });
+}
+
+qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_operand* R_host,
+                              const qm_probe_cfg* cfg, void* const* l_stage, void* const* r_stage,
+                              qm_metric_result* out_host, qm_metric_result* out_dev, void* const* ws,
+                              const size_t* ws_bytes, void* stream) {
+  if (n > 0 && (!L_host || !R_host || !cfg || !l_stage || !r_stage || !out_host || !out_dev || !ws || !ws_bytes))
+    return QM_ERR_INVALID_ARG;
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  int32_t issued = 0;
+  qm_status st = run_batch(n, user, [&](int32_t i, cudaStream_t s) {
+    qm_status e = enqueue_host_probe(&L_host[i], &R_host[i], &cfg[i], l_stage[i], r_stage[i], out_host + i,
+                                     out_dev + i, ws[i], ws_bytes[i], s);
+    if (e == QM_OK) ++issued;
+    return e;
+  });
+  QM_CUDA_OK(cudaStreamSynchronize(user));
+  if (st != QM_OK) return st;
+  for (int32_t i = 0; i < issued; ++i) {
+    st = host_record_status(out_host + i);
+    if (st != QM_OK) return st;
+  }
   return QM_OK;
 }
 

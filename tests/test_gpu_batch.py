@@ -1,0 +1,88 @@
+"""qm_probe_batch / qm_probe_batch_host: the probes of a measurement pass issued together give
+the records of the same probes issued one by one (same kernels, fixed summation order)."""
+import ctypes as C
+
+import pytest
+import torch
+
+import paper_2408_02897_b200 as qm
+from paper_2408_02897_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+
+def _ops():
+    shapes = [(300, 200, 128, "e4m3", "tensor", "tensor"), (256, 128, 64, "int8", "channel", "tensor"),
+              (130, 264, 256, "e5m2", "tensor", "channel"), (512, 384, 192, "e4m3", "channel", "channel"),
+              (64, 64, 1024, "int8", "tensor", "tensor")]
+    out = []
+    for i, (M, N, K, fmt, gl, gr) in enumerate(shapes):
+        rng = workloads._rng(100 + i)
+        out.append((workloads.normal(rng, (M, K)), workloads.normal(rng, (K, N), 0.05), fmt, gl, gr))
+    return out
+
+
+def _same(a, b):
+    return a.record() == b.record() and a.device_error == b.device_error
+
+
+def test_batch_equals_single_probes():
+    ops = _ops()
+    dev = [(L.cuda(), R.cuda()) for L, R, *_ in ops]
+    single = [qm.qm_probe_layer(qm.operand_of(Ld, -1), qm.operand_of(Rd, -2), f, f, gl, gr)
+              for (Ld, Rd), (_, _, f, gl, gr) in zip(dev, ops)]
+    batch = qm.ProbeBatch([(qm.operand_of(Ld, -1), qm.operand_of(Rd, -2), f, f, gl, gr)
+                           for (Ld, Rd), (_, _, f, gl, gr) in zip(dev, ops)])
+    for _ in range(3):                      # workspaces are reused without clearing by the caller
+        batch.launch()
+        torch.cuda.synchronize()
+        assert all(_same(g, s) for g, s in zip(batch.results(), single))
+    batch.launch_serial()
+    torch.cuda.synchronize()
+    assert all(_same(g, s) for g, s in zip(batch.results(), single))
+
+
+def test_batch_orders_after_and_before_the_callers_stream():
+    L0, R0, f, gl, gr = _ops()[0]
+    Ld, Rd = torch.zeros_like(L0, device="cuda"), R0.cuda()
+    want = qm.qm_probe_layer(qm.operand_of(L0.cuda(), -1), qm.operand_of(Rd, -2), f, f, gl, gr)
+    batch = qm.ProbeBatch([(qm.operand_of(Ld, -1), qm.operand_of(Rd, -2), f, f, gl, gr)] * 4)
+    s = torch.cuda.Stream()
+    src = L0.cuda()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        Ld.copy_(src)                       # the batch must see this write ...
+        batch.launch(stream=s)
+        snapshot = batch.out.clone()        # ... and this read must see the batch's records
+    s.synchronize()
+    sz = C.sizeof(qm.MetricResult)
+    raw = snapshot.cpu().numpy().tobytes()
+    for i in range(4):
+        assert _same(qm.MetricResult.from_buffer_copy(raw[i * sz:(i + 1) * sz]), want)
+
+
+def test_host_batch_equals_single_probes():
+    ops = _ops()
+    single = [qm.qm_probe_layer(qm.operand_of(L.cuda(), -1), qm.operand_of(R.cuda(), -2), f, f, gl, gr)
+              for L, R, f, gl, gr in ops]
+    hb = qm.HostProbeBatch([(L.pin_memory(), -1, R.pin_memory(), -2, f, f, gl, gr) for L, R, f, gl, gr in ops])
+    for _ in range(2):
+        assert all(_same(g, s) for g, s in zip(hb.run(), single))
+    assert hb.h2d_bytes == sum(L.numel() * 2 + R.numel() * 2 for L, R, *_ in ops)
+
+
+def test_empty_and_bad_batches():
+    lib = qm.lib()
+    assert lib.qm_probe_batch(0, None, None, None, None, None, None, None) == 0
+    assert lib.qm_probe_batch(-1, None, None, None, None, None, None, None) != 0
+    assert lib.qm_probe_batch(2, None, None, None, None, None, None, None) != 0
+    # a refused probe in the middle: the ones before it still complete, the call reports the error
+    L0, R0, f, gl, gr = _ops()[0]
+    Ld, Rd = L0.cuda(), R0.cuda()
+    want = qm.qm_probe_layer(qm.operand_of(Ld, -1), qm.operand_of(Rd, -2), f, f, gl, gr)
+    batch = qm.ProbeBatch([(qm.operand_of(Ld, -1), qm.operand_of(Rd, -2), f, f, gl, gr)] * 3)
+    batch.ws_bytes[1] = 16                  # too small
+    with pytest.raises(qm.QmError):
+        batch.launch()
+    torch.cuda.synchronize()
+    assert _same(batch.results()[0], want)
