@@ -95,6 +95,34 @@ typedef struct {
   uint32_t reserved;
 } qm_metric_result;
 
+/* Power sums of all elements of one tensor (Experiments section: "mean, variance,
+ * skew and Kurtosis" of the matmul inputs of the baseline).  With n = count,
+ * mu = sum1/n and the raw moments r_k = sum_k/n:  variance m2 = r2 - mu^2,
+ * m3 = r3 - 3 mu r2 + 2 mu^3,  m4 = r4 - 4 mu r3 + 6 mu^2 r2 - 3 mu^4,
+ * skew = m3 / m2^1.5, kurtosis = m4 / m2^2 (3 for a normal law). */
+typedef struct {
+  double sum1, sum2, sum3, sum4;
+  double max_abs;
+  uint64_t count;
+  uint32_t device_error;   /* QM_DEVERR_NONFINITE when a NaN or Inf was seen                */
+  uint32_t reserved;
+} qm_tensor_stats_result;
+
+/* Eq. 2, RE = |v - v~| / |v|, over the non-zero elements of one tensor under Eq. 1,
+ * split as in the Results section: an element is OVERFLOW when |v/delta| exceeds the
+ * largest expressible magnitude (it is capped), UNDERFLOW when it is not zero but its
+ * code is, ROUNDING otherwise.  err2_* are sums of (v - v~)^2 per class. */
+typedef struct {
+  double sum_re;           /* over all non-zero elements (an underflow contributes 1)     */
+  double sum_re_round;     /* over the rounding class                                     */
+  double max_re_round;
+  double err2_round, err2_overflow, err2_underflow;
+  double sum_x2;
+  uint64_t count, n_nonzero, n_overflow, n_underflow;
+  uint32_t device_error;
+  uint32_t reserved;
+} qm_quant_error_result;
+
 typedef struct {
   int32_t fmt_l, fmt_r;    /* qm_format per operand                                       */
   int32_t gran_l, gran_r;  /* qm_gran per operand                                         */
@@ -200,6 +228,27 @@ qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host
                               const qm_probe_cfg* cfg, void* l_stage, void* r_stage,
                               qm_metric_result* out_host, qm_metric_result* out_dev,
                               void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Single-tensor passes beside the probe, one read of the tensor each.
+ * qm_tensor_stats: the power sums from which mean, variance, skew and kurtosis of
+ * the tensor follow (Experiments section), and max|x|.  Powers are formed in fp32
+ * (|x| up to 2^31 keeps x^4 finite), summed in fp32 over 32 elements and in fp64
+ * from there on.
+ * qm_quantize_error: Eq. 2 and the clipping / rounding split of the Results
+ * section for the codes qm_quantize would produce with these scales.  `delta`
+ * (device) holds finished Eq. 1 scales as written by qm_scale or qm_quantize:
+ * one value (QM_GRAN_TENSOR) or batch * noncontract values (QM_GRAN_CHANNEL).
+ * `out` (device) receives the record.  `ws` is device scratch of at least
+ * qm_stats_workspace_bytes() bytes, 256-byte aligned; its contents on entry do
+ * not matter and concurrent calls must not share it.  The operand needs a unit
+ * stride in one of its two dimensions and fewer than 2^32 groups of 8 elements.
+ */
+size_t qm_stats_workspace_bytes(void);
+qm_status qm_tensor_stats(const qm_operand* x, qm_tensor_stats_result* out, void* ws, size_t ws_bytes,
+                          void* stream);
+qm_status qm_quantize_error(const qm_operand* x, int32_t fmt, int32_t gran, const float* delta,
+                            qm_quant_error_result* out, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * The probes of one measurement pass (the per-layer loop of the Methodology

@@ -47,6 +47,36 @@ class MetricResult(C.Structure):
                 "snr_db": 10.0 * math.log10(sr / sd) if sd > 0 and sr > 0 else float("inf")}
 
 
+class TensorStats(C.Structure):
+    _fields_ = [("sum1", C.c_double), ("sum2", C.c_double), ("sum3", C.c_double), ("sum4", C.c_double),
+                ("max_abs", C.c_double), ("count", C.c_uint64), ("device_error", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+    def derived(self):
+        """mean, variance, skew, kurtosis from the power sums (population moments)."""
+        n = self.count
+        if n == 0:
+            return {"mean": 0.0, "variance": 0.0, "skew": 0.0, "kurtosis": 0.0}
+        mu, r2, r3, r4 = self.sum1 / n, self.sum2 / n, self.sum3 / n, self.sum4 / n
+        m2 = r2 - mu * mu
+        m3 = r3 - 3 * mu * r2 + 2 * mu ** 3
+        m4 = r4 - 4 * mu * r3 + 6 * mu * mu * r2 - 3 * mu ** 4
+        ok = m2 > 0
+        return {"mean": mu, "variance": m2, "skew": m3 / m2 ** 1.5 if ok else 0.0,
+                "kurtosis": m4 / (m2 * m2) if ok else 0.0}
+
+
+class QuantError(C.Structure):
+    _fields_ = [("sum_re", C.c_double), ("sum_re_round", C.c_double), ("max_re_round", C.c_double),
+                ("err2_round", C.c_double), ("err2_overflow", C.c_double), ("err2_underflow", C.c_double),
+                ("sum_x2", C.c_double), ("count", C.c_uint64), ("n_nonzero", C.c_uint64),
+                ("n_overflow", C.c_uint64), ("n_underflow", C.c_uint64), ("device_error", C.c_uint32),
+                ("reserved", C.c_uint32)]
+
+    def record(self):
+        return {k: getattr(self, k) for k, _ in self._fields_ if k not in ("device_error", "reserved")}
+
+
 class ProbeCfg(C.Structure):
     _fields_ = [("fmt_l", C.c_int32), ("fmt_r", C.c_int32), ("gran_l", C.c_int32), ("gran_r", C.c_int32),
                 ("round", C.c_int32), ("ref", C.c_int32)]
@@ -76,6 +106,9 @@ def lib():
             "qm_probe_layer": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, SZ, P]),
             "qm_operand_span_bytes": (SZ, [OP]),
             "qm_probe_layer_host": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, C.POINTER(MetricResult), P, P, SZ, P]),
+            "qm_stats_workspace_bytes": (SZ, []),
+            "qm_tensor_stats": (I32, [OP, P, P, SZ, P]),
+            "qm_quantize_error": (I32, [OP, I32, I32, P, P, P, SZ, P]),
             "qm_probe_batch": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), P, C.POINTER(P), C.POINTER(SZ), P]),
             "qm_probe_batch_host": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), C.POINTER(P), C.POINTER(P),
                                           C.POINTER(MetricResult), P, C.POINTER(P), C.POINTER(SZ), P]),
@@ -213,6 +246,31 @@ def qm_metric_noalloc(ref, q, den, out=None, stream=None):
     _check(lib().qm_metric_noalloc(_ptr(ref), _ptr(q), _ptr(den), ref.numel(), _ptr(out), _stream(stream)),
            "qm_metric_noalloc")
     return _read_result(out)
+
+
+def _stats_ws():
+    n = lib().qm_stats_workspace_bytes()
+    return torch.empty(n, dtype=torch.uint8, device="cuda"), n
+
+
+def qm_tensor_stats(op, ws=None, stream=None):
+    """Power sums and max|x| of a tensor -> TensorStats (synchronises to read the record)."""
+    ws, n = (ws, ws.numel()) if ws is not None else _stats_ws()
+    out = torch.empty(C.sizeof(TensorStats), dtype=torch.uint8, device="cuda")
+    _check(lib().qm_tensor_stats(C.byref(op), _ptr(out), _ptr(ws), n, _stream(stream)), "qm_tensor_stats")
+    return TensorStats.from_buffer_copy(out.cpu().numpy().tobytes())
+
+
+def qm_quantize_error(op, fmt, gran, delta=None, ws=None, stream=None):
+    """Eq. 2 sums and the clipping / rounding split of an operand -> QuantError.  delta=None
+    takes the Eq. 1 scales of the operand itself (qm_scale)."""
+    if delta is None:
+        delta = qm_scale(op, fmt, gran, stream)
+    ws, n = (ws, ws.numel()) if ws is not None else _stats_ws()
+    out = torch.empty(C.sizeof(QuantError), dtype=torch.uint8, device="cuda")
+    _check(lib().qm_quantize_error(C.byref(op), FMT[fmt], GRAN[gran], _ptr(delta), _ptr(out), _ptr(ws), n,
+                                   _stream(stream)), "qm_quantize_error")
+    return QuantError.from_buffer_copy(out.cpu().numpy().tobytes())
 
 
 def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref):

@@ -313,6 +313,30 @@ size_t qm_operand_span_bytes(const qm_operand* x) {
   return (size_t)(last + 1) * (v.dtype == QM_DT_BF16 ? 2 : 4);
 }
 
+size_t qm_stats_workspace_bytes(void) { return stats_workspace_bytes(); }
+
+qm_status qm_tensor_stats(const qm_operand* x, qm_tensor_stats_result* out, void* ws, size_t ws_bytes,
+                          void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (!out || !ws) return QM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255) return QM_ERR_ALIGNMENT;
+  if (ws_bytes < stats_workspace_bytes()) return QM_ERR_WORKSPACE_TOO_SMALL;
+  return launch_tensor_stats(v, out, ws, static_cast<cudaStream_t>(stream));
+}
+
+qm_status qm_quantize_error(const qm_operand* x, int32_t fmt, int32_t gran, const float* delta,
+                            qm_quant_error_result* out, void* ws, size_t ws_bytes, void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (!valid_fmt(fmt) || !valid_gran(gran) || !delta || !out || !ws) return QM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255) return QM_ERR_ALIGNMENT;
+  if (ws_bytes < stats_workspace_bytes()) return QM_ERR_WORKSPACE_TOO_SMALL;
+  return launch_quantize_error(v, fmt, gran, delta, out, ws, static_cast<cudaStream_t>(stream));
+}
+
 // copies in, probe, record out: everything qm_probe_layer_host puts into the stream
 static qm_status enqueue_host_probe(const qm_operand* L_host, const qm_operand* R_host, const qm_probe_cfg* cfg,
                                     void* l_stage, void* r_stage, qm_metric_result* out_host,

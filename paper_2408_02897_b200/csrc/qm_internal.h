@@ -81,6 +81,13 @@ qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, 
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
                                      void* abs_copy, uint32_t* err_word, cudaStream_t s);
 
+// ---- single-tensor passes (tensor_stats.cu) --------------------------------
+size_t stats_workspace_bytes();
+qm_status launch_tensor_stats(const View& x, qm_tensor_stats_result* out, void* ws, cudaStream_t s);
+// delta: finished Eq. 1 scales (1 value, or one per batch element and non-contracting index)
+qm_status launch_quantize_error(const View& x, int fmt, int gran, const float* delta,
+                                qm_quant_error_result* out, void* ws, cudaStream_t s);
+
 // ---- metric (metric.cu) ----------------------------------------------------
 // One partial record per CTA: {sum_be, max_be, sum_diff2, sum_ref2, sum_den2} as doubles.
 constexpr int kPartialDoubles = 5;

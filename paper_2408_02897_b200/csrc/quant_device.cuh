@@ -1,0 +1,172 @@
+// Device helpers shared by the streaming kernels (scale, quantize, tensor statistics, Eq. 2
+// error split): element loads, the exact quotient of Eq. 1, the 8-bit conversions, small
+// reductions.  Included by .cu files only; everything sits in the including file's anonymous
+// namespace.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "qm_internal.h"
+
+namespace qm {
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------- element helpers
+// |x| as an order-preserving unsigned integer: for IEEE formats the bit pattern with the sign
+// cleared orders like the magnitude, and Inf / NaN patterns sort above every finite value, so
+// an integer max also carries "non-finite seen" to the end.  bf16 patterns are widened to the
+// fp32 pattern (shift by 16) so one code path serves both input types.
+__device__ __forceinline__ uint32_t absbits_f32(uint32_t w) { return w & 0x7fffffffu; }
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Two quantized bytes from t = x / delta: t0 in bits 0..7, t1 in bits 8..15.
+// RTNE, saturating at the largest finite magnitude.
+template <int FMT>
+__device__ __forceinline__ uint32_t quant2(float t0, float t1) {
+  if (FMT == QM_FMT_INT8) {
+    int a = __float2int_rn(t0), b = __float2int_rn(t1);      // round to nearest even
+    a = max(-127, min(127, a));
+    b = max(-127, min(127, b));
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8);
+  } else {
+    uint16_t r;
+    if (FMT == QM_FMT_E4M3)
+      asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(t1), "f"(t0));
+    else
+      asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(t1), "f"(t0));
+    return r;
+  }
+}
+
+// 8 consecutive elements held as fp32.
+struct Vec8 { float v[8]; };
+
+template <typename T> struct Loader;
+template <> struct Loader<__nv_bfloat16> {
+  static __device__ __forceinline__ Vec8 load8(const void* p) {
+    uint4 w = __ldg(reinterpret_cast<const uint4*>(p));
+    Vec8 r;
+    r.v[0] = bf16_lo(w.x); r.v[1] = bf16_hi(w.x); r.v[2] = bf16_lo(w.y); r.v[3] = bf16_hi(w.y);
+    r.v[4] = bf16_lo(w.z); r.v[5] = bf16_hi(w.z); r.v[6] = bf16_lo(w.w); r.v[7] = bf16_hi(w.w);
+    return r;
+  }
+  static __device__ __forceinline__ float load1(const void* p, int64_t i) {
+    return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p) + i) << 16);
+  }
+};
+template <> struct Loader<float> {
+  static __device__ __forceinline__ Vec8 load8(const void* p) {
+    float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    Vec8 r;
+    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w;
+    r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+    return r;
+  }
+  static __device__ __forceinline__ float load1(const void* p, int64_t i) {
+    return __ldg(reinterpret_cast<const float*>(p) + i);
+  }
+};
+
+__device__ __forceinline__ uint32_t absmax8(const Vec8& x, uint32_t acc) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc = max(acc, absbits_f32(__float_as_uint(x.v[i])));
+  return acc;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);   // round to nearest even
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// x / delta, correctly rounded (the IEEE quotient Eq. 1 asks for), for many x under one delta.
+// With r = RN(1/delta) computed once per scaling group, a product and two residual corrections
+//   q0 = x r;  q1 = q0 + (x - q0 delta) r;  q = q1 + (x - q1 delta) r      (residuals exact by FMA)
+// give RN(x / delta): q1 is within one ulp of the quotient, and one more correction of a
+// faithful quotient with the correctly rounded reciprocal rounds correctly (Markstein's
+// theorem).  This needs the intermediate values inside the normal range, so it is used only for
+// 2^-60 <= delta <= 2^60, where any |x| small enough to leave that range quantizes to zero in
+// every format; other deltas take the division instruction sequence.
+struct Quotient {
+  float delta, recip;
+  bool fast;
+  __device__ __forceinline__ explicit Quotient(float d) : delta(d) {
+    fast = d >= 8.6736174e-19f && d <= 1.1529215e18f;        // 2^-60 .. 2^60
+    recip = fast ? __frcp_rn(d) : 0.f;
+  }
+  __device__ __forceinline__ float operator()(float x) const {
+    if (!fast) return __fdiv_rn(x, delta);
+    const float q0 = x * recip;
+    const float q1 = fmaf(fmaf(-q0, delta, x), recip, q0);
+    const float q = fmaf(fmaf(-q1, delta, x), recip, q1);
+    return copysignf(q, x);                                   // keeps the sign of a zero input
+  }
+};
+
+template <int FMT>
+__device__ __forceinline__ uint2 quant8(const Vec8& x, const Quotient& quot) {
+  float t[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) t[i] = quot(x.v[i]);
+  uint2 r;
+  r.x = quant2<FMT>(t[0], t[1]) | (quant2<FMT>(t[2], t[3]) << 16);
+  r.y = quant2<FMT>(t[4], t[5]) | (quant2<FMT>(t[6], t[7]) << 16);
+  return r;
+}
+
+__device__ __forceinline__ uint4 abs_bf16x8(const Vec8& x) {
+  uint4 r;
+  r.x = pack_bf16x2(fabsf(x.v[0]), fabsf(x.v[1]));
+  r.y = pack_bf16x2(fabsf(x.v[2]), fabsf(x.v[3]));
+  r.z = pack_bf16x2(fabsf(x.v[4]), fabsf(x.v[5]));
+  r.w = pack_bf16x2(fabsf(x.v[6]), fabsf(x.v[7]));
+  return r;
+}
+__device__ __forceinline__ uint4 to_bf16x8(const Vec8& x) {
+  uint4 r;
+  r.x = pack_bf16x2(x.v[0], x.v[1]); r.y = pack_bf16x2(x.v[2], x.v[3]);
+  r.z = pack_bf16x2(x.v[4], x.v[5]); r.w = pack_bf16x2(x.v[6], x.v[7]);
+  return r;
+}
+
+__device__ __forceinline__ uint32_t warp_max(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+__device__ __forceinline__ uint32_t block_max(uint32_t v) {
+  __shared__ uint32_t s[32];
+  v = warp_max(v);
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) s[w] = v;
+  __syncthreads();
+  if (w == 0) {
+    v = lane < (int)(blockDim.x >> 5) ? s[lane] : 0u;
+    v = warp_max(v);
+  }
+  return v;   // valid in warp 0
+}
+
+// Division of a 32-bit index by a launch-time constant without a divide instruction
+// (multiply-high and shift; the magic numbers come from the host).
+struct FastDiv {
+  uint32_t d, m, s;
+  __host__ explicit FastDiv(uint32_t div = 1) : d(div), m(0), s(0) {
+    if (d > 1) {
+      while ((1ull << s) < d) ++s;                          // s = ceil(log2 d)
+      m = (uint32_t)((((1ull << s) - d) << 32) / d + 1);
+    }
+  }
+  __device__ __forceinline__ uint32_t div(uint32_t n) const {
+    if (d == 1) return n;
+    const uint32_t t = __umulhi(m, n);
+    return (t + ((n - t) >> 1)) >> (s - 1);
+  }
+};
+
+}  // namespace
+}  // namespace qm
