@@ -23,8 +23,15 @@ def tensor(shape, dtype, seed, scale=1.0, dist="t"):
     return torch.from_numpy(x.astype(np.float32)).to(dtype)
 
 
+def to_dev(t):
+    """The tensor on the GPU with the strides it has on the CPU (a view of its base tensor)."""
+    if t.is_contiguous():
+        return t.cuda()
+    return torch.as_strided(t._base.cuda(), t.shape, t.stride(), t.storage_offset())
+
+
 def check_stats(t, contract_dim=-1):
-    got = qm.qm_tensor_stats(qm.operand_of(t.cuda(), contract_dim))
+    got = qm.qm_tensor_stats(qm.operand_of(to_dev(t), contract_dim))
     x = t.float().numpy().astype(np.float64)
     want = oracle.tensor_stats(t.float().numpy())
     assert got.device_error == 0
@@ -80,7 +87,7 @@ def test_stats_zero_constant_and_nonfinite():
 
 
 def check_error(t, contract_dim, fmt, gran, delta=None):
-    td = t.cuda()
+    td = to_dev(t)
     op = qm.operand_of(td, contract_dim)
     x = as3(oriented(t, contract_dim))
     if delta is None:
@@ -106,7 +113,8 @@ def test_error_contiguous(fmt, gran, dtype):
     t = tensor((96, 200), dtype, 21) * torch.from_numpy(10.0 ** rng.uniform(-3, 1, (96, 1)).astype(np.float32)).to(dtype)
     t[5] = 0
     got, want = check_error(t, -1, fmt, gran)
-    assert want["n_underflow"] > 0 or fmt == "e5m2"
+    if fmt == "int8" and gran == "tensor":
+        assert want["n_underflow"] > 0              # the case does exercise the underflow class
 
 
 @pytest.mark.parametrize("fmt", FMTS)
