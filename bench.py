@@ -175,12 +175,32 @@ def scale_quantize_rates(qm, hbm_gbs, rows=16384, cols=4096, iters=10):
     t_quant = timed(lambda: raw_quant(op_rows, 0, delta, None, codes))
     t_fused = timed(lambda: raw_quant(op_rows, 1, None, dch, codes))
     t_trans = timed(lambda: raw_quant(op_cols, 0, delta, None, codes_t))
+    ws_n = L.qm_stats_workspace_bytes()
+    ws = torch.empty(ws_n, dtype=torch.uint8, device="cuda")
+    rec = torch.empty(128, dtype=torch.uint8, device="cuda")
+
+    def raw_stats():
+        rc = L.qm_tensor_stats(C.byref(op_rows), C.c_void_p(rec.data_ptr()), C.c_void_p(ws.data_ptr()), ws_n, st)
+        assert rc == 0, rc
+
+    def raw_error(gran, dl):
+        rc = L.qm_quantize_error(C.byref(op_rows), 1, gran, C.c_void_p(dl.data_ptr()), C.c_void_p(rec.data_ptr()),
+                                 C.c_void_p(ws.data_ptr()), ws_n, st)
+        assert rc == 0, rc
+
+    t_stats = timed(raw_stats)
+    t_err = timed(lambda: raw_error(0, delta))
+    t_err_ch = timed(lambda: raw_error(1, dch))
     out = {"tensor": f"bf16 [{rows} x {cols}] ({n * 2 / 1e6:.0f} MB)", "hbm_peak_gbs": hbm_gbs,
            "scale_tensor_gbs": 2 * n / t_scale / 1e9,                 # 2 B/elem read
            "quantize_gbs": 3 * n / t_quant / 1e9,                     # 2 B read + 1 B code
            "scale_quantize_rows_gbs": 3 * n / t_fused / 1e9,          # fused per-row scale + codes, input read once
-           "quantize_transpose_gbs": 3 * n / t_trans / 1e9}
-    for k in ("scale_tensor", "quantize", "scale_quantize_rows", "quantize_transpose"):
+           "quantize_transpose_gbs": 3 * n / t_trans / 1e9,
+           "tensor_stats_gbs": 2 * n / t_stats / 1e9,                  # 2 B/elem read, power sums + max
+           "quantize_error_gbs": 2 * n / t_err / 1e9,                  # 2 B/elem read, Eq. 2 split, one scale
+           "quantize_error_rows_gbs": 2 * n / t_err_ch / 1e9}         # one scale per row
+    for k in ("scale_tensor", "quantize", "scale_quantize_rows", "quantize_transpose", "tensor_stats",
+              "quantize_error", "quantize_error_rows"):
         out[k + "_frac_of_hbm"] = out[k + "_gbs"] / hbm_gbs
     return out
 

@@ -52,6 +52,86 @@ struct Acc {
 // which entries of a record combine by max instead of sum
 template <int KIND> __device__ __forceinline__ bool is_max(int i) { return KIND == kStats ? i == 4 : i == 9; }
 
+// Per-thread sums of one batch of up to four groups of 8 elements: fp32 inside the batch.
+template <int KIND, int FMT>
+struct Batch {
+  float f[7];
+  uint32_t n[3];
+  uint32_t mx;
+  __device__ __forceinline__ Batch() : mx(0) {
+#pragma unroll
+    for (int i = 0; i < 7; ++i) f[i] = 0.f;
+    n[0] = n[1] = n[2] = 0;
+  }
+  // statistics: f = {sum x, sum x^2, sum x^3, sum x^4}; padded entries are zero and add nothing.
+  // Two elements per instruction (packed fp32 pairs): p[k] holds the even-lane and odd-lane halves
+  // of the k-th power sum, folded into f by fold_stats().
+  uint64_t p2[4] = {0ull, 0ull, 0ull, 0ull};
+  __device__ __forceinline__ void stats(const Vec8& v) {
+    mx = absmax8(v, mx);
+#pragma unroll
+    for (int e = 0; e < 8; e += 2) {
+      uint64_t x, x2;
+      asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "f"(v.v[e]), "f"(v.v[e + 1]));
+      asm("mul.rn.f32x2 %0, %1, %1;" : "=l"(x2) : "l"(x));
+      asm("add.rn.f32x2 %0, %0, %1;" : "+l"(p2[0]) : "l"(x));
+      asm("add.rn.f32x2 %0, %0, %1;" : "+l"(p2[1]) : "l"(x2));
+      asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(p2[2]) : "l"(x2), "l"(x));
+      asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(p2[3]) : "l"(x2));
+    }
+  }
+  __device__ __forceinline__ void fold_stats() {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float a, b;
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(p2[k]));
+      f[k] = a + b;
+    }
+  }
+  // Eq. 2 split: f = {sum RE, sum RE rounding, err2 rounding, err2 overflow, err2 underflow,
+  // sum x^2, max RE rounding}; n = {non-zero, overflow, underflow}.  Branch-free per element.
+  __device__ __forceinline__ void error2(float xa, float xb, float ta, float tb, float da, float db) {
+    float ga, gb;
+    decode2<FMT>(quant2<FMT>(ta, tb), ga, gb);
+    const float qmaxv = fmt_qmax(FMT);
+    const float xs[2] = {xa, xb}, ts[2] = {ta, tb}, gs[2] = {ga, gb}, ds[2] = {da, db};
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const float x = xs[h];
+      const bool nz = x != 0.f;
+      const float err = fabsf(fmaf(-gs[h], ds[h], x));        // |x - value(code) delta|, one rounding
+      float rcp;
+      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fabsf(x)));
+      const float re = nz ? err * rcp : 0.f;
+      const float e2 = err * err;
+      const bool over = fabsf(ts[h]) > qmaxv;
+      const bool under = nz && !over && gs[h] == 0.f;
+      const bool rnd = nz && !over && !under;
+      n[0] += nz; n[1] += over; n[2] += under;
+      f[0] += re;
+      f[5] = fmaf(x, x, f[5]);
+      f[3] += over ? e2 : 0.f;
+      f[4] += under ? e2 : 0.f;
+      f[2] += rnd ? e2 : 0.f;
+      const float rr = rnd ? re : 0.f;
+      f[1] += rr;
+      f[6] = fmaxf(f[6], rr);
+    }
+  }
+  __device__ __forceinline__ void flush(Acc& acc) {
+    if (KIND == kStats) {
+      fold_stats();
+      acc.d[0] += (double)f[0]; acc.d[1] += (double)f[1]; acc.d[2] += (double)f[2]; acc.d[3] += (double)f[3];
+      acc.d[4] = fmax(acc.d[4], (double)mx);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 6; ++i) acc.d[i] += (double)f[i];
+      acc.d[6] += (double)n[0]; acc.d[7] += (double)n[1]; acc.d[8] += (double)n[2];
+      acc.d[9] = fmax(acc.d[9], (double)f[6]);
+    }
+  }
+};
+
 template <typename T, int KIND, int FMT>
 __global__ void __launch_bounds__(kThreads)
 tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __restrict__ counter,
@@ -60,97 +140,71 @@ tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __res
   Acc acc;
 #pragma unroll
   for (int i = 0; i < kRec; ++i) acc.d[i] = 0.0;
-  const float qmaxv = fmt_qmax(FMT);
   const uint32_t stride = gridDim.x * kThreads;
-  for (uint32_t g0 = blockIdx.x * kThreads + threadIdx.x; g0 < p.total_groups; g0 += 4 * stride) {
-    Vec8 v[4];
-    float dl[4][8];
-    int live[4];
+  const bool whole_groups = (p.inner & 7) == 0;               // no ragged tail anywhere
+  const bool flat = p.outer == 1 && p.groups_per_line == p.total_groups;
+
+  // where group g starts, and which deltas it takes
+  auto locate = [&](uint32_t g, uint32_t& b, uint32_t& o, uint32_t& j) -> int64_t {
+    if (flat) { b = 0; o = 0; j = g; return (int64_t)g * 8; }
+    const uint32_t line = p.by_gpl.div(g);
+    j = g - line * p.groups_per_line;
+    b = p.by_outer.div(line);
+    o = line - b * p.outer;
+    return (int64_t)b * p.batch_stride + (int64_t)o * p.line_stride + (int64_t)j * 8;
+  };
+  auto process = [&](Batch<KIND, FMT>& bt, const Vec8& v, uint32_t b, uint32_t o, uint32_t j, int live) {
+    if (KIND == kStats) { bt.stats(v); return; }
+    if (p.delta_mode != 2) {
+      const float d = p.delta_mode == 0 ? __ldg(p.delta) : __ldg(p.delta + (int64_t)b * p.delta_batch + o);
+      const Quotient q(d);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t g = g0 + u * stride;
-      live[u] = 0;
-      if (g < p.total_groups) {
-        const uint32_t line = p.by_gpl.div(g), j = g - line * p.groups_per_line;
-        const uint32_t b = p.by_outer.div(line), o = line - b * p.outer;
-        const int64_t off = (int64_t)b * p.batch_stride + (int64_t)o * p.line_stride + (int64_t)j * 8;
+      for (int e = 0; e < 8; e += 2) bt.error2(v.v[e], v.v[e + 1], q(v.v[e]), q(v.v[e + 1]), d, d);
+    } else {
+      const float* dp = p.delta + (int64_t)b * p.delta_batch + (int64_t)j * 8;
+      float d[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) d[e] = e < live ? __ldg(dp + e) : 1.f;
+#pragma unroll
+      for (int e = 0; e < 8; e += 2)
+        bt.error2(v.v[e], v.v[e + 1], Quotient(d[e])(v.v[e]), Quotient(d[e + 1])(v.v[e + 1]), d[e], d[e + 1]);
+    }
+  };
+
+  for (uint32_t g0 = blockIdx.x * kThreads + threadIdx.x; g0 < p.total_groups; g0 += 4 * stride) {
+    Batch<KIND, FMT> bt;
+    const bool full = whole_groups && (uint64_t)g0 + 3ull * stride < p.total_groups;
+    if (full) {
+      // all four loads are issued before any arithmetic
+      Vec8 v[4];
+      uint32_t b[4], o[4], j[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int64_t off = locate(g0 + u * stride, b[u], o[u], j[u]);
+        v[u] = Loader<T>::load8(reinterpret_cast<const char*>(p.x) + off * (int64_t)sizeof(T));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) process(bt, v[u], b[u], o[u], j[u], 8);
+    } else {
+      for (int u = 0; u < 4; ++u) {
+        const uint64_t g = (uint64_t)g0 + (uint64_t)u * stride;
+        if (g >= p.total_groups) break;
+        uint32_t b, o, j;
+        const int64_t off = locate((uint32_t)g, b, o, j);
         const int64_t left = p.inner - (int64_t)j * 8;
-        live[u] = left < 8 ? (int)left : 8;
+        const int live = left < 8 ? (int)left : 8;
         const char* base = reinterpret_cast<const char*>(p.x) + off * (int64_t)sizeof(T);
-        if (live[u] == 8) {
-          v[u] = Loader<T>::load8(base);
+        Vec8 v;
+        if (live == 8) {
+          v = Loader<T>::load8(base);
         } else {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) v[u].v[e] = e < live[u] ? Loader<T>::load1(base, e) : 0.f;
+          for (int e = 0; e < 8; ++e) v.v[e] = e < live ? Loader<T>::load1(base, e) : 0.f;
         }
-        if (KIND == kError) {
-          if (p.delta_mode == 2) {
-            const float* d = p.delta + (int64_t)b * p.delta_batch + (int64_t)j * 8;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) dl[u][e] = e < live[u] ? __ldg(d + e) : 1.f;
-          } else {
-            const float d = p.delta_mode == 0 ? __ldg(p.delta) : __ldg(p.delta + (int64_t)b * p.delta_batch + o);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) dl[u][e] = d;
-          }
-        }
+        process(bt, v, b, o, j, live);
       }
     }
-    if (KIND == kStats) {
-      float s1 = 0.f, s2 = 0.f, s3 = 0.f, s4 = 0.f;
-      uint32_t mx = 0;
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (live[u] == 0) continue;
-        mx = absmax8(v[u], mx);          // padded entries are zero and change nothing
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float x = v[u].v[e], x2 = x * x;
-          s1 += x; s2 += x2; s3 = fmaf(x2, x, s3); s4 = fmaf(x2, x2, s4);
-        }
-      }
-      acc.d[0] += (double)s1; acc.d[1] += (double)s2; acc.d[2] += (double)s3; acc.d[3] += (double)s4;
-      acc.d[4] = fmax(acc.d[4], (double)mx);
-    } else {
-      float sre = 0.f, srr = 0.f, e2r = 0.f, e2o = 0.f, e2u = 0.f, sx2 = 0.f, mrr = 0.f;
-      uint32_t nnz = 0, nov = 0, nun = 0;
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (live[u] == 0) continue;
-        const bool one_delta = p.delta_mode != 2;
-        const Quotient q0(dl[u][0]);
-#pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-          const float xa = v[u].v[e], xb = v[u].v[e + 1];
-          const float da = dl[u][e], db = dl[u][e + 1];
-          float ta, tb;
-          if (one_delta) { ta = q0(xa); tb = q0(xb); }
-          else { ta = Quotient(da)(xa); tb = Quotient(db)(xb); }
-          float ga, gb;
-          decode2<FMT>(quant2<FMT>(ta, tb), ga, gb);
-          const float xs[2] = {xa, xb}, ts[2] = {ta, tb}, gs[2] = {ga, gb}, ds[2] = {da, db};
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            const float x = xs[h];
-            if (x != 0.f) {                                   // padded entries are zero
-              const float err = fabsf(fmaf(-gs[h], ds[h], x));  // |x - value(code) delta|, one rounding
-              const float re = __fdividef(err, fabsf(x));
-              const bool over = fabsf(ts[h]) > qmaxv;
-              const bool under = !over && gs[h] == 0.f;
-              ++nnz;
-              sre += re;
-              sx2 = fmaf(x, x, sx2);
-              if (over) { ++nov; e2o = fmaf(err, err, e2o); }
-              else if (under) { ++nun; e2u = fmaf(err, err, e2u); }
-              else { srr += re; e2r = fmaf(err, err, e2r); mrr = fmaxf(mrr, re); }
-            }
-          }
-        }
-      }
-      acc.d[0] += (double)sre; acc.d[1] += (double)srr; acc.d[2] += (double)e2r; acc.d[3] += (double)e2o;
-      acc.d[4] += (double)e2u; acc.d[5] += (double)sx2; acc.d[6] += (double)nnz; acc.d[7] += (double)nov;
-      acc.d[8] += (double)nun; acc.d[9] = fmax(acc.d[9], (double)mrr);
-    }
+    bt.flush(acc);
   }
 
   // block record
@@ -245,19 +299,27 @@ qm_status make_lines(const View& x, bool channel_delta, const float* delta, Line
   return QM_OK;
 }
 
-int pass_blocks(const Lines& p) {
+// One wave of resident blocks (or fewer when the tensor is small).
+int pass_blocks(const Lines& p, int resident_per_sm) {
   const int64_t want = ((int64_t)p.total_groups + 4 * kThreads - 1) / (4 * kThreads);
-  const int64_t cap = (int64_t)sm_count() * 8 < kMaxBlocks ? (int64_t)sm_count() * 8 : kMaxBlocks;
+  int64_t cap = (int64_t)sm_count() * resident_per_sm;
+  if (cap > kMaxBlocks) cap = kMaxBlocks;
   return (int)(want < 1 ? 1 : (want > cap ? cap : want));
 }
 
 template <typename T, int KIND, int FMT>
 qm_status launch_pass(const Lines& p, void* result, uint64_t count, void* ws, cudaStream_t s) {
+  static int resident = 0;                       // per instantiation; the same on every device
+  if (resident == 0) {
+    int nb = 0;
+    QM_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, tensor_pass_kernel<T, KIND, FMT>, kThreads, 0));
+    resident = nb > 0 ? nb : 1;
+  }
   uint32_t* counter = static_cast<uint32_t*>(ws);
   double* partials = reinterpret_cast<double*>(static_cast<char*>(ws) + kCounterBytes);
   QM_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), s));
-  QM_CUDA_OK(launch_pdl(tensor_pass_kernel<T, KIND, FMT>, dim3(pass_blocks(p)), dim3(kThreads), 0, s, p, partials,
-                        counter, result, count));
+  QM_CUDA_OK(launch_pdl(tensor_pass_kernel<T, KIND, FMT>, dim3(pass_blocks(p, resident)), dim3(kThreads), 0, s, p,
+                        partials, counter, result, count));
   count_launch();
   return QM_OK;
 }
