@@ -133,7 +133,7 @@ struct Batch {
 };
 
 template <typename T, int KIND, int FMT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, KIND == kError ? 3 : 1)
 tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __restrict__ counter,
                    void* __restrict__ result, uint64_t count) {
   pdl_prologue();
@@ -171,22 +171,25 @@ tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __res
     }
   };
 
-  for (uint32_t g0 = blockIdx.x * kThreads + threadIdx.x; g0 < p.total_groups; g0 += 4 * stride) {
+  // loads in flight per thread: four for the bandwidth-bound statistics, two for the
+  // arithmetic-bound error split (fewer registers, more resident warps)
+  constexpr int U = KIND == kError ? 2 : 4;
+  for (uint32_t g0 = blockIdx.x * kThreads + threadIdx.x; g0 < p.total_groups; g0 += U * stride) {
     Batch<KIND, FMT> bt;
-    const bool full = whole_groups && (uint64_t)g0 + 3ull * stride < p.total_groups;
+    const bool full = whole_groups && (uint64_t)g0 + (uint64_t)(U - 1) * stride < p.total_groups;
     if (full) {
-      // all four loads are issued before any arithmetic
-      Vec8 v[4];
-      uint32_t b[4], o[4], j[4];
+      // all loads of the batch are issued before any arithmetic
+      Vec8 v[U];
+      uint32_t b[U], o[U], j[U];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < U; ++u) {
         const int64_t off = locate(g0 + u * stride, b[u], o[u], j[u]);
         v[u] = Loader<T>::load8(reinterpret_cast<const char*>(p.x) + off * (int64_t)sizeof(T));
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) process(bt, v[u], b[u], o[u], j[u], 8);
+      for (int u = 0; u < U; ++u) process(bt, v[u], b[u], o[u], j[u], 8);
     } else {
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < U; ++u) {
         const uint64_t g = (uint64_t)g0 + (uint64_t)u * stride;
         if (g >= p.total_groups) break;
         uint32_t b, o, j;
@@ -301,7 +304,7 @@ qm_status make_lines(const View& x, bool channel_delta, const float* delta, Line
 
 // One wave of resident blocks (or fewer when the tensor is small).
 int pass_blocks(const Lines& p, int resident_per_sm) {
-  const int64_t want = ((int64_t)p.total_groups + 4 * kThreads - 1) / (4 * kThreads);
+  const int64_t want = ((int64_t)p.total_groups + 2 * kThreads - 1) / (2 * kThreads);
   int64_t cap = (int64_t)sm_count() * resident_per_sm;
   if (cap > kMaxBlocks) cap = kMaxBlocks;
   return (int)(want < 1 ? 1 : (want > cap ? cap : want));
