@@ -68,9 +68,10 @@ struct Batch {
   // of the k-th power sum, folded into f by fold_stats().
   uint64_t p2[4] = {0ull, 0ull, 0ull, 0ull};
   __device__ __forceinline__ void stats(const Vec8& v) {
-    mx = absmax8(v, mx);
 #pragma unroll
     for (int e = 0; e < 8; e += 2) {
+      // max |x| as a three-input fp32 max (a NaN input shows up in the sums instead)
+      asm("max.f32 %0, %0, %1, %2;" : "+f"(f[4]) : "f"(fabsf(v.v[e])), "f"(fabsf(v.v[e + 1])));
       uint64_t x, x2;
       asm("mov.b64 %0, {%1, %2};" : "=l"(x) : "f"(v.v[e]), "f"(v.v[e + 1]));
       asm("mul.rn.f32x2 %0, %1, %1;" : "=l"(x2) : "l"(x));
@@ -122,7 +123,7 @@ struct Batch {
     if (KIND == kStats) {
       fold_stats();
       acc.d[0] += (double)f[0]; acc.d[1] += (double)f[1]; acc.d[2] += (double)f[2]; acc.d[3] += (double)f[3];
-      acc.d[4] = fmax(acc.d[4], (double)mx);
+      acc.d[4] = fmax(acc.d[4], (double)f[4]);
     } else {
 #pragma unroll
       for (int i = 0; i < 6; ++i) acc.d[i] += (double)f[i];
@@ -260,11 +261,11 @@ tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __res
   if (lane != 0) return;
   if (KIND == kStats) {
     qm_tensor_stats_result* r = static_cast<qm_tensor_stats_result*>(result);
-    const uint32_t mx = (uint32_t)tot[4];
     r->sum1 = tot[0]; r->sum2 = tot[1]; r->sum3 = tot[2]; r->sum4 = tot[3];
-    r->max_abs = (double)__uint_as_float(mx);
+    r->max_abs = tot[4];
     r->count = count;
-    r->device_error = mx >= 0x7f800000u ? QM_DEVERR_NONFINITE : 0u;
+    // a NaN or Inf element (or a power that left the fp32 range) makes sum x^4 NaN or Inf
+    r->device_error = (tot[3] != tot[3] || tot[3] > 1.7e308 || tot[4] > 3.5e38) ? QM_DEVERR_NONFINITE : 0u;
     r->reserved = 0;
   } else {
     qm_quant_error_result* r = static_cast<qm_quant_error_result*>(result);

@@ -20,7 +20,7 @@ def main():
     ap.add_argument("--fmt", default="e4m3")
     ap.add_argument("--gran", default="tensor")
     ap.add_argument("--iters", type=int, default=3)
-    ap.add_argument("--stage", default="probe", choices=["probe", "quantize"])
+    ap.add_argument("--stage", default="probe", choices=["probe", "quantize", "stats"])
     ap.add_argument("--r-layout", default="kn", choices=["kn", "nk"], help="R stored [K,N] or [N,K]")
     a = ap.parse_args()
     rng = workloads._rng(11)
@@ -36,6 +36,12 @@ def main():
         torch.cuda.synchronize()
         r = plan.result()
         print("mean_be", r.derived()["mean_be"], "device_error", r.device_error)
+    elif a.stage == "stats":
+        # the single-tensor passes on the left operand
+        for _ in range(a.iters):
+            st = qm.qm_tensor_stats(Lop)
+            er = qm.qm_quantize_error(Lop, a.fmt, a.gran)
+        print("kurtosis", st.derived()["kurtosis"], "mean RE", er.sum_re / max(er.n_nonzero, 1))
     else:
         for _ in range(a.iters):
             qm.qm_quantize(Lop, a.fmt, a.gran, None, want_abs=True)
