@@ -12,7 +12,9 @@ cardinalities, tie enumeration, closed-form SQNR, brute-force triple loops,
 on-grid zero error, scale invariance, a hand-computed 2x2x2 case; for the tensor statistics
 and the Eq. 2 split (stats.py): closed-form moments of small integer arrays and of uniform /
 exponential laws, scipy's skew and kurtosis, hand-worked INT8 / E4M3 examples, the half-ulp
-bound on rounding RE, the class identities (counts and squared errors add up).
+bound on rounding RE, the class identities (counts and squared errors add up); for stochastic
+rounding (rng.py, probe._quantize_stochastic): the published known-answer vectors of
+Philox4x32-10, round-up frequency = distance fraction, unbiasedness, grid values fixed.
 Parity unpinned: the paper prints no numeric value of Eq. 3 for any input, so
 the metric is pinned only by those mathematical checks, not by a paper value.
 """

@@ -16,6 +16,7 @@ test share.
 """
 import numpy as np
 
+from .rng import element_uniforms
 from .formats import decode_table, positive_grid, qmax
 
 
@@ -60,8 +61,11 @@ def _expand(delta, x):
     return delta[..., None]
 
 
-def quantize(x, fmt, delta):
+def quantize(x, fmt, delta, rounding="rtne", seed=0, stream=0):
     """Eq. 1, left half, with the saturation rule of the Methodology section.
+
+    rounding == "stochastic" (second rounding mode of the Methodology section): see
+    _quantize_stochastic.  What follows describes the default, round-to-nearest-even.
 
     t = x / delta in float32; the code is the grid value nearest to t, a tie
     going to the value whose code is even (round-to-nearest-even); |t| above the
@@ -76,6 +80,10 @@ def quantize(x, fmt, delta):
     t = (x / _expand(delta, x)).astype(np.float32)      # IEEE float32 division
     if not np.all(np.isfinite(t)):
         raise ValueError("non-finite input")
+    if rounding == "stochastic":
+        return _quantize_stochastic(t, fmt, seed, stream)
+    if rounding != "rtne":
+        raise ValueError(rounding)
     g = positive_grid(fmt)                               # g[c] = value of code c
     mid = (g[:-1] + g[1:]) / 2.0                         # exact in float64
     a = np.abs(t.astype(np.float64))
@@ -88,6 +96,33 @@ def quantize(x, fmt, delta):
     else:
         # FP8 is sign-magnitude with IEEE conventions (the FP8 rules the paper cites): the sign
         # bit of the input survives rounding, so a negative value that rounds to zero is -0.
+        code = np.where(np.signbit(t), idx + 128, idx)
+    return code.astype(np.uint8)
+
+
+def _quantize_stochastic(t, fmt, seed, stream):
+    """Stochastic rounding of t = x / delta onto the format's grid.
+
+    With lo <= |t| <= hi the two neighbouring expressible magnitudes (|t| first capped at the
+    largest one: the saturation rule), the result is hi with probability
+    p = (|t| - lo) / (hi - lo) and lo otherwise, so its expectation is t.  The draw of element
+    number i (C order over the operand in its [.., nc, c] orientation) is the uniform number
+    u_i of rng.element_uniforms(seed, stream): hi iff u_i < p.  A value on the grid has p = 0 and
+    never moves; the sign is kept (FP8 keeps it on a zero result as RTNE does).
+    All of it is exact in float64: |t| - lo and hi - lo are exact differences of float32 values.
+    """
+    g = positive_grid(fmt)
+    a = np.minimum(np.abs(t.astype(np.float64)), g[-1])
+    lo_i = np.searchsorted(g, a, side="right") - 1        # largest grid value <= a
+    hi_i = np.minimum(lo_i + 1, len(g) - 1)
+    lo, hi = g[lo_i], g[hi_i]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        p = np.where(hi > lo, (a - lo) / (hi - lo), 0.0)
+    u = element_uniforms(t.shape, seed, stream)
+    idx = np.where(u < p, hi_i, lo_i)
+    if fmt == "int8":
+        code = np.where(np.signbit(t) & (idx > 0), 256 - idx, idx)
+    else:
         code = np.where(np.signbit(t), idx + 128, idx)
     return code.astype(np.uint8)
 
@@ -163,14 +198,16 @@ def derived(rec):
     }
 
 
-def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False):
+def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False, round_l="rtne", round_r="rtne", seed=0):
     """The whole probe for L [.., M, K] and R [.., K, N].
 
     rows: optional index array of output rows to evaluate (row-sampled mode;
     scales are still computed over the whole operands).  With full=True the
-    intermediate arrays are returned too.
+    intermediate arrays are returned too.  round_l / round_r choose the rounding mode per
+    operand (the paper rounds gradients stochastically); stochastic draws are numbered over
+    the whole operand in its [.., nc, c] orientation, stream 0 for L and 1 for R.
     """
-    l = _as_f32(l)
+    l = l_full = _as_f32(l)
     rt = np.swapaxes(_as_f32(r), -1, -2)
     dl = scale(l, fmt_l, gran_l)
     dr = scale(rt, fmt_r, gran_r)
@@ -179,8 +216,11 @@ def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False):
         dl_rows = dl if dl.shape == (1,) else dl[..., rows]
     else:
         dl_rows = dl
-    cl = quantize(l, fmt_l, dl_rows)
-    cr = quantize(rt, fmt_r, dr)
+    if round_l == "stochastic" and rows is not None:
+        cl = quantize(_as_f32(l_full), fmt_l, dl, "stochastic", seed, 0)[..., rows, :]
+    else:
+        cl = quantize(l, fmt_l, dl_rows, round_l, seed, 0)
+    cr = quantize(rt, fmt_r, dr, round_r, seed, 1)
     acc = gemm_lp(cl, fmt_l, cr, fmt_r)
     q = descale(acc, dl_rows, dr)
     c = gemm_ref(l, rt)
