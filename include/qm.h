@@ -59,7 +59,10 @@ typedef enum { QM_DT_F32 = 0, QM_DT_BF16 = 1 } qm_dtype;
 /* Scale granularity (Methodology, 4th bullet): one number for the whole tensor,
  * or one per index of the non-contracting dimension (and per batch element). */
 typedef enum { QM_GRAN_TENSOR = 0, QM_GRAN_CHANNEL = 1 } qm_gran;
-typedef enum { QM_ROUND_RTNE = 0 } qm_round;
+/* Rounding function of Eq. 1 (Methodology, 2nd bullet: round-to-nearest-even and stochastic
+ * rounding).  In qm_probe_cfg.round the two STOCHASTIC flags may be OR-ed: the paper rounds
+ * only the gradient operand stochastically, and which side that is depends on the product. */
+typedef enum { QM_ROUND_RTNE = 0, QM_ROUND_STOCHASTIC_L = 1, QM_ROUND_STOCHASTIC_R = 2 } qm_round;
 /* How the high-precision side of Eq. 3 is evaluated:
  *  BF16_FP32ACC: bf16 operands on the tensor cores, fp32 accumulation (every
  *                bf16 x bf16 product is exact in fp32);
@@ -126,8 +129,9 @@ typedef struct {
 typedef struct {
   int32_t fmt_l, fmt_r;    /* qm_format per operand                                       */
   int32_t gran_l, gran_r;  /* qm_gran per operand                                         */
-  int32_t round;           /* qm_round                                                    */
+  int32_t round;           /* qm_round flags                                              */
   int32_t ref;             /* qm_ref                                                      */
+  uint64_t seed;           /* of the stochastic draws; unused with QM_ROUND_RTNE          */
 } qm_probe_cfg;
 
 /* Row length in bytes of a code tensor whose contracting extent is `contract`. */
@@ -161,6 +165,25 @@ qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta,
 qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t round,
                       const float* delta, float* delta_out, uint8_t* codes,
                       void* abs_copy, void* kmaj_copy, void* stream);
+
+/*
+ * Eq. 1 with stochastic rounding (Methodology, 2nd bullet).  t = x / delta as in
+ * qm_quantize; with lo <= |t| <= hi the neighbouring expressible magnitudes (|t|
+ * capped at the largest one first), the code is hi's with probability
+ * (|t| - lo) / (hi - lo) and lo's otherwise, so the expectation is t; values on
+ * the grid never move and the sign is kept.  The paper does not say where the
+ * random numbers come from.  Here element number i of the operand (numbered
+ * batch-major, then noncontract, then contract, whatever the strides) uses
+ * u = (w >> 8) / 2^24 with w = word (i mod 4) of Philox4x32-10 (Salmon et al.,
+ * SC'11) on counter (i div 4: low word, high word, stream_id, 0) and key
+ * (seed: low word, high word); hi iff u (hi - lo) < |t| - lo.  The same
+ * (seed, stream_id) therefore reproduces the same codes on any layout.
+ * Other arguments as for qm_quantize (round is implied; qm_quantize itself
+ * accepts QM_ROUND_RTNE only).
+ */
+qm_status qm_quantize_stochastic(const qm_operand* x, int32_t fmt, int32_t gran, uint64_t seed,
+                                 uint32_t stream_id, const float* delta, float* delta_out,
+                                 uint8_t* codes, void* abs_copy, void* kmaj_copy, void* stream);
 
 /*
  * The 8-bit product and its descaling (Methodology, 3rd bullet):
@@ -209,6 +232,8 @@ qm_status qm_metric(const float* ref, const float* q, const float* den, int64_t 
  * share it.
  * QM_REF_BF16_FP32ACC needs bf16 operands and K a multiple of 16;
  * QM_REF_FP32 takes fp32 or bf16 operands of any shape.
+ * cfg->round: an operand flagged stochastic is quantized as by
+ * qm_quantize_stochastic with cfg->seed and stream_id 0 (L) or 1 (R).
  */
 size_t qm_workspace_bytes(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg);
 qm_status qm_probe_layer(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,

@@ -79,7 +79,7 @@ class QuantError(C.Structure):
 
 class ProbeCfg(C.Structure):
     _fields_ = [("fmt_l", C.c_int32), ("fmt_r", C.c_int32), ("gran_l", C.c_int32), ("gran_r", C.c_int32),
-                ("round", C.c_int32), ("ref", C.c_int32)]
+                ("round", C.c_int32), ("ref", C.c_int32), ("seed", C.c_uint64)]
 
 
 _lib = None
@@ -98,6 +98,7 @@ def lib():
             "qm_code_ld": (I64, [I64]),
             "qm_scale": (I32, [OP, I32, I32, P, P]),
             "qm_quantize": (I32, [OP, I32, I32, I32, P, P, P, P, P, P]),
+            "qm_quantize_stochastic": (I32, [OP, I32, I32, C.c_uint64, C.c_uint32, P, P, P, P, P, P]),
             "qm_gemm": (I32, [P, I32, P, I32, P, I32, P, I32, I64, I64, I64, I64, P, P, I32, P]),
             "qm_gemm_ref": (I32, [P, P, I64, I64, I64, I64, P, P]),
             "qm_metric_workspace_bytes": (SZ, [I64]),
@@ -181,8 +182,9 @@ def qm_scale(op, fmt, gran, stream=None):
     return delta
 
 
-def qm_quantize(op, fmt, gran, delta=None, want_abs=False, want_kmaj=False, stream=None):
-    """Codes of an operand.  delta=None fuses the scale step.  Returns (codes, delta, abs, kmaj)."""
+def qm_quantize(op, fmt, gran, delta=None, want_abs=False, want_kmaj=False, stream=None, stochastic=None):
+    """Codes of an operand.  delta=None fuses the scale step.  Returns (codes, delta, abs, kmaj).
+    stochastic=(seed, stream_id) rounds stochastically (qm_quantize_stochastic) instead of RTNE."""
     ldc = qm_code_ld(op.contract)
     codes = torch.empty((op.batch, op.noncontract, ldc), dtype=torch.uint8, device="cuda")
     shape = (op.batch, op.noncontract, op.contract)
@@ -191,8 +193,13 @@ def qm_quantize(op, fmt, gran, delta=None, want_abs=False, want_kmaj=False, stre
     dout = None
     if delta is None:
         dout = torch.empty(_n_delta(op, gran), dtype=torch.float32, device="cuda")
-    _check(lib().qm_quantize(C.byref(op), FMT[fmt], GRAN[gran], 0, _ptr(delta), _ptr(dout), _ptr(codes),
-                             _ptr(ab), _ptr(km), _stream(stream)), "qm_quantize")
+    if stochastic is not None:
+        _check(lib().qm_quantize_stochastic(C.byref(op), FMT[fmt], GRAN[gran], stochastic[0], stochastic[1],
+                                            _ptr(delta), _ptr(dout), _ptr(codes), _ptr(ab), _ptr(km),
+                                            _stream(stream)), "qm_quantize_stochastic")
+    else:
+        _check(lib().qm_quantize(C.byref(op), FMT[fmt], GRAN[gran], 0, _ptr(delta), _ptr(dout), _ptr(codes),
+                                 _ptr(ab), _ptr(km), _stream(stream)), "qm_quantize")
     return codes, (delta if delta is not None else dout), ab, km
 
 
@@ -273,9 +280,13 @@ def qm_quantize_error(op, fmt, gran, delta=None, ws=None, stream=None):
     return QuantError.from_buffer_copy(out.cpu().numpy().tobytes())
 
 
-def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref):
+ROUND = {"rtne": 0, "stochastic_l": 1, "stochastic_r": 2, "stochastic_both": 3}
+
+
+def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding="rtne", seed=0):
     c = ProbeCfg()
-    c.fmt_l, c.fmt_r, c.gran_l, c.gran_r, c.round, c.ref = FMT[fmt_l], FMT[fmt_r], GRAN[gran_l], GRAN[gran_r], 0, REF[ref]
+    c.fmt_l, c.fmt_r, c.gran_l, c.gran_r, c.ref = FMT[fmt_l], FMT[fmt_r], GRAN[gran_l], GRAN[gran_r], REF[ref]
+    c.round, c.seed = ROUND[rounding], seed
     return c
 
 
@@ -290,8 +301,8 @@ def qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
 class ProbePlan:
     """Pre-allocated workspace and result buffer for repeated probes of one shape."""
 
-    def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
-        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref)
+    def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", rounding="rtne", seed=0):
+        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed)
         self.ws_bytes = qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
         self.out = torch.zeros(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
@@ -304,9 +315,10 @@ class ProbePlan:
         return _read_result(self.out)
 
 
-def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None):
-    """The whole probe for one product; returns the MetricResult (synchronises to read it)."""
-    plan = ProbePlan(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
+def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None, rounding="rtne", seed=0):
+    """The whole probe for one product; returns the MetricResult (synchronises to read it).
+    rounding: "rtne", or "stochastic_l" / "stochastic_r" / "stochastic_both" with `seed`."""
+    plan = ProbePlan(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed)
     plan.launch(L_op, R_op, stream)
     return plan.result()
 

@@ -138,7 +138,7 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
   if (st != QM_OK) return st;
   if (!valid_fmt(cfg->fmt_l) || !valid_fmt(cfg->fmt_r) || !valid_gran(cfg->gran_l) || !valid_gran(cfg->gran_r))
     return QM_ERR_INVALID_ARG;
-  if (cfg->round != QM_ROUND_RTNE) return QM_ERR_UNSUPPORTED;
+  if (cfg->round & ~(QM_ROUND_STOCHASTIC_L | QM_ROUND_STOCHASTIC_R)) return QM_ERR_INVALID_ARG;
   if (cfg->ref != QM_REF_BF16_FP32ACC && cfg->ref != QM_REF_FP32) return QM_ERR_INVALID_ARG;
   if (L->c != R->c || L->batch != R->batch) return QM_ERR_INVALID_ARG;
   if ((cfg->fmt_l == QM_FMT_INT8) != (cfg->fmt_r == QM_FMT_INT8)) return QM_ERR_UNSUPPORTED;
@@ -151,14 +151,15 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
 
 // scale + quantize of one operand inside the probe
 qm_status prepare_operand(const View& x, int fmt, int gran, uint32_t* amax, float* delta, uint8_t* codes,
-                          void* abs_copy, void* kmaj_copy, uint32_t* err_word, cudaStream_t s) {
-  if (gran == QM_GRAN_CHANNEL && x.c_contig())
+                          void* abs_copy, void* kmaj_copy, uint32_t* err_word, const StochasticDraw* draw,
+                          cudaStream_t s) {
+  if (!draw && gran == QM_GRAN_CHANNEL && x.c_contig())
     return launch_scale_quantize_rows(x, fmt, delta, codes, abs_copy, err_word, s);
   qm_status st = launch_absmax(x, gran, amax, s);
   if (st != QM_OK) return st;
   // the quantize kernel turns max|x| into delta itself
   return launch_quantize(x, fmt, gran, reinterpret_cast<const float*>(amax), true, delta, err_word, codes,
-                         abs_copy, kmaj_copy, s);
+                         abs_copy, kmaj_copy, s, draw);
 }
 
 }  // namespace
@@ -183,28 +184,42 @@ qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta,
   return launch_finalize_delta(delta, n, fmt, nullptr, s);
 }
 
-qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t round, const float* delta,
-                      float* delta_out, uint8_t* codes, void* abs_copy, void* kmaj_copy, void* stream) {
+static qm_status quantize_entry(const qm_operand* x, int32_t fmt, int32_t gran, const StochasticDraw* draw,
+                                const float* delta, float* delta_out, uint8_t* codes, void* abs_copy,
+                                void* kmaj_copy, void* stream) {
   View v;
   qm_status st = to_view(x, &v);
   if (st != QM_OK) return st;
   if (!valid_fmt(fmt) || !valid_gran(gran) || !codes) return QM_ERR_INVALID_ARG;
-  if (round != QM_ROUND_RTNE) return QM_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(codes) & 15) || (reinterpret_cast<uintptr_t>(abs_copy) & 15) ||
       (reinterpret_cast<uintptr_t>(kmaj_copy) & 15))
     return QM_ERR_ALIGNMENT;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (delta) return launch_quantize(v, fmt, gran, delta, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s);
+  if (delta)
+    return launch_quantize(v, fmt, gran, delta, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s, draw);
   if (!delta_out) return QM_ERR_INVALID_ARG;
   const int64_t n = delta_count(v, gran);
-  if (gran == QM_GRAN_CHANNEL && v.c_contig() && !kmaj_copy)
+  if (!draw && gran == QM_GRAN_CHANNEL && v.c_contig() && !kmaj_copy)
     return launch_scale_quantize_rows(v, fmt, delta_out, codes, abs_copy, nullptr, s);
   QM_CUDA_OK(cudaMemsetAsync(delta_out, 0, sizeof(float) * n, s));
   st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta_out), s);
   if (st != QM_OK) return st;
   st = launch_finalize_delta(delta_out, n, fmt, nullptr, s);
   if (st != QM_OK) return st;
-  return launch_quantize(v, fmt, gran, delta_out, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s);
+  return launch_quantize(v, fmt, gran, delta_out, false, nullptr, nullptr, codes, abs_copy, kmaj_copy, s, draw);
+}
+
+qm_status qm_quantize(const qm_operand* x, int32_t fmt, int32_t gran, int32_t round, const float* delta,
+                      float* delta_out, uint8_t* codes, void* abs_copy, void* kmaj_copy, void* stream) {
+  if (round != QM_ROUND_RTNE) return QM_ERR_UNSUPPORTED;   // stochastic rounding: qm_quantize_stochastic
+  return quantize_entry(x, fmt, gran, nullptr, delta, delta_out, codes, abs_copy, kmaj_copy, stream);
+}
+
+qm_status qm_quantize_stochastic(const qm_operand* x, int32_t fmt, int32_t gran, uint64_t seed, uint32_t stream_id,
+                                 const float* delta, float* delta_out, uint8_t* codes, void* abs_copy,
+                                 void* kmaj_copy, void* stream) {
+  const StochasticDraw draw{seed, stream_id};
+  return quantize_entry(x, fmt, gran, &draw, delta, delta_out, codes, abs_copy, kmaj_copy, stream);
 }
 
 qm_status qm_gemm(const uint8_t* codes_l, int32_t fmt_l, const float* delta_l, int32_t gran_l,
@@ -284,9 +299,12 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   void* ar = w.tc ? base + w.off_ar : nullptr;
   void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
-  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err, s);
+  const StochasticDraw draw_l{cfg->seed, 0u}, draw_r{cfg->seed, 1u};
+  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err,
+                       (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, s);
   if (st != QM_OK) return st;
-  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err, s);
+  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err,
+                       (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, s);
   if (st != QM_OK) return st;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {

@@ -74,9 +74,11 @@ qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_
 // codes (+ optional |x| and x as bf16, contraction-major).  `delta` holds finished deltas, or,
 // with from_amax, the max|x| bit patterns of launch_absmax: the kernel then does the division
 // itself, writes the deltas to delta_out and raises QM_DEVERR_NONFINITE in err_word (optional).
+// draw != nullptr: stochastic rounding with these draws instead of round-to-nearest-even.
+struct StochasticDraw { uint64_t seed; uint32_t stream; };
 qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, bool from_amax,
                           float* delta_out, uint32_t* err_word, uint8_t* codes, void* abs_copy,
-                          void* kmaj_copy, cudaStream_t s);
+                          void* kmaj_copy, cudaStream_t s, const StochasticDraw* draw = nullptr);
 // Single pass per row: absmax, delta, codes (contiguous contraction, per-channel).
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
                                      void* abs_copy, uint32_t* err_word, cudaStream_t s);

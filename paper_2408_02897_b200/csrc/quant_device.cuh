@@ -117,6 +117,92 @@ __device__ __forceinline__ uint2 quant8(const Vec8& x, const Quotient& quot) {
   return r;
 }
 
+// ---------------------------------------------------------------- stochastic rounding
+// Second rounding mode of the Methodology section.  The uniform number of element i of an operand
+// is word (i mod 4) of Philox4x32-10 (Salmon et al., SC'11) with counter (i div 4 as two words,
+// stream, 0) and the seed's two words as key; u = (word >> 8) / 2^24.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t (&out)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Rounding mode of one quantize launch, passed by value.
+struct Rounding {
+  int stochastic;
+  uint32_t k0, k1;      // seed, low and high word
+  uint32_t stream;      // which operand of the probe draws (0 = left, 1 = right)
+};
+
+// t = x / delta moved onto the format's grid: with lo <= |t| <= hi the neighbouring expressible
+// magnitudes (|t| capped at the largest one first), hi when u (hi - lo) < |t| - lo and lo
+// otherwise.  Both sides of the comparison are exact in fp32 (hi - lo is a power of two and
+// |t| - lo a difference inside one binade), so the decision equals the one taken in exact
+// arithmetic.  The sign of t is kept.
+template <int FMT>
+__device__ __forceinline__ float sr_value(float t, uint32_t word) {
+  const float a = fminf(fabsf(t), fmt_qmax(FMT));
+  const float u = (float)(word >> 8) * 5.9604644775390625e-8f;          // 2^-24, exact
+  float lo, spacing;
+  if (FMT == QM_FMT_INT8) {
+    lo = floorf(a);
+    spacing = 1.f;
+  } else {
+    constexpr int m = FMT == QM_FMT_E4M3 ? 3 : 2;                        // mantissa bits
+    constexpr int emin = FMT == QM_FMT_E4M3 ? -6 : -14;                  // smallest normal exponent
+    const float min_normal = __uint_as_float((uint32_t)(127 + emin) << 23);
+    if (a >= min_normal) {
+      const uint32_t bits = __float_as_uint(a) & ~((1u << (23 - m)) - 1u);   // mantissa cut to m bits
+      lo = __uint_as_float(bits);
+      spacing = __uint_as_float(((bits >> 23) - m) << 23);
+    } else {
+      spacing = __uint_as_float((uint32_t)(127 + emin - m) << 23);       // the subnormal step
+      lo = floorf(a * __uint_as_float((uint32_t)(127 - emin + m) << 23)) * spacing;
+    }
+  }
+  const float r = (u * spacing < a - lo) ? lo + spacing : lo;
+  return copysignf(r, t);
+}
+
+// Eight consecutive elements whose first has number idx0 in the operand.
+template <int FMT>
+__device__ __forceinline__ uint2 quant8_sr(const Vec8& x, const Quotient& quot, const Rounding& rnd,
+                                           uint64_t idx0) {
+  uint32_t w[12];
+  const uint64_t blk = idx0 >> 2;
+  const int first = (int)(idx0 & 3);
+#pragma unroll
+  for (int b = 0; b < 3; ++b) {
+    if (b < 2 || first != 0) {
+      const uint64_t c = blk + b;
+      philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), rnd.stream, 0u, rnd.k0, rnd.k1,
+                    *reinterpret_cast<uint32_t(*)[4]>(&w[4 * b]));
+    } else {
+      w[8] = w[9] = w[10] = w[11] = 0u;
+    }
+  }
+  float t[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    // word first + i without dynamic indexing of the register array
+    uint32_t word = 0;
+#pragma unroll
+    for (int f = 0; f < 4; ++f)
+      if (first == f) word = w[f + i];
+    t[i] = sr_value<FMT>(quot(x.v[i]), word);
+  }
+  uint2 r;
+  r.x = quant2<FMT>(t[0], t[1]) | (quant2<FMT>(t[2], t[3]) << 16);
+  r.y = quant2<FMT>(t[4], t[5]) | (quant2<FMT>(t[6], t[7]) << 16);
+  return r;
+}
+
 __device__ __forceinline__ uint4 abs_bf16x8(const Vec8& x) {
   uint4 r;
   r.x = pack_bf16x2(fabsf(x.v[0]), fabsf(x.v[1]));

@@ -176,7 +176,8 @@ template <typename T, int FMT>
 __global__ void __launch_bounds__(kThreads)
 quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_nc, int64_t batch,
                      int64_t s_b, const DeltaSrc ds, const FastDiv by_chunks, const FastDiv by_nc,
-                     uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy) {
+                     uint8_t* __restrict__ codes, int64_t ldc, __nv_bfloat16* __restrict__ abs_copy,
+                     const Rounding rnd) {
   pdl_prologue();
   const uint32_t chunks_per_row = (uint32_t)(ldc >> 4);     // 16 codes per chunk, padding included
   const uint32_t total = (uint32_t)(nc * batch) * chunks_per_row;   // < 2^32, checked by the host
@@ -200,7 +201,15 @@ quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_n
         v1.v[j] = k0 + 8 + j < c ? Loader<T>::load1(p, 8 + j) : 0.f;
       }
     }
-    uint2 q0 = quant8<FMT>(v0, quot), q1 = quant8<FMT>(v1, quot);
+    uint2 q0, q1;
+    if (rnd.stochastic) {
+      const uint64_t e0 = (uint64_t)row * (uint64_t)c + (uint64_t)k0;   // number of the chunk's first element
+      q0 = quant8_sr<FMT>(v0, quot, rnd, e0);
+      q1 = quant8_sr<FMT>(v1, quot, rnd, e0 + 8);
+    } else {
+      q0 = quant8<FMT>(v0, quot);
+      q1 = quant8<FMT>(v1, quot);
+    }
     *reinterpret_cast<uint4*>(codes + row * ldc + k0) = make_uint4(q0.x, q0.y, q1.x, q1.y);
     if (abs_copy) {
       __nv_bfloat16* a = abs_copy + row * c + k0;
@@ -381,7 +390,8 @@ __global__ void __launch_bounds__(kThreads)
 quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
                           const DeltaSrc ds,
                           uint8_t* __restrict__ codes, int64_t ldc,
-                          __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy) {
+                          __nv_bfloat16* __restrict__ abs_copy, __nv_bfloat16* __restrict__ kmaj_copy,
+                          const Rounding rnd) {
   pdl_prologue();
   __shared__ float tile[64][65];     // +1 column spreads the transposed accesses over the banks
   const int64_t b = blockIdx.z;
@@ -419,7 +429,9 @@ quantize_transpose_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_
     for (int j = 0; j < 8; ++j) v.v[j] = tile[tx * 8 + j][nrow];
     const Quotient quot(ds.per_channel ? ds.get(b * nc + nn, blockIdx.y == 0 && tx == 0) : d_tensor);
     const int64_t orow = b * nc + nn;
-    *reinterpret_cast<uint2*>(codes + orow * ldc + k0) = quant8<FMT>(v, quot);
+    *reinterpret_cast<uint2*>(codes + orow * ldc + k0) =
+        rnd.stochastic ? quant8_sr<FMT>(v, quot, rnd, (uint64_t)orow * (uint64_t)c + (uint64_t)k0)
+                       : quant8<FMT>(v, quot);
     if (abs_copy || kmaj_copy) {
       if (k0 + 8 <= c && (c & 7) == 0) {
         if (abs_copy) *reinterpret_cast<uint4*>(abs_copy + orow * c + k0) = abs_bf16x8(v);
@@ -556,7 +568,8 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
 
 template <typename T, int FMT>
 qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax, float* delta_out,
-                     uint32_t* err_word, uint8_t* codes, void* abs_copy, void* kmaj_copy, cudaStream_t s) {
+                     uint32_t* err_word, uint8_t* codes, void* abs_copy, void* kmaj_copy, const Rounding& rnd,
+                     cudaStream_t s) {
   const T* p = static_cast<const T*>(x.data);
   const int64_t ldc = qm_code_ld(x.c);
   DeltaSrc ds;
@@ -565,7 +578,8 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
   if (x.c_contig()) {
     const int64_t total = x.nc * x.batch * (ldc >> 4);
     if (total >= (1ll << 32) || x.nc >= (1ll << 32)) return QM_ERR_UNSUPPORTED;   // 32-bit chunk index
-    const bool dense = x.dtype == QM_DT_BF16 && x.s_nc == x.c && (x.c & 15) == 0 &&
+    // (stochastic rounding takes the general kernels: the draws cost more than the fast paths save)
+    const bool dense = !rnd.stochastic && x.dtype == QM_DT_BF16 && x.s_nc == x.c && (x.c & 15) == 0 &&
                        (x.batch == 1 || x.s_b == x.nc * x.c);
     if (dense) {
       const uint4* src = reinterpret_cast<const uint4*>(x.data);
@@ -583,7 +597,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
     } else
     launch_pdl(quantize_rows_kernel<T, FMT>, dim3(grid_for(total, 16)), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
-        codes, ldc, static_cast<__nv_bfloat16*>(abs_copy));
+        codes, ldc, static_cast<__nv_bfloat16*>(abs_copy), rnd);
     if (kmaj_copy) {
       // already contraction-major: a strided copy honours the parameter
       if (x.dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;
@@ -593,7 +607,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
                                      x.c * 2, x.nc, cudaMemcpyDeviceToDevice, s));
     }
   } else {
-    if (x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
+    if (!rnd.stochastic && x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
         ((x.nc + 63) / 64) * ((x.c + 255) / 256) * x.batch >= 4 * (int64_t)sm_count()) {
       dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
       launch_pdl(quantize_transpose_bf16_kernel<FMT>, dim3(grid), dim3(kThreads), 0, s, 
@@ -606,7 +620,7 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
     dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((ldc + 63) / 64), (unsigned)x.batch);
     launch_pdl(quantize_transpose_kernel<T, FMT>, dim3(grid), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc, static_cast<__nv_bfloat16*>(abs_copy),
-        static_cast<__nv_bfloat16*>(kmaj_copy));
+        static_cast<__nv_bfloat16*>(kmaj_copy), rnd);
   }
   count_launch();
   QM_CUDA_OK(cudaGetLastError());
@@ -668,8 +682,13 @@ qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_
 
 qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, bool from_amax,
                           float* delta_out, uint32_t* err_word, uint8_t* codes, void* abs_copy,
-                          void* kmaj_copy, cudaStream_t s) {
-#define QM_ARGS x, gran, delta, from_amax, delta_out, err_word, codes, abs_copy, kmaj_copy, s
+                          void* kmaj_copy, cudaStream_t s, const StochasticDraw* draw) {
+  Rounding rnd{};
+  if (draw) {
+    rnd.stochastic = 1;
+    rnd.k0 = (uint32_t)draw->seed; rnd.k1 = (uint32_t)(draw->seed >> 32); rnd.stream = draw->stream;
+  }
+#define QM_ARGS x, gran, delta, from_amax, delta_out, err_word, codes, abs_copy, kmaj_copy, rnd, s
 #define QM_Q(T)                                                    \
   (fmt == QM_FMT_INT8   ? quantize_t<T, QM_FMT_INT8>(QM_ARGS)      \
    : fmt == QM_FMT_E4M3 ? quantize_t<T, QM_FMT_E4M3>(QM_ARGS)      \

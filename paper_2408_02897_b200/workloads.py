@@ -30,6 +30,12 @@ def student_t(rng, shape, nu, dtype=torch.bfloat16):
     return torch.from_numpy(x).to(dtype)
 
 
+def lognormal_signed(rng, shape, mu, sigma, dtype=torch.bfloat16):
+    """Gradient-like values: log-normal magnitudes (the paper finds gradients log-normal), random signs."""
+    x = np.exp(rng.normal(mu, sigma, shape)) * rng.choice([-1.0, 1.0], shape)
+    return torch.from_numpy(x.astype(np.float32)).to(dtype)
+
+
 def op(name, L, cl, R, cr, fmt_l, fmt_r, gran_l="tensor", gran_r="tensor", ref="bf16"):
     return dict(name=name, L=L, cl=cl, R=R, cr=cr, fmt_l=fmt_l, fmt_r=fmt_r, gran_l=gran_l,
                 gran_r=gran_r, ref=ref)

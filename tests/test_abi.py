@@ -27,10 +27,29 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(L, n), n
 
 
-def test_struct_layouts_match_header():
-    assert C.sizeof(binding.MetricResult) == 56
-    assert C.sizeof(binding.Operand) == 64
-    assert C.sizeof(binding.ProbeCfg) == 24
+def test_struct_layouts_match_header(tmp_path):
+    """The ctypes mirrors have the sizes and field offsets a C compiler gives the header's structs."""
+    import subprocess
+    pairs = [("qm_metric_result", binding.MetricResult), ("qm_operand", binding.Operand),
+             ("qm_probe_cfg", binding.ProbeCfg), ("qm_tensor_stats_result", binding.TensorStats),
+             ("qm_quant_error_result", binding.QuantError)]
+    lines = []
+    for cname, cls in pairs:
+        lines.append(f'printf("{cname} %zu", sizeof({cname}));')
+        for fname, _ in cls._fields_:
+            lines.append(f'printf(" %zu", offsetof({cname}, {fname}));')
+        lines.append('printf("\\n");')
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "qm.h"\nint main(void) {\n' + "\n".join(lines) + "\nreturn 0; }\n")
+    exe = tmp_path / "layout"
+    inc = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include")
+    subprocess.check_call(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe)])
+    out = subprocess.check_output([str(exe)], text=True).strip().splitlines()
+    for (cname, cls), line in zip(pairs, out):
+        w = line.split()
+        assert w[0] == cname and int(w[1]) == C.sizeof(cls), line
+        assert [int(x) for x in w[2:]] == [getattr(cls, f).offset for f, _ in cls._fields_], line
+    assert C.sizeof(binding.MetricResult) == 56 and C.sizeof(binding.ProbeCfg) == 32
 
 
 def test_host_side_argument_checks():
