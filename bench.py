@@ -175,6 +175,12 @@ def scale_quantize_rates(qm, hbm_gbs, rows=16384, cols=4096, iters=10):
     t_quant = timed(lambda: raw_quant(op_rows, 0, delta, None, codes))
     t_fused = timed(lambda: raw_quant(op_rows, 1, None, dch, codes))
     t_trans = timed(lambda: raw_quant(op_cols, 0, delta, None, codes_t))
+    def raw_quant_sr(op, cod):
+        rc = L.qm_quantize_stochastic(C.byref(op), 1, 0, 12345, 0, C.c_void_p(delta.data_ptr()), None,
+                                      C.c_void_p(cod.data_ptr()), None, None, st)
+        assert rc == 0, rc
+
+    t_sr = timed(lambda: raw_quant_sr(op_rows, codes))
     ws_n = L.qm_stats_workspace_bytes()
     ws = torch.empty(ws_n, dtype=torch.uint8, device="cuda")
     rec = torch.empty(128, dtype=torch.uint8, device="cuda")
@@ -196,10 +202,11 @@ def scale_quantize_rates(qm, hbm_gbs, rows=16384, cols=4096, iters=10):
            "quantize_gbs": 3 * n / t_quant / 1e9,                     # 2 B read + 1 B code
            "scale_quantize_rows_gbs": 3 * n / t_fused / 1e9,          # fused per-row scale + codes, input read once
            "quantize_transpose_gbs": 3 * n / t_trans / 1e9,
+           "quantize_stochastic_gbs": 3 * n / t_sr / 1e9,              # 2 B read + 1 B code, Philox draws
            "tensor_stats_gbs": 2 * n / t_stats / 1e9,                  # 2 B/elem read, power sums + max
            "quantize_error_gbs": 2 * n / t_err / 1e9,                  # 2 B/elem read, Eq. 2 split, one scale
            "quantize_error_rows_gbs": 2 * n / t_err_ch / 1e9}         # one scale per row
-    for k in ("scale_tensor", "quantize", "scale_quantize_rows", "quantize_transpose", "tensor_stats",
+    for k in ("scale_tensor", "quantize", "scale_quantize_rows", "quantize_transpose", "quantize_stochastic", "tensor_stats",
               "quantize_error", "quantize_error_rows"):
         out[k + "_frac_of_hbm"] = out[k + "_gbs"] / hbm_gbs
     return out
