@@ -27,7 +27,7 @@ def _as_f32(x):
     return x
 
 
-def scale(x, fmt, gran):
+def scale(x, fmt, gran, batch_groups=None):
     """Eq. 1, right half: delta = max|X| / qmax, one delta per scaling group.
 
     gran == "tensor": one number for the whole (batched) tensor, shape [1].
@@ -35,6 +35,15 @@ def scale(x, fmt, gran):
     (and per matmul-batch element), shape x.shape[:-1]  ("finer levels of
     granularity on non-contracting dimensions", Methodology 4th bullet).
     An all-zero group gets delta = 1.  Non-finite input is an error.
+
+    batch_groups (channel granularity of a batched [b, nc, c] operand only): the granularity
+    levels of the Results section share scales along the matmul-batch axis.  Batch element
+    number b belongs to group b mod batch_groups and all elements of a group share their
+    per-channel scales: batch_groups = 1 is the paper's "channel" (one scale tensor over the
+    non-batch, non-contracting dimension), batch_groups = number of heads with the batch laid
+    out [examples][heads] is its "fine-grained" (batch dimensions included, except the axis of
+    the individual examples).  None: every batch element has its own scales.  The returned
+    array still has shape x.shape[:-1], with shared entries repeated.
     """
     x = _as_f32(x)
     if not np.all(np.isfinite(x)):
@@ -44,6 +53,12 @@ def scale(x, fmt, gran):
         amax = np.array([a.max() if a.size else 0.0], dtype=np.float32)
     elif gran == "channel":
         amax = a.max(axis=-1).astype(np.float32) if a.shape[-1] else np.zeros(a.shape[:-1], np.float32)
+        if batch_groups is not None:
+            if x.ndim != 3 or batch_groups < 1 or x.shape[0] % batch_groups:
+                raise ValueError("batch_groups must divide the batch of a [b, nc, c] operand")
+            g = batch_groups
+            shared = amax.reshape(x.shape[0] // g, g, x.shape[1]).max(axis=0)      # over the examples
+            amax = np.broadcast_to(shared, (x.shape[0] // g, g, x.shape[1])).reshape(x.shape[:2]).copy()
     else:
         raise ValueError(gran)
     delta = amax / np.float32(qmax(fmt))          # one float32 division
@@ -198,7 +213,8 @@ def derived(rec):
     }
 
 
-def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False, round_l="rtne", round_r="rtne", seed=0):
+def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False, round_l="rtne", round_r="rtne", seed=0,
+          groups_l=None, groups_r=None):
     """The whole probe for L [.., M, K] and R [.., K, N].
 
     rows: optional index array of output rows to evaluate (row-sampled mode;
@@ -206,11 +222,12 @@ def probe(l, r, fmt_l, fmt_r, gran_l, gran_r, rows=None, full=False, round_l="rt
     intermediate arrays are returned too.  round_l / round_r choose the rounding mode per
     operand (the paper rounds gradients stochastically); stochastic draws are numbered over
     the whole operand in its [.., nc, c] orientation, stream 0 for L and 1 for R.
+    groups_l / groups_r: batch_groups of scale() for an operand with channel granularity.
     """
     l = l_full = _as_f32(l)
     rt = np.swapaxes(_as_f32(r), -1, -2)
-    dl = scale(l, fmt_l, gran_l)
-    dr = scale(rt, fmt_r, gran_r)
+    dl = scale(l, fmt_l, gran_l, groups_l if gran_l == "channel" else None)
+    dr = scale(rt, fmt_r, gran_r, groups_r if gran_r == "channel" else None)
     if rows is not None:
         l = l[..., rows, :]
         dl_rows = dl if dl.shape == (1,) else dl[..., rows]

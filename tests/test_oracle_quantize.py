@@ -223,3 +223,38 @@ def test_division_is_fp32_not_reciprocal_multiply():
     # a tie produced only by exact division: 7.5 / 3 = 2.5 -> 2
     x = np.array([[7.5, 381.0]], np.float32)
     assert oracle.dequantize(oracle.quantize(x, "int8", d), "int8")[0, 0] == 2.0
+
+
+# ------------------------------------------------------------------ scales shared along the batch
+def test_batch_groups_match_the_granularity_levels_of_the_results_section():
+    """'channel' = one scale per non-contracting index shared by the whole matmul batch;
+    'fine-grained' = also per head, shared by the examples.  Hand-built case: batch laid out
+    [examples = 2][heads = 3], one row, so the maxima can be read off."""
+    x = np.zeros((6, 1, 4), np.float32)
+    peaks = [1.0, 20.0, 3.0, 40.0, 5.0, 6.0]            # b = e * 3 + h
+    for b, p in enumerate(peaks):
+        x[b, 0, b % 4] = -p
+    own = oracle.scale(x, "int8", "channel")
+    assert np.array_equal(own[:, 0] * 127, np.float32(peaks))
+    fine = oracle.scale(x, "int8", "channel", batch_groups=3)       # per head: max over the two examples
+    assert np.allclose(fine[:, 0] * 127, [40.0, 20.0, 6.0, 40.0, 20.0, 6.0])
+    chan = oracle.scale(x, "int8", "channel", batch_groups=1)       # shared by the whole batch
+    assert np.allclose(chan[:, 0] * 127, [40.0] * 6)
+    assert np.array_equal(oracle.scale(x, "int8", "channel", batch_groups=6), own)
+    with pytest.raises(ValueError):
+        oracle.scale(x, "int8", "channel", batch_groups=4)
+
+
+def test_batch_groups_equal_a_per_channel_scale_of_the_regrouped_tensor():
+    rng = np.random.default_rng(12)
+    E, H, S, D = 3, 4, 10, 16
+    x = rng.standard_normal((E * H, S, D)).astype(np.float32) * 10.0 ** rng.uniform(-2, 1, (E * H, 1, 1)).astype(np.float32)
+    got = oracle.scale(x, "e4m3", "channel", batch_groups=H)
+    # the same numbers from the textbook route: move the examples next to the contraction and take
+    # an ordinary per-row absmax
+    regrouped = x.reshape(E, H, S, D).transpose(1, 2, 0, 3).reshape(H, S, E * D)
+    want = oracle.scale(regrouped, "e4m3", "channel")               # [H, S]
+    assert np.array_equal(got.reshape(E, H, S), np.broadcast_to(want, (E, H, S)))
+    # coarser sharing never gives a smaller scale, and quantization error cannot shrink with it
+    own = oracle.scale(x, "e4m3", "channel")
+    assert np.all(got >= own) and np.all(oracle.scale(x, "e4m3", "channel", 1) >= got)
