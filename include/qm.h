@@ -132,6 +132,8 @@ typedef struct {
   int32_t round;           /* qm_round flags                                              */
   int32_t ref;             /* qm_ref                                                      */
   uint64_t seed;           /* of the stochastic draws; unused with QM_ROUND_RTNE          */
+  int32_t batch_groups_l;  /* QM_GRAN_CHANNEL on a batched operand: see qm_scale_shared;  */
+  int32_t batch_groups_r;  /* 0 = every batch element has its own scales                  */
 } qm_probe_cfg;
 
 /* Row length in bytes of a code tensor whose contracting extent is `contract`. */
@@ -146,6 +148,21 @@ int64_t qm_code_ld(int64_t contract);
  * makes the group's delta NaN/Inf.
  */
 qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta, void* stream);
+
+/*
+ * Per-channel scales shared along the matmul batch (the granularity levels of the
+ * Results section).  Batch element b belongs to group b % batch_groups, and the
+ * batch elements of a group share one scale per non-contracting index, taken
+ * over all of them:  batch_groups = 1 is the paper's "channel" level (a scale
+ * tensor over the non-batch, non-contracting dimension), batch_groups = number
+ * of heads, for a batch laid out [examples][heads], is its "fine-grained" level
+ * (batch dimensions included, except the axis of the individual examples), and
+ * batch_groups = batch is QM_GRAN_CHANNEL of qm_scale.  batch_groups must divide
+ * the batch.  `delta` receives batch * noncontract values, shared ones repeated,
+ * so it can be handed to qm_quantize / qm_gemm with QM_GRAN_CHANNEL as it is.
+ */
+qm_status qm_scale_shared(const qm_operand* x, int32_t fmt, int32_t batch_groups, float* delta,
+                          void* stream);
 
 /*
  * Eq. 1 (left half) and the saturation rule: code = sat(RTNE(x / delta)), the

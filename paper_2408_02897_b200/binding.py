@@ -79,7 +79,8 @@ class QuantError(C.Structure):
 
 class ProbeCfg(C.Structure):
     _fields_ = [("fmt_l", C.c_int32), ("fmt_r", C.c_int32), ("gran_l", C.c_int32), ("gran_r", C.c_int32),
-                ("round", C.c_int32), ("ref", C.c_int32), ("seed", C.c_uint64)]
+                ("round", C.c_int32), ("ref", C.c_int32), ("seed", C.c_uint64),
+                ("batch_groups_l", C.c_int32), ("batch_groups_r", C.c_int32)]
 
 
 _lib = None
@@ -97,6 +98,7 @@ def lib():
         sig = {
             "qm_code_ld": (I64, [I64]),
             "qm_scale": (I32, [OP, I32, I32, P, P]),
+            "qm_scale_shared": (I32, [OP, I32, I32, P, P]),
             "qm_quantize": (I32, [OP, I32, I32, I32, P, P, P, P, P, P]),
             "qm_quantize_stochastic": (I32, [OP, I32, I32, C.c_uint64, C.c_uint32, P, P, P, P, P, P]),
             "qm_gemm": (I32, [P, I32, P, I32, P, I32, P, I32, I64, I64, I64, I64, P, P, I32, P]),
@@ -179,6 +181,14 @@ def qm_scale(op, fmt, gran, stream=None):
     """Eq. 1 scales of an operand -> float32 CUDA tensor (1 or batch*noncontract values)."""
     delta = torch.empty(_n_delta(op, gran), dtype=torch.float32, device="cuda")
     _check(lib().qm_scale(C.byref(op), FMT[fmt], GRAN[gran], _ptr(delta), _stream(stream)), "qm_scale")
+    return delta
+
+
+def qm_scale_shared(op, fmt, batch_groups, stream=None):
+    """Per-channel Eq. 1 scales shared along the matmul batch (batch element b in group b % batch_groups)
+    -> float32 CUDA tensor of batch*noncontract values, usable wherever "channel" scales are."""
+    delta = torch.empty(op.batch * op.noncontract, dtype=torch.float32, device="cuda")
+    _check(lib().qm_scale_shared(C.byref(op), FMT[fmt], batch_groups, _ptr(delta), _stream(stream)), "qm_scale_shared")
     return delta
 
 
@@ -283,8 +293,9 @@ def qm_quantize_error(op, fmt, gran, delta=None, ws=None, stream=None):
 ROUND = {"rtne": 0, "stochastic_l": 1, "stochastic_r": 2, "stochastic_both": 3}
 
 
-def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding="rtne", seed=0):
+def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding="rtne", seed=0, groups=(0, 0)):
     c = ProbeCfg()
+    c.batch_groups_l, c.batch_groups_r = groups
     c.fmt_l, c.fmt_r, c.gran_l, c.gran_r, c.ref = FMT[fmt_l], FMT[fmt_r], GRAN[gran_l], GRAN[gran_r], REF[ref]
     c.round, c.seed = ROUND[rounding], seed
     return c
@@ -301,8 +312,9 @@ def qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
 class ProbePlan:
     """Pre-allocated workspace and result buffer for repeated probes of one shape."""
 
-    def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", rounding="rtne", seed=0):
-        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed)
+    def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", rounding="rtne", seed=0,
+                 groups=(0, 0)):
+        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed, groups)
         self.ws_bytes = qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
         self.out = torch.zeros(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
@@ -315,10 +327,12 @@ class ProbePlan:
         return _read_result(self.out)
 
 
-def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None, rounding="rtne", seed=0):
+def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None, rounding="rtne", seed=0,
+                   groups=(0, 0)):
     """The whole probe for one product; returns the MetricResult (synchronises to read it).
-    rounding: "rtne", or "stochastic_l" / "stochastic_r" / "stochastic_both" with `seed`."""
-    plan = ProbePlan(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed)
+    rounding: "rtne", or "stochastic_l" / "stochastic_r" / "stochastic_both" with `seed`.
+    groups: batch_groups of (L, R) for channel scales shared along the batch (0 = not shared)."""
+    plan = ProbePlan(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed, groups)
     plan.launch(L_op, R_op, stream)
     return plan.result()
 

@@ -139,6 +139,9 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
   if (!valid_fmt(cfg->fmt_l) || !valid_fmt(cfg->fmt_r) || !valid_gran(cfg->gran_l) || !valid_gran(cfg->gran_r))
     return QM_ERR_INVALID_ARG;
   if (cfg->round & ~(QM_ROUND_STOCHASTIC_L | QM_ROUND_STOCHASTIC_R)) return QM_ERR_INVALID_ARG;
+  if (cfg->batch_groups_l < 0 || cfg->batch_groups_r < 0) return QM_ERR_INVALID_ARG;
+  if ((cfg->batch_groups_l && L->batch % cfg->batch_groups_l) || (cfg->batch_groups_r && R->batch % cfg->batch_groups_r))
+    return QM_ERR_INVALID_ARG;
   if (cfg->ref != QM_REF_BF16_FP32ACC && cfg->ref != QM_REF_FP32) return QM_ERR_INVALID_ARG;
   if (L->c != R->c || L->batch != R->batch) return QM_ERR_INVALID_ARG;
   if ((cfg->fmt_l == QM_FMT_INT8) != (cfg->fmt_r == QM_FMT_INT8)) return QM_ERR_UNSUPPORTED;
@@ -152,11 +155,16 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
 // scale + quantize of one operand inside the probe
 qm_status prepare_operand(const View& x, int fmt, int gran, uint32_t* amax, float* delta, uint8_t* codes,
                           void* abs_copy, void* kmaj_copy, uint32_t* err_word, const StochasticDraw* draw,
-                          cudaStream_t s) {
-  if (!draw && gran == QM_GRAN_CHANNEL && x.c_contig())
+                          int batch_groups, cudaStream_t s) {
+  const bool shared = gran == QM_GRAN_CHANNEL && batch_groups > 0 && batch_groups < x.batch;
+  if (!draw && !shared && gran == QM_GRAN_CHANNEL && x.c_contig())
     return launch_scale_quantize_rows(x, fmt, delta, codes, abs_copy, err_word, s);
   qm_status st = launch_absmax(x, gran, amax, s);
   if (st != QM_OK) return st;
+  if (shared) {
+    st = launch_share_amax(amax, x.batch, batch_groups, x.nc, s);
+    if (st != QM_OK) return st;
+  }
   // the quantize kernel turns max|x| into delta itself
   return launch_quantize(x, fmt, gran, reinterpret_cast<const float*>(amax), true, delta, err_word, codes,
                          abs_copy, kmaj_copy, s, draw);
@@ -181,6 +189,24 @@ qm_status qm_scale(const qm_operand* x, int32_t fmt, int32_t gran, float* delta,
   QM_CUDA_OK(cudaMemsetAsync(delta, 0, sizeof(float) * n, s));
   st = launch_absmax(v, gran, reinterpret_cast<uint32_t*>(delta), s);
   if (st != QM_OK) return st;
+  return launch_finalize_delta(delta, n, fmt, nullptr, s);
+}
+
+qm_status qm_scale_shared(const qm_operand* x, int32_t fmt, int32_t batch_groups, float* delta, void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (!valid_fmt(fmt) || !delta) return QM_ERR_INVALID_ARG;
+  if (batch_groups < 1 || v.batch % batch_groups) return QM_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t n = v.nc * v.batch;
+  QM_CUDA_OK(cudaMemsetAsync(delta, 0, sizeof(float) * n, s));
+  st = launch_absmax(v, QM_GRAN_CHANNEL, reinterpret_cast<uint32_t*>(delta), s);
+  if (st != QM_OK) return st;
+  if (batch_groups < v.batch) {
+    st = launch_share_amax(reinterpret_cast<uint32_t*>(delta), v.batch, batch_groups, v.nc, s);
+    if (st != QM_OK) return st;
+  }
   return launch_finalize_delta(delta, n, fmt, nullptr, s);
 }
 
@@ -301,10 +327,10 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
   const StochasticDraw draw_l{cfg->seed, 0u}, draw_r{cfg->seed, 1u};
   st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err,
-                       (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, s);
+                       (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, cfg->batch_groups_l, s);
   if (st != QM_OK) return st;
   st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err,
-                       (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, s);
+                       (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, cfg->batch_groups_r, s);
   if (st != QM_OK) return st;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {

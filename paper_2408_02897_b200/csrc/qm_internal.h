@@ -68,6 +68,9 @@ void profile_events(cudaEvent_t* start, cudaEvent_t* stop);
 // amax: uint32 buffer (1 or batch*nc entries) that must be zero on entry; on exit it holds
 // the bit pattern of max|x| per group.
 qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream_t s);
+// In place on the per-(batch element, channel) maxima of launch_absmax: entries of batch elements
+// b with equal b % groups are replaced by their common maximum (scales shared along the batch).
+qm_status launch_share_amax(uint32_t* amax_bits, int64_t batch, int64_t groups, int64_t nc, cudaStream_t s);
 // In place: bit pattern of max|x| -> delta = max|x| / qmax (1 where max|x| == 0).
 // err_word (optional): gets QM_DEVERR_NONFINITE or-ed in when a group max is NaN/Inf.
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s);

@@ -135,6 +135,19 @@ absmax_cols_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, 
   if (col < nc && m) atomicMax(amax + b * nc + col, m);
 }
 
+// Per-channel maxima shared along the batch: batch element b belongs to group b % groups, and
+// every (group, channel) entry becomes the maximum over the group's batch elements (integer max
+// of the order-preserving bit patterns), written back to each of them.  One thread per entry.
+__global__ void share_amax_kernel(uint32_t* __restrict__ amax, int64_t batch, int64_t groups, int64_t nc) {
+  pdl_prologue();
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= groups * nc) return;
+  const int64_t g = i / nc, ch = i - g * nc;
+  uint32_t m = 0;
+  for (int64_t b = g; b < batch; b += groups) m = max(m, amax[b * nc + ch]);
+  for (int64_t b = g; b < batch; b += groups) amax[b * nc + ch] = m;
+}
+
 __global__ void finalize_delta_kernel(float* __restrict__ delta, int64_t n, float qmax,
                                       uint32_t* __restrict__ err_word) {
   pdl_prologue();
@@ -671,6 +684,14 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
 qm_status launch_absmax(const View& x, int gran, uint32_t* amax_bits, cudaStream_t s) {
   return x.dtype == QM_DT_BF16 ? absmax_t<__nv_bfloat16>(x, gran, amax_bits, s)
                                : absmax_t<float>(x, gran, amax_bits, s);
+}
+
+qm_status launch_share_amax(uint32_t* amax_bits, int64_t batch, int64_t groups, int64_t nc, cudaStream_t s) {
+  const int64_t n = groups * nc;
+  launch_pdl(share_amax_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, s, amax_bits, batch, groups, nc);
+  count_launch();
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
 }
 
 qm_status launch_finalize_delta(float* delta, int64_t n, int fmt, uint32_t* err_word, cudaStream_t s) {
