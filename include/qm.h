@@ -257,6 +257,22 @@ qm_status qm_probe_layer(const qm_operand* L, const qm_operand* R, const qm_prob
                          qm_metric_result* out, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Two formats in one pass.  The paper sweeps the 8-bit formats over the same
+ * tensors (Table 1): the reference product L.R and the denominator product
+ * |L|.|R| do not depend on the format, so this call computes them once and keeps
+ * one 8-bit accumulator per format beside them.  cfg_a and cfg_b must agree in
+ * everything except fmt_l / fmt_r, use QM_REF_BF16_FP32ACC, and at most one of
+ * them may be the INT8 format.  out[0] receives the record of cfg_a, out[1]
+ * that of cfg_b; each equals what qm_probe_layer gives for that configuration.
+ * `ws`: at least qm_workspace_bytes2(...) bytes, otherwise as for qm_probe_layer.
+ */
+size_t qm_workspace_bytes2(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg_a,
+                           const qm_probe_cfg* cfg_b);
+qm_status qm_probe_layer2(const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg_a,
+                          const qm_probe_cfg* cfg_b, qm_metric_result* out, void* ws, size_t ws_bytes,
+                          void* stream);
+
+/*
  * Same probe for operands that live in HOST memory (pinned memory makes the
  * copies asynchronous).  L->data and R->data are host pointers; l_stage and
  * r_stage are device buffers the caller owns, large enough for the operands'

@@ -107,6 +107,8 @@ def lib():
             "qm_metric": (I32, [P, P, P, I64, P, P, SZ, P]),
             "qm_workspace_bytes": (SZ, [OP, OP, C.POINTER(ProbeCfg)]),
             "qm_probe_layer": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, SZ, P]),
+            "qm_workspace_bytes2": (SZ, [OP, OP, C.POINTER(ProbeCfg), C.POINTER(ProbeCfg)]),
+            "qm_probe_layer2": (I32, [OP, OP, C.POINTER(ProbeCfg), C.POINTER(ProbeCfg), P, P, SZ, P]),
             "qm_operand_span_bytes": (SZ, [OP]),
             "qm_probe_layer_host": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, C.POINTER(MetricResult), P, P, SZ, P]),
             "qm_stats_workspace_bytes": (SZ, []),
@@ -325,6 +327,34 @@ class ProbePlan:
 
     def result(self):
         return _read_result(self.out)
+
+
+class ProbePlan2:
+    """Workspace and the two result records of a two-format probe (qm_probe_layer2).
+    fmts_a / fmts_b are (fmt_l, fmt_r) of the two configurations; everything else is shared."""
+
+    def __init__(self, L_op, R_op, fmts_a, fmts_b, gran_l, gran_r, rounding="rtne", seed=0, groups=(0, 0)):
+        self.cfg_a = _cfg(fmts_a[0], fmts_a[1], gran_l, gran_r, "bf16", rounding, seed, groups)
+        self.cfg_b = _cfg(fmts_b[0], fmts_b[1], gran_l, gran_r, "bf16", rounding, seed, groups)
+        self.ws_bytes = lib().qm_workspace_bytes2(C.byref(L_op), C.byref(R_op), C.byref(self.cfg_a), C.byref(self.cfg_b))
+        if self.ws_bytes == 0:
+            raise QmError(2, "qm_workspace_bytes2: the two configurations cannot share a pass")
+        self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
+        self.out = torch.zeros(2 * C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
+
+    def launch(self, L_op, R_op, stream=None):
+        _check(lib().qm_probe_layer2(C.byref(L_op), C.byref(R_op), C.byref(self.cfg_a), C.byref(self.cfg_b),
+                                     _ptr(self.out), _ptr(self.ws), self.ws_bytes, _stream(stream)), "qm_probe_layer2")
+
+    def results(self):
+        return _records(self.out.cpu().numpy().tobytes(), 2)
+
+
+def qm_probe_layer2(L_op, R_op, fmts_a, fmts_b, gran_l, gran_r, stream=None, rounding="rtne", seed=0, groups=(0, 0)):
+    """Both formats' records of one product from a single pass; returns [MetricResult, MetricResult]."""
+    plan = ProbePlan2(L_op, R_op, fmts_a, fmts_b, gran_l, gran_r, rounding, seed, groups)
+    plan.launch(L_op, R_op, stream)
+    return plan.results()
 
 
 def qm_probe_layer(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", stream=None, rounding="rtne", seed=0,

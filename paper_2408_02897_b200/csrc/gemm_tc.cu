@@ -49,7 +49,7 @@ constexpr uint32_t kBLp = kHalfN * kBlockK;                       //  4 KB
 constexpr int kMaxStages = 8;
 constexpr int kRefAhead = 2;               // k-blocks of reference MMAs issued before the hand-back wait
 
-enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2 };
+enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2, kProbe2 = 3 };
 
 // Stage layout: left-operand tiles first (L, |L|, codes), then the right-operand halves.
 template <int MODE> struct Cfg;
@@ -58,6 +58,16 @@ template <> struct Cfg<kProbe> {
   static constexpr uint32_t kOffL = 0, kOffLa = kABf16, kOffCl = 2 * kABf16;
   static constexpr uint32_t kOffR = 2 * kABf16 + kALp, kOffRa = kOffR + kBBf16, kOffCr = kOffRa + kBBf16;
   static constexpr uint32_t kStageBytes = kOffCr + kBLp;          // 60 KB
+  static constexpr uint32_t kTmemCols = 512;
+};
+// Two 8-bit formats in one pass: the reference and denominator products are shared, each format
+// has its own code tiles and its own accumulator.
+template <> struct Cfg<kProbe2> {
+  static constexpr int kStages = 3;
+  static constexpr uint32_t kOffL = 0, kOffLa = kABf16, kOffCl = 2 * kABf16, kOffCl2 = kOffCl + kALp;
+  static constexpr uint32_t kOffR = kOffCl2 + kALp, kOffRa = kOffR + kBBf16, kOffCr = kOffRa + kBBf16;
+  static constexpr uint32_t kOffCr2 = kOffCr + kBLp;
+  static constexpr uint32_t kStageBytes = kOffCr2 + kBLp;         // 72 KB
   static constexpr uint32_t kTmemCols = 512;
 };
 template <> struct Cfg<kLpOnly> {
@@ -86,6 +96,10 @@ struct KernelArgs {
   uint64_t count;                        // Probe: batch * M * N
   uint32_t* err_word;
   uint32_t idesc_lp;                     // instruction descriptor of the 8-bit MMA
+  // Probe2: scales and descriptor of the second format (granularities are shared); its record
+  // is result[1] and its per-CTA records follow the first format's gridDim.x records
+  const float* dl2; const float* dr2;
+  uint32_t idesc_lp2;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -270,7 +284,8 @@ struct Shared {
   uint32_t is_last;
   uint32_t pad;
   float delta_r[2][kBlockN];
-  double red[5][kEpiWarps];
+  float delta_r2[2][kBlockN];    // Probe2: column scales of the second format
+  double red[10][kEpiWarps];
 };
 
 // Named barrier 1 over the 256 epilogue threads, returning the OR of `flag` over all of them.
@@ -383,12 +398,15 @@ __device__ __forceinline__ void stats16(const uint32_t* rc, const uint32_t* rd, 
   }
 }
 
-template <int MODE, int LPKIND>
+template <int MODE, int LPKIND, int LPKIND2>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUtensorMap map_r,
           const __grid_constant__ CUtensorMap map_la, const __grid_constant__ CUtensorMap map_ra,
           const __grid_constant__ CUtensorMap map_cl, const __grid_constant__ CUtensorMap map_cr,
+          const __grid_constant__ CUtensorMap map_cl2, const __grid_constant__ CUtensorMap map_cr2,
           const KernelArgs a) {
+  constexpr bool kAnyProbe = MODE == kProbe || MODE == kProbe2;
+  constexpr int kFormats = MODE == kProbe2 ? 2 : 1;
   using C = Cfg<MODE>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -403,9 +421,9 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   const int num_kb = (int)((a.K + kBlockK - 1) / kBlockK);
   volatile uint32_t* abort_flag = &sh->abort_flag;
 
-  if (warp == 0 && lane < 6) {
+  if (warp == 0 && lane < 8) {
     // fetch the tensor maps into the descriptor cache while the CTA sets itself up
-    const CUtensorMap* maps[6] = {&map_l, &map_r, &map_la, &map_ra, &map_cl, &map_cr};
+    const CUtensorMap* maps[8] = {&map_l, &map_r, &map_la, &map_ra, &map_cl, &map_cr, &map_cl2, &map_cr2};
     asm volatile("prefetch.tensormap [%0];" ::"l"(maps[lane]) : "memory");
   }
   if (threadIdx.x == 0) {
@@ -454,17 +472,21 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
           const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
           const int k0 = kb * kBlockK;
-          if (MODE == kProbe || MODE == kRefOnly) {
+          if (kAnyProbe || MODE == kRefOnly) {
             tma_load_3d(base + C::kOffL, &map_l, bar, k0, r0, tc.b);
             tma_load_3d(base + C::kOffR, &map_r, bar, k0, c0, tc.b);
           }
-          if (MODE == kProbe) {
+          if (kAnyProbe) {
             tma_load_3d(base + C::kOffLa, &map_la, bar, k0, r0, tc.b);
             tma_load_3d(base + C::kOffRa, &map_ra, bar, k0, c0, tc.b);
           }
-          if (MODE == kProbe || MODE == kLpOnly) {
+          if (kAnyProbe || MODE == kLpOnly) {
             tma_load_3d(base + C::kOffCl, &map_cl, bar, k0, r0, tc.b);
             tma_load_3d(base + C::kOffCr, &map_cr, bar, k0, c0, tc.b);
+          }
+          if constexpr (MODE == kProbe2) {
+            tma_load_3d(base + C::kOffCl2, &map_cl2, bar, k0, r0, tc.b);
+            tma_load_3d(base + C::kOffCr2, &map_cr2, bar, k0, c0, tc.b);
           }
         }
       }
@@ -485,8 +507,8 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
         // and hand them back; the denominator and 8-bit MMAs of those k-blocks follow that
         // signal.
         const uint32_t col_ref = MODE == kProbe ? ((3 * it) & 3) * 128u : 0u;
-        const uint32_t col_den = ((3 * it + 1) & 3) * 128u;
-        const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : 0u;
+        const uint32_t col_den = MODE == kProbe ? ((3 * it + 1) & 3) * 128u : 128u;
+        const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : (MODE == kProbe2 ? 256u : 0u);
         auto issue_ref = [&](uint32_t base, int kb) {
           const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
 #pragma unroll
@@ -505,7 +527,45 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
             mma_pair<LPKIND>(tmem_base + col_lp, dl + 2 * k, dr + 2 * k, a.idesc_lp, (kb | k) != 0, lead);
         };
+        // Probe2: the second format's accumulator takes the fourth block (columns 384..511), so
+        // nothing rotates.  The reference and denominator blocks come back when both epilogues
+        // have copied them out (tmem_empty), the two 8-bit blocks when they have finished the tile
+        // (lp_done); the reference and denominator MMAs of as many k-blocks as there are stages
+        // are therefore issued between the two signals.
+        auto issue_lp2 = [&](uint32_t base, int kb) {
+          if constexpr (MODE == kProbe2) {
+            const uint64_t dl = smem_desc(base + C::kOffCl2, 64), dr = smem_desc(base + C::kOffCr2, 64);
+#pragma unroll
+            for (int k = 0; k < kBlockK / 32; ++k)
+              mma_pair<LPKIND2>(tmem_base + 384u, dl + 2 * k, dr + 2 * k, a.idesc_lp2, (kb | k) != 0, lead);
+          }
+        };
         int kb = 0;
+        if (MODE == kProbe2) {
+          if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
+          tc_fence_after();
+          const int n_ahead = num_kb < kStages ? num_kb : kStages;
+          for (int j = 0; j < n_ahead && ok; ++j) {
+            const int s = (g + j) % kStages;
+            if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, a.err_word)) ok = false;
+            tc_fence_after();
+            if (ok) {
+              const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+              issue_ref(base, j);
+              issue_den(base, j);
+            }
+          }
+          if (!ok) break;
+          if (it > 0 && !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, a.err_word)) break;
+          tc_fence_after();
+          for (; kb < n_ahead; ++kb, ++g) {
+            const int s = g % kStages;
+            const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+            issue_lp(base, kb);
+            issue_lp2(base, kb);
+            tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+          }
+        }
         if (MODE == kProbe) {
           const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
           for (int j = 0; j < n_ahead && ok; ++j) {
@@ -516,7 +576,9 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           }
           if (!ok) break;
         }
-        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word)) break;
+        if (MODE != kProbe2 && it > 0 &&
+            !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word))
+          break;
         tc_fence_after();
         if (MODE == kProbe) {
           const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
@@ -534,9 +596,10 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           if (!mbar_wait_warp(smem_u32(&sh->full[s]), use & 1, abort_flag, a.err_word)) { ok = false; break; }
           tc_fence_after();
           const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-          if (MODE == kProbe || MODE == kRefOnly) issue_ref(base, kb);
-          if (MODE == kProbe) issue_den(base, kb);
-          if (MODE == kProbe || MODE == kLpOnly) issue_lp(base, kb);
+          if (kAnyProbe || MODE == kRefOnly) issue_ref(base, kb);
+          if (kAnyProbe) issue_den(base, kb);
+          if (kAnyProbe || MODE == kLpOnly) issue_lp(base, kb);
+          issue_lp2(base, kb);
           tc_commit_pair(smem_u32(&sh->empty[s]), lead);        // frees the stage in both CTAs
         }
         // The next tile's reference block is this tile's free one, last read by the epilogue of
@@ -557,26 +620,85 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
     const float dr_tensor = (MODE != kRefOnly && !a.pc_r) ? __ldg(a.dr) : 1.f;
     const bool per_col = MODE != kRefOnly && a.pc_r;
     const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
-    double sbe = 0, mbe = 0, sd2 = 0, sr2 = 0, sn2 = 0;
+    double acc[kFormats][5];                       // per format: sum BE, max BE, sum diff^2, sum C^2, sum D^2
+#pragma unroll
+    for (int f = 0; f < kFormats; ++f)
+#pragma unroll
+      for (int i = 0; i < 5; ++i) acc[f][i] = 0.0;
+    [[maybe_unused]] const float dl_tensor2 = (MODE == kProbe2 && !a.pc_l) ? __ldg(a.dl2) : 1.f;
+    [[maybe_unused]] const float dr_tensor2 = (MODE == kProbe2 && !a.pc_r) ? __ldg(a.dr2) : 1.f;
+    auto add_stats = [&](int f, const Stats2& st) {
+      float x0, x1;
+      unpack2(st.be, x0, x1); acc[f][0] += (double)x0 + (double)x1;
+      unpack2(st.d2, x0, x1); acc[f][2] += (double)x0 + (double)x1;
+      unpack2(st.r2, x0, x1); acc[f][3] += (double)x0 + (double)x1;
+      unpack2(st.n2, x0, x1); acc[f][4] += (double)x0 + (double)x1;
+      acc[f][1] = fmax(acc[f][1], (double)st.mx);
+    };
     uint32_t it = 0;
     for (int t = pair; t < a.num_tiles; t += num_pairs, ++it) {
       const TileCoord tc = tile_coord(t, a);
       float* dr_s = sh->delta_r[it & 1];
+      [[maybe_unused]] float* dr_s2 = sh->delta_r2[it & 1];
       if (per_col && et < kBlockN) {
         const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
         dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
+        if (MODE == kProbe2) dr_s2[et] = col < a.N ? __ldg(a.dr2 + (int64_t)tc.b * a.N + col) : 0.f;
       }
       const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
       const bool row_ok = row < a.M;
       float dlv = dl_tensor;
       if (MODE != kRefOnly && a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
+      [[maybe_unused]] float dlv2 = dl_tensor2;
+      if (MODE == kProbe2 && a.pc_l) dlv2 = row_ok ? __ldg(a.dl2 + (int64_t)tc.b * a.M + row) : 0.f;
 
       const bool ok = mbar_wait(smem_u32(&sh->tmem_full), it & 1, abort_flag, a.err_word);
       // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
       if (epi_barrier_any(!ok)) break;
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      if (MODE == kProbe) {
+      if (MODE == kProbe2) {
+        // Fixed blocks: reference 0, denominator 128, first format 256, second format 384.  Copy
+        // this warp's 64 reference and denominator columns into registers and hand those two
+        // blocks back (the next tile's reference and denominator MMAs start), walk both 8-bit
+        // blocks in chunks of 16 columns, then report the tile finished (lp_done).
+        const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;
+        uint32_t rc[64], rd[64], rq[16];
+        tmem_ld32(lane_addr + 0u + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
+        tmem_ld32(lane_addr + 0u + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
+        tmem_ld32(lane_addr + 128u + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
+        tmem_ld32(lane_addr + 128u + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+        Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f}, st2{0ull, 0ull, 0ull, 0ull, 0.f};
+        const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
+        const uint64_t ndl2b = pack2(-dlv2, -dlv2), drt2b = pack2(dr_tensor2, dr_tensor2);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int cc0 = h * 64 + c * 16;
+          const int64_t col0 = colw + c * 16;
+          if (col0 < a.N) {                       // uniform across the warp
+            const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
+            tmem_ld16(lane_addr + 256u + cc0, rq);
+            tmem_ld_wait();
+            if (n_live == 16) stats16<LPKIND, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
+            else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
+            tmem_ld16(lane_addr + 384u + cc0, rq);
+            tmem_ld_wait();
+            if (n_live == 16) stats16<LPKIND2, false>(&rc[c * 16], &rd[c * 16], rq, ndl2b, dr_s2 + cc0, per_col, drt2b, 16, st2);
+            else stats16<LPKIND2, true>(&rc[c * 16], &rd[c * 16], rq, ndl2b, dr_s2 + cc0, per_col, drt2b, n_live, st2);
+          }
+        }
+        if (row_ok) {
+          add_stats(0, st);
+          if constexpr (kFormats == 2) add_stats(1, st2);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
+      } else if (MODE == kProbe) {
         // Accumulator blocks of this tile (they rotate so that the next tile's MMAs never wait
         // for this arithmetic): copy this warp's 64 columns of the reference and denominator
         // blocks into registers, hand those two blocks back to the MMA lane, then walk the
@@ -607,14 +729,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
           }
         }
-        if (row_ok) {
-          float x0, x1;
-          unpack2(st.be, x0, x1); sbe += (double)x0 + (double)x1;
-          unpack2(st.d2, x0, x1); sd2 += (double)x0 + (double)x1;
-          unpack2(st.r2, x0, x1); sr2 += (double)x0 + (double)x1;
-          unpack2(st.n2, x0, x1); sn2 += (double)x0 + (double)x1;
-          mbe = fmax(mbe, (double)st.mx);
-        }
+        if (row_ok) add_stats(0, st);
         tc_fence_before();                        // the 8-bit block's loads are complete as well
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
@@ -646,35 +761,38 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           }
         }
       }
-      if (MODE != kProbe) {
+      if (!kAnyProbe) {
         // this warp has finished reading the accumulator of the tile: tell the leader's MMA lane
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
       }
     }
-    if (MODE == kProbe) {
+    if (kAnyProbe) {
+      // per format: warp sums -> CTA record -> (last CTA) fixed-order sum of all records
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        sbe += __shfl_xor_sync(0xffffffffu, sbe, o);
-        mbe = fmax(mbe, __shfl_xor_sync(0xffffffffu, mbe, o));
-        sd2 += __shfl_xor_sync(0xffffffffu, sd2, o);
-        sr2 += __shfl_xor_sync(0xffffffffu, sr2, o);
-        sn2 += __shfl_xor_sync(0xffffffffu, sn2, o);
-      }
-      if (lane == 0) {
-        sh->red[0][warp - 2] = sbe; sh->red[1][warp - 2] = mbe; sh->red[2][warp - 2] = sd2;
-        sh->red[3][warp - 2] = sr2; sh->red[4][warp - 2] = sn2;
+      for (int f = 0; f < kFormats; ++f) {
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+          double x = acc[f][i];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const double y = __shfl_xor_sync(0xffffffffu, x, o);
+            x = i == 1 ? fmax(x, y) : x + y;
+          }
+          if (lane == 0) sh->red[f * 5 + i][warp - 2] = x;
+        }
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (et == 0) {
-        double r[5] = {0, 0, 0, 0, 0};
-        for (int i = 0; i < kEpiWarps; ++i) {
-          r[0] += sh->red[0][i]; r[1] = fmax(r[1], sh->red[1][i]); r[2] += sh->red[2][i];
-          r[3] += sh->red[3][i]; r[4] += sh->red[4][i];
+        for (int f = 0; f < kFormats; ++f) {
+          double* rec = a.partials + ((int64_t)f * gridDim.x + blockIdx.x) * kPartialDoubles;
+          for (int i = 0; i < 5; ++i) {
+            double x = 0.0;
+            for (int w = 0; w < kEpiWarps; ++w) x = i == 1 ? fmax(x, sh->red[f * 5 + i][w]) : x + sh->red[f * 5 + i][w];
+            __stcg(rec + i, x);
+          }
         }
-        double* rec = a.partials + (int64_t)blockIdx.x * kPartialDoubles;
-        for (int i = 0; i < 5; ++i) __stcg(rec + i, r[i]);
         __threadfence();
         const uint32_t prev = atomicAdd(a.done_counter, 1u);
         sh->is_last = prev == gridDim.x - 1 ? 1u : 0u;
@@ -683,26 +801,29 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       if (sh->is_last && warp == 2) {
         // last CTA: every record is visible; fixed-order sum (lane l takes records l, l+32, ...)
         __threadfence();
-        double r[5] = {0, 0, 0, 0, 0};
-        for (int i = lane; i < (int)gridDim.x; i += 32) {
-          const double* rec = a.partials + (int64_t)i * kPartialDoubles;
-          r[0] += __ldcg(rec); r[1] = fmax(r[1], __ldcg(rec + 1)); r[2] += __ldcg(rec + 2);
-          r[3] += __ldcg(rec + 3); r[4] += __ldcg(rec + 4);
-        }
+        for (int f = 0; f < kFormats; ++f) {
+          double r[5] = {0, 0, 0, 0, 0};
+          for (int i = lane; i < (int)gridDim.x; i += 32) {
+            const double* rec = a.partials + ((int64_t)f * gridDim.x + i) * kPartialDoubles;
+            r[0] += __ldcg(rec); r[1] = fmax(r[1], __ldcg(rec + 1)); r[2] += __ldcg(rec + 2);
+            r[3] += __ldcg(rec + 3); r[4] += __ldcg(rec + 4);
+          }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          r[0] += __shfl_xor_sync(0xffffffffu, r[0], o);
-          r[1] = fmax(r[1], __shfl_xor_sync(0xffffffffu, r[1], o));
-          r[2] += __shfl_xor_sync(0xffffffffu, r[2], o);
-          r[3] += __shfl_xor_sync(0xffffffffu, r[3], o);
-          r[4] += __shfl_xor_sync(0xffffffffu, r[4], o);
-        }
-        if (lane == 0) {
-          a.result->sum_be = r[0]; a.result->max_be = r[1]; a.result->sum_diff2 = r[2];
-          a.result->sum_ref2 = r[3]; a.result->sum_den2 = r[4];
-          a.result->count = a.count;
-          a.result->device_error = a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u;
-          a.result->reserved = 0;
+          for (int o = 16; o > 0; o >>= 1) {
+            r[0] += __shfl_xor_sync(0xffffffffu, r[0], o);
+            r[1] = fmax(r[1], __shfl_xor_sync(0xffffffffu, r[1], o));
+            r[2] += __shfl_xor_sync(0xffffffffu, r[2], o);
+            r[3] += __shfl_xor_sync(0xffffffffu, r[3], o);
+            r[4] += __shfl_xor_sync(0xffffffffu, r[4], o);
+          }
+          if (lane == 0) {
+            qm_metric_result* out = a.result + f;
+            out->sum_be = r[0]; out->max_be = r[1]; out->sum_diff2 = r[2];
+            out->sum_ref2 = r[3]; out->sum_den2 = r[4];
+            out->count = a.count;
+            out->device_error = a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u;
+            out->reserved = 0;
+          }
         }
       }
     }
@@ -799,9 +920,10 @@ int grid_size(GemmShape g) {
   return 2 * (int)(tiles < pairs ? tiles : pairs);
 }
 
-template <int MODE, int LPKIND>
+// maps: eight tensor maps (L, R, |L|, |R|, codes L, codes R, second-format codes L, R).
+template <int MODE, int LPKIND, int LPKIND2 = LPKIND>
 qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cudaStream_t s) {
-  auto kern = tc_kernel<MODE, LPKIND>;
+  auto kern = tc_kernel<MODE, LPKIND, LPKIND2>;
   static bool attr_done = false;     // per instantiation
   if (!attr_done) {
     QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<MODE>()));
@@ -836,9 +958,10 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  if (MODE == kProbe) profile_events(&ev0, &ev1);
+  if (MODE == kProbe || MODE == kProbe2) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
-  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka));
+  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6], maps[7],
+                                ka));
   if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
   count_launch();
   return QM_OK;
@@ -846,13 +969,13 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
 
 }  // namespace
 
-int tc_probe_records(GemmShape g) { return grid_size(g); }
+int tc_probe_records(GemmShape g) { return grid_size(g); }   // per format
 
 qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   if (!shape_ok(p.g)) return QM_ERR_UNSUPPORTED;
   const GemmShape g = p.g;
   const int64_t ldc = qm_code_ld(g.K);
-  CUtensorMap maps[6];
+  CUtensorMap maps[8];
   bool ok = make_map(&maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
             make_map(&maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
             make_map(&maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
@@ -860,12 +983,27 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
             make_map(&maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
             make_map(&maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
+  const bool two = p.cl2 != nullptr;
+  if (two) {
+    ok = make_map(&maps[6], p.cl2, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+         make_map(&maps[7], p.cr2, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
+    if (!ok) return QM_ERR_CUDA;
+  } else {
+    maps[6] = maps[4]; maps[7] = maps[5];
+  }
   KernelArgs ka{};
   fill_tiles(&ka, g);
   ka.dl = p.dl; ka.pc_l = p.gran_l == QM_GRAN_CHANNEL; ka.dr = p.dr; ka.pc_r = p.gran_r == QM_GRAN_CHANNEL;
   ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
   ka.count = (uint64_t)(g.M * g.N * g.batch);
   ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+  if (two) {
+    // the first format is an FP8 one (the caller orders them), the second FP8 or INT8
+    if (p.fmt_l == QM_FMT_INT8) return QM_ERR_UNSUPPORTED;
+    ka.dl2 = p.dl2; ka.dr2 = p.dr2; ka.idesc_lp2 = lp_idesc(p.fmt_l2, p.fmt_r2);
+    return p.fmt_l2 == QM_FMT_INT8 ? launch<kProbe2, kKindF8, kKindI8>(maps, ka, g, s)
+                                   : launch<kProbe2, kKindF8, kKindF8>(maps, ka, g, s);
+  }
   return p.fmt_l == QM_FMT_INT8 ? launch<kProbe, kKindI8>(maps, ka, g, s)
                                 : launch<kProbe, kKindF8>(maps, ka, g, s);
 }
@@ -875,11 +1013,11 @@ qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int g
                             float* out_descaled, void* out_raw, uint32_t* err_word, cudaStream_t s) {
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
   const int64_t ldc = qm_code_ld(g.K);
-  CUtensorMap maps[6];
+  CUtensorMap maps[8];
   bool ok = make_map(&maps[4], cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
             make_map(&maps[5], cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
-  maps[0] = maps[1] = maps[2] = maps[3] = maps[4];
+  maps[0] = maps[1] = maps[2] = maps[3] = maps[6] = maps[7] = maps[4];
   KernelArgs ka{};
   fill_tiles(&ka, g);
   ka.dl = dl; ka.pc_l = gran_l == QM_GRAN_CHANNEL; ka.dr = dr; ka.pc_r = gran_r == QM_GRAN_CHANNEL;
@@ -892,11 +1030,11 @@ qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int g
 qm_status launch_tc_gemm_ref(const void* l, const void* r, GemmShape g, float* out, uint32_t* err_word,
                              cudaStream_t s) {
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
-  CUtensorMap maps[6];
+  CUtensorMap maps[8];
   bool ok = make_map(&maps[0], l, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
             make_map(&maps[1], r, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K);
   if (!ok) return QM_ERR_CUDA;
-  maps[2] = maps[3] = maps[4] = maps[5] = maps[0];
+  maps[2] = maps[3] = maps[4] = maps[5] = maps[6] = maps[7] = maps[0];
   KernelArgs ka{};
   fill_tiles(&ka, g);
   ka.out_descaled = out; ka.err_word = err_word;

@@ -350,6 +350,133 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   return launch_metric_finalize(part, w.n_part, (uint64_t)(g.M * g.N * g.batch), err, out, s);
 }
 
+// ---- two formats in one pass -------------------------------------------------------------------
+}  // extern "C"
+namespace {
+struct Workspace2 {
+  Workspace a;                 // everything of the first format's probe
+  size_t off_dl2, off_dr2, off_cl2, off_cr2, off_part2, total;
+};
+// Orders the two configurations so that an FP8 one comes first; returns false when they cannot
+// share a pass.
+bool order2(const qm_probe_cfg* ca, const qm_probe_cfg* cb, const qm_probe_cfg** first, const qm_probe_cfg** second,
+            bool* swapped) {
+  if (!ca || !cb) return false;
+  if (ca->gran_l != cb->gran_l || ca->gran_r != cb->gran_r || ca->round != cb->round || ca->seed != cb->seed ||
+      ca->batch_groups_l != cb->batch_groups_l || ca->batch_groups_r != cb->batch_groups_r)
+    return false;
+  if (ca->ref != QM_REF_BF16_FP32ACC || cb->ref != QM_REF_BF16_FP32ACC) return false;
+  const bool a_int = ca->fmt_l == QM_FMT_INT8, b_int = cb->fmt_l == QM_FMT_INT8;
+  if (a_int && b_int) return false;
+  *swapped = a_int;
+  *first = a_int ? cb : ca;
+  *second = a_int ? ca : cb;
+  return true;
+}
+Workspace2 plan2(const View& L, const View& R, const qm_probe_cfg& first) {
+  Workspace2 w{};
+  w.a = plan(L, R, first);
+  size_t o = w.a.total;
+  auto take = [&](size_t bytes) { size_t at = o; o += align256(bytes); return at; };
+  w.off_dl2 = take(sizeof(float) * delta_count(L, first.gran_l));
+  w.off_dr2 = take(sizeof(float) * delta_count(R, first.gran_r));
+  const int64_t ldc = qm_code_ld(L.c);
+  w.off_cl2 = take((size_t)(L.batch * L.nc * ldc));
+  w.off_cr2 = take((size_t)(R.batch * R.nc * ldc));
+  w.off_part2 = take(sizeof(double) * kPartialDoubles * 2 * (size_t)w.a.n_part);
+  w.total = o;
+  return w;
+}
+// absmax once, then the codes of both formats from the same maxima
+qm_status prepare_operand2(const View& x, int fmt_a, int fmt_b, int gran, uint32_t* amax, float* delta_a,
+                           float* delta_b, uint8_t* codes_a, uint8_t* codes_b, void* abs_copy, void* kmaj_copy,
+                           uint32_t* err_word, const StochasticDraw* draw, int batch_groups, cudaStream_t s) {
+  qm_status st = launch_absmax(x, gran, amax, s);
+  if (st != QM_OK) return st;
+  if (gran == QM_GRAN_CHANNEL && batch_groups > 0 && batch_groups < x.batch) {
+    st = launch_share_amax(amax, x.batch, batch_groups, x.nc, s);
+    if (st != QM_OK) return st;
+  }
+  st = launch_quantize(x, fmt_a, gran, reinterpret_cast<const float*>(amax), true, delta_a, err_word, codes_a,
+                       abs_copy, kmaj_copy, s, draw);
+  if (st != QM_OK) return st;
+  return launch_quantize(x, fmt_b, gran, reinterpret_cast<const float*>(amax), true, delta_b, err_word, codes_b,
+                         nullptr, nullptr, s, draw);
+}
+}  // namespace
+extern "C" {
+
+size_t qm_workspace_bytes2(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg_a,
+                           const qm_probe_cfg* cfg_b) {
+  const qm_probe_cfg *c1, *c2;
+  bool swapped;
+  View L, R;
+  if (!order2(cfg_a, cfg_b, &c1, &c2, &swapped)) return 0;
+  if (check_probe(Lo, Ro, c1, &L, &R) != QM_OK || check_probe(Lo, Ro, c2, &L, &R) != QM_OK) return 0;
+  return plan2(L, R, *c1).total;
+}
+
+qm_status qm_probe_layer2(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg_a,
+                          const qm_probe_cfg* cfg_b, qm_metric_result* out, void* ws, size_t ws_bytes,
+                          void* stream) {
+  const qm_probe_cfg *c1, *c2;
+  bool swapped;
+  if (!cfg_a || !cfg_b) return QM_ERR_INVALID_ARG;
+  if (!order2(cfg_a, cfg_b, &c1, &c2, &swapped)) return QM_ERR_UNSUPPORTED;
+  View L, R;
+  qm_status st = check_probe(Lo, Ro, c1, &L, &R);
+  if (st == QM_OK) st = check_probe(Lo, Ro, c2, &L, &R);
+  if (st != QM_OK) return st;
+  if (!out || !ws) return QM_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(ws) & 255) return QM_ERR_ALIGNMENT;
+  const Workspace2 w = plan2(L, R, *c1);
+  if (ws_bytes < w.total) return QM_ERR_WORKSPACE_TOO_SMALL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  uint32_t* err = reinterpret_cast<uint32_t*>(base + w.a.off_err);
+  QM_CUDA_OK(cudaMemsetAsync(base, 0, w.a.off_dl, s));      // error word, CTA counter, both max|x| buffers
+  uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.a.off_ml);
+  uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.a.off_mr);
+  float* dl = reinterpret_cast<float*>(base + w.a.off_dl);
+  float* dr = reinterpret_cast<float*>(base + w.a.off_dr);
+  float* dl2 = reinterpret_cast<float*>(base + w.off_dl2);
+  float* dr2 = reinterpret_cast<float*>(base + w.off_dr2);
+  void* kl = L.c_contig() ? nullptr : base + w.a.off_kl;
+  void* kr = R.c_contig() ? nullptr : base + w.a.off_kr;
+  const StochasticDraw draw_l{c1->seed, 0u}, draw_r{c1->seed, 1u};
+  st = prepare_operand2(L, c1->fmt_l, c2->fmt_l, c1->gran_l, ml, dl, dl2, base + w.a.off_cl, base + w.off_cl2,
+                        base + w.a.off_al, kl, err, (c1->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr,
+                        c1->batch_groups_l, s);
+  if (st != QM_OK) return st;
+  st = prepare_operand2(R, c1->fmt_r, c2->fmt_r, c1->gran_r, mr, dr, dr2, base + w.a.off_cr, base + w.off_cr2,
+                        base + w.a.off_ar, kr, err, (c1->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr,
+                        c1->batch_groups_r, s);
+  if (st != QM_OK) return st;
+  TcProbeArgs p{};
+  p.l = kl ? kl : L.data; p.l_ld = kl ? L.c : L.s_nc; p.l_sb = kl ? L.nc * L.c : L.s_b;
+  p.r = kr ? kr : R.data; p.r_ld = kr ? R.c : R.s_nc; p.r_sb = kr ? R.nc * R.c : R.s_b;
+  p.l_abs = base + w.a.off_al; p.r_abs = base + w.a.off_ar;
+  p.cl = base + w.a.off_cl; p.cr = base + w.a.off_cr; p.cl2 = base + w.off_cl2; p.cr2 = base + w.off_cr2;
+  p.fmt_l = c1->fmt_l; p.fmt_r = c1->fmt_r; p.fmt_l2 = c2->fmt_l; p.fmt_r2 = c2->fmt_r;
+  p.dl = dl; p.dr = dr; p.dl2 = dl2; p.dr2 = dr2; p.gran_l = c1->gran_l; p.gran_r = c1->gran_r;
+  p.g = GemmShape{L.nc, R.nc, L.c, L.batch};
+  p.partials = reinterpret_cast<double*>(base + w.off_part2);
+  p.err_word = err; p.done_counter = err + 1;
+  // the kernel writes record 0 for its first format: give it scratch records when the caller's
+  // order is the other way round, and copy them across
+  if (!swapped) {
+    p.result = out;
+    return launch_tc_probe(p, s);
+  }
+  qm_metric_result* tmp = reinterpret_cast<qm_metric_result*>(base + w.a.off_part);   // unused by this path
+  p.result = tmp;
+  st = launch_tc_probe(p, s);
+  if (st != QM_OK) return st;
+  QM_CUDA_OK(cudaMemcpyAsync(out, tmp + 1, sizeof(qm_metric_result), cudaMemcpyDeviceToDevice, s));
+  QM_CUDA_OK(cudaMemcpyAsync(out + 1, tmp, sizeof(qm_metric_result), cudaMemcpyDeviceToDevice, s));
+  return QM_OK;
+}
+
 size_t qm_operand_span_bytes(const qm_operand* x) {
   View v;
   if (to_view(x, &v) != QM_OK) return 0;

@@ -129,6 +129,12 @@ struct TcProbeArgs {
   uint32_t* done_counter;                   // zero on entry; counts finished CTAs
   qm_metric_result* result;                 // written by the last CTA to finish
   uint32_t* err_word;
+  // Two formats in one pass (cl2 != nullptr): codes and scales of the second format, same
+  // granularities; `result` then points at two records and `partials` holds 2 x tc_probe_records.
+  // The first format must be an FP8 one.
+  const uint8_t* cl2 = nullptr; const uint8_t* cr2 = nullptr;
+  int fmt_l2 = 0, fmt_r2 = 0;
+  const float* dl2 = nullptr; const float* dr2 = nullptr;
 };
 int tc_probe_records(GemmShape g);
 qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
