@@ -844,6 +844,219 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
   }
 }
 
+// ------------------------------------------------------------------ plain products on 256 x 256 tiles
+// qm_gemm and qm_gemm_ref on wide outputs.  One accumulator per tile leaves room for 256-column
+// tiles, which halves the MMA instructions and the left-operand traffic per flop, and for two
+// accumulator buffers (2 x 256 tensor-memory columns), so the epilogue of one tile runs under the
+// main loop of the next.  A k-block is 128 BYTES of contraction per row for every operand type
+// (64 bf16 or 128 codes), so all tiles are 128-byte-swizzled 16 KB blocks: a stage is this CTA's
+// 128 left rows and its 128-row half of the right tile, 32 KB, six stages.  Roles, barriers,
+// bounded waits and the exit protocol are those of tc_kernel.
+constexpr int kWideN = 256;
+constexpr int kWideHalfN = 128;
+constexpr int kWideStages = 6;
+constexpr uint32_t kWideTile = 128 * 128;                 // 16 KB
+constexpr uint32_t kWideStageBytes = 2 * kWideTile;
+
+struct SharedWide {
+  uint64_t full[kWideStages];
+  uint64_t empty[kWideStages];
+  uint64_t tmem_full[2];         // per CTA, per accumulator buffer
+  uint64_t tmem_empty[2];        // leader, per accumulator buffer
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+  float delta_r[2][kWideN];
+};
+
+// KIND: kKindF16 (bf16 x bf16 -> fp32 output), kKindF8 / kKindI8 (descaled and/or raw output)
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_gemm_wide_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const KernelArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  SharedWide* sh = reinterpret_cast<SharedWide*>(tiles + (size_t)kWideStages * kWideStageBytes);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  constexpr int kElemsPerBlock = KIND == kKindF16 ? 64 : 128;          // contraction elements per k-block
+  const int num_kb = (int)((a.K + kElemsPerBlock - 1) / kElemsPerBlock);
+  volatile uint32_t* abort_flag = &sh->abort_flag;
+
+  if (warp == 0 && lane < 2) {
+    const CUtensorMap* maps[2] = {&map_a, &map_b};
+    asm volatile("prefetch.tensormap [%0];" ::"l"(maps[lane]) : "memory");
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kWideStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->tmem_full[b]), 1);
+      mbar_init(smem_u32(&sh->tmem_empty[b]), 2 * kEpiWarps);
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&sh->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync();
+  pdl_prologue();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      uint32_t g = 0;
+      bool ok = true;
+      for (int t = pair; t < a.num_tiles && ok; t += num_pairs) {
+        const TileCoord tc = tile_coord(t, a);
+        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;
+        const int c0 = tc.n_tile * kWideN + (int)rank * kWideHalfN;
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kWideStages;
+          const uint32_t use = g / kWideStages;
+          if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, a.err_word)) {
+            ok = false;
+            break;
+          }
+          if (rank == 0) mbar_expect_tx(smem_u32(&sh->full[s]), 2 * kWideStageBytes);
+          const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
+          const uint32_t base = smem_u32(tiles + (size_t)s * kWideStageBytes);
+          tma_load_3d(base, &map_a, bar, kb * kElemsPerBlock, r0, tc.b);
+          tma_load_3d(base + kWideTile, &map_b, bar, kb * kElemsPerBlock, c0, tc.b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA, converged warp)
+    if (rank == 0) {
+      const bool lead = elect_one();
+      const uint32_t idesc = KIND == kKindF16 ? make_idesc(1, 1, 1, kPairM, kWideN) : a.idesc_lp;
+      uint32_t g = 0, it = 0;
+      bool ok = true;
+      for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
+        const uint32_t buf = it & 1;
+        // the buffer was last used by tile it-2: wait until both epilogues have drained it
+        if (it >= 2 && !mbar_wait_warp(smem_u32(&sh->tmem_empty[buf]), ((it >> 1) - 1) & 1, abort_flag, a.err_word))
+          break;
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kWideStages;
+          if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kWideStages) & 1, abort_flag, a.err_word)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t base = smem_u32(tiles + (size_t)s * kWideStageBytes);
+          const uint64_t da = smem_desc(base, 128), db = smem_desc(base + kWideTile, 128);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)             // 32 bytes of contraction per instruction
+            mma_pair<KIND>(tmem_base + buf * kWideN, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0, lead);
+          tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+        }
+        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full[buf]), lead);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int q = warp & 3;
+    const int h = (warp - 2) >> 2;                // which 128-column half of the tile
+    const int et = (warp - 2) * 32 + lane;        // 0..255
+    const float dl_tensor = (KIND != kKindF16 && !a.pc_l) ? __ldg(a.dl) : 1.f;
+    const float dr_tensor = (KIND != kKindF16 && !a.pc_r) ? __ldg(a.dr) : 1.f;
+    const bool per_col = KIND != kKindF16 && a.pc_r;
+    // 16-byte stores need 16-byte aligned rows: output bases aligned and N a multiple of 4
+    const bool vec_ok = (a.N & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out_descaled) & 15) == 0 &&
+                        (reinterpret_cast<uintptr_t>(a.out_raw) & 15) == 0;
+    uint32_t it = 0;
+    for (int t = pair; t < a.num_tiles; t += num_pairs, ++it) {
+      const TileCoord tc = tile_coord(t, a);
+      const uint32_t buf = it & 1;
+      float* dr_s = sh->delta_r[buf];
+      if (per_col) {
+        const int64_t col = (int64_t)tc.n_tile * kWideN + et;
+        dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
+      }
+      const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
+      const bool row_ok = row < a.M;
+      float dlv = dl_tensor;
+      if (KIND != kKindF16 && a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
+      const bool ok = mbar_wait(smem_u32(&sh->tmem_full[buf]), (it >> 1) & 1, abort_flag, a.err_word);
+      if (epi_barrier_any(!ok)) break;            // also publishes delta_r
+      tc_fence_after();
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + buf * kWideN;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        const int cc0 = h * 128 + c * 32;
+        const int64_t col0 = (int64_t)tc.n_tile * kWideN + cc0;
+        if (col0 >= a.N) break;                   // uniform across the warp
+        const int n_live = (int)(a.N - col0 < 32 ? a.N - col0 : 32);
+        uint32_t r[32];
+        tmem_ld32(lane_addr + cc0, r);
+        tmem_ld_wait();
+        if (row_ok) {
+          const int64_t o = ((int64_t)tc.b * a.M + row) * a.N + col0;
+          if (n_live == 32 && vec_ok) {
+            // 128 bytes per thread and chunk: whole lines
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              if (KIND == kKindF16) {
+                *reinterpret_cast<uint4*>(a.out_descaled + o + j) = make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+              } else {
+                if (a.out_raw)
+                  *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(a.out_raw) + o + j) =
+                      make_uint4(r[j], r[j + 1], r[j + 2], r[j + 3]);
+                if (a.out_descaled) {
+                  float4 v;
+                  float* pv = &v.x;
+#pragma unroll
+                  for (int e = 0; e < 4; ++e) {
+                    const float acc = KIND == kKindI8 ? (float)(int)r[j + e] : __uint_as_float(r[j + e]);
+                    pv[e] = acc * (dlv * (per_col ? dr_s[cc0 + j + e] : dr_tensor));
+                  }
+                  *reinterpret_cast<float4*>(a.out_descaled + o + j) = v;
+                }
+              }
+            }
+          } else {
+            for (int j = 0; j < n_live; ++j) {
+              if (KIND == kKindF16) {
+                a.out_descaled[o + j] = __uint_as_float(r[j]);
+              } else {
+                const float acc = KIND == kKindI8 ? (float)(int)r[j] : __uint_as_float(r[j]);
+                if (a.out_descaled) a.out_descaled[o + j] = acc * (dlv * (per_col ? dr_s[cc0 + j] : dr_tensor));
+                if (a.out_raw) reinterpret_cast<uint32_t*>(a.out_raw)[o + j] = r[j];
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->tmem_empty[buf]), 0));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -864,19 +1077,20 @@ EncodeTiledFn encode_fn() {
 
 // Tensor map over [batch][rows][K] with the contracting index contiguous; box = 64 x box_rows x 1,
 // swizzle span = row width of the box (128 bytes for bf16, 64 bytes for codes).
+// wide: 128-byte boxes and swizzle for the codes as well (the 256 x 256 tile kernel).
 bool make_map(CUtensorMap* m, const void* base, bool bf16, int box_rows, int64_t K, int64_t rows, int64_t batch,
-              int64_t ld_elems, int64_t sb_elems) {
+              int64_t ld_elems, int64_t sb_elems, bool wide = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const uint64_t es = bf16 ? 2 : 1;
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
   cuuint64_t sb = batch > 1 ? (cuuint64_t)sb_elems * es : (cuuint64_t)rows * ld_elems * es;
   cuuint64_t strides[2] = {(cuuint64_t)ld_elems * es, sb};
-  cuuint32_t box[3] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows, 1};
+  cuuint32_t box[3] = {(cuuint32_t)((wide && !bf16) ? 2 * kBlockK : kBlockK), (cuuint32_t)box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
                   const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                  (bf16 || wide) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -967,6 +1181,41 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   return QM_OK;
 }
 
+// The 256 x 256 tile kernel: worth it once the output is at least one such tile wide.
+bool use_wide(GemmShape g) { return g.N >= kWideN; }
+
+template <int KIND>
+qm_status launch_wide(const CUtensorMap& ma, const CUtensorMap& mb, KernelArgs ka, GemmShape g, cudaStream_t s) {
+  auto kern = tc_gemm_wide_kernel<KIND>;
+  constexpr size_t smem = (size_t)kWideStages * kWideStageBytes + sizeof(SharedWide) + 1024;
+  static bool attr_done = false;
+  if (!attr_done) {
+    QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attr_done = true;
+  }
+  ka.tiles_m = (int32_t)((g.M + kPairM - 1) / kPairM);
+  ka.tiles_n = (int32_t)((g.N + kWideN - 1) / kWideN);
+  const int64_t tiles = (int64_t)ka.tiles_m * ka.tiles_n * g.batch;
+  if (tiles >= (1ll << 31)) return QM_ERR_UNSUPPORTED;
+  ka.num_tiles = (int32_t)tiles;
+  const int pairs = max_pairs();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(2 * (tiles < pairs ? tiles : pairs)));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, ma, mb, ka));
+  count_launch();
+  return QM_OK;
+}
+
 }  // namespace
 
 int tc_probe_records(GemmShape g) { return grid_size(g); }   // per format
@@ -1014,6 +1263,19 @@ qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int g
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
   const int64_t ldc = qm_code_ld(g.K);
   CUtensorMap maps[8];
+  if (use_wide(g)) {
+    if (!make_map(&maps[0], cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc, true) ||
+        !make_map(&maps[1], cr, false, kWideHalfN, g.K, g.N, g.batch, ldc, g.N * ldc, true))
+      return QM_ERR_CUDA;
+    KernelArgs kw{};
+    kw.M = g.M; kw.N = g.N; kw.K = g.K;
+    kw.dl = dl; kw.pc_l = gran_l == QM_GRAN_CHANNEL; kw.dr = dr; kw.pc_r = gran_r == QM_GRAN_CHANNEL;
+    kw.out_descaled = out_descaled; kw.out_raw = out_raw; kw.err_word = err_word;
+    const uint32_t fa = fmt_l == QM_FMT_E4M3 ? 0u : 1u, fb = fmt_r == QM_FMT_E4M3 ? 0u : 1u;
+    kw.idesc_lp = fmt_l == QM_FMT_INT8 ? make_idesc(2, 1, 1, kPairM, kWideN) : make_idesc(1, fa, fb, kPairM, kWideN);
+    return fmt_l == QM_FMT_INT8 ? launch_wide<kKindI8>(maps[0], maps[1], kw, g, s)
+                                : launch_wide<kKindF8>(maps[0], maps[1], kw, g, s);
+  }
   bool ok = make_map(&maps[4], cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
             make_map(&maps[5], cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
@@ -1031,6 +1293,15 @@ qm_status launch_tc_gemm_ref(const void* l, const void* r, GemmShape g, float* o
                              cudaStream_t s) {
   if (!shape_ok(g)) return QM_ERR_UNSUPPORTED;
   CUtensorMap maps[8];
+  if (use_wide(g)) {
+    if (!make_map(&maps[0], l, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K, true) ||
+        !make_map(&maps[1], r, true, kWideHalfN, g.K, g.N, g.batch, g.K, g.N * g.K, true))
+      return QM_ERR_CUDA;
+    KernelArgs kw{};
+    kw.M = g.M; kw.N = g.N; kw.K = g.K;
+    kw.out_descaled = out; kw.err_word = err_word;
+    return launch_wide<kKindF16>(maps[0], maps[1], kw, g, s);
+  }
   bool ok = make_map(&maps[0], l, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
             make_map(&maps[1], r, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K);
   if (!ok) return QM_ERR_CUDA;

@@ -115,3 +115,31 @@ def test_metric_reduction(n):
     for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
         assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k]) + 1e-30, (k, got[k], want[k])
     assert abs(got["max_be"] - want["max_be"]) <= 1e-6 * want["max_be"]
+
+
+# ------------------------------------------------------------------ 256-column tiles (outputs at least 256 wide)
+@pytest.mark.parametrize("shape", [(1, 300, 600, 144), (2, 130, 258, 272), (1, 4096, 3072, 256), (3, 256, 512, 1040)])
+@pytest.mark.parametrize("gran", [("tensor", "tensor"), ("channel", "channel")])
+def test_int8_gemm_exact_on_wide_outputs(shape, gran):
+    # ragged last tile, a width that is not a multiple of 4 (scalar stores), a contraction that is
+    # not a multiple of the 128-code k-block, several tiles per CTA pair (both accumulator buffers
+    # reused), batches
+    b, M, N, K = shape
+    acc, want, out, raw, _ = run_gemm("int8", "int8", b, M, N, K, gran[0], gran[1], False, 27)
+    assert np.array_equal(raw.astype(np.int64), acc.astype(np.int64))
+    assert np.allclose(out, want, rtol=3e-7, atol=0)
+
+
+@pytest.mark.parametrize("fmts", [("e4m3", "e4m3"), ("e5m2", "e4m3")])
+def test_fp8_gemm_exact_on_wide_outputs(fmts):
+    acc, want, out, raw, _ = run_gemm(fmts[0], fmts[1], 1, 2304, 2560, 400, "channel", "tensor", False, 28, small=True)
+    assert np.array_equal(raw.view(np.float32).astype(np.float64), acc)
+
+
+def test_reference_product_wide_many_tiles():
+    rng = np.random.default_rng(29)
+    l = torch.from_numpy(rng.integers(-4, 5, (1, 4096, 192)).astype(np.float32)).to(torch.bfloat16)
+    r = torch.from_numpy(rng.integers(-4, 5, (1, 2816, 192)).astype(np.float32)).to(torch.bfloat16)
+    out = qm.qm_gemm_ref(l.cuda(), r.cuda()).cpu().numpy()
+    want = l.float().numpy().astype(np.float64) @ np.swapaxes(r.float().numpy().astype(np.float64), -1, -2)
+    assert np.array_equal(out.astype(np.float64), want)          # small integers: every sum exact
