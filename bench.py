@@ -136,6 +136,56 @@ def time_oracle_sample(ops, rows_per_op, seed=7):
     return flops, dt
 
 
+def gemm_rates(qm, n=8192, iters=10):
+    """T(FL)OP/s of the stand-alone products qm_gemm (E4M3, INT8) and qm_gemm_ref (bf16) at n^3, and,
+    as the achievable reference of the same run, of the library GEMMs torch reaches (harness only)."""
+    import ctypes as C
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(iters):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / iters * 1e-3
+
+    x = torch.randn(n, n, device="cuda").to(torch.bfloat16)
+    w = (torch.randn(n, n, device="cuda") * 0.02).to(torch.bfloat16)
+    opx, opw = qm.operand_of(x, -1), qm.operand_of(w, -1)
+    F = 2.0 * n ** 3
+    L = qm.lib()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    out = torch.empty((1, n, n), dtype=torch.float32, device="cuda")
+    res = {"shape": f"{n}^3, fp32 output written"}
+    for fmt in ("e4m3", "int8"):
+        cx, dx, _, _ = qm.qm_quantize(opx, fmt, "tensor")
+        cw, dw, _, _ = qm.qm_quantize(opw, fmt, "tensor")
+
+        def run():
+            rc = L.qm_gemm(C.c_void_p(cx.data_ptr()), qm.FMT[fmt], C.c_void_p(dx.data_ptr()), 0,
+                           C.c_void_p(cw.data_ptr()), qm.FMT[fmt], C.c_void_p(dw.data_ptr()), 0, n, n, n, 1,
+                           C.c_void_p(out.data_ptr()), None, 0, st)
+            assert rc == 0, rc
+        res[f"qm_gemm_{fmt}_tops"] = F / timed(run) / 1e12
+    res["qm_gemm_ref_bf16_tflops"] = F / timed(lambda: qm.qm_gemm_ref(x[None], w[None])) / 1e12
+    del out
+    try:
+        res["library_bf16_tflops"] = F / timed(lambda: torch.matmul(x, w.t())) / 1e12
+        xf, wf = x.to(torch.float8_e4m3fn), w.to(torch.float8_e4m3fn)
+        one = torch.ones((), device="cuda")
+        res["library_e4m3_tflops"] = F / timed(lambda: torch._scaled_mm(xf, wf.t(), scale_a=one, scale_b=one,
+                                                                        out_dtype=torch.bfloat16)) / 1e12
+        xi = torch.randint(-127, 127, (n, n), device="cuda", dtype=torch.int8)
+        res["library_int8_tops"] = F / timed(lambda: torch._int_mm(xi, xi.t())) / 1e12
+    except Exception as e:      # the library reference is context only
+        res["library_note"] = repr(e)[:120]
+    return res
+
+
 def scale_quantize_rates(qm, hbm_gbs, rows=16384, cols=4096, iters=10):
     """Algorithmic GB/s of the scale / quantize kernels on one FFN-activation-sized bf16 tensor
     (rows x cols, 134 MB: larger than L2), each timed with CUDA events after a warm-up."""
@@ -381,7 +431,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "roofline": roofline,
             "pct_of_composite_tensor_peak": 100.0 * value / peak_tflops,
-            "scale_quantize": sq,
+            "scale_quantize": sq, "gemm": gemm_rates(qm),
             "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
     if not args.no_cpu_baseline and world == 1:
         f, s = time_oracle_sample(ops, args.oracle_rows)
