@@ -33,7 +33,7 @@ from paper_2408_02897_b200 import workloads  # noqa: E402
 # dram__bytes_read + dram__bytes_write for M=4096 N=2304 K=768 E4M3, and the library's kernel
 # revision the counters were taken at.  Traffic grows with the operand bytes (every operand is
 # read from DRAM once), so a launch of another shape is scaled by its operand bytes.
-NCU_TC = {"revision": "tc-pair-rot4-refahead", "dram_bytes": 24.648e6, "shape": (4096, 2304, 768)}
+NCU_TC = {"revision": "tc-pair-rot4-refahead-2", "dram_bytes": 24.648e6, "shape": (4096, 2304, 768)}
 
 
 def tc_operand_bytes(M, N, K, b=1):

@@ -20,7 +20,7 @@ def main():
     ap.add_argument("--fmt", default="e4m3")
     ap.add_argument("--gran", default="tensor")
     ap.add_argument("--iters", type=int, default=3)
-    ap.add_argument("--stage", default="probe", choices=["probe", "quantize", "stats"])
+    ap.add_argument("--stage", default="probe", choices=["probe", "quantize", "stats", "gemm"])
     ap.add_argument("--r-layout", default="kn", choices=["kn", "nk"], help="R stored [K,N] or [N,K]")
     a = ap.parse_args()
     rng = workloads._rng(11)
@@ -36,6 +36,19 @@ def main():
         torch.cuda.synchronize()
         r = plan.result()
         print("mean_be", r.derived()["mean_be"], "device_error", r.device_error)
+    elif a.stage == "gemm":
+        # the stand-alone products: 8-bit codes of both operands, then qm_gemm and qm_gemm_ref
+        Rk = R.transpose(-1, -2).contiguous() if a.r_layout == "kn" else R
+        Rk_op = qm.operand_of(Rk, -1)
+        cl, dl, _, _ = qm.qm_quantize(Lop, a.fmt, a.gran)
+        cr, dr, _, _ = qm.qm_quantize(Rk_op, a.fmt, a.gran)
+        L3 = L if L.dim() == 3 else L[None]
+        R3 = Rk if Rk.dim() == 3 else Rk[None]
+        for _ in range(a.iters):
+            out, _ = qm.qm_gemm(cl, a.fmt, dl, a.gran, cr, a.fmt, dr, a.gran, a.K)
+            ref = qm.qm_gemm_ref(L3, R3)
+        torch.cuda.synchronize()
+        print("rel diff of the two products", float((out - ref).norm() / ref.norm()))
     elif a.stage == "stats":
         # the single-tensor passes on the left operand
         for _ in range(a.iters):
