@@ -547,6 +547,7 @@ qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host
 namespace {
 constexpr int kBatchStreams = 3;
 struct BatchStreams {
+  std::mutex issue;            // one batch at a time is put into the streams (host side only)
   bool ready = false;
   cudaStream_t s[kBatchStreams];
   cudaEvent_t fork, join[kBatchStreams];
@@ -582,6 +583,8 @@ qm_status run_batch(int32_t n, cudaStream_t user, F issue) {
   qm_status st = batch_streams(&b);
   if (st != QM_OK) return st;
   const int used = n < kBatchStreams ? n : kBatchStreams;
+  // the fork and join events are reused by every call: calls from several host threads take turns
+  std::lock_guard<std::mutex> lock(b->issue);
   QM_CUDA_OK(cudaEventRecord(b->fork, user));
   for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
   for (int32_t i = 0; i < n && st == QM_OK; ++i) st = issue(i, b->s[i % kBatchStreams]);
@@ -609,6 +612,7 @@ qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_oper
                               const size_t* ws_bytes, void* stream) {
   if (n > 0 && (!L_host || !R_host || !cfg || !l_stage || !r_stage || !out_host || !out_dev || !ws || !ws_bytes))
     return QM_ERR_INVALID_ARG;
+  if (n == 0) return QM_OK;
   cudaStream_t user = static_cast<cudaStream_t>(stream);
   int32_t issued = 0;
   qm_status st = run_batch(n, user, [&](int32_t i, cudaStream_t s) {

@@ -96,3 +96,17 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", "/nonexistent/libqm.so")
     with pytest.raises(qm.QmError):
         binding.lib()
+
+
+def test_batch_and_two_format_argument_checks_need_no_gpu():
+    L = qm.lib()
+    assert L.qm_probe_batch(0, None, None, None, None, None, None, None) == 0       # empty batch: nothing to do
+    assert L.qm_probe_batch(-1, None, None, None, None, None, None, None) == 1
+    assert L.qm_probe_batch(3, None, None, None, None, None, None, None) == 1
+    assert L.qm_probe_batch_host(0, None, None, None, None, None, None, None, None, None, None) == 0
+    assert L.qm_probe_layer2(None, None, None, None, None, None, 0, None) == 1
+    assert L.qm_workspace_bytes2(None, None, None, None) == 0
+    assert L.qm_stats_workspace_bytes() >= 4096
+    op = binding.Operand()
+    assert L.qm_tensor_stats(C.byref(op), None, None, 0, None) == 1                   # null data
+    assert L.qm_scale_shared(C.byref(op), 1, 1, None, None) == 1
