@@ -104,3 +104,20 @@ def test_config5_attention_batched():
         check_full(pick(ops, name), n_rows=16)
     ops = workloads.attention_ops(workloads._rng(62), 512, 512, 64, "int8")
     check_full(pick(ops, "qk-dq-int8"), n_rows=16)
+
+
+def test_config2_whole_records_through_the_batch_entry_point():
+    """The benchmark's workload in the benchmark's launch configuration (one qm_probe_batch call for
+    the step's eight probes): every whole-matrix record against the oracle's full probe."""
+    ops = workloads.config2()
+    dev = [(o["L"].cuda(), o["R"].cuda()) for o in ops]
+    batch = qm.ProbeBatch([(qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"]), o["fmt_l"], o["fmt_r"],
+                            o["gran_l"], o["gran_r"], o["ref"]) for o, (Ld, Rd) in zip(ops, dev)])
+    for _ in range(2):
+        batch.launch()
+    torch.cuda.synchronize()
+    for o, got in zip(ops, batch.results()):
+        assert got.device_error == 0
+        L, R = workloads.orient(o)
+        want = oracle.probe(L, R, o["fmt_l"], o["fmt_r"], o["gran_l"], o["gran_r"])
+        assert_record_close(got.record(), want, what=o["name"], K=L.shape[-1])
