@@ -380,6 +380,10 @@ int64_t qm_kernel_launches(void);
 const char* qm_kernel_revision(void);
 qm_status qm_profile_enable(int32_t on);
 qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
+/* The same interval launch by launch, without ending it: for launch i (in issue order, up to
+ * `cap`) its start relative to the first recorded launch's start and its duration, both in
+ * milliseconds; *launches receives the number recorded so far. */
+qm_status qm_profile_samples(double* start_ms, double* dur_ms, int32_t cap, int32_t* launches);
 
 #ifdef __cplusplus
 }

@@ -8,11 +8,11 @@ from .binding import (FMT, GRAN, REF, QmError, MetricResult, lib, qm_code_ld, qm
                       qm_gemm, qm_gemm_ref, qm_metric, qm_tensor_stats, qm_quantize_error, TensorStats, QuantError, qm_metric_noalloc, qm_probe_layer, qm_probe_layer2, ProbePlan2, qm_probe_layer_host,
                       qm_workspace_bytes, operand_of, ProbePlan, ProbeBatch, HostProbeBatch,
                       kernel_launches,
-                      profile_enable, profile_read)
+                      profile_enable, profile_read, profile_samples)
 
 __all__ = ["FMT", "GRAN", "REF", "QmError", "MetricResult", "lib", "qm_code_ld", "qm_scale", "qm_scale_shared",
            "qm_quantize", "qm_gemm", "qm_gemm_ref", "qm_metric", "qm_tensor_stats", "qm_quantize_error",
            "TensorStats", "QuantError", "qm_metric_noalloc", "qm_probe_layer",
            "qm_probe_layer_host", "qm_probe_layer2", "ProbePlan2", "qm_workspace_bytes", "operand_of", "ProbePlan", "ProbeBatch",
            "HostProbeBatch", "kernel_launches",
-           "profile_enable", "profile_read"]
+           "profile_enable", "profile_read", "profile_samples"]

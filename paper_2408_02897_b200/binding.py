@@ -126,6 +126,7 @@ def lib():
             "qm_kernel_launches": (I64, []),
             "qm_profile_enable": (I32, [I32]),
             "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),
+            "qm_profile_samples": (I32, [C.POINTER(C.c_double), C.POINTER(C.c_double), I32, C.POINTER(I32)]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -482,6 +483,14 @@ def kernel_launches():
 
 def profile_enable(on=True):
     _check(lib().qm_profile_enable(1 if on else 0), "qm_profile_enable")
+
+
+def profile_samples(cap=4096):
+    """[(start_ms, duration_ms)] of the fused probe launches recorded since profiling was enabled or
+    last read, starts relative to the first one; does not end the interval."""
+    st, du, n = (C.c_double * cap)(), (C.c_double * cap)(), C.c_int32(0)
+    _check(lib().qm_profile_samples(st, du, cap, C.byref(n)), "qm_profile_samples")
+    return [(st[i], du[i]) for i in range(min(n.value, cap))]
 
 
 def profile_read():

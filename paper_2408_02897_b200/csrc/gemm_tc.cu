@@ -29,6 +29,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
+#include <mutex>
 
 #include "qm_internal.h"
 
@@ -1057,6 +1058,364 @@ tc_gemm_wide_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   }
 }
 
+// ------------------------------------------------------------------ several probes in one launch
+// The probes of a batch as ONE persistent launch of the fused probe kernel.  A launch per probe
+// pays, each time, the kernel's set-up and drain, the launch gap, and the last wave of a tile
+// count that is not a multiple of the 74 CTA pairs; here the tiles of all probes form one
+// sequence.  The host orders the probes by descending contraction length (tile cost) and the
+// sequence is dealt to the pairs back and forth (round r gives pair p position r P + p when r is
+// even and r P + P-1-p when it is odd), which for descending costs balances the pairs to within
+// one tile of the cheapest kind.  Everything inside a tile is the probe mode of tc_kernel
+// (rotating accumulators, reference MMAs ahead of the hand-back, overlapped epilogue); the
+// operand maps, scales, shapes and the 8-bit MMA kind are read per tile from a table in the
+// kernel's parameter space.  A pair's positions increase, so it meets each probe in one run:
+// when the probe changes, the epilogue warps reduce their statistics and write the CTA's record
+// of the probe they leave.
+constexpr int kMaxGroup = 16;
+
+struct GroupProblem {
+  CUtensorMap maps[6];        // L, R, |L|, |R|, codes L, codes R
+  KernelArgs a;               // num_tiles, tiles_m, tiles_n: of this probe
+  int32_t tile_begin;         // position of its first tile in the sequence
+  int32_t kind;               // kKindF8 or kKindI8
+  int32_t pad[2];
+};
+struct GroupTable {
+  int32_t n, total_tiles;
+  int32_t pad[14];
+  GroupProblem p[kMaxGroup];
+};
+
+// position of pair `pair` in round r of the back-and-forth deal
+__device__ __forceinline__ int group_position(int r, int pair, int num_pairs) {
+  return r * num_pairs + ((r & 1) ? num_pairs - 1 - pair : pair);
+}
+// which probe a position belongs to (tile_begin is ascending)
+__device__ __forceinline__ int group_find(const GroupTable& tab, int pos) {
+  int pi = 0;
+  while (pi + 1 < tab.n && pos >= tab.p[pi + 1].tile_begin) ++pi;
+  return pi;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+tc_group_kernel(const __grid_constant__ GroupTable tab) {
+  using C = Cfg<kProbe>;
+  constexpr int kStages = C::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Shared* sh = reinterpret_cast<Shared*>(tiles + (size_t)kStages * C::kStageBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  volatile uint32_t* abort_flag = &sh->abort_flag;
+  uint32_t* const err0 = tab.p[0].a.err_word;                 // where a timed-out wait is reported
+
+  if (warp == 0) {
+    // fetch the tensor maps of this pair's first tile into the descriptor cache
+    const int pos = group_position(0, pair, num_pairs);
+    if (pos < tab.total_tiles && lane < 6)
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tab.p[group_find(tab, pos)].maps[lane]) : "memory");
+  }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&sh->tmem_full), 1);
+    mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
+    mbar_init(smem_u32(&sh->lp_done), 2 * kEpiWarps);
+    sh->abort_flag = 0;
+    sh->is_last = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(&sh->tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync();
+  pdl_prologue();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      uint32_t g = 0;
+      bool ok = true;
+      for (int r = 0; ok; ++r) {
+        const int pos = group_position(r, pair, num_pairs);
+        if (pos >= tab.total_tiles) {
+          if (r * num_pairs >= tab.total_tiles) break;          // no round reaches further
+          continue;
+        }
+        const GroupProblem& pr = tab.p[group_find(tab, pos)];
+        const TileCoord tc = tile_coord(pos - pr.tile_begin, pr.a);
+        const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;
+        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;
+        for (int kb = 0; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          const uint32_t use = g / kStages;
+          if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, err0)) {
+            ok = false;
+            break;
+          }
+          if (rank == 0) mbar_expect_tx(smem_u32(&sh->full[s]), 2 * C::kStageBytes);
+          const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
+          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          const int k0 = kb * kBlockK;
+          tma_load_3d(base + C::kOffL, &pr.maps[0], bar, k0, r0, tc.b);
+          tma_load_3d(base + C::kOffR, &pr.maps[1], bar, k0, c0, tc.b);
+          tma_load_3d(base + C::kOffLa, &pr.maps[2], bar, k0, r0, tc.b);
+          tma_load_3d(base + C::kOffRa, &pr.maps[3], bar, k0, c0, tc.b);
+          tma_load_3d(base + C::kOffCl, &pr.maps[4], bar, k0, r0, tc.b);
+          tma_load_3d(base + C::kOffCr, &pr.maps[5], bar, k0, c0, tc.b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader CTA, converged warp)
+    if (rank == 0) {
+      const bool lead = elect_one();
+      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
+      uint32_t g = 0, it = 0;
+      bool ok = true;
+      for (int r = 0; ok; ++r) {
+        const int pos = group_position(r, pair, num_pairs);
+        if (pos >= tab.total_tiles) {
+          if (r * num_pairs >= tab.total_tiles) break;
+          continue;
+        }
+        const GroupProblem& pr = tab.p[group_find(tab, pos)];
+        const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+        const uint32_t idesc_lp = pr.a.idesc_lp;
+        const bool is_i8 = pr.kind == kKindI8;
+        const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
+        const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
+        auto issue_ref = [&](uint32_t base, int kb) {
+          const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)
+            mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+        };
+        auto issue_rest = [&](uint32_t base, int kb) {
+          const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)
+            mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+          const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 32; ++k) {
+            if (is_i8) mma_pair<kKindI8>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
+            else mma_pair<kKindF8>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
+          }
+        };
+        // reference MMAs of the first k-blocks go ahead of the hand-back of the previous tile
+        int kb = 0;
+        const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
+        for (int j = 0; j < n_ahead && ok; ++j) {
+          const int s = (g + j) % kStages;
+          if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, err0)) ok = false;
+          tc_fence_after();
+          if (ok) issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
+        }
+        if (!ok) break;
+        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, err0)) break;
+        tc_fence_after();
+        for (; kb < n_ahead; ++kb, ++g) {
+          const int s = g % kStages;
+          issue_rest(smem_u32(tiles + (size_t)s * C::kStageBytes), kb);
+          tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+        }
+        for (; kb < num_kb; ++kb, ++g) {
+          const int s = g % kStages;
+          if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages) & 1, abort_flag, err0)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          issue_ref(base, kb);
+          issue_rest(base, kb);
+          tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+        }
+        if (ok && it > 0 && !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, err0)) ok = false;
+        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full), lead);
+        ++it;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    const int q = warp & 3;
+    const int h = (warp - 2) >> 2;
+    const int et = (warp - 2) * 32 + lane;
+    const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
+    double acc[5] = {0, 0, 0, 0, 0};               // of the probe in hand: sum BE, max BE, sum diff^2, C^2, D^2
+    int cur = -1;                                  // the probe in hand
+    // reduce the statistics of probe `pi` over the CTA and write its record (all 256 threads call)
+    auto flush = [&](int pi) {
+#pragma unroll
+      for (int i = 0; i < 5; ++i) {
+        double x = acc[i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const double y = __shfl_xor_sync(0xffffffffu, x, o);
+          x = i == 1 ? fmax(x, y) : x + y;
+        }
+        if (lane == 0) sh->red[i][warp - 2] = x;
+        acc[i] = 0.0;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (et < 5) {
+        double x = 0.0;
+        for (int w = 0; w < kEpiWarps; ++w) x = et == 1 ? fmax(x, sh->red[et][w]) : x + sh->red[et][w];
+        __stcg(tab.p[pi].a.partials + (int64_t)blockIdx.x * kPartialDoubles + et, x);
+        __threadfence();
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");       // red[] may be reused
+    };
+    uint32_t it = 0;
+    uint32_t met = 0;                              // bit pi: this CTA has had tiles of probe pi
+    bool live = true;
+    for (int r = 0; live; ++r) {
+      const int pos = group_position(r, pair, num_pairs);
+      if (pos >= tab.total_tiles) {
+        if (r * num_pairs >= tab.total_tiles) break;
+        continue;
+      }
+      const int pi = group_find(tab, pos);
+      if (pi != cur) {
+        if (cur >= 0) flush(cur);
+        cur = pi;
+        met |= 1u << pi;
+      }
+      const GroupProblem& pr = tab.p[pi];
+      const KernelArgs& a = pr.a;
+      const TileCoord tc = tile_coord(pos - pr.tile_begin, a);
+      const bool per_col = a.pc_r != 0;
+      const float dr_tensor = per_col ? 1.f : __ldg(a.dr);
+      float* dr_s = sh->delta_r[it & 1];
+      if (per_col && et < kBlockN) {
+        const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
+        dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
+      }
+      const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
+      const bool row_ok = row < a.M;
+      float dlv;
+      if (a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
+      else dlv = __ldg(a.dl);
+
+      const bool ok = mbar_wait(smem_u32(&sh->tmem_full), it & 1, abort_flag, err0);
+      if (epi_barrier_any(!ok)) { live = false; break; }
+      tc_fence_after();
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+      const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
+      const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
+      const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;
+      uint32_t rc[64], rd[64], rq[16];
+      tmem_ld32(lane_addr + col_ref + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
+      tmem_ld32(lane_addr + col_ref + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
+      tmem_ld32(lane_addr + col_den + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
+      tmem_ld32(lane_addr + col_den + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+      Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f};
+      const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
+      const bool is_i8 = pr.kind == kKindI8;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int cc0 = h * 64 + c * 16;
+        const int64_t col0 = colw + c * 16;
+        if (col0 < a.N) {
+          tmem_ld16(lane_addr + col_lp + cc0, rq);
+          tmem_ld_wait();
+          const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
+          if (is_i8) {
+            if (n_live == 16) stats16<kKindI8, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
+            else stats16<kKindI8, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
+          } else {
+            if (n_live == 16) stats16<kKindF8, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
+            else stats16<kKindF8, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
+          }
+        }
+      }
+      if (row_ok) {
+        float x0, x1;
+        unpack2(st.be, x0, x1); acc[0] += (double)x0 + (double)x1;
+        unpack2(st.d2, x0, x1); acc[2] += (double)x0 + (double)x1;
+        unpack2(st.r2, x0, x1); acc[3] += (double)x0 + (double)x1;
+        unpack2(st.n2, x0, x1); acc[4] += (double)x0 + (double)x1;
+        acc[1] = fmax(acc[1], (double)st.mx);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
+      ++it;
+    }
+    if (cur >= 0) flush(cur);
+    // the records of the probes this CTA never met are zero
+    if (et == 0) {
+      for (int pi = 0; pi < tab.n; ++pi) {
+        if (met & (1u << pi)) continue;
+        double* rec = tab.p[pi].a.partials + (int64_t)blockIdx.x * kPartialDoubles;
+        for (int i = 0; i < 5; ++i) __stcg(rec + i, 0.0);
+      }
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (et == 0) {
+      __threadfence();
+      const uint32_t prev = atomicAdd(tab.p[0].a.done_counter, 1u);
+      sh->is_last = prev == gridDim.x - 1 ? 1u : 0u;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (sh->is_last) {
+      // last CTA: every record of every probe is visible; each epilogue warp takes probes
+      // warp-2, warp-2+8, ...; fixed-order sum (lane l takes records l, l+32, ...)
+      __threadfence();
+      const uint32_t timed_out = err0 ? (*reinterpret_cast<volatile uint32_t*>(err0) & QM_DEVERR_TIMEOUT) : 0u;
+      for (int pi = warp - 2; pi < tab.n; pi += kEpiWarps) {
+        const KernelArgs& a = tab.p[pi].a;
+        double s5[5] = {0, 0, 0, 0, 0};
+        for (int i = lane; i < (int)gridDim.x; i += 32) {
+          const double* rec = a.partials + (int64_t)i * kPartialDoubles;
+          s5[0] += __ldcg(rec); s5[1] = fmax(s5[1], __ldcg(rec + 1)); s5[2] += __ldcg(rec + 2);
+          s5[3] += __ldcg(rec + 3); s5[4] += __ldcg(rec + 4);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          s5[0] += __shfl_xor_sync(0xffffffffu, s5[0], o);
+          s5[1] = fmax(s5[1], __shfl_xor_sync(0xffffffffu, s5[1], o));
+          s5[2] += __shfl_xor_sync(0xffffffffu, s5[2], o);
+          s5[3] += __shfl_xor_sync(0xffffffffu, s5[3], o);
+          s5[4] += __shfl_xor_sync(0xffffffffu, s5[4], o);
+        }
+        if (lane == 0) {
+          a.result->sum_be = s5[0]; a.result->max_be = s5[1]; a.result->sum_diff2 = s5[2];
+          a.result->sum_ref2 = s5[3]; a.result->sum_den2 = s5[4];
+          a.result->count = a.count;
+          a.result->device_error =
+              (a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u) | timed_out;
+          a.result->reserved = 0;
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  __syncwarp();
+  cluster_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -1218,7 +1577,77 @@ qm_status launch_wide(const CUtensorMap& ma, const CUtensorMap& mb, KernelArgs k
 
 }  // namespace
 
-int tc_probe_records(GemmShape g) { return grid_size(g); }   // per format
+int tc_group_max() { return kMaxGroup; }
+
+qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
+  if (n < 1 || n > kMaxGroup) return QM_ERR_INVALID_ARG;
+  // descending contraction length = descending tile cost
+  int order[kMaxGroup];
+  for (int i = 0; i < n; ++i) order[i] = i;
+  for (int i = 1; i < n; ++i)
+    for (int j = i; j > 0 && ps[order[j]].g.K > ps[order[j - 1]].g.K; --j) {
+      const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
+    }
+  static GroupTable tab;               // 15 KB: kept off the stack; guarded by the mutex below
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  tab.n = n;
+  int64_t total = 0;
+  for (int k = 0; k < n; ++k) {
+    const TcProbeArgs& p = ps[order[k]];
+    if (!shape_ok(p.g) || p.cl2) return QM_ERR_UNSUPPORTED;
+    const GemmShape g = p.g;
+    const int64_t ldc = qm_code_ld(g.K);
+    GroupProblem& gp = tab.p[k];
+    const bool ok = make_map(&gp.maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
+                    make_map(&gp.maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
+                    make_map(&gp.maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
+                    make_map(&gp.maps[3], p.r_abs, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K) &&
+                    make_map(&gp.maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+                    make_map(&gp.maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
+    if (!ok) return QM_ERR_CUDA;
+    KernelArgs ka{};
+    fill_tiles(&ka, g);
+    ka.dl = p.dl; ka.pc_l = p.gran_l == QM_GRAN_CHANNEL; ka.dr = p.dr; ka.pc_r = p.gran_r == QM_GRAN_CHANNEL;
+    ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
+    ka.count = (uint64_t)(g.M * g.N * g.batch);
+    ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+    gp.a = ka;
+    gp.kind = p.fmt_l == QM_FMT_INT8 ? kKindI8 : kKindF8;
+    gp.tile_begin = (int32_t)total;
+    total += ka.num_tiles;
+    if (total >= (1ll << 31)) return QM_ERR_UNSUPPORTED;
+  }
+  tab.total_tiles = (int32_t)total;
+  static bool attr_done = false;
+  if (!attr_done) {
+    QM_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)smem_bytes<kProbe>()));
+    attr_done = true;
+  }
+  const int pairs = max_pairs();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(2 * (total < pairs ? total : pairs)));
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem_bytes<kProbe>();
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  profile_events(&ev0, &ev1);
+  if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
+  QM_CUDA_OK(cudaLaunchKernelEx(&cfg, tc_group_kernel, tab));
+  if (ev1) QM_CUDA_OK(cudaEventRecord(ev1, s));
+  count_launch();
+  return QM_OK;
+}
+
+int tc_probe_records(GemmShape) { return 2 * max_pairs(); }   // per format; the grouped launch uses the whole grid
 
 qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   if (!shape_ok(p.g)) return QM_ERR_UNSUPPORTED;

@@ -300,8 +300,15 @@ size_t qm_workspace_bytes(const qm_operand* Lo, const qm_operand* Ro, const qm_p
   return plan(L, R, *cfg).total;
 }
 
-qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
-                         qm_metric_result* out, void* ws, size_t ws_bytes, void* stream) {
+// The probe in phases that may be issued apart, on different streams (same arguments every time):
+// kClear clears the workspace words, kPrepareL / kPrepareR run scale + quantize of one operand
+// (after kClear), kProducts the products and the Eq. 3 reduction (after both).  With `defer` set and a tensor-core configuration, kProducts only describes the
+// fused kernel's work in *defer (for a grouped launch) instead of launching it.
+enum { kClear = 1, kPrepareL = 2, kPrepareR = 4, kPrepare = kClear | kPrepareL | kPrepareR, kProducts = 8 };
+static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
+                              qm_metric_result* out, void* ws, size_t ws_bytes, void* stream, int phases,
+                              TcProbeArgs* defer, bool* deferred) {
+  if (deferred) *deferred = false;
   View L, R;
   qm_status st = check_probe(Lo, Ro, cfg, &L, &R);
   if (st != QM_OK) return st;
@@ -318,7 +325,7 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   uint8_t* cr = base + w.off_cr;
   double* part = reinterpret_cast<double*>(base + w.off_part);
   // the error word, the finished-CTA counter and both max|x| buffers are adjacent: one clear
-  QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
+  if (phases & kClear) QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
   uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.off_ml);
   uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.off_mr);
   void* al = w.tc ? base + w.off_al : nullptr;
@@ -326,12 +333,17 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
   void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
   const StochasticDraw draw_l{cfg->seed, 0u}, draw_r{cfg->seed, 1u};
-  st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err,
-                       (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, cfg->batch_groups_l, s);
-  if (st != QM_OK) return st;
-  st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err,
-                       (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, cfg->batch_groups_r, s);
-  if (st != QM_OK) return st;
+  if (phases & kPrepareL) {
+    st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err,
+                         (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, cfg->batch_groups_l, s);
+    if (st != QM_OK) return st;
+  }
+  if (phases & kPrepareR) {
+    st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err,
+                         (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, cfg->batch_groups_r, s);
+    if (st != QM_OK) return st;
+  }
+  if (!(phases & kProducts)) return QM_OK;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {
     TcProbeArgs p{};
@@ -343,11 +355,21 @@ qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_pr
     p.g = g; p.partials = part; p.err_word = err;
     p.done_counter = err + 1;               // second word of the cleared error slot
     p.result = out;
+    if (defer) {
+      *defer = p;
+      *deferred = true;
+      return QM_OK;
+    }
     return launch_tc_probe(p, s);           // the last CTA writes the record
   }
   st = launch_simt_probe(L, R, cl, cfg->fmt_l, dl, cfg->gran_l, cr, cfg->fmt_r, dr, cfg->gran_r, part, s);
   if (st != QM_OK) return st;
   return launch_metric_finalize(part, w.n_part, (uint64_t)(g.M * g.N * g.batch), err, out, s);
+}
+
+qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
+                         qm_metric_result* out, void* ws, size_t ws_bytes, void* stream) {
+  return probe_phases(Lo, Ro, cfg, out, ws, ws_bytes, stream, kPrepare | kProducts, nullptr, nullptr);
 }
 
 // ---- two formats in one pass -------------------------------------------------------------------
@@ -545,7 +567,8 @@ qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host
 
 // ---- batches of probes over the library's own streams ------------------------------------------
 namespace {
-constexpr int kBatchStreams = 3;
+constexpr int kBatchStreams = 8;      // streams of the pool
+constexpr int kHostBatchStreams = 3;  // of which the host-operand batches use this many
 struct BatchStreams {
   std::mutex issue;            // one batch at a time is put into the streams (host side only)
   bool ready = false;
@@ -582,12 +605,12 @@ qm_status run_batch(int32_t n, cudaStream_t user, F issue) {
   BatchStreams* b = nullptr;
   qm_status st = batch_streams(&b);
   if (st != QM_OK) return st;
-  const int used = n < kBatchStreams ? n : kBatchStreams;
+  const int used = n < kHostBatchStreams ? n : kHostBatchStreams;
   // the fork and join events are reused by every call: calls from several host threads take turns
   std::lock_guard<std::mutex> lock(b->issue);
   QM_CUDA_OK(cudaEventRecord(b->fork, user));
   for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
-  for (int32_t i = 0; i < n && st == QM_OK; ++i) st = issue(i, b->s[i % kBatchStreams]);
+  for (int32_t i = 0; i < n && st == QM_OK; ++i) st = issue(i, b->s[i % kHostBatchStreams]);
   for (int j = 0; j < used; ++j) {
     QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
     QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
@@ -601,9 +624,76 @@ extern "C" {
 qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,
                          qm_metric_result* out, void* const* ws, const size_t* ws_bytes, void* stream) {
   if (n > 0 && (!L || !R || !cfg || !out || !ws || !ws_bytes)) return QM_ERR_INVALID_ARG;
-  return run_batch(n, static_cast<cudaStream_t>(stream), [&](int32_t i, cudaStream_t s) {
-    return qm_probe_layer(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], s);
-  });
+  cudaStream_t user = static_cast<cudaStream_t>(stream);
+  if (n < 0) return QM_ERR_INVALID_ARG;
+  if (n == 0) return QM_OK;
+  BatchStreams* b = nullptr;
+  qm_status st = batch_streams(&b);
+  if (st != QM_OK) return st;
+  std::lock_guard<std::mutex> lock(b->issue);
+  // Scale + quantize of every OPERAND is a chain of two or three short, latency-bound kernels, and
+  // all 2n chains are independent: the workspace words of every probe are cleared on the caller's
+  // stream, then the chains are spread over the library's streams so that they run beside one
+  // another.  Probes that do not take the fused tensor-core kernel (fp32 reference) run whole on
+  // one of those streams.  A refused probe ends the issue there; the ones before it complete.
+  std::vector<int32_t> fused;
+  int32_t good = 0;
+  for (; good < n && st == QM_OK; ++good)
+    if (cfg[good].ref == QM_REF_BF16_FP32ACC)
+      st = probe_phases(&L[good], &R[good], &cfg[good], out + good, ws[good], ws_bytes[good], user, kClear, nullptr,
+                        nullptr);
+  if (st != QM_OK) --good;
+  QM_CUDA_OK(cudaEventRecord(b->fork, user));
+  const int used = 2 * good < kBatchStreams ? 2 * good : kBatchStreams;
+  for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
+  // One chunk: all chains, then the caller's stream waits for the library's streams and takes the
+  // fused kernels as one persistent launch.  (Two chunks, the second one's chains running under
+  // the first one's launch, measured slower: the chains wait for the SMs the launch holds.)
+  const int32_t chunk = good;
+  std::vector<TcProbeArgs> args;
+  for (int32_t c0 = 0; c0 < good; c0 += chunk) {
+    const int32_t c1 = c0 + chunk < good ? c0 + chunk : good;
+    fused.clear();
+    for (int32_t i = c0; i < c1; ++i) {
+      cudaStream_t sl = b->s[(2 * i) % kBatchStreams], sr = b->s[(2 * i + 1) % kBatchStreams];
+      qm_status e;
+      if (cfg[i].ref == QM_REF_BF16_FP32ACC) {
+        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepareL, nullptr, nullptr);
+        if (e == QM_OK)
+          e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sr, kPrepareR, nullptr, nullptr);
+        if (e == QM_OK) fused.push_back(i);
+      } else {
+        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepare | kProducts, nullptr, nullptr);
+      }
+      if (e != QM_OK && st == QM_OK) st = e;
+    }
+    for (int j = 0; j < used; ++j) {
+      QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
+      QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
+    }
+    // up to tc_group_max() probes per persistent launch
+    auto flush_group = [&]() -> qm_status {
+      if (args.empty()) return QM_OK;
+      const qm_status e = args.size() == 1 ? launch_tc_probe(args[0], user)
+                                           : launch_tc_probe_group(args.data(), (int)args.size(), user);
+      args.clear();
+      return e;
+    };
+    for (int32_t i : fused) {
+      TcProbeArgs p{};
+      bool deferred = false;
+      const qm_status e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], user, kProducts, &p, &deferred);
+      if (e != QM_OK) { if (st == QM_OK) st = e; continue; }
+      if (deferred) args.push_back(p);
+      if ((int)args.size() == tc_group_max()) {
+        const qm_status g = flush_group();
+        if (g != QM_OK && st == QM_OK) st = g;
+      }
+    }
+    const qm_status g = flush_group();
+    if (g != QM_OK && st == QM_OK) st = g;
+  }
+  return st;
 }
 
 qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_operand* R_host,
@@ -656,6 +746,21 @@ qm_status qm_profile_enable(int32_t on) {
   std::lock_guard<std::mutex> lock(qm::g_prof_mutex);
   qm::g_prof_on = on != 0;
   qm::g_prof_used = 0;
+  return QM_OK;
+}
+
+qm_status qm_profile_samples(double* start_ms, double* dur_ms, int32_t cap, int32_t* launches) {
+  if (!start_ms || !dur_ms || !launches || cap < 0) return QM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(qm::g_prof_mutex);
+  const int32_t n = (int32_t)(qm::g_prof_used / 2);
+  for (int32_t i = 0; i < n && i < cap; ++i) {
+    QM_CUDA_OK(cudaEventSynchronize(qm::g_prof_events[2 * i + 1]));
+    float t0 = 0, t1 = 0;
+    QM_CUDA_OK(cudaEventElapsedTime(&t0, qm::g_prof_events[0], qm::g_prof_events[2 * i]));
+    QM_CUDA_OK(cudaEventElapsedTime(&t1, qm::g_prof_events[2 * i], qm::g_prof_events[2 * i + 1]));
+    start_ms[i] = t0; dur_ms[i] = t1;
+  }
+  *launches = n;
   return QM_OK;
 }
 

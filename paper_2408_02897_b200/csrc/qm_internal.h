@@ -138,6 +138,10 @@ struct TcProbeArgs {
 };
 int tc_probe_records(GemmShape g);
 qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
+// Up to tc_group_max() one-format probes as one persistent launch (every probe's operands must be
+// prepared already; each writes its own record; the first probe's done_counter counts the CTAs).
+int tc_group_max();
+qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s);
 qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
                             const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
                             GemmShape g, float* out_descaled, void* out_raw, uint32_t* err_word,

