@@ -738,7 +738,7 @@ int32_t qm_version(void) { return 100; }
 
 const char* qm_last_cuda_error(void) { return qm::g_last_error; }
 
-const char* qm_kernel_revision(void) { return "tc-pair-rot4-refahead-2"; }
+const char* qm_kernel_revision(void) { return "tc-group-rot4-refahead-2"; }
 
 int64_t qm_kernel_launches(void) { return (int64_t)qm::g_launches.load(); }
 

@@ -20,9 +20,20 @@ def main():
     ap.add_argument("--fmt", default="e4m3")
     ap.add_argument("--gran", default="tensor")
     ap.add_argument("--iters", type=int, default=3)
-    ap.add_argument("--stage", default="probe", choices=["probe", "quantize", "stats", "gemm"])
+    ap.add_argument("--stage", default="probe", choices=["probe", "quantize", "stats", "gemm", "batch"])
     ap.add_argument("--r-layout", default="kn", choices=["kn", "nk"], help="R stored [K,N] or [N,K]")
     a = ap.parse_args()
+    if a.stage == "batch":
+        # the benchmark's step: the eight probes of the BERT-base forward workload as one batch
+        ops = workloads.config2()
+        dev = [(o["L"].cuda(), o["R"].cuda()) for o in ops]
+        batch = qm.ProbeBatch([(qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"]), o["fmt_l"], o["fmt_r"],
+                                o["gran_l"], o["gran_r"], o["ref"]) for o, (Ld, Rd) in zip(ops, dev)])
+        for _ in range(a.iters):
+            batch.launch()
+        torch.cuda.synchronize()
+        print("mean_be", [round(r.derived()["mean_be"], 6) for r in batch.results()])
+        return
     rng = workloads._rng(11)
     lead = (a.batch,) if a.batch > 1 else ()
     L = workloads.normal(rng, lead + (a.M, a.K)).cuda()
