@@ -305,6 +305,8 @@ def main():
     ap.add_argument("--workload", default="bert_base_fwd")
     ap.add_argument("--oracle-rows", type=int, default=4096)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the scale/quantize and stand-alone GEMM rate blocks (profiling runs)")
     args = ap.parse_args()
 
     ops, desc = build_workload(args.workload)
@@ -397,7 +399,7 @@ def main():
         return
 
     peaks = load_peaks()
-    sq = scale_quantize_rates(qm, peaks["hbm_gbs"])
+    sq = None if args.no_extras else scale_quantize_rates(qm, peaks["hbm_gbs"])
     # composite tensor bound of the fused kernel: per 2MNK, one product at the 8-bit rate
     # (2 x bf16) and two at the bf16 rate  ->  3 / (1/(2P) + 2/P) = 1.2 P in summed flops
     peak_tflops = 1.2 * peaks["bf16_tflops"]
@@ -426,7 +428,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(launches), "roofline": roofline,
             "pct_of_composite_tensor_peak": 100.0 * value / peak_tflops,
-            "scale_quantize": sq, "gemm": gemm_rates(qm),
+            "scale_quantize": sq, "gemm": None if args.no_extras else gemm_rates(qm),
             "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
     if not args.no_cpu_baseline and world == 1:
         f, s = time_oracle_sample(ops, args.oracle_rows)
