@@ -311,20 +311,24 @@ qm_status qm_quantize_error(const qm_operand* x, int32_t fmt, int32_t gran, cons
 /*
  * The probes of one measurement pass (the per-layer loop of the Methodology
  * section: every matmul of a network is probed on its own), issued together.
- * Probe i is qm_probe_layer(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i]):
- * the probes are independent, so the library spreads them over a few streams of
+ * Probe i computes what qm_probe_layer(&L[i], &R[i], &cfg[i], out + i, ws[i],
+ * ws_bytes[i]) computes.  The probes are independent, so the library runs the
+ * scale/quantize kernels of all operands beside one another on a few streams of
  * its own (created on the first call on each device, kept until the process
- * exits) and the scale/quantize kernels of one probe run beside the fused
- * kernel of another.  All of it is ordered after the work already in `stream`,
+ * exits) and then the fused kernels of all tensor-core probes as one persistent
+ * launch over the tiles of all of them (the sums of a record are then taken
+ * over another tile-to-CTA assignment than in qm_probe_layer and may differ in
+ * the last bits).  All of it is ordered after the work already in `stream`,
  * and work put into `stream` after the call waits for every probe.  `out` is a
  * device array of n records; the n workspaces must be distinct and sized per
  * probe.  With qm_probe_batch_host the operands live in host memory as for
  * qm_probe_layer_host (l_stage[i], r_stage[i]: distinct device staging buffers),
- * the copies of one probe overlap the kernels of another, out_host receives the
- * n records and the call waits for them; the first device-detected condition
- * is returned.  n == 0 is a no-op.  On an argument error of probe i the probes
- * before it have been issued and are waited for as described; the rest are not.
- * Make the first call on a device outside any stream capture.
+ * whole probes are spread over the library's streams so that the copies of one
+ * overlap the kernels of another, out_host receives the n records and the call
+ * waits for them; the first device-detected condition is returned.  n == 0 is a
+ * no-op.  On an argument error of probe i the probes before it are completed
+ * as described; the rest are not issued.  Make the first call on a device
+ * outside any stream capture.
  */
 qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,
                          qm_metric_result* out, void* const* ws, const size_t* ws_bytes, void* stream);
