@@ -154,6 +154,23 @@ qm_status noalloc_scratch(double** out) {
 }
 
 }  // namespace
+// ---- clearing the control words of several workspaces in one launch --------------------------
+namespace {
+__global__ void clear_many_kernel(const ClearList list) {
+  pdl_prologue();
+  const int w = blockIdx.x;                      // gridDim.y blocks per region
+  uint32_t* p = static_cast<uint32_t*>(list.ptr[w]);
+  for (uint32_t i = blockIdx.y * blockDim.x + threadIdx.x; i < list.words[w]; i += gridDim.y * blockDim.x) p[i] = 0u;
+}
+}  // namespace
+
+qm_status launch_clear_many(const ClearList& list, cudaStream_t s) {
+  if (list.n < 1 || list.n > kClearMax) return QM_ERR_INVALID_ARG;
+  QM_CUDA_OK(launch_pdl(clear_many_kernel, dim3((unsigned)list.n, 8), dim3(256), 0, s, list));
+  count_launch();
+  return QM_OK;
+}
+
 }  // namespace qm
 
 extern "C" qm_status qm_metric_noalloc(const float* ref, const float* q, const float* den, int64_t count,

@@ -304,10 +304,27 @@ size_t qm_workspace_bytes(const qm_operand* Lo, const qm_operand* Ro, const qm_p
 // kClear clears the workspace words, kPrepareL / kPrepareR run scale + quantize of one operand
 // (after kClear), kProducts the products and the Eq. 3 reduction (after both).  With `defer` set and a tensor-core configuration, kProducts only describes the
 // fused kernel's work in *defer (for a grouped launch) instead of launching it.
+// What one prepared operand leaves behind that does not depend on the 8-bit format: the max|x|
+// bit patterns, the |x| copy and (for a strided contraction) the contraction-major copy.  Inside
+// a batch a later probe whose operand is the same tensor under the same scale grouping borrows
+// them and runs only its own quantize kernel.
+struct OperandShare {
+  const uint32_t* amax = nullptr;
+  void* abs_copy = nullptr;
+  void* kmaj_copy = nullptr;
+};
+struct ProbeShare {
+  const OperandShare* from_l = nullptr;   // borrow (inputs)
+  const OperandShare* from_r = nullptr;
+  OperandShare* own_l = nullptr;          // what this probe's own chains produce (outputs)
+  OperandShare* own_r = nullptr;
+};
+
 enum { kClear = 1, kPrepareL = 2, kPrepareR = 4, kPrepare = kClear | kPrepareL | kPrepareR, kProducts = 8 };
 static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
                               qm_metric_result* out, void* ws, size_t ws_bytes, void* stream, int phases,
-                              TcProbeArgs* defer, bool* deferred) {
+                              TcProbeArgs* defer, bool* deferred, const ProbeShare* share = nullptr,
+                              ClearList* clear_later = nullptr) {
   if (deferred) *deferred = false;
   View L, R;
   qm_status st = check_probe(Lo, Ro, cfg, &L, &R);
@@ -325,7 +342,12 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
   uint8_t* cr = base + w.off_cr;
   double* part = reinterpret_cast<double*>(base + w.off_part);
   // the error word, the finished-CTA counter and both max|x| buffers are adjacent: one clear
-  if (phases & kClear) QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
+  if ((phases & kClear) && clear_later && clear_later->n < kClearMax) {
+    clear_later->ptr[clear_later->n] = base;                 // cleared with others by one kernel
+    clear_later->words[clear_later->n++] = (uint32_t)(w.off_dl / 4);
+  } else if (phases & kClear) {
+    QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
+  }
   uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.off_ml);
   uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.off_mr);
   void* al = w.tc ? base + w.off_al : nullptr;
@@ -333,16 +355,26 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
   void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
   const StochasticDraw draw_l{cfg->seed, 0u}, draw_r{cfg->seed, 1u};
+  const StochasticDraw* dl_draw = (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr;
+  const StochasticDraw* dr_draw = (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr;
+  const OperandShare* from_l = share ? share->from_l : nullptr;
+  const OperandShare* from_r = share ? share->from_r : nullptr;
+  if (share && share->own_l) *share->own_l = OperandShare{ml, al, kl};
+  if (share && share->own_r) *share->own_r = OperandShare{mr, ar, kr};
   if (phases & kPrepareL) {
-    st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err,
-                         (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr, cfg->batch_groups_l, s);
+    st = from_l ? launch_quantize(L, cfg->fmt_l, cfg->gran_l, reinterpret_cast<const float*>(from_l->amax), true, dl,
+                                  err, cl, nullptr, nullptr, s, dl_draw)
+                : prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err, dl_draw, cfg->batch_groups_l, s);
     if (st != QM_OK) return st;
   }
   if (phases & kPrepareR) {
-    st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err,
-                         (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr, cfg->batch_groups_r, s);
+    st = from_r ? launch_quantize(R, cfg->fmt_r, cfg->gran_r, reinterpret_cast<const float*>(from_r->amax), true, dr,
+                                  err, cr, nullptr, nullptr, s, dr_draw)
+                : prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err, dr_draw, cfg->batch_groups_r, s);
     if (st != QM_OK) return st;
   }
+  if (from_l) { al = from_l->abs_copy; kl = from_l->kmaj_copy; }
+  if (from_r) { ar = from_r->abs_copy; kr = from_r->kmaj_copy; }
   if (!(phases & kProducts)) return QM_OK;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {
@@ -596,6 +628,28 @@ qm_status batch_streams(BatchStreams** out) {
   return QM_OK;
 }
 
+// The earlier probe (j < i) of a batch whose operand on side `side` (0 = L, 1 = R) is the very
+// tensor of probe i's, scaled in the same groups, and that has prepared it itself through the
+// absmax -> quantize route (so that its max|x| array exists); -1 if there is none.
+int find_lender(const qm_operand* ops, const qm_probe_cfg* cfg, int i, int side, const std::vector<int>& lender) {
+  const qm_operand& x = ops[i];
+  const int gran = side ? cfg[i].gran_r : cfg[i].gran_l;
+  const int groups = side ? cfg[i].batch_groups_r : cfg[i].batch_groups_l;
+  const bool grouped = gran == QM_GRAN_CHANNEL && groups > 0 && groups < x.batch;
+  // per-channel scales of a contiguous contraction take the single-pass kernel, which keeps no maxima
+  if (gran == QM_GRAN_CHANNEL && !grouped && (x.stride_c == 1 || x.contract == 1)) return -1;
+  for (int j = 0; j < i; ++j) {
+    if (cfg[j].ref != QM_REF_BF16_FP32ACC || lender[2 * j + side] >= 0) continue;
+    const qm_operand& y = ops[j];
+    const int gj = side ? cfg[j].gran_r : cfg[j].gran_l, pj = side ? cfg[j].batch_groups_r : cfg[j].batch_groups_l;
+    if (y.data == x.data && y.dtype == x.dtype && y.noncontract == x.noncontract && y.contract == x.contract &&
+        y.stride_nc == x.stride_nc && y.stride_c == x.stride_c && y.batch == x.batch &&
+        y.stride_batch == x.stride_batch && gj == gran && pj == groups)
+      return j;
+  }
+  return -1;
+}
+
 // Runs issue(i, stream_i) for i < n round-robin over the library's streams, between a fork from
 // and a join back into the caller's stream.  The join happens even when a probe was refused.
 template <typename F>
@@ -638,11 +692,16 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
   // one of those streams.  A refused probe ends the issue there; the ones before it complete.
   std::vector<int32_t> fused;
   int32_t good = 0;
+  ClearList clears{};
   for (; good < n && st == QM_OK; ++good)
     if (cfg[good].ref == QM_REF_BF16_FP32ACC)
       st = probe_phases(&L[good], &R[good], &cfg[good], out + good, ws[good], ws_bytes[good], user, kClear, nullptr,
-                        nullptr);
+                        nullptr, nullptr, &clears);
   if (st != QM_OK) --good;
+  if (clears.n > 0) {
+    const qm_status e = launch_clear_many(clears, user);
+    if (e != QM_OK) return e;
+  }
   QM_CUDA_OK(cudaEventRecord(b->fork, user));
   const int used = 2 * good < kBatchStreams ? 2 * good : kBatchStreams;
   for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
@@ -650,6 +709,9 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
   // fused kernels as one persistent launch.  (Two chunks, the second one's chains running under
   // the first one's launch, measured slower: the chains wait for the SMs the launch holds.)
   const int32_t chunk = good;
+  std::vector<OperandShare> own(2 * (size_t)n);
+  std::vector<int> lender(2 * (size_t)n, -1);     // per operand: the probe it borrows from, or -1
+  std::vector<ProbeShare> shares((size_t)n);
   std::vector<TcProbeArgs> args;
   for (int32_t c0 = 0; c0 < good; c0 += chunk) {
     const int32_t c1 = c0 + chunk < good ? c0 + chunk : good;
@@ -658,9 +720,19 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
       cudaStream_t sl = b->s[(2 * i) % kBatchStreams], sr = b->s[(2 * i + 1) % kBatchStreams];
       qm_status e;
       if (cfg[i].ref == QM_REF_BF16_FP32ACC) {
-        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepareL, nullptr, nullptr);
+        // An operand that an earlier probe of the batch has already prepared (the same tensor under
+        // the same scale grouping: a sweep of formats over one layer) borrows that probe's max|x|,
+        // |x| copy and contraction-major copy and only quantizes, on the lender's stream.
+        ProbeShare sh;
+        sh.own_l = &own[2 * i]; sh.own_r = &own[2 * i + 1];
+        const int dl_i = find_lender(L, cfg, i, 0, lender), dr_i = find_lender(R, cfg, i, 1, lender);
+        lender[2 * i] = dl_i; lender[2 * i + 1] = dr_i;
+        if (dl_i >= 0) { sh.from_l = &own[2 * dl_i]; sl = b->s[(2 * dl_i) % kBatchStreams]; }
+        if (dr_i >= 0) { sh.from_r = &own[2 * dr_i + 1]; sr = b->s[(2 * dr_i + 1) % kBatchStreams]; }
+        shares[i] = sh;
+        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepareL, nullptr, nullptr, &sh);
         if (e == QM_OK)
-          e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sr, kPrepareR, nullptr, nullptr);
+          e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sr, kPrepareR, nullptr, nullptr, &sh);
         if (e == QM_OK) fused.push_back(i);
       } else {
         e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepare | kProducts, nullptr, nullptr);
@@ -682,7 +754,8 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
     for (int32_t i : fused) {
       TcProbeArgs p{};
       bool deferred = false;
-      const qm_status e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], user, kProducts, &p, &deferred);
+      const qm_status e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], user, kProducts, &p, &deferred,
+                                       &shares[i]);
       if (e != QM_OK) { if (st == QM_OK) st = e; continue; }
       if (deferred) args.push_back(p);
       if ((int)args.size() == tc_group_max()) {

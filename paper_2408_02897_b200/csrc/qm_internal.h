@@ -103,6 +103,12 @@ qm_status launch_metric_partials(const float* ref, const float* q, const float* 
 qm_status launch_metric_finalize(const double* partials, int n, uint64_t count,
                                  const uint32_t* err_word, qm_metric_result* out, cudaStream_t s);
 
+// Zeroes up to kClearMax regions of 32-bit words (4-byte aligned) in one launch: the control words
+// of the workspaces of a batch.
+constexpr int kClearMax = 32;
+struct ClearList { int n; void* ptr[kClearMax]; uint32_t words[kClearMax]; };
+qm_status launch_clear_many(const ClearList& list, cudaStream_t s);
+
 // ---- CUDA-core GEMMs (gemm_simt.cu) ---------------------------------------
 struct GemmShape { int64_t M, N, K, batch; };
 qm_status launch_simt_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,

@@ -91,3 +91,34 @@ def test_empty_and_bad_batches():
         batch.launch()
     torch.cuda.synchronize()
     assert _same(batch.results()[0], want)
+
+
+def test_format_sweep_over_the_same_tensors_borrows_prepared_operands():
+    """Probes of one batch that quantize the very same tensors into different formats share the
+    format-independent part of the preparation; every record must still be the single probe's."""
+    rng = workloads._rng(120)
+    X = workloads.normal(rng, (520, 256)).cuda()              # activations, contraction contiguous
+    W = workloads.normal(rng, (256, 392), 0.05).cuda()        # weights stored [K, N]: contraction strided
+    Q = workloads.normal(rng, (6, 136, 64)).cuda()            # batched, for shared channel scales
+    Kt = workloads.normal(rng, (6, 200, 64)).cuda()
+    cases = []
+    for gl, gr in (("tensor", "tensor"), ("channel", "channel"), ("tensor", "channel")):
+        for f in ("e4m3", "int8", "e5m2"):
+            cases.append((qm.operand_of(X, -1), qm.operand_of(W, -2), f, f, gl, gr, {}))
+    for f in ("e4m3", "int8"):
+        cases.append((qm.operand_of(Q, -1), qm.operand_of(Kt, -1), f, f, "channel", "channel", {"groups": (2, 2)}))
+        cases.append((qm.operand_of(X, -1), qm.operand_of(W, -2), f, f, "tensor", "tensor",
+                      {"rounding": "stochastic_r", "seed": 3}))
+    single = [qm.qm_probe_layer(Lo, Ro, fl, fr, gl, gr, **kw) for Lo, Ro, fl, fr, gl, gr, kw in cases]
+    batch = qm.ProbeBatch([c[:6] for c in cases])
+    for i, c in enumerate(cases):                             # per-probe extras of the configuration
+        kw = c[6]
+        batch.cfg[i].round = qm.binding.ROUND[kw.get("rounding", "rtne")]
+        batch.cfg[i].seed = kw.get("seed", 0)
+        batch.cfg[i].batch_groups_l, batch.cfg[i].batch_groups_r = kw.get("groups", (0, 0))
+    for _ in range(2):
+        batch.launch()
+        torch.cuda.synchronize()
+        got = batch.results()
+        for i, (g, s) in enumerate(zip(got, single)):
+            assert _same(g, s), (i, cases[i][2:], g.record(), s.record())
