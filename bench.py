@@ -327,7 +327,15 @@ def main():
     qm.lib()   # fail now if the CUDA library is missing
 
     # ---- inputs resident in HBM; one workspace and one result record per probe
-    dev_tensors = [(o["L"].cuda(), o["R"].cuda()) for o in ops]
+    # (a tensor that several probes of the step share, here the same layer probed in two formats,
+    # is resident once)
+    on_dev = {}
+
+    def resident(t):
+        if id(t) not in on_dev:
+            on_dev[id(t)] = t.cuda()
+        return on_dev[id(t)]
+    dev_tensors = [(resident(o["L"]), resident(o["R"])) for o in ops]
     batch = qm.ProbeBatch([(qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"]), o["fmt_l"], o["fmt_r"],
                             o["gran_l"], o["gran_r"], o["ref"]) for o, (Ld, Rd) in zip(ops, dev_tensors)])
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB L2
