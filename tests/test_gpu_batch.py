@@ -122,3 +122,30 @@ def test_format_sweep_over_the_same_tensors_borrows_prepared_operands():
         got = batch.results()
         for i, (g, s) in enumerate(zip(got, single)):
             assert _same(g, s), (i, cases[i][2:], g.record(), s.record())
+
+
+def test_large_mixed_batch_spans_several_grouped_launches():
+    """More probes than one grouped launch takes (16), shapes from a single tile to many, one
+    k-block to many, batched operands, both reference modes in one batch."""
+    rng = workloads._rng(130)
+    shapes = [(64, 64, 64), (256, 128, 64), (300, 200, 128), (1000, 520, 192), (128, 1024, 320), (520, 136, 1040)]
+    cases = []
+    for i in range(21):
+        M, N, K = shapes[i % len(shapes)]
+        fmt = ("e4m3", "int8", "e5m2")[i % 3]
+        gran = ("tensor", "channel")[(i // 3) % 2]
+        ref = "fp32" if i in (4, 11) else "bf16"
+        if i % 7 == 6:
+            L, R = workloads.normal(rng, (3, M, K)), workloads.normal(rng, (3, N, K), 0.1)
+            cases.append((L.cuda(), -1, R.cuda(), -1, fmt, gran, ref))
+        else:
+            L, R = workloads.student_t(rng, (M, K), 4.0), workloads.normal(rng, (K, N), 0.05)
+            cases.append((L.cuda(), -1, R.cuda(), -2, fmt, gran, ref))
+    probes = [(qm.operand_of(L, cl), qm.operand_of(R, cr), f, f, g, g, ref) for L, cl, R, cr, f, g, ref in cases]
+    single = [qm.qm_probe_layer(*p) for p in probes]
+    batch = qm.ProbeBatch(probes)
+    for _ in range(2):
+        batch.launch()
+        torch.cuda.synchronize()
+        for i, (g, s) in enumerate(zip(batch.results(), single)):
+            assert _same(g, s), (i, cases[i][4:], g.record(), s.record())
