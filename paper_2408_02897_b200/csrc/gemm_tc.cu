@@ -1097,6 +1097,63 @@ __device__ __forceinline__ int group_find(const GroupTable& tab, int pos) {
   return pi;
 }
 
+// The MMAs of one tile of the grouped kernel (leader CTA, converged warp); g counts k-blocks,
+// `it` tiles of this pair.  Returns false when a wait gave up.
+template <int LPK>
+__device__ __forceinline__ bool group_mma_tile(Shared* sh, uint8_t* tiles, uint32_t tmem_base, uint32_t& g, uint32_t it,
+                                               int num_kb, uint32_t idesc_lp, bool lead,
+                                               volatile uint32_t* abort_flag, uint32_t* err0) {
+  using C = Cfg<kProbe>;
+  constexpr int kStages = C::kStages;
+  constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
+  const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
+  const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
+  auto issue_ref = [&](uint32_t base, int kb) {
+    const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
+#pragma unroll
+    for (int k = 0; k < kBlockK / 16; ++k)
+      mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+  };
+  auto issue_rest = [&](uint32_t base, int kb) {
+    const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
+#pragma unroll
+    for (int k = 0; k < kBlockK / 16; ++k)
+      mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+    const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
+#pragma unroll
+    for (int k = 0; k < kBlockK / 32; ++k)
+      mma_pair<LPK>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
+  };
+  // reference MMAs of the first k-blocks go ahead of the hand-back of the previous tile
+  int kb = 0;
+  const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
+  for (int j = 0; j < n_ahead; ++j) {
+    const int s = (g + j) % kStages;
+    if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, err0)) return false;
+    tc_fence_after();
+    issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
+  }
+  if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, err0)) return false;
+  tc_fence_after();
+  for (; kb < n_ahead; ++kb, ++g) {
+    const int s = g % kStages;
+    issue_rest(smem_u32(tiles + (size_t)s * C::kStageBytes), kb);
+    tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+  }
+  for (; kb < num_kb; ++kb, ++g) {
+    const int s = g % kStages;
+    if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages) & 1, abort_flag, err0)) return false;
+    tc_fence_after();
+    const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+    issue_ref(base, kb);
+    issue_rest(base, kb);
+    tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+  }
+  if (it > 0 && !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, err0)) return false;
+  tc_commit_pair(smem_u32(&sh->tmem_full), lead);
+  return true;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 tc_group_kernel(const __grid_constant__ GroupTable tab) {
   using C = Cfg<kProbe>;
@@ -1193,56 +1250,10 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         }
         const GroupProblem& pr = tab.p[group_find(tab, pos)];
         const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
-        const uint32_t idesc_lp = pr.a.idesc_lp;
-        const bool is_i8 = pr.kind == kKindI8;
-        const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
-        const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
-        auto issue_ref = [&](uint32_t base, int kb) {
-          const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)
-            mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
-        };
-        auto issue_rest = [&](uint32_t base, int kb) {
-          const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 16; ++k)
-            mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
-          const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k) {
-            if (is_i8) mma_pair<kKindI8>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
-            else mma_pair<kKindF8>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
-          }
-        };
-        // reference MMAs of the first k-blocks go ahead of the hand-back of the previous tile
-        int kb = 0;
-        const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
-        for (int j = 0; j < n_ahead && ok; ++j) {
-          const int s = (g + j) % kStages;
-          if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, err0)) ok = false;
-          tc_fence_after();
-          if (ok) issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
-        }
+        ok = pr.kind == kKindI8
+                 ? group_mma_tile<kKindI8>(sh, tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, abort_flag, err0)
+                 : group_mma_tile<kKindF8>(sh, tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, abort_flag, err0);
         if (!ok) break;
-        if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, err0)) break;
-        tc_fence_after();
-        for (; kb < n_ahead; ++kb, ++g) {
-          const int s = g % kStages;
-          issue_rest(smem_u32(tiles + (size_t)s * C::kStageBytes), kb);
-          tc_commit_pair(smem_u32(&sh->empty[s]), lead);
-        }
-        for (; kb < num_kb; ++kb, ++g) {
-          const int s = g % kStages;
-          if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages) & 1, abort_flag, err0)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-          issue_ref(base, kb);
-          issue_rest(base, kb);
-          tc_commit_pair(smem_u32(&sh->empty[s]), lead);
-        }
-        if (ok && it > 0 && !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, err0)) ok = false;
-        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full), lead);
         ++it;
       }
     }
