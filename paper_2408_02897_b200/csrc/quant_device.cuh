@@ -241,7 +241,7 @@ __device__ __forceinline__ uint32_t block_max(uint32_t v) {
 // (multiply-high and shift; the magic numbers come from the host).
 struct FastDiv {
   uint32_t d, m, s;
-  __host__ explicit FastDiv(uint32_t div = 1) : d(div), m(0), s(0) {
+  __host__ FastDiv(uint32_t div = 1) : d(div), m(0), s(0) {
     if (d > 1) {
       while ((1ull << s) < d) ++s;                          // s = ceil(log2 d)
       m = (uint32_t)((((1ull << s) - d) << 32) / d + 1);
