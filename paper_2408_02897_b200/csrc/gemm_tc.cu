@@ -1239,7 +1239,6 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     // ------------------------------------------------------------ MMA issuer (leader CTA, converged warp)
     if (rank == 0) {
       const bool lead = elect_one();
-      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
       uint32_t g = 0, it = 0;
       bool ok = true;
       for (int r = 0; ok; ++r) {
