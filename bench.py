@@ -85,7 +85,7 @@ class ClockSampler:
              "clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"],
+                                          "-i", str(self.index), "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -299,7 +299,8 @@ def run_reference(args, ops, desc):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=500,
+                    help="timed steps (0.4 ms each: the default keeps the GPU under load long enough for the clock samples)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="bert_base_fwd")
@@ -311,7 +312,7 @@ def main():
 
     ops, desc = build_workload(args.workload)
     if args.impl == "reference":
-        if args.steps == 20 and args.warmup == 3:
+        if args.steps == 500 and args.warmup == 3:
             args.steps, args.warmup = 3, 1
         run_reference(args, ops, desc)
         return
