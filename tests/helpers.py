@@ -31,10 +31,8 @@ def gpu_probe(o):
 
 
 def _derived(rec):
-    n = max(rec["count"], 1)
-    sd, sr, sn = rec["sum_diff2"], rec["sum_ref2"], rec["sum_den2"]
-    return {"mean_be": rec["sum_be"] / n, "normwise_be": (sd / sn) ** 0.5 if sn > 0 else 0.0,
-            "rel_l2": (sd / sr) ** 0.5 if sr > 0 else 0.0}
+    d = oracle.derived(rec)
+    return {k: d[k] for k in ("mean_be", "normwise_be", "rel_l2")}
 
 
 def assert_record_close(got, want, rtol=1e-4, rtol_max=1e-3, what="", K=None):

@@ -58,6 +58,7 @@ def test_ref_and_den_brute_force():
 
 def test_hand_computed_2x2x2():
     be = codes_l = codes_r = None
+    lit = {}
     for line in open(os.path.join(GOLDEN, "hand_2x2x2.txt")):
         if line.startswith("be "):
             be = [Fraction(t) for t in line.split()[1:]]
@@ -65,6 +66,8 @@ def test_hand_computed_2x2x2():
             codes_l = [int(t) for t in line.split()[1:]]
         elif line.startswith("codes_r_kxn "):
             codes_r = [int(t) for t in line.split()[1:]]
+        elif not line.startswith("#") and len(line.split()) == 2:
+            lit[line.split()[0]] = float(line.split()[1])
     L = np.array([[127, -63.5], [0.5, 2.5]], np.float32)
     R = np.array([[1.5, 127], [-3.5, 10.25]], np.float32)
     rec, full = oracle.probe(L, R, "int8", "int8", "tensor", "tensor", full=True)
@@ -80,10 +83,18 @@ def test_hand_computed_2x2x2():
     assert abs(rec["sum_diff2"] - (97.25 ** 2 + 10.875 ** 2 + 69.125 ** 2)) < 1e-9
     assert rec["sum_ref2"] == 412.75 ** 2 + 15478.125 ** 2 + 64 + 89.125 ** 2
     assert rec["sum_den2"] == 412.75 ** 2 + 16779.875 ** 2 + 9.5 ** 2 + 89.125 ** 2
+    # the record's sums and every derived scalar against the stored hand-worked literals
+    for k in ("sum_diff2", "sum_ref2", "sum_den2"):
+        assert abs(rec[k] - lit[k]) <= 1e-15 * lit[k], k
     dv = oracle.derived(rec)
-    assert abs(dv["mean_be"] - float(sum(be)) / 4) < 1e-15
-    assert abs(dv["rel_l2"] - (rec["sum_diff2"] / rec["sum_ref2"]) ** 0.5) < 1e-15
-    assert abs(dv["snr_db"] - 10 * np.log10(rec["sum_ref2"] / rec["sum_diff2"])) < 1e-12
+    assert set(dv) == {"mean_be", "max_be", "normwise_be", "rel_l2", "snr_db"}
+    for k in dv:
+        assert abs(dv[k] - lit[k]) <= 1e-14 * abs(lit[k]), (k, dv[k], lit[k])
+    # degenerate records: an exact product has infinite SNR and zero errors, an empty one is all zero
+    exact = oracle.derived({"sum_be": 0.0, "max_be": 0.0, "sum_diff2": 0.0, "sum_ref2": 5.0, "sum_den2": 7.0, "count": 3})
+    assert exact["snr_db"] == float("inf") and exact["rel_l2"] == 0 and exact["normwise_be"] == 0 and exact["mean_be"] == 0
+    empty = oracle.derived({"sum_be": 0.0, "max_be": 0.0, "sum_diff2": 0.0, "sum_ref2": 0.0, "sum_den2": 0.0, "count": 0})
+    assert empty["mean_be"] == 0 and empty["rel_l2"] == 0 and empty["normwise_be"] == 0
 
 
 @pytest.mark.parametrize("fmt", FMTS)
