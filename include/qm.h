@@ -98,6 +98,15 @@ typedef struct {
   uint32_t reserved;
 } qm_metric_result;
 
+/* The scalars the probe reports, all from one statistics record (host arithmetic on a host
+ * copy of the record): mean and max of the inner-product-level backward error of Eq. 3, its
+ * norm-wise form sqrt(sum (C-Q)^2 / sum D^2), the relative L2 error sqrt(sum (C-Q)^2 / sum C^2)
+ * and the signal-to-noise ratio 10 log10(sum C^2 / sum (C-Q)^2) in dB (+inf for an exact
+ * product).  A ratio whose denominator sum is zero is reported as 0; count == 0 gives mean 0.
+ * rec and out are HOST pointers. */
+typedef struct { double mean_be, max_be, normwise_be, rel_l2, snr_db; } qm_metric_scalars_t;
+qm_status qm_metric_scalars(const qm_metric_result* rec, qm_metric_scalars_t* out);
+
 /* Power sums of all elements of one tensor (Experiments section: "mean, variance,
  * skew and Kurtosis" of the matmul inputs of the baseline).  With n = count,
  * mu = sum1/n and the raw moments r_k = sum_k/n:  variance m2 = r2 - mu^2,
@@ -110,6 +119,13 @@ typedef struct {
   uint32_t device_error;   /* QM_DEVERR_NONFINITE when a NaN or Inf was seen                */
   uint32_t reserved;
 } qm_tensor_stats_result;
+
+/* "mean, variance, skew and Kurtosis" (Experiments section) from the power sums of a record, by
+ * the formulas above: population central moments, kurtosis as the plain fourth standardised
+ * moment.  Evaluated in long double; an empty or constant tensor gives skew = kurtosis = 0.
+ * rec and out are HOST pointers. */
+typedef struct { double mean, variance, skew, kurtosis; } qm_tensor_moments_t;
+qm_status qm_tensor_moments(const qm_tensor_stats_result* rec, qm_tensor_moments_t* out);
 
 /* Eq. 2, RE = |v - v~| / |v|, over the non-zero elements of one tensor under Eq. 1,
  * split as in the Results section: an element is OVERFLOW when |v/delta| exceeds the
@@ -379,9 +395,6 @@ qm_status qm_metric_noalloc(const float* ref, const float* q, const float* den, 
  * Events are host objects; no device memory is involved.
  */
 int64_t qm_kernel_launches(void);
-/* Tag of the fused tensor-core kernel's current design; changes whenever that kernel changes,
- * so that stored profiler counters can be recognised as stale. */
-const char* qm_kernel_revision(void);
 qm_status qm_profile_enable(int32_t on);
 qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
 /* The same interval launch by launch, without ending it: for launch i (in issue order, up to

@@ -92,9 +92,13 @@ def quantize(x, fmt, delta, rounding="rtne", seed=0, stream=0):
     grid values, so no conversion instruction is involved.
     """
     x = _as_f32(x)
-    t = (x / _expand(delta, x)).astype(np.float32)      # IEEE float32 division
-    if not np.all(np.isfinite(t)):
+    if not (np.all(np.isfinite(x)) and np.all(np.isfinite(np.asarray(delta)))):
         raise ValueError("non-finite input")
+    with np.errstate(over="ignore"):
+        # IEEE float32 division.  With a scale that is not the tensor's own (a stale or shared one)
+        # the quotient of finite numbers can exceed the float32 range; it is then a magnitude above
+        # the largest expressible value and saturates like any other (the saturation rule).
+        t = (x / _expand(delta, x)).astype(np.float32)
     if rounding == "stochastic":
         return _quantize_stochastic(t, fmt, seed, stream)
     if rounding != "rtne":

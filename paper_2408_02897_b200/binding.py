@@ -4,7 +4,6 @@ Tensors are torch CUDA tensors (torch is used for device memory and streams); an
 product L.R is described by `operand_of(tensor, contract_dim)`.
 """
 import ctypes as C
-import math
 import os
 
 import torch
@@ -39,12 +38,19 @@ class MetricResult(C.Structure):
         return {k: getattr(self, k) for k in ("sum_be", "max_be", "sum_diff2", "sum_ref2", "sum_den2", "count")}
 
     def derived(self):
-        n = max(self.count, 1)
-        sd, sr, sn = self.sum_diff2, self.sum_ref2, self.sum_den2
-        return {"mean_be": self.sum_be / n, "max_be": self.max_be,
-                "normwise_be": math.sqrt(sd / sn) if sn > 0 else 0.0,
-                "rel_l2": math.sqrt(sd / sr) if sr > 0 else 0.0,
-                "snr_db": 10.0 * math.log10(sr / sd) if sd > 0 and sr > 0 else float("inf")}
+        """mean BE, max BE, norm-wise BE, relative L2, SNR [dB] of the record (qm_metric_scalars)."""
+        out = MetricScalars()
+        _check(lib().qm_metric_scalars(C.byref(self), C.byref(out)), "qm_metric_scalars")
+        return {k: getattr(out, k) for k, _ in out._fields_}
+
+
+class MetricScalars(C.Structure):
+    _fields_ = [("mean_be", C.c_double), ("max_be", C.c_double), ("normwise_be", C.c_double),
+                ("rel_l2", C.c_double), ("snr_db", C.c_double)]
+
+
+class TensorMoments(C.Structure):
+    _fields_ = [("mean", C.c_double), ("variance", C.c_double), ("skew", C.c_double), ("kurtosis", C.c_double)]
 
 
 class TensorStats(C.Structure):
@@ -53,17 +59,10 @@ class TensorStats(C.Structure):
                 ("reserved", C.c_uint32)]
 
     def derived(self):
-        """mean, variance, skew, kurtosis from the power sums (population moments)."""
-        n = self.count
-        if n == 0:
-            return {"mean": 0.0, "variance": 0.0, "skew": 0.0, "kurtosis": 0.0}
-        mu, r2, r3, r4 = self.sum1 / n, self.sum2 / n, self.sum3 / n, self.sum4 / n
-        m2 = r2 - mu * mu
-        m3 = r3 - 3 * mu * r2 + 2 * mu ** 3
-        m4 = r4 - 4 * mu * r3 + 6 * mu * mu * r2 - 3 * mu ** 4
-        ok = m2 > 0
-        return {"mean": mu, "variance": m2, "skew": m3 / m2 ** 1.5 if ok else 0.0,
-                "kurtosis": m4 / (m2 * m2) if ok else 0.0}
+        """mean, variance, skew, kurtosis of the tensor (qm_tensor_moments)."""
+        out = TensorMoments()
+        _check(lib().qm_tensor_moments(C.byref(self), C.byref(out)), "qm_tensor_moments")
+        return {k: getattr(out, k) for k, _ in out._fields_}
 
 
 class QuantError(C.Structure):
@@ -105,6 +104,8 @@ def lib():
             "qm_gemm_ref": (I32, [P, P, I64, I64, I64, I64, P, P]),
             "qm_metric_workspace_bytes": (SZ, [I64]),
             "qm_metric": (I32, [P, P, P, I64, P, P, SZ, P]),
+            "qm_metric_scalars": (I32, [C.POINTER(MetricResult), C.POINTER(MetricScalars)]),
+            "qm_tensor_moments": (I32, [C.POINTER(TensorStats), C.POINTER(TensorMoments)]),
             "qm_workspace_bytes": (SZ, [OP, OP, C.POINTER(ProbeCfg)]),
             "qm_probe_layer": (I32, [OP, OP, C.POINTER(ProbeCfg), P, P, SZ, P]),
             "qm_workspace_bytes2": (SZ, [OP, OP, C.POINTER(ProbeCfg), C.POINTER(ProbeCfg)]),
@@ -122,7 +123,6 @@ def lib():
             "qm_last_cuda_error": (C.c_char_p, []),
             "qm_metric_noalloc": (I32, [P, P, P, I64, P, P]),
             "qm_metric_noalloc_max_count": (I64, []),
-            "qm_kernel_revision": (C.c_char_p, []),
             "qm_kernel_launches": (I64, []),
             "qm_profile_enable": (I32, [I32]),
             "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),

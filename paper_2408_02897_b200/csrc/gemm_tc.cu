@@ -1493,8 +1493,23 @@ void fill_tiles(KernelArgs* ka, GemmShape g) {
 }
 
 // CTA pairs that can be resident at once (one per TPC unless the device says fewer).
-int g_max_pairs = 0;
-int max_pairs() { return g_max_pairs > 0 ? g_max_pairs : sm_count() / 2; }
+int g_max_pairs[kMaxDevices] = {};     // per device; 0 = not yet queried
+int max_pairs() {
+  const int dev = current_device();
+  return dev >= 0 && g_max_pairs[dev] > 0 ? g_max_pairs[dev] : sm_count() / 2;
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device.
+template <typename K>
+qm_status allow_smem(K kern, size_t bytes, bool (&done)[kMaxDevices]) {
+  const int dev = current_device();
+  if (dev < 0) return QM_ERR_UNSUPPORTED;
+  if (!done[dev]) {
+    QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    done[dev] = true;
+  }
+  return QM_OK;
+}
 
 // CTAs to launch: two per tile, at most the resident number of pairs.
 int grid_size(GemmShape g) {
@@ -1507,12 +1522,11 @@ int grid_size(GemmShape g) {
 template <int MODE, int LPKIND, int LPKIND2 = LPKIND>
 qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cudaStream_t s) {
   auto kern = tc_kernel<MODE, LPKIND, LPKIND2>;
-  static bool attr_done = false;     // per instantiation
-  if (!attr_done) {
-    QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<MODE>()));
-    attr_done = true;
-  }
-  if (MODE == kProbe && g_max_pairs == 0) {
+  static bool attr_done[kMaxDevices] = {};     // per instantiation
+  const qm_status as = allow_smem(kern, smem_bytes<MODE>(), attr_done);
+  if (as != QM_OK) return as;
+  const int dev = current_device();
+  if (MODE == kProbe && g_max_pairs[dev] == 0) {
     // the probe configuration has the largest footprint: its residency bounds the grid of all modes
     cudaLaunchConfig_t q{};
     q.gridDim = dim3((unsigned)(2 * (sm_count() / 2))); q.blockDim = dim3(kThreads);
@@ -1523,9 +1537,9 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
     q.attrs = qa; q.numAttrs = 1;
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &q) == cudaSuccess && n > 0)
-      g_max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+      g_max_pairs[dev] = n < sm_count() / 2 ? n : sm_count() / 2;
     else
-      g_max_pairs = sm_count() / 2;
+      g_max_pairs[dev] = sm_count() / 2;
     (void)cudaGetLastError();
   }
   cudaLaunchConfig_t cfg{};
@@ -1557,11 +1571,9 @@ template <int KIND>
 qm_status launch_wide(const CUtensorMap& ma, const CUtensorMap& mb, KernelArgs ka, GemmShape g, cudaStream_t s) {
   auto kern = tc_gemm_wide_kernel<KIND>;
   constexpr size_t smem = (size_t)kWideStages * kWideStageBytes + sizeof(SharedWide) + 1024;
-  static bool attr_done = false;
-  if (!attr_done) {
-    QM_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attr_done = true;
-  }
+  static bool attr_done[kMaxDevices] = {};
+  const qm_status as = allow_smem(kern, smem, attr_done);
+  if (as != QM_OK) return as;
   ka.tiles_m = (int32_t)((g.M + kPairM - 1) / kPairM);
   ka.tiles_n = (int32_t)((g.N + kWideN - 1) / kWideN);
   const int64_t tiles = (int64_t)ka.tiles_m * ka.tiles_n * g.batch;
@@ -1629,12 +1641,9 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     if (total >= (1ll << 31)) return QM_ERR_UNSUPPORTED;
   }
   tab.total_tiles = (int32_t)total;
-  static bool attr_done = false;
-  if (!attr_done) {
-    QM_CUDA_OK(cudaFuncSetAttribute(tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)smem_bytes<kProbe>()));
-    attr_done = true;
-  }
+  static bool attr_done[kMaxDevices] = {};
+  const qm_status as = allow_smem(tc_group_kernel, smem_bytes<kProbe>(), attr_done);
+  if (as != QM_OK) return as;
   const int pairs = max_pairs();
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(2 * (total < pairs ? total : pairs)));

@@ -136,7 +136,6 @@ static __device__ __align__(256) double g_noalloc_partials[kNoAllocRecords * kPa
 
 // In host code the array's name is only a handle for the runtime, not a device address: the
 // address the kernels need is looked up once per device (with that device current) and cached.
-constexpr int kMaxDevices = 64;
 double* g_noalloc_ptr[kMaxDevices] = {};
 
 qm_status noalloc_scratch(double** out) {

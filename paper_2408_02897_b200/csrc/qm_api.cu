@@ -18,15 +18,22 @@ void note_cuda_error(cudaError_t e, const char* where) {
   (void)cudaGetLastError();   // do not let a non-sticky error be blamed on a later call
 }
 
+int current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
+  static std::atomic<int> n[kMaxDevices];
+  const int dev = current_device();
+  if (dev < 0) return 148;
+  int v = n[dev].load(std::memory_order_relaxed);
+  if (v == 0) {
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n[dev].store(v, std::memory_order_relaxed);
   }
-  return n;
+  return v;
 }
 
 bool pdl_enabled() {
@@ -609,11 +616,10 @@ struct BatchStreams {
 };
 // One set per device, created on first use (never inside a stream capture) and kept.
 qm_status batch_streams(BatchStreams** out) {
-  static BatchStreams pool[64];
+  static BatchStreams pool[kMaxDevices];
   static std::mutex mu;
-  int dev = 0;
-  QM_CUDA_OK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return QM_ERR_UNSUPPORTED;
+  const int dev = current_device();
+  if (dev < 0) return QM_ERR_UNSUPPORTED;
   std::lock_guard<std::mutex> lock(mu);
   BatchStreams& b = pool[dev];
   if (!b.ready) {
@@ -810,8 +816,6 @@ const char* qm_status_string(int32_t st) {
 int32_t qm_version(void) { return 100; }
 
 const char* qm_last_cuda_error(void) { return qm::g_last_error; }
-
-const char* qm_kernel_revision(void) { return "tc-group-rot4-refahead-2"; }
 
 int64_t qm_kernel_launches(void) { return (int64_t)qm::g_launches.load(); }
 

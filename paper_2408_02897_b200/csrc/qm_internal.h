@@ -33,7 +33,11 @@ void note_cuda_error(cudaError_t e, const char* where);
     }                                                      \
   } while (0)
 
-int sm_count();
+// One-time host state (function attributes, occupancy, SM counts, stream pools, symbol addresses)
+// is kept per device, indexed by the current device's ordinal.
+constexpr int kMaxDevices = 64;
+int current_device();   // the ordinal, or -1 when it cannot be read or is not below kMaxDevices
+int sm_count();         // of the current device
 
 // Programmatic dependent launch.  Every kernel of the probe's chain is launched with the
 // attribute that lets its CTAs be scheduled while the kernel before it in the stream is still

@@ -102,7 +102,10 @@ struct Quotient {
     const float q0 = x * recip;
     const float q1 = fmaf(fmaf(-q0, delta, x), recip, q0);
     const float q = fmaf(fmaf(-q1, delta, x), recip, q1);
-    return copysignf(q, x);                                   // keeps the sign of a zero input
+    // A delta handed in from elsewhere (stale, shared) can make x * recip overflow; the corrections
+    // then evaluate inf - inf.  fminf returns its non-NaN operand, so that case comes out as the
+    // largest float and saturates in the conversion, as the division would.
+    return copysignf(fminf(fabsf(q), 3.402823466e38f), x);    // keeps the sign of a zero input
   }
 };
 

@@ -101,9 +101,18 @@ struct Batch {
       const float x = xs[h];
       const bool nz = x != 0.f;
       const float err = fabsf(fmaf(-gs[h], ds[h], x));        // |x - value(code) delta|, one rounding
-      float rcp;
-      asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(fabsf(x)));
-      const float re = nz ? err * rcp : 0.f;
+      // |x| below the normal range (a subnormal bf16 or fp32 element) would be flushed by the
+      // approximate reciprocal: those rare elements take the division, which also makes the RE
+      // of an underflowed one (err == |x|) exactly 1
+      const float ax = fabsf(x);
+      float re;
+      if (ax >= 1e-36f) {
+        float rcp;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rcp) : "f"(ax));
+        re = err * rcp;
+      } else {
+        re = nz ? __fdiv_rn(err, ax) : 0.f;
+      }
       const float e2 = err * err;
       const bool over = fabsf(ts[h]) > qmaxv;
       const bool under = nz && !over && gs[h] == 0.f;
@@ -313,12 +322,15 @@ int pass_blocks(const Lines& p, int resident_per_sm) {
 
 template <typename T, int KIND, int FMT>
 qm_status launch_pass(const Lines& p, void* result, uint64_t count, void* ws, cudaStream_t s) {
-  static int resident = 0;                       // per instantiation; the same on every device
-  if (resident == 0) {
+  static int resident_of[kMaxDevices] = {};      // per instantiation and device
+  const int dev = current_device();
+  if (dev < 0) return QM_ERR_UNSUPPORTED;
+  if (resident_of[dev] == 0) {
     int nb = 0;
     QM_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, tensor_pass_kernel<T, KIND, FMT>, kThreads, 0));
-    resident = nb > 0 ? nb : 1;
+    resident_of[dev] = nb > 0 ? nb : 1;
   }
+  const int resident = resident_of[dev];
   uint32_t* counter = static_cast<uint32_t*>(ws);
   double* partials = reinterpret_cast<double*>(static_cast<char*>(ws) + kCounterBytes);
   QM_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), s));

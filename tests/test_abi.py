@@ -32,7 +32,8 @@ def test_struct_layouts_match_header(tmp_path):
     import subprocess
     pairs = [("qm_metric_result", binding.MetricResult), ("qm_operand", binding.Operand),
              ("qm_probe_cfg", binding.ProbeCfg), ("qm_tensor_stats_result", binding.TensorStats),
-             ("qm_quant_error_result", binding.QuantError)]
+             ("qm_quant_error_result", binding.QuantError), ("qm_metric_scalars_t", binding.MetricScalars),
+             ("qm_tensor_moments_t", binding.TensorMoments)]
     lines = []
     for cname, cls in pairs:
         lines.append(f'printf("{cname} %zu", sizeof({cname}));')
@@ -110,3 +111,40 @@ def test_batch_and_two_format_argument_checks_need_no_gpu():
     op = binding.Operand()
     assert L.qm_tensor_stats(C.byref(op), None, None, 0, None) == 1                   # null data
     assert L.qm_scale_shared(C.byref(op), 1, 1, None, None) == 1
+
+
+def test_derived_scalars_come_from_the_library():
+    """qm_metric_scalars on the record of the hand-computed 2x2x2 case (tests/golden/hand_2x2x2.txt
+    holds the record's sums and the scalars worked out by hand), and qm_tensor_moments on small
+    arrays whose moments are known in closed form."""
+    lit = {}
+    for line in open(os.path.join(ROOT, "tests", "golden", "hand_2x2x2.txt")):
+        w = line.split()
+        if len(w) == 2 and not line.startswith("#"):
+            lit[w[0]] = float(w[1])
+    rec = binding.MetricResult(4 * lit["mean_be"], lit["max_be"], lit["sum_diff2"], lit["sum_ref2"], lit["sum_den2"], 4, 0, 0)
+    got = rec.derived()
+    assert set(got) == {"mean_be", "max_be", "normwise_be", "rel_l2", "snr_db"}
+    for k, v in got.items():
+        assert abs(v - lit[k]) <= 1e-14 * abs(lit[k]), (k, v, lit[k])
+    exact = binding.MetricResult(0.0, 0.0, 0.0, 5.0, 7.0, 3, 0, 0).derived()
+    assert exact["snr_db"] == float("inf") and exact["rel_l2"] == 0 and exact["normwise_be"] == 0
+    empty = binding.MetricResult(0.0, 0.0, 0.0, 0.0, 0.0, 0, 0, 0).derived()
+    assert all(empty[k] == 0 for k in ("mean_be", "max_be", "normwise_be", "rel_l2"))
+    L = qm.lib()
+    assert L.qm_metric_scalars(None, None) == 1 and L.qm_tensor_moments(None, None) == 1
+
+    def moments(xs):
+        t = binding.TensorStats(sum(xs), sum(x ** 2 for x in xs), sum(x ** 3 for x in xs), sum(x ** 4 for x in xs),
+                                max(abs(x) for x in xs), len(xs), 0, 0)
+        return t.derived()
+    m = moments([1, 2, 3, 4])                     # mean 5/2, variance 5/4, symmetric, m4 = 41/16
+    assert m["mean"] == 2.5 and m["variance"] == 1.25 and m["skew"] == 0.0 and abs(m["kurtosis"] - 1.64) < 1e-15
+    m = moments([0, 0, 0, 4])                     # mean 1, m2 = 3, m3 = 6, m4 = 21
+    assert m["mean"] == 1 and m["variance"] == 3 and abs(m["skew"] - 6 / 3 ** 1.5) < 1e-15 and abs(m["kurtosis"] - 21 / 9) < 1e-15
+    m = moments([7, 7, 7])                        # constant tensor: no spread, skew and kurtosis reported as 0
+    assert m == {"mean": 7.0, "variance": 0.0, "skew": 0.0, "kurtosis": 0.0}
+    # a badly centred tensor (mean / sigma = 1e4): the extended-precision evaluation keeps the variance
+    xs = [10000 + d for d in (-1, 0, 1)] * 5
+    m = moments(xs)
+    assert abs(m["variance"] - 2 / 3) < 1e-6 and abs(m["skew"]) < 1e-3

@@ -214,3 +214,20 @@ def test_extreme_scales_take_the_division_path():
         t = torch.from_numpy(x[0]).cuda()
         codes, _, _, _ = qm.qm_quantize(qm.operand_of(t, -1), "e4m3", "tensor", torch.from_numpy(dd).cuda())
         assert np.array_equal(codes.cpu().numpy(), want), d
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_supplied_scale_that_overflows_the_quotient_saturates(fmt, dtype):
+    """A scale handed in from elsewhere can make x / delta exceed the float32 range; such elements
+    saturate at the largest expressible value (codes against the oracle, bit for bit)."""
+    t = make((40, 64), dtype, 9)
+    t[0, 0] = 3e38; t[1, 5] = -3e38; t[2, 7] = 1e30; t[3, 3] = -2.5e35
+    for dv in (1e-12, 3e-9, 2.0 ** -70):          # the corrected-reciprocal path and the division path
+        d = np.array([dv], dtype=np.float32)
+        x = as3(oriented(t, -1))
+        want = oracle.quantize(x, fmt, d)
+        codes, _, _, _ = qm.qm_quantize(qm.operand_of(t.cuda(), -1), fmt, "tensor", torch.from_numpy(d).cuda())
+        assert np.array_equal(codes.cpu().numpy()[..., :64], want)
+        v = oracle.dequantize(want, fmt)
+        assert v[0, 0, 0] == oracle.qmax(fmt) and v[0, 1, 5] == -oracle.qmax(fmt)

@@ -133,6 +133,26 @@ def test_error_with_outside_scale_overflows(fmt):
     assert want["n_overflow"] > 0 and want["err2_overflow"] > 0
 
 
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_error_with_subnormal_elements(fmt, dtype):
+    """Non-zero elements below the normal range of float32 (bf16 subnormals are float32 subnormals):
+    their code is zero, so each is an underflow with RE exactly 1 and the sums stay finite."""
+    t = tensor((32, 64), dtype, 27)
+    sub = torch.tensor([1e-39, -3e-40, 2.0 ** -133, -2.0 ** -130], dtype=torch.float32).to(dtype)
+    assert (sub != 0).all()
+    t[3, 10:14] = sub
+    t[7, 0] = sub[0]
+    got, want = check_error(t, -1, fmt, "tensor")
+    assert want["n_underflow"] >= 5 and np.isfinite(got.sum_re)
+    check_error(t, -1, fmt, "channel")
+    # a tensor made only of such elements: scales are subnormal themselves, codes are not zero
+    tiny = (tensor((8, 64), torch.float32, 28) * 1e-39).to(dtype)
+    check_error(tiny, -1, fmt, "tensor")
+    got_s, _ = check_stats(t)
+    assert got_s.device_error == 0
+
+
 def test_error_large_dense_and_repeatable():
     t = tensor((2048, 4096), torch.bfloat16, 26, scale=0.02)
     got, _ = check_error(t, -1, "e4m3", "tensor")

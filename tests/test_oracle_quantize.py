@@ -258,3 +258,20 @@ def test_batch_groups_equal_a_per_channel_scale_of_the_regrouped_tensor():
     # coarser sharing never gives a smaller scale, and quantization error cannot shrink with it
     own = oracle.scale(x, "e4m3", "channel")
     assert np.all(got >= own) and np.all(oracle.scale(x, "e4m3", "channel", 1) >= got)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_quotient_beyond_float32_saturates(fmt):
+    """Finite inputs under a much smaller outside scale: x / delta overflows float32, which is a
+    magnitude above the largest expressible value and must saturate (Methodology, saturation rule),
+    with the sign kept; non-finite inputs or scales remain errors."""
+    x = np.array([[3e38, -3e38, 1e30, -0.0, 2e-30]], dtype=np.float32)
+    d = np.array([1e-30], dtype=np.float32)
+    v = oracle.dequantize(oracle.quantize(x, fmt, d), fmt)
+    top = oracle.qmax(fmt)
+    assert v[0, 0] == top and v[0, 1] == -top and v[0, 2] == top and v[0, 3] == 0
+    assert v[0, 4] == 2.0
+    with pytest.raises(ValueError):
+        oracle.quantize(np.array([[np.inf]], dtype=np.float32), fmt, d)
+    with pytest.raises(ValueError):
+        oracle.quantize(x, fmt, np.array([np.nan], dtype=np.float32))
