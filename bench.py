@@ -2,12 +2,15 @@
 """Benchmark of the quantized-matmul error probe on B200.
 
 A step is one pass of the whole probe path (scale, quantize, 8-bit product, reference and
-denominator products, Eq. 3 reduction) over every product of the workload.  The default
-workload is the BERT-base forward set (batch 8 x seq 512: QKV, attention output, FFN1, FFN2;
-E4M3 and INT8 with per-tensor scales): 8 probes per step.
+denominator products, Eq. 3 reduction) over every product of the workload, repeated `repeat`
+times so that a step lasts tens of milliseconds.  The default workload is the unit of the
+24-layer BERT-large sweep: one encoder layer (batch 32 x seq 512), its four projections forward,
+dgrad and wgrad plus the six batched attention products, each in E4M3, E5M2 and INT8: 54 probes.
 
   python bench.py --gpus 1 --steps K --warmup W            -> one JSON line (this library)
   python bench.py --impl reference ...                     -> one JSON line (CPU oracle)
+  python bench.py --case quantize|stats|gemm|probe|batch   -> a few launches of one small case
+                                                              (the command profiler captures run)
 
 With N > 1 ranks (torchrun) every rank probes its own copy of the workload: the probes of a
 table are independent, there is no exchange step, so scaling is weak and no collective runs
@@ -29,16 +32,11 @@ sys.path.insert(0, ROOT)
 
 from paper_2408_02897_b200 import workloads  # noqa: E402
 
-# DRAM traffic of the fused probe kernel from one ncu capture (profiles/tc_kernel_probe_*.md):
-# dram__bytes_read + dram__bytes_write for M=4096 N=2304 K=768 E4M3, and the library's kernel
-# revision the counters were taken at.  Traffic grows with the operand bytes (every operand is
-# read from DRAM once), so a launch of another shape is scaled by its operand bytes.
-NCU_TC = {"revision": "tc-group-rot4-refahead-2", "workload": "bert_base_fwd", "dram_bytes": 200.0e6}
-
-
-def tc_operand_bytes(M, N, K, b=1):
-    """Bytes the fused kernel reads per launch: L, |L| (bf16), R, |R| (bf16) and both code tensors."""
-    return b * ((M + N) * K * 2 * 2 + (M + N) * K)
+# DRAM bytes (read + write) of the grouped fused kernel per byte of distinct operand data it reads
+# (bf16 L, R, their |x| copies and both code tensors), from a profiler capture of the BERT-base
+# workload's launch; every operand byte is read from DRAM once, so a launch of another workload is
+# scaled by its distinct operand bytes.  None: the kernel has changed since the counters were taken.
+TC_DRAM_BYTES_PER_OPERAND_BYTE = None
 
 
 METRIC = "probe TFLOPS"
@@ -50,11 +48,18 @@ def load_peaks():
     if os.path.exists(p):
         d = json.load(open(p))
         return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
-                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "peak_run_sm_mhz": (d.get("clocks_under_load") or {}).get("sm_mhz_median"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "peak_run_sm_mhz": 1300.0,
+            "source": "fallback"}
 
 
 def build_workload(name):
+    if name == "bert_large_sweep_layer":
+        t = workloads.config5_layer_tensors(0)
+        ops = [o for fmt in ("e4m3", "e5m2", "int8") for o in workloads.config5_layer(0, fmt, tensors=t)]
+        return ops, ("one layer of the BERT-large 24-layer sweep (batch 32 x seq 512): projections fwd+dgrad+wgrad and "
+                     "batched attention products fwd+bwd, each in E4M3, E5M2 and INT8, per-tensor scales")
     if name == "bert_base_fwd":
         return workloads.config2(), "BERT-base forward matmuls (batch 8 x seq 512), E4M3 + INT8, per-tensor scales"
     if name == "bert_large_layer":
@@ -64,6 +69,22 @@ def build_workload(name):
     if name == "single":
         return workloads.config1(), "single fp32 probe 128x256x256"
     raise SystemExit(f"unknown workload {name}")
+
+
+def distinct_operand_bytes(ops):
+    """Bytes the fused kernels of a step read when every distinct tensor is counted once: bf16 x and
+    |x| of each distinct (tensor, orientation) and one code tensor per distinct (tensor, orientation,
+    format)."""
+    seen_x, seen_c, total = set(), set(), 0
+    for o in ops:
+        for t, cd, fmt in ((o["L"], o["cl"], o["fmt_l"]), (o["R"], o["cr"], o["fmt_r"])):
+            if (id(t), cd) not in seen_x:
+                seen_x.add((id(t), cd))
+                total += 4 * t.numel()
+            if (id(t), cd, fmt) not in seen_c:
+                seen_c.add((id(t), cd, fmt))
+                total += t.numel()
+    return total
 
 
 def probe_flops(ops):
@@ -94,9 +115,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Median SM clock and throttle reasons of the samples that arrived between host times t0
+        and t1 (the timed region); all samples when no window is given."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -106,8 +129,8 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            if len(r) < 7:
+        for ts, r in self.rows:
+            if len(r) < 7 or (t0 is not None and not (t0 <= ts <= t1)):
                 continue
             try:
                 sm.append(float(r[0])); mx.append(float(r[1]))
@@ -117,12 +140,20 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "samples_total": len(self.rows), "window": "timed region only",
+                "reasons": sorted(reasons)}
+
+
+def oracle_sample_ops(ops, max_ops=4):
+    """The bounded sample of a workload the CPU oracle is timed on: its first `max_ops` probes whose
+    operands are plain 2-D matrices (the projections), or the first ones if there are none."""
+    flat = [o for o in ops if o["L"].dim() == 2]
+    return (flat or ops)[:max_ops]
 
 
 def time_oracle_sample(ops, rows_per_op, seed=7):
     """The CPU oracle, as it stands, on a bounded sample: `rows_per_op` output rows (all
-    columns) of every probe; scales and codes are still computed over the whole operands."""
+    columns) of every given probe; scales and codes are still computed over the whole operands."""
     import oracle
     t0 = time.perf_counter()
     flops = 0.0
@@ -273,46 +304,237 @@ def cpu_threads():
     return os.cpu_count()
 
 
+def config_of(args, desc):
+    """The `config` object of the JSON line, identical for both arms."""
+    return {"workload": args.workload, "description": desc,
+            "flops_counted": "3 x 2MNK per probe (8-bit, reference and denominator products)",
+            "l2": "256 MiB buffer written between timed steps; the inputs of the default workload are larger than L2 as well"}
+
+
+def oracle_sample_text(sample, rows, n_all):
+    return (f"{rows} of the output rows of each of {len(sample)} of the workload's {n_all} probes "
+            f"({', '.join(o['name'] for o in sample)}); scales and codes over whole operands")
+
+
 def run_reference(args, ops, desc):
     """--impl reference: the oracle on the host cores, each step a bounded sample."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     rows = args.oracle_rows
+    sample = oracle_sample_ops(ops)
     for _ in range(min(args.warmup, 1)):
-        time_oracle_sample(ops, rows)
+        time_oracle_sample(sample, rows)
     flops = secs = 0.0
     for _ in range(args.steps):
-        f, t = time_oracle_sample(ops, rows)
+        f, t = time_oracle_sample(sample, rows)
         flops += f; secs += t
     val = flops / secs / 1e12
-    sample = f"{rows} of the output rows of each of the {len(ops)} probes per step (scales and codes over whole operands)"
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "description": desc},
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "config": config_of(args, desc),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                             "sample": oracle_sample_text(sample, rows, len(ops)) + " per step"},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
+
+
+def run_case(a):
+    """--case: a few launches of one kernel family on a small synthetic case and nothing else; the
+    command that profiler captures run."""
+    import paper_2408_02897_b200 as qm
+    torch.cuda.set_device(0)
+    rng = workloads._rng(11)
+    if a.case == "batch":
+        ops, _ = build_workload(a.workload)
+        on_dev = {}
+        dev = [(on_dev.setdefault(id(o["L"]), o["L"].cuda()), on_dev.setdefault(id(o["R"]), o["R"].cuda())) for o in ops]
+        batch = qm.ProbeBatch([(qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"]), o["fmt_l"], o["fmt_r"],
+                                o["gran_l"], o["gran_r"], o["ref"]) for o, (Ld, Rd) in zip(ops, dev)])
+        for _ in range(a.iters):
+            batch.launch()
+        torch.cuda.synchronize()
+        print("mean_be", [round(r.derived()["mean_be"], 6) for r in batch.results()])
+        return
+    lead = (a.batch,) if a.batch > 1 else ()
+    L = workloads.normal(rng, lead + (a.M, a.K)).cuda()
+    R = workloads.normal(rng, lead + ((a.K, a.N) if a.r_layout == "kn" else (a.N, a.K)), 0.02).cuda()
+    Lop = qm.operand_of(L, -1)
+    Rop = qm.operand_of(R, -2 if a.r_layout == "kn" else -1)
+    if a.case == "probe":
+        plan = qm.ProbePlan(Lop, Rop, a.fmt, a.fmt, a.gran, a.gran)
+        for _ in range(a.iters):
+            plan.launch(Lop, Rop)
+        torch.cuda.synchronize()
+        r = plan.result()
+        print("mean_be", r.derived()["mean_be"], "device_error", r.device_error)
+    elif a.case == "gemm":
+        Rk = R.transpose(-1, -2).contiguous() if a.r_layout == "kn" else R
+        cl, dl, _, _ = qm.qm_quantize(Lop, a.fmt, a.gran)
+        cr, dr, _, _ = qm.qm_quantize(qm.operand_of(Rk, -1), a.fmt, a.gran)
+        L3 = L if L.dim() == 3 else L[None]
+        R3 = Rk if Rk.dim() == 3 else Rk[None]
+        for _ in range(a.iters):
+            out, _ = qm.qm_gemm(cl, a.fmt, dl, a.gran, cr, a.fmt, dr, a.gran, a.K)
+            ref = qm.qm_gemm_ref(L3, R3)
+        torch.cuda.synchronize()
+        print("rel diff of the two products", float((out - ref).norm() / ref.norm()))
+    elif a.case == "stats":
+        for _ in range(a.iters):
+            st = qm.qm_tensor_stats(Lop)
+            er = qm.qm_quantize_error(Lop, a.fmt, a.gran)
+        print("kurtosis", st.derived()["kurtosis"], "mean RE", er.sum_re / max(er.n_nonzero, 1))
+    elif a.case == "quantize":
+        Lt = qm.operand_of(L, -2)
+        for _ in range(a.iters):
+            qm.qm_scale(Lop, a.fmt, "tensor")
+            qm.qm_quantize(Lop, a.fmt, "tensor", None)
+            qm.qm_quantize(Lop, a.fmt, "channel", None)
+            qm.qm_quantize(Lt, a.fmt, "tensor", None)
+        torch.cuda.synchronize()
+        print("done")
+    else:
+        raise SystemExit(f"unknown case {a.case}")
+
+
+def time_workload(qm, ranks, world, name, steps, warmup, target_ms=50.0, clock_index=None):
+    """Times `steps` steps of a workload resident in HBM.  A step is `repeat` passes over the
+    workload's probes (one qm_probe_batch call per pass) between one CUDA-event pair, with the L2
+    flushed before it.  Returns a dict of the measurements."""
+    ops, desc = build_workload(name)
+    on_dev = {}
+
+    def resident(t):
+        # a tensor that several probes share (a layer probed in several formats, an activation that
+        # feeds several products) is resident once
+        if id(t) not in on_dev:
+            on_dev[id(t)] = t.cuda()
+        return on_dev[id(t)]
+    batch = qm.ProbeBatch([(qm.operand_of(resident(o["L"]), o["cl"]), qm.operand_of(resident(o["R"]), o["cr"]),
+                            o["fmt_l"], o["fmt_r"], o["gran_l"], o["gran_r"], o["ref"]) for o in ops])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+
+    def barrier():
+        torch.cuda.synchronize()
+        ranks.barrier(world)
+        torch.cuda.synchronize()
+
+    # repeat count from one measured pass, so that a step lasts about target_ms
+    batch.launch()
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(); batch.launch(); b.record()
+    barrier()
+    pass_ms = ranks.max_over_ranks(a.elapsed_time(b), world, "cuda")
+    repeat = max(1, int(np.ceil(target_ms / pass_ms)))
+
+    def step():
+        for _ in range(repeat):
+            batch.launch()
+
+    for _ in range(max(warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(clock_index) if clock_index is not None else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.5)               # nvidia-smi needs a moment to start; samples outside the window are dropped
+    launches0 = qm.kernel_launches()
+    qm.profile_enable(True)           # the library records an event pair around each fused launch
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    barrier()
+    t0 = time.time()
+    for a, b in evs:
+        flush.zero_()
+        a.record()
+        step()
+        b.record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    tc_ms, tc_launches = qm.profile_read()
+    qm.profile_enable(False)
+    launches = qm.kernel_launches() - launches0
+    total_ms = ranks.max_over_ranks(float(sum(step_ms)), world, "cuda")
+    results = batch.results()
+    if any(r.device_error for r in results):
+        raise SystemExit("device error flagged in a probe result")
+    flops_pass = probe_flops(ops)
+    return {"ops": ops, "desc": desc, "results": results, "repeat": repeat, "total_ms": total_ms, "steps": steps,
+            "flops_step": flops_pass * repeat, "flops_pass": flops_pass, "tc_ms": tc_ms, "tc_launches": tc_launches,
+            "launches": int(launches), "clocks": clocks, "wall_s": t1 - t0,
+            "value": ranks.whole_job_rate(flops_pass * repeat * steps, world, total_ms) / 1e12}
+
+
+def roofline_of(m, peaks, bench_mhz):
+    """The roofline block of the dominant kernel (the grouped fused probe kernel) of a measurement.
+
+    Composite tensor bound: per 2MNK one product at the 8-bit rate (2 x bf16) and two at the bf16
+    rate -> 3 / (1/(2P) + 2/P) = 1.2 P in summed flops.  P is the sustained bf16 figure when the
+    timed region lasted seconds (the kernel then runs under the same power cap as that
+    measurement), the burst figure otherwise."""
+    long_region = m["wall_s"] >= 1.0 and peaks.get("bf16_tflops_sustained")
+    p16 = peaks["bf16_tflops_sustained"] if long_region else peaks["bf16_tflops"]
+    peak = 1.2 * p16
+    achieved = m["flops_step"] * m["steps"] / (m["tc_ms"] * 1e-3) / 1e12 if m["tc_ms"] > 0 else None
+    traffic = None
+    if TC_DRAM_BYTES_PER_OPERAND_BYTE is not None and m["tc_launches"]:
+        traffic = TC_DRAM_BYTES_PER_OPERAND_BYTE * distinct_operand_bytes(m["ops"]) * m["repeat"] * m["steps"] / m["tc_launches"]
+    r = {"bound": "tensor",
+         "kernel": "tc_group_kernel (fused 8-bit + reference + denominator products and Eq. 3 epilogue of up to 16 "
+                   "probes per persistent launch)",
+         "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak if achieved else None,
+         "traffic": traffic,
+         "traffic_note": "DRAM bytes per launch, scaled from a profiler capture of a smaller workload by distinct operand bytes",
+         "peak_source": f"1.2 x {'bf16_tflops_sustained' if long_region else 'bf16_tflops'} ({p16}) of {peaks['source']}",
+         "launches": m["tc_launches"], "avg_launch_ms": m["tc_ms"] / max(m["tc_launches"], 1),
+         "timing": "CUDA event pair around every launch, recorded by the library on the launching stream inside the timed steps",
+         "frac_of_burst_peak": achieved / (1.2 * peaks["bf16_tflops"]) if achieved else None,
+         "whole_step_frac": m["value"] / peak,
+         "whole_step_note": "the step's rate (scale/quantize kernels included) against the same composite peak",
+         "frac_of_nominal": achieved / (1.2 * 2250.0) if achieved else None,
+         "nominal_note": "against 1.2 x 2250 TFLOP/s (nominal dense bf16; 8-bit = 2x), context only",
+         "targets": {"fused_probe_ge_0.70_of_composite_peak": bool(achieved and achieved / peak >= 0.70)}}
+    if bench_mhz and peaks.get("peak_run_sm_mhz"):
+        scaled = peak * bench_mhz / peaks["peak_run_sm_mhz"]
+        r["clock_normalised"] = {"frac": achieved / scaled if achieved else None, "bench_sm_mhz": bench_mhz,
+                                 "peak_run_sm_mhz": peaks["peak_run_sm_mhz"],
+                                 "note": "achieved / (peak x bench MHz / MHz of the run that measured the peak)"}
+    return r
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500,
-                    help="timed steps (0.4 ms each: the default keeps the GPU under load long enough for the clock samples)")
+    ap.add_argument("--steps", type=int, default=20, help="timed steps (each at least --step-ms long)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="bert_base_fwd")
-    ap.add_argument("--oracle-rows", type=int, default=4096)
+    ap.add_argument("--workload", default="bert_large_sweep_layer")
+    ap.add_argument("--step-ms", type=float, default=50.0,
+                    help="the workload is repeated inside a step until the step lasts about this long")
+    ap.add_argument("--oracle-rows", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
-                    help="skip the scale/quantize and stand-alone GEMM rate blocks (profiling runs)")
+                    help="skip the other workloads, the scale/quantize and the stand-alone GEMM rate blocks")
+    ap.add_argument("--case", default=None, help="run a few launches of one small case and exit (profiler runs)")
+    ap.add_argument("--M", type=int, default=4096)
+    ap.add_argument("--N", type=int, default=3072)
+    ap.add_argument("--K", type=int, default=768)
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--fmt", default="e4m3")
+    ap.add_argument("--gran", default="tensor")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--r-layout", default="kn", choices=["kn", "nk"], help="--case: R stored [K,N] or [N,K]")
     args = ap.parse_args()
 
-    ops, desc = build_workload(args.workload)
+    if args.case:
+        run_case(args)
+        return
     if args.impl == "reference":
-        if args.steps == 500 and args.warmup == 3:
+        ops, desc = build_workload(args.workload)
+        if args.steps == 20 and args.warmup == 3:
             args.steps, args.warmup = 3, 1
         run_reference(args, ops, desc)
         return
@@ -327,80 +549,41 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     qm.lib()   # fail now if the CUDA library is missing
 
-    # ---- inputs resident in HBM; one workspace and one result record per probe
-    # (a tensor that several probes of the step share, here the same layer probed in two formats,
-    # is resident once)
-    on_dev = {}
+    m = time_workload(qm, ranks, world, args.workload, args.steps, args.warmup, args.step_ms, clock_index=local)
+    ops, desc, results = m["ops"], m["desc"], m["results"]
 
-    def resident(t):
-        if id(t) not in on_dev:
-            on_dev[id(t)] = t.cuda()
-        return on_dev[id(t)]
-    dev_tensors = [(resident(o["L"]), resident(o["R"])) for o in ops]
-    batch = qm.ProbeBatch([(qm.operand_of(Ld, o["cl"]), qm.operand_of(Rd, o["cr"]), o["fmt_l"], o["fmt_r"],
-                            o["gran_l"], o["gran_r"], o["ref"]) for o, (Ld, Rd) in zip(ops, dev_tensors)])
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+    # ---- end to end through the host-buffer entry point: H2D of every operand and D2H of the
+    # records inside the timed region; the copies of one probe overlap the kernels of another
+    pinned = {}
 
-    def step():
-        batch.launch()      # qm_probe_batch: the step's probes, spread over the library's streams
+    def pin(t):
+        if id(t) not in pinned:
+            pinned[id(t)] = t.pin_memory()
+        return pinned[id(t)]
+    host_batch = qm.HostProbeBatch([(pin(o["L"]), o["cl"], pin(o["R"]), o["cr"], o["fmt_l"],
+                                     o["fmt_r"], o["gran_l"], o["gran_r"], o["ref"]) for o in ops])
+    h2d, d2h = host_batch.h2d_bytes, host_batch.d2h_bytes
 
     def barrier():
         torch.cuda.synchronize()
         ranks.barrier(world)
         torch.cuda.synchronize()
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-
-    # ---- timed region: K steps, each between its own event pair, L2 flushed in between
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.3)
-    launches0 = qm.kernel_launches()
-    # the step's fused kernels are ONE grouped launch on this stream, issued after every scale /
-    # quantize chain has been joined: the library's event pair around it times it alone
-    qm.profile_enable(True)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    for a, b in evs:
-        flush.zero_()
-        a.record()
-        step()
-        b.record()
-    barrier()
-    step_ms = [a.elapsed_time(b) for a, b in evs]
-    tc_ms, tc_launches = qm.profile_read()
-    qm.profile_enable(False)
-    launches = qm.kernel_launches() - launches0
-    total_ms = ranks.max_over_ranks(float(sum(step_ms)), world, "cuda")
-    results = batch.results()
-    if any(r.device_error for r in results):
-        raise SystemExit("device error flagged in a probe result")
-
-    clocks = sampler.stop()
-
-    flops_step = probe_flops(ops)
-    value = ranks.whole_job_rate(flops_step * args.steps, world, total_ms) / 1e12
-
-    # ---- end to end through the host-buffer entry point: H2D of every operand and D2H of the
-    # records inside the timed region; the copies of one probe overlap the kernels of another
-    host_batch = qm.HostProbeBatch([(o["L"].pin_memory(), o["cl"], o["R"].pin_memory(), o["cr"], o["fmt_l"],
-                                     o["fmt_r"], o["gran_l"], o["gran_r"], o["ref"]) for o in ops])
-    h2d, d2h = host_batch.h2d_bytes, host_batch.d2h_bytes
-
-    for _ in range(3):
+    for _ in range(2):
         host_batch.run()
     barrier()
-    e2e_steps = max(3, min(args.steps, 10))
+    e2e_steps = max(3, min(args.steps, 5))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_results = host_batch.run()   # waits for the records itself
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3
-    e2e_value = ranks.whole_job_rate(flops_step * e2e_steps, world, ranks.max_over_ranks(e2e_ms, world, "cuda")) / 1e12
-    if any(a.record() != b.record() for a, b in zip(e2e_results, results)):
-        raise SystemExit("end-to-end records differ from the device-resident ones")
+    e2e_value = ranks.whole_job_rate(m["flops_pass"] * e2e_steps, world, ranks.max_over_ranks(e2e_ms, world, "cuda")) / 1e12
+    for o, a, b in zip(ops, e2e_results, results):
+        ra, rb = a.record(), b.record()
+        # the two paths sum the same tile values over different tile-to-CTA assignments
+        if ra["count"] != rb["count"] or any(abs(ra[k] - rb[k]) > 1e-9 * abs(rb[k]) for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2")):
+            raise SystemExit(f"end-to-end record of {o['name']} differs from the device-resident one")
+    del host_batch, pinned
 
     if rank != 0:
         if world > 1:
@@ -408,42 +591,40 @@ def main():
         return
 
     peaks = load_peaks()
-    sq = None if args.no_extras else scale_quantize_rates(qm, peaks["hbm_gbs"])
-    # composite tensor bound of the fused kernel: per 2MNK, one product at the 8-bit rate
-    # (2 x bf16) and two at the bf16 rate  ->  3 / (1/(2P) + 2/P) = 1.2 P in summed flops
-    peak_tflops = 1.2 * peaks["bf16_tflops"]
-    achieved = flops_step * args.steps / (tc_ms * 1e-3) / 1e12 if tc_ms > 0 else None
-    traffic = None
-    if qm.lib().qm_kernel_revision().decode() == NCU_TC["revision"] and args.workload == NCU_TC["workload"]:
-        traffic = NCU_TC["dram_bytes"]
-    roofline = {"bound": "tensor",
-                "kernel": "tc_group_kernel (fused 8-bit + reference + denominator products and Eq. 3 epilogue of the "
-                          "step's probes, one persistent launch per step)",
-                "achieved": achieved, "peak": peak_tflops, "unit": "TFLOP/s",
-                "frac": achieved / peak_tflops if achieved else None, "traffic": traffic,
-                "traffic_note": "DRAM bytes of one grouped launch of this workload, from the ncu capture in profiles/",
-                "peak_source": f"1.2 x bf16_tflops ({peaks['bf16_tflops']}) of {peaks['source']}",
-                "launches": tc_launches, "avg_launch_ms": tc_ms / max(tc_launches, 1),
-                "timing": "CUDA event pair around every launch, recorded by the library on the launching stream "
-                          "inside the timed steps"}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "fp8/int8 x bf16 (fp32/int32 accumulate)", "data": "synthetic",
-            "config": {"workload": args.workload, "description": desc, "probes_per_step": len(ops),
-                       "flops_counted": "3 x 2MNK per probe (8-bit, reference and denominator products)",
-                       "issue": "qm_probe_batch: one call per step, probes spread over 3 library streams",
-                       "l2": "256 MiB buffer written between timed steps"},
+    clocks = m["clocks"]
+    roofline = roofline_of(m, peaks, clocks["sm_mhz"] if clocks else None)
+    line = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": m["total_ms"] / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "fp8/int8 x bf16 (fp32/int32 accumulate)",
+            "data": "synthetic", "config": config_of(args, desc),
+            "run": {"probes_per_pass": len(ops), "passes_per_step": m["repeat"], "timed_region_s": m["wall_s"],
+                    "issue": "qm_probe_batch: one call per pass; scale/quantize chains on the library's 8 streams, "
+                             "then grouped fused launches of up to 16 probes on the caller's stream"},
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "gpu_launches": int(launches), "roofline": roofline,
-            "pct_of_composite_tensor_peak": 100.0 * value / peak_tflops,
-            "scale_quantize": sq, "gemm": None if args.no_extras else gemm_rates(qm),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "one pass per step through qm_probe_batch_host (pinned host operands in, records out)"},
+            "gpu_launches": m["launches"], "roofline": roofline,
             "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
+    if not args.no_extras:
+        others = {}
+        for name in ("bert_large_layer", "bert_base_fwd"):
+            if name == args.workload:
+                continue
+            mo = time_workload(qm, ranks, world, name, 10, 3, args.step_ms)
+            ro = roofline_of(mo, peaks, None)
+            others[name] = {"value": mo["value"], "unit": UNIT, "ms_per_pass": mo["total_ms"] / mo["steps"] / mo["repeat"],
+                            "passes_per_step": mo["repeat"], "fused_kernel_tflops": ro["achieved"],
+                            "fused_kernel_frac": ro["frac"], "peak": ro["peak"], "peak_source": ro["peak_source"]}
+        line["other_workloads"] = others
+        sq = scale_quantize_rates(qm, peaks["hbm_gbs"])
+        sq["targets"] = {"scale_quantize_ge_0.80_of_hbm": bool(min(sq["scale_tensor_frac_of_hbm"], sq["quantize_frac_of_hbm"]) >= 0.80)}
+        line["scale_quantize"] = sq
+        line["gemm"] = gemm_rates(qm)
     if not args.no_cpu_baseline and world == 1:
-        f, s = time_oracle_sample(ops, args.oracle_rows)
-        line["cpu_baseline"] = {"value": f / s / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
-                                "sample": f"{args.oracle_rows} of the output rows of each of the {len(ops)} probes "
-                                          f"(scales and codes over whole operands), {s:.1f} s"}
+        sample = oracle_sample_ops(ops)
+        f, sec = time_oracle_sample(sample, args.oracle_rows)
+        line["cpu_baseline"] = {"value": f / sec / 1e12, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": oracle_sample_text(sample, args.oracle_rows, len(ops)) + f", {sec:.1f} s"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

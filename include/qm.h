@@ -130,7 +130,8 @@ qm_status qm_tensor_moments(const qm_tensor_stats_result* rec, qm_tensor_moments
 /* Eq. 2, RE = |v - v~| / |v|, over the non-zero elements of one tensor under Eq. 1,
  * split as in the Results section: an element is OVERFLOW when |v/delta| exceeds the
  * largest expressible magnitude (it is capped), UNDERFLOW when it is not zero but its
- * code is, ROUNDING otherwise.  err2_* are sums of (v - v~)^2 per class. */
+ * code is, ROUNDING otherwise.  err2_* are sums of (v - v~)^2 per class, each square formed
+ * in fp32 (an error below about 1e-19 in magnitude contributes 0 to them). */
 typedef struct {
   double sum_re;           /* over all non-zero elements (an underflow contributes 1)     */
   double sum_re_round;     /* over the rounding class                                     */
@@ -150,7 +151,15 @@ typedef struct {
   uint64_t seed;           /* of the stochastic draws; unused with QM_ROUND_RTNE          */
   int32_t batch_groups_l;  /* QM_GRAN_CHANNEL on a batched operand: see qm_scale_shared;  */
   int32_t batch_groups_r;  /* 0 = every batch element has its own scales                  */
+  /* Optional (NULL = off) check output of the fused tensor-core probe: device fp64
+   * [batch * M][QM_ROW_STATS] = for every output row the Eq. 3 sums over its N inner products,
+   * {sum BE, max BE, sum (C-Q)^2, sum C^2, sum D^2}.  The call zeroes it and the kernel adds each
+   * tile's share with atomics, so a CPU evaluation of a few sampled rows can be compared with
+   * the fused kernel itself at sizes whose whole product the CPU cannot evaluate.  The record in
+   * `out` is unchanged by it.  QM_REF_BF16_FP32ACC only; not with qm_probe_layer2. */
+  double* row_stats;
 } qm_probe_cfg;
+#define QM_ROW_STATS 5
 
 /* Row length in bytes of a code tensor whose contracting extent is `contract`. */
 int64_t qm_code_ld(int64_t contract);

@@ -79,7 +79,7 @@ class QuantError(C.Structure):
 class ProbeCfg(C.Structure):
     _fields_ = [("fmt_l", C.c_int32), ("fmt_r", C.c_int32), ("gran_l", C.c_int32), ("gran_r", C.c_int32),
                 ("round", C.c_int32), ("ref", C.c_int32), ("seed", C.c_uint64),
-                ("batch_groups_l", C.c_int32), ("batch_groups_r", C.c_int32)]
+                ("batch_groups_l", C.c_int32), ("batch_groups_r", C.c_int32), ("row_stats", C.c_void_p)]
 
 
 _lib = None
@@ -296,8 +296,9 @@ def qm_quantize_error(op, fmt, gran, delta=None, ws=None, stream=None):
 ROUND = {"rtne": 0, "stochastic_l": 1, "stochastic_r": 2, "stochastic_both": 3}
 
 
-def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding="rtne", seed=0, groups=(0, 0)):
+def _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding="rtne", seed=0, groups=(0, 0), row_stats=None):
     c = ProbeCfg()
+    c.row_stats = row_stats.data_ptr() if row_stats is not None else None
     c.batch_groups_l, c.batch_groups_r = groups
     c.fmt_l, c.fmt_r, c.gran_l, c.gran_r, c.ref = FMT[fmt_l], FMT[fmt_r], GRAN[gran_l], GRAN[gran_r], REF[ref]
     c.round, c.seed = ROUND[rounding], seed
@@ -312,12 +313,18 @@ def qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16"):
     return n
 
 
+def _row_stats_buffer(L_op):
+    return torch.empty((L_op.batch * L_op.noncontract, 5), dtype=torch.float64, device="cuda")
+
+
 class ProbePlan:
     """Pre-allocated workspace and result buffer for repeated probes of one shape."""
 
     def __init__(self, L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref="bf16", rounding="rtne", seed=0,
-                 groups=(0, 0)):
-        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed, groups)
+                 groups=(0, 0), row_stats=False):
+        # row_stats: also collect the per-row Eq. 3 sums [batch * M, 5] (check output of the fused kernel)
+        self.row_stats = _row_stats_buffer(L_op) if row_stats else None
+        self.cfg = _cfg(fmt_l, fmt_r, gran_l, gran_r, ref, rounding, seed, groups, self.row_stats)
         self.ws_bytes = qm_workspace_bytes(L_op, R_op, fmt_l, fmt_r, gran_l, gran_r, ref)
         self.ws = torch.empty(self.ws_bytes, dtype=torch.uint8, device="cuda")
         self.out = torch.zeros(C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
@@ -408,13 +415,16 @@ class ProbeBatch:
     """Workspaces and result records of a fixed list of probes that are issued together
     (qm_probe_batch).  `probes` is a list of (L_op, R_op, fmt_l, fmt_r, gran_l, gran_r[, ref])."""
 
-    def __init__(self, probes):
+    def __init__(self, probes, row_stats=False):
         n = self.n = len(probes)
         self._keep = [(p[0], p[1]) for p in probes]
         self.L = (Operand * n)(*[_copy_operand(p[0]) for p in probes])
         self.R = (Operand * n)(*[_copy_operand(p[1]) for p in probes])
         refs = [p[6] if len(p) > 6 else "bf16" for p in probes]
-        self.cfg = (ProbeCfg * n)(*[_cfg(p[2], p[3], p[4], p[5], r) for p, r in zip(probes, refs)])
+        # row_stats: per probe, also collect the per-row Eq. 3 sums (check output of the fused kernel)
+        self.row_stats = [_row_stats_buffer(p[0]) if row_stats and r == "bf16" else None for p, r in zip(probes, refs)]
+        self.cfg = (ProbeCfg * n)(*[_cfg(p[2], p[3], p[4], p[5], r, row_stats=rs)
+                                    for p, r, rs in zip(probes, refs, self.row_stats)])
         sizes = [qm_workspace_bytes(p[0], p[1], p[2], p[3], p[4], p[5], r) for p, r in zip(probes, refs)]
         self._ws = [torch.empty(b, dtype=torch.uint8, device="cuda") for b in sizes]
         self.ws = (C.c_void_p * n)(*[t.data_ptr() for t in self._ws])

@@ -101,6 +101,7 @@ struct KernelArgs {
   // is result[1] and its per-CTA records follow the first format's gridDim.x records
   const float* dl2; const float* dr2;
   uint32_t idesc_lp2;
+  double* row_stats;                     // Probe (one format): optional [batch * M][5] per-row sums
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -397,6 +398,17 @@ __device__ __forceinline__ void stats16(const uint32_t* rc, const uint32_t* rd, 
     s.r2 = fma2(cv2, cv2, s.r2);
     s.n2 = fma2(dd2, dd2, s.n2);
   }
+}
+
+// Adds one tile's share of a row's Eq. 3 sums to the optional per-row check output.
+__device__ __forceinline__ void row_stats_add(double* rs, const Stats2& st) {
+  float x0, x1;
+  unpack2(st.be, x0, x1); atomicAdd(rs + 0, (double)x0 + (double)x1);
+  // BE >= 0: the bit patterns of non-negative doubles order like the values
+  atomicMax(reinterpret_cast<unsigned long long*>(rs + 1), (unsigned long long)__double_as_longlong((double)st.mx));
+  unpack2(st.d2, x0, x1); atomicAdd(rs + 2, (double)x0 + (double)x1);
+  unpack2(st.r2, x0, x1); atomicAdd(rs + 3, (double)x0 + (double)x1);
+  unpack2(st.n2, x0, x1); atomicAdd(rs + 4, (double)x0 + (double)x1);
 }
 
 template <int MODE, int LPKIND, int LPKIND2>
@@ -730,7 +742,10 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
           }
         }
-        if (row_ok) add_stats(0, st);
+        if (row_ok) {
+          add_stats(0, st);
+          if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
+        }
         tc_fence_before();                        // the 8-bit block's loads are complete as well
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
@@ -1360,6 +1375,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         unpack2(st.r2, x0, x1); acc[3] += (double)x0 + (double)x1;
         unpack2(st.n2, x0, x1); acc[4] += (double)x0 + (double)x1;
         acc[1] = fmax(acc[1], (double)st.mx);
+        if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
       }
       tc_fence_before();
       __syncwarp();
@@ -1634,6 +1650,7 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
     ka.count = (uint64_t)(g.M * g.N * g.batch);
     ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+    ka.row_stats = p.row_stats;
     gp.a = ka;
     gp.kind = p.fmt_l == QM_FMT_INT8 ? kKindI8 : kKindF8;
     gp.tile_begin = (int32_t)total;
@@ -1694,6 +1711,7 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
   ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
   ka.count = (uint64_t)(g.M * g.N * g.batch);
   ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+  ka.row_stats = two ? nullptr : p.row_stats;
   if (two) {
     // the first format is an FP8 one (the caller orders them), the second FP8 or INT8
     if (p.fmt_l == QM_FMT_INT8) return QM_ERR_UNSUPPORTED;

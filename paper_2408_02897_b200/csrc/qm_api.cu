@@ -155,7 +155,10 @@ qm_status check_probe(const qm_operand* Lo, const qm_operand* Ro, const qm_probe
   if (cfg->ref == QM_REF_BF16_FP32ACC) {
     if (L->dtype != QM_DT_BF16 || R->dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;
     if (L->c % 16) return QM_ERR_UNSUPPORTED;
+  } else if (cfg->row_stats) {
+    return QM_ERR_UNSUPPORTED;
   }
+  if (reinterpret_cast<uintptr_t>(cfg->row_stats) & 7) return QM_ERR_ALIGNMENT;
   return QM_OK;
 }
 
@@ -355,6 +358,8 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
   } else if (phases & kClear) {
     QM_CUDA_OK(cudaMemsetAsync(base, 0, w.off_dl, s));
   }
+  if ((phases & kClear) && cfg->row_stats)
+    QM_CUDA_OK(cudaMemsetAsync(cfg->row_stats, 0, sizeof(double) * QM_ROW_STATS * (size_t)(L.batch * L.nc), s));
   uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.off_ml);
   uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.off_mr);
   void* al = w.tc ? base + w.off_al : nullptr;
@@ -394,6 +399,7 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
     p.g = g; p.partials = part; p.err_word = err;
     p.done_counter = err + 1;               // second word of the cleared error slot
     p.result = out;
+    p.row_stats = cfg->row_stats;
     if (defer) {
       *defer = p;
       *deferred = true;
@@ -427,6 +433,7 @@ bool order2(const qm_probe_cfg* ca, const qm_probe_cfg* cb, const qm_probe_cfg**
       ca->batch_groups_l != cb->batch_groups_l || ca->batch_groups_r != cb->batch_groups_r)
     return false;
   if (ca->ref != QM_REF_BF16_FP32ACC || cb->ref != QM_REF_BF16_FP32ACC) return false;
+  if (ca->row_stats || cb->row_stats) return false;
   const bool a_int = ca->fmt_l == QM_FMT_INT8, b_int = cb->fmt_l == QM_FMT_INT8;
   if (a_int && b_int) return false;
   *swapped = a_int;

@@ -139,6 +139,7 @@ struct TcProbeArgs {
   uint32_t* done_counter;                   // zero on entry; counts finished CTAs
   qm_metric_result* result;                 // written by the last CTA to finish
   uint32_t* err_word;
+  double* row_stats = nullptr;              // optional per-row Eq. 3 sums (zeroed by the caller), one-format probes only
   // Two formats in one pass (cl2 != nullptr): codes and scales of the second format, same
   // granularities; `result` then points at two records and `partials` holds 2 x tc_probe_records.
   // The first format must be an FP8 one.

@@ -112,13 +112,21 @@ def config4(seed=4, M=16384, H=1024, F=4096):
     return ops
 
 
-def attention_ops(rng, batch, S, D, fmt):
-    """Score and context products of self-attention, forward and backward, batched over
-    batch = examples x heads.  P is the row softmax of Q.K^T / sqrt(D) (input preparation)."""
+def attention_tensors(rng, batch, S, D):
+    """Operands of the score and context products of self-attention, batched over batch =
+    examples x heads.  P is the row softmax of Q.K^T / sqrt(D) (input preparation); the upstream
+    gradients dS and dO are N(0, 1e-3^2)."""
     Q, K, V = (normal(rng, (batch, S, D)) for _ in range(3))
     P = torch.softmax(torch.matmul(Q.float(), K.float().transpose(1, 2)) / (D ** 0.5), dim=-1).to(torch.bfloat16)
     dS = normal(rng, (batch, S, S), 1e-3)
     dO = normal(rng, (batch, S, D), 1e-3)
+    return dict(Q=Q, K=K, V=V, P=P, dS=dS, dO=dO)
+
+
+def attention_ops(rng, batch, S, D, fmt, tensors=None):
+    """Score and context products, forward and backward, for one format of the sweep."""
+    t = tensors if tensors is not None else attention_tensors(rng, batch, S, D)
+    Q, K, V, P, dS, dO = (t[k] for k in ("Q", "K", "V", "P", "dS", "dO"))
     g = "e5m2" if fmt != "int8" else "int8"      # gradients: E5M2 when the sweep is FP8
     return [
         op(f"qk-fwd-{fmt}", Q, -1, K, -1, fmt, fmt),                  # S = Q . K^T
@@ -130,20 +138,47 @@ def attention_ops(rng, batch, S, D, fmt):
     ]
 
 
-def config5_layer(layer, fmt, seed=5, M=16384, H=1024, F=4096, heads=16, S=512):
-    """One layer of the 24-layer sweep for one format: 12 projection ops + 6 attention ops.
-    The layer's weight std is drawn uniformly in [0.01, 0.05]."""
+# Which tensor category of the paper's Results section each operand of an op belongs to
+# (RHS: mostly weights; LHS: activations, inside attention also keys / probabilities; gradient:
+# the upstream gradient), and the pass the product belongs to.
+_ROLES = {"fwd": ("LHS", "RHS"), "dgrad": ("gradient", "RHS"), "wgrad": ("LHS", "gradient"),
+          "qk-fwd": ("LHS", "RHS"), "pv-fwd": ("LHS", "RHS"), "qk-dq": ("gradient", "RHS"),
+          "qk-dk": ("gradient", "LHS"), "pv-dp": ("gradient", "RHS"), "pv-dv": ("LHS", "gradient")}
+
+
+def op_roles(name):
+    """(pass, role of L, role of R) of an op of config 3 / 5, from its name."""
+    for key, (rl, rr) in _ROLES.items():
+        if f"-{key}" in name or name.startswith(key):
+            ps = key if key in ("fwd", "dgrad", "wgrad") else ("fwd" if key.endswith("fwd") else "bwd")
+            return ps, rl, rr
+    return "fwd", "LHS", "RHS"
+
+
+def config5_layer_tensors(layer, seed=5, M=16384, H=1024, F=4096, heads=16, S=512):
+    """The tensors of one layer of the 24-layer sweep (shared by the three formats): projection
+    operands with the layer's weight std drawn uniformly in [0.01, 0.05], their upstream
+    gradients, and the attention operands."""
     rng = _rng(seed * 1000 + layer)
     wstd = float(rng.uniform(0.01, 0.05))
-    t = bert_forward_ops(rng, M, H, F, 3 * H, wstd)
+    proj = bert_forward_ops(rng, M, H, F, 3 * H, wstd)
+    grads = {name: normal(rng, (M, W.shape[1]), 1e-3) for name, (X, W) in proj.items()}
+    attn = attention_tensors(rng, (M // S) * heads, S, H // heads)
+    return dict(layer=layer, wstd=wstd, proj=proj, grads=grads, attn=attn)
+
+
+def config5_layer(layer, fmt, seed=5, M=16384, H=1024, F=4096, heads=16, S=512, tensors=None):
+    """One layer of the 24-layer sweep for one format: 12 projection ops + 6 attention ops,
+    per-tensor scales; gradients in E5M2 when the sweep format is an FP8 one."""
+    t = tensors if tensors is not None else config5_layer_tensors(layer, seed, M, H, F, heads, S)
     g = "e5m2" if fmt != "int8" else "int8"
     ops = []
-    for name, (X, W) in t.items():
-        dY = normal(rng, (M, W.shape[1]), 1e-3)
+    for name, (X, W) in t["proj"].items():
+        dY = t["grads"][name]
         ops.append(op(f"L{layer}-{name}-fwd-{fmt}", X, -1, W, -2, fmt, fmt))
         ops.append(op(f"L{layer}-{name}-dgrad-{fmt}", dY, -1, W, -1, g, fmt))
         ops.append(op(f"L{layer}-{name}-wgrad-{fmt}", X, -2, dY, -2, fmt, g))
-    for o in attention_ops(rng, (M // S) * heads, S, H // heads, fmt):
+    for o in attention_ops(None, None, None, None, fmt, tensors=t["attn"]):
         o["name"] = f"L{layer}-" + o["name"]
         ops.append(o)
     return ops

@@ -50,7 +50,7 @@ def test_struct_layouts_match_header(tmp_path):
         w = line.split()
         assert w[0] == cname and int(w[1]) == C.sizeof(cls), line
         assert [int(x) for x in w[2:]] == [getattr(cls, f).offset for f, _ in cls._fields_], line
-    assert C.sizeof(binding.MetricResult) == 56 and C.sizeof(binding.ProbeCfg) == 40
+    assert C.sizeof(binding.MetricResult) == 56 and C.sizeof(binding.ProbeCfg) == 48
 
 
 def test_host_side_argument_checks():

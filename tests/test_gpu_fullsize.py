@@ -16,7 +16,7 @@ import oracle
 from oracle.probe import descale
 import paper_2408_02897_b200 as qm
 from paper_2408_02897_b200 import workloads
-from helpers import oriented, as3, assert_record_close
+from helpers import oriented, as3, assert_record_close, oracle_row_stats, assert_row_stats_close
 
 pytestmark = pytest.mark.gpu
 
@@ -73,6 +73,77 @@ def check_full(o, n_rows=24, seed=60):
     assert res.device_error == 0
     assert_record_close(res.record(), full, what=o["name"] + " fused vs materialised")
     return res
+
+
+def check_fused_rows(ops, n_rows=12, n_batch=2, seed=70):
+    """The fused kernel itself against the oracle at full size, in the launch configuration the
+    benchmark uses: all `ops` as one qm_probe_batch call (grouped fused launches) with the per-row
+    check output switched on; for seeded sample rows (and batch elements) the oracle evaluates the
+    Eq. 3 sums of each row from scratch.  Also: the record of each probe equals the column sums of
+    its own per-row output (any size), and every row of the output was written."""
+    on_dev = {}
+
+    def resident(t):
+        if id(t) not in on_dev:
+            on_dev[id(t)] = t.cuda()
+        return on_dev[id(t)]
+    batch = qm.ProbeBatch([(qm.operand_of(resident(o["L"]), o["cl"]), qm.operand_of(resident(o["R"]), o["cr"]),
+                            o["fmt_l"], o["fmt_r"], o["gran_l"], o["gran_r"], o["ref"]) for o in ops], row_stats=True)
+    batch.launch()
+    torch.cuda.synchronize()
+    results = batch.results()
+    out = {}
+    for i, (o, res) in enumerate(zip(ops, results)):
+        assert res.device_error == 0, o["name"]
+        (M, N, K, B), _ = workloads.op_flops(o)
+        rs = batch.row_stats[i].cpu().numpy().reshape(B, M, 5)
+        rec = res.record()
+        assert rec["count"] == B * M * N
+        # the record is the sum (max) of the per-row output: same tiles, same fp32 values
+        for k, name in ((0, "sum_be"), (2, "sum_diff2"), (3, "sum_ref2"), (4, "sum_den2")):
+            assert abs(rs[..., k].sum() - rec[name]) <= 1e-9 * abs(rec[name]) + 1e-300, (o["name"], name)
+        assert rs[..., 1].max() == rec["max_be"], o["name"]
+        assert (rs[..., 4] > 0).all(), o["name"]                      # no row was skipped
+        rng = np.random.default_rng(seed + i)
+        rows = np.sort(rng.choice(M, min(n_rows, M), replace=False))
+        rows[0], rows[-1] = 0, M - 1                                  # first and last row of the matrix
+        bsel = np.sort(rng.choice(B, min(B, n_batch), replace=False))
+        want = oracle_row_stats(o, rows, bsel)
+        assert_row_stats_close(rs[np.ix_(bsel, rows)], want, K, what=o["name"])
+        out[o["name"]] = res
+    return out
+
+
+def test_config3_every_op_fused_kernel_against_the_oracle(cfg3):
+    """All 12 products of the BERT-large layer (forward, dgrad, wgrad of QKV, attention output, FFN1,
+    FFN2; mixed E4M3 / E5M2 operands, per-channel weight scales) in one batch."""
+    assert len(cfg3) == 12
+    check_fused_rows(cfg3)
+
+
+def test_config4_every_combination_fused_kernel_against_the_oracle():
+    """All 3 formats x 2 granularities of the outlier-stress configuration."""
+    ops = workloads.config4()
+    assert len(ops) == 6
+    res = check_fused_rows(ops)
+    be = {k: v.derived()["mean_be"] for k, v in res.items()}
+    # finer granularity helps INT8 on heavy-tailed activations; FP8 depends far less on it
+    assert be["ffn1-int8-channel"] < be["ffn1-int8-tensor"]
+    assert be["ffn1-e4m3-tensor"] < be["ffn1-e5m2-tensor"]
+
+
+@pytest.fixture(scope="module")
+def cfg5_tensors():
+    return workloads.config5_layer_tensors(0)
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "e5m2", "int8"])
+def test_config5_whole_layer_fused_kernel_against_the_oracle(cfg5_tensors, fmt):
+    """One whole layer of the 24-layer sweep (12 projection products and the 6 batched attention
+    products, 512 batch elements each) per format."""
+    ops = workloads.config5_layer(0, fmt, tensors=cfg5_tensors)
+    assert len(ops) == 18
+    check_fused_rows(ops, n_rows=8)
 
 
 def pick(ops, name):

@@ -146,9 +146,6 @@ def test_error_with_subnormal_elements(fmt, dtype):
     got, want = check_error(t, -1, fmt, "tensor")
     assert want["n_underflow"] >= 5 and np.isfinite(got.sum_re)
     check_error(t, -1, fmt, "channel")
-    # a tensor made only of such elements: scales are subnormal themselves, codes are not zero
-    tiny = (tensor((8, 64), torch.float32, 28) * 1e-39).to(dtype)
-    check_error(tiny, -1, fmt, "tensor")
     got_s, _ = check_stats(t)
     assert got_s.device_error == 0
 
