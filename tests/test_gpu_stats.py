@@ -99,8 +99,12 @@ def check_error(t, contract_dim, fmt, gran, delta=None):
     assert got.device_error == 0
     for k in ("count", "n_nonzero", "n_overflow", "n_underflow"):
         assert getattr(got, k) == want[k], (k, getattr(got, k), want[k])
+    # the kernel squares in float32: a square below the normal range (2^-126) is lost there, so a sum
+    # of squares carries that much absolute slack per element
+    tiny = want["count"] * 2.0 ** -126
     for k in ("sum_re", "sum_re_round", "err2_round", "err2_overflow", "err2_underflow", "sum_x2"):
-        assert abs(getattr(got, k) - want[k]) <= 1e-5 * abs(want[k]) + 1e-300, (k, getattr(got, k), want[k])
+        slack = tiny if k.startswith("err2") or k == "sum_x2" else 1e-300
+        assert abs(getattr(got, k) - want[k]) <= 1e-5 * abs(want[k]) + slack, (k, getattr(got, k), want[k])
     assert abs(got.max_re_round - want["max_re_round"]) <= 1e-6 * want["max_re_round"] + 1e-300
     return got, want
 
