@@ -411,6 +411,22 @@ qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
  * milliseconds; *launches receives the number recorded so far. */
 qm_status qm_profile_samples(double* start_ms, double* dur_ms, int32_t cap, int32_t* launches);
 
+/*
+ * Testing aids for the bounded device waits (no counterpart in the paper).
+ * Every barrier wait inside the fused probe kernel gives up after a time limit
+ * (one second by default): the kernel then raises QM_DEVERR_TIMEOUT in the
+ * record, lets its outstanding loads and tensor-core work finish, frees its
+ * tensor memory and returns, and the context stays usable.
+ * qm_debug_set_wait_limit_ns sets that limit for later launches (0 restores
+ * the default).  qm_debug_stop_producer_after(k) makes the loading warp of
+ * every CTA of later launches stop after its first k k-blocks (64-deep slices
+ * of the contraction), so that the warps waiting for the next slice run into
+ * the limit; 0xffffffff (the default) switches the hook off.  Both are
+ * process-wide and meant for tests only.
+ */
+void qm_debug_set_wait_limit_ns(uint64_t ns);
+void qm_debug_stop_producer_after(uint32_t k_blocks);
+
 #ifdef __cplusplus
 }
 #endif

@@ -124,6 +124,8 @@ def lib():
             "qm_metric_noalloc": (I32, [P, P, P, I64, P, P]),
             "qm_metric_noalloc_max_count": (I64, []),
             "qm_kernel_launches": (I64, []),
+            "qm_debug_set_wait_limit_ns": (None, [C.c_uint64]),
+            "qm_debug_stop_producer_after": (None, [C.c_uint32]),
             "qm_profile_enable": (I32, [I32]),
             "qm_profile_read": (I32, [C.POINTER(C.c_double), C.POINTER(I32)]),
             "qm_profile_samples": (I32, [C.POINTER(C.c_double), C.POINTER(C.c_double), I32, C.POINTER(I32)]),

@@ -28,6 +28,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <atomic>
 #include <cstdlib>
 #include <mutex>
 
@@ -50,17 +51,10 @@ constexpr uint32_t kBLp = kHalfN * kBlockK;                       //  4 KB
 constexpr int kMaxStages = 8;
 constexpr int kRefAhead = 2;               // k-blocks of reference MMAs issued before the hand-back wait
 
-enum Mode { kProbe = 0, kLpOnly = 1, kRefOnly = 2, kProbe2 = 3 };
+enum Mode { kLpOnly = 1, kRefOnly = 2, kProbe2 = 3 };
 
 // Stage layout: left-operand tiles first (L, |L|, codes), then the right-operand halves.
 template <int MODE> struct Cfg;
-template <> struct Cfg<kProbe> {
-  static constexpr int kStages = 3;
-  static constexpr uint32_t kOffL = 0, kOffLa = kABf16, kOffCl = 2 * kABf16;
-  static constexpr uint32_t kOffR = 2 * kABf16 + kALp, kOffRa = kOffR + kBBf16, kOffCr = kOffRa + kBBf16;
-  static constexpr uint32_t kStageBytes = kOffCr + kBLp;          // 60 KB
-  static constexpr uint32_t kTmemCols = 512;
-};
 // Two 8-bit formats in one pass: the reference and denominator products are shared, each format
 // has its own code tiles and its own accumulator.
 template <> struct Cfg<kProbe2> {
@@ -102,6 +96,7 @@ struct KernelArgs {
   const float* dl2; const float* dr2;
   uint32_t idesc_lp2;
   double* row_stats;                     // Probe (one format): optional [batch * M][5] per-row sums
+  const uint32_t* err_also[2];           // Probe (one format): further error words to report in the record, or null
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -418,7 +413,7 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           const __grid_constant__ CUtensorMap map_cl, const __grid_constant__ CUtensorMap map_cr,
           const __grid_constant__ CUtensorMap map_cl2, const __grid_constant__ CUtensorMap map_cr2,
           const KernelArgs a) {
-  constexpr bool kAnyProbe = MODE == kProbe || MODE == kProbe2;
+  constexpr bool kAnyProbe = MODE == kProbe2;
   constexpr int kFormats = MODE == kProbe2 ? 2 : 1;
   using C = Cfg<MODE>;
   constexpr int kStages = C::kStages;
@@ -512,16 +507,8 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
       uint32_t g = 0, it = 0;
       bool ok = true;
       for (int t = pair; t < a.num_tiles && ok; t += num_pairs, ++it) {
-        // Probe: the three accumulators rotate through the four 128-column blocks of tensor
-        // memory (see the epilogue).  The reference block of this tile has been free since the
-        // epilogue of tile it-2 ended (awaited before tile it-1 was committed, below), so the
-        // reference MMAs of the first k-blocks are issued at once and keep the tensor pipe busy
-        // while both epilogues copy the previous tile's reference and denominator blocks out
-        // and hand them back; the denominator and 8-bit MMAs of those k-blocks follow that
-        // signal.
-        const uint32_t col_ref = MODE == kProbe ? ((3 * it) & 3) * 128u : 0u;
-        const uint32_t col_den = MODE == kProbe ? ((3 * it + 1) & 3) * 128u : 128u;
-        const uint32_t col_lp = MODE == kProbe ? ((3 * it + 2) & 3) * 128u : (MODE == kProbe2 ? 256u : 0u);
+        const uint32_t col_ref = 0u, col_den = 128u;
+        const uint32_t col_lp = MODE == kProbe2 ? 256u : 0u;
         auto issue_ref = [&](uint32_t base, int kb) {
           const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
 #pragma unroll
@@ -579,30 +566,10 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
             tc_commit_pair(smem_u32(&sh->empty[s]), lead);
           }
         }
-        if (MODE == kProbe) {
-          const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
-          for (int j = 0; j < n_ahead && ok; ++j) {
-            const int s = (g + j) % kStages;
-            if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, a.err_word)) ok = false;
-            tc_fence_after();
-            if (ok) issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
-          }
-          if (!ok) break;
-        }
         if (MODE != kProbe2 && it > 0 &&
             !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, a.err_word))
           break;
         tc_fence_after();
-        if (MODE == kProbe) {
-          const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
-          for (; kb < n_ahead; ++kb, ++g) {
-            const int s = g % kStages;
-            const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-            issue_den(base, kb);
-            issue_lp(base, kb);
-            tc_commit_pair(smem_u32(&sh->empty[s]), lead);
-          }
-        }
         for (; kb < num_kb; ++kb, ++g) {
           const int s = g % kStages;
           const uint32_t use = g / kStages;
@@ -615,12 +582,6 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           issue_lp2(base, kb);
           tc_commit_pair(smem_u32(&sh->empty[s]), lead);        // frees the stage in both CTAs
         }
-        // The next tile's reference block is this tile's free one, last read by the epilogue of
-        // tile it-1: wait for that epilogue here, where the barrier cannot yet have moved on to
-        // this tile's phase.
-        if (MODE == kProbe && ok && it > 0 &&
-            !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, a.err_word))
-          ok = false;
         if (ok) tc_commit_pair(smem_u32(&sh->tmem_full), lead); // this tile's accumulators are complete
       }
     }
@@ -709,44 +670,6 @@ tc_kernel(const __grid_constant__ CUtensorMap map_l, const __grid_constant__ CUt
           if constexpr (kFormats == 2) add_stats(1, st2);
         }
         tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
-      } else if (MODE == kProbe) {
-        // Accumulator blocks of this tile (they rotate so that the next tile's MMAs never wait
-        // for this arithmetic): copy this warp's 64 columns of the reference and denominator
-        // blocks into registers, hand those two blocks back to the MMA lane, then walk the
-        // 8-bit block in chunks of 16 columns.
-        const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
-        const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
-        const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;      // first column of this warp
-        uint32_t rc[64], rd[64], rq[16];
-        tmem_ld32(lane_addr + col_ref + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
-        tmem_ld32(lane_addr + col_ref + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
-        tmem_ld32(lane_addr + col_den + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
-        tmem_ld32(lane_addr + col_den + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
-        Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f};
-        const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int cc0 = h * 64 + c * 16;
-          const int64_t col0 = colw + c * 16;
-          if (col0 < a.N) {                       // uniform across the warp
-            tmem_ld16(lane_addr + col_lp + cc0, rq);
-            tmem_ld_wait();
-            const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
-            if (n_live == 16) stats16<LPKIND, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
-            else stats16<LPKIND, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
-          }
-        }
-        if (row_ok) {
-          add_stats(0, st);
-          if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
-        }
-        tc_fence_before();                        // the 8-bit block's loads are complete as well
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
       } else {
@@ -1073,23 +996,71 @@ tc_gemm_wide_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   }
 }
 
-// ------------------------------------------------------------------ several probes in one launch
-// The probes of a batch as ONE persistent launch of the fused probe kernel.  A launch per probe
-// pays, each time, the kernel's set-up and drain, the launch gap, and the last wave of a tile
-// count that is not a multiple of the 74 CTA pairs; here the tiles of all probes form one
-// sequence.  The host orders the probes by descending contraction length (tile cost) and the
-// sequence is dealt to the pairs back and forth (round r gives pair p position r P + p when r is
-// even and r P + P-1-p when it is odd), which for descending costs balances the pairs to within
-// one tile of the cheapest kind.  Everything inside a tile is the probe mode of tc_kernel
-// (rotating accumulators, reference MMAs ahead of the hand-back, overlapped epilogue); the
-// operand maps, scales, shapes and the 8-bit MMA kind are read per tile from a table in the
-// kernel's parameter space.  A pair's positions increase, so it meets each probe in one run:
-// when the probe changes, the epilogue warps reduce their statistics and write the CTA's record
-// of the probe they leave.
+// ------------------------------------------------------------------ the fused probe kernel
+// One persistent launch computes the Eq. 3 records of up to kMaxGroup probes (one probe is a
+// group of one).  A launch per probe pays, each time, the kernel's set-up and drain, the launch
+// gap, and the last wave of a tile count that is not a multiple of the 74 CTA pairs; here the
+// tiles of all probes form one sequence.  The host orders the probes by descending contraction
+// length (tile cost) and the sequence is dealt to the pairs back and forth (round r gives pair p
+// position r P + p when r is even and r P + P-1-p when it is odd), which for descending costs
+// balances the pairs to within one tile of the cheapest kind.  The operand maps, scales, shapes
+// and the 8-bit MMA kind are read per tile from a table in the kernel's parameter space.  A
+// pair's positions increase, so it meets each probe in one run: when the probe changes, the
+// epilogue warps reduce their statistics and write the CTA's record of the probe they leave.
+//
+// Roles in each CTA (384 threads):
+//   warp 0       TMA producer: per 64-deep k-block the bf16 tiles of L and R and both code tiles
+//                (36 KB per CTA) into a ring of kTmaStages stages; a CTA's loads complete on its
+//                own `full` barrier.
+//   warps 2, 3   converters: the denominator product of Eq. 3 multiplies |L| by |R|.  Its operand
+//                tiles are not loaded: once a stage has landed these warps copy its L and R tiles
+//                with the sign bits cleared (the swizzled layout is elementwise-transparent) into
+//                a second ring of kAbsStages stages (24 KB per CTA), make the copies visible to
+//                the tensor core's reads (fence.proxy.async) and arrive on the leader's `ready`
+//                barrier.  The tensor cores are bound by the bytes an SM pulls from L2 per flop;
+//                this takes 24 of 60 KB per k-block off that path, and no |x| copy exists in HBM.
+//   warp 1       allocates tensor memory; in the leader CTA it runs the MMA loop converged and one
+//                elected lane issues the pair's MMAs once `ready` says that both CTAs' tiles and
+//                their sign-cleared copies are in place; tcgen05.commit frees the stage in both
+//                CTAs (`empty`), which the producer (TMA ring) and the converters (|x| ring) await.
+//   warps 4..11  epilogue (see below).
+// Three accumulators live side by side in tensor memory: the reference L.R (bf16, kind::f16), the
+// denominator |L|.|R| (bf16, kind::f16) and the 8-bit product (kind::f8f6f4 or kind::i8), 128
+// columns each, rotating from tile to tile through the four 128-column blocks so that the next
+// tile's MMAs overlap this tile's epilogue; no M x N matrix ever goes to HBM.
 constexpr int kMaxGroup = 16;
+constexpr int kConvWarps = 2;
+constexpr int kProbeThreads = 32 * (2 + kConvWarps + kEpiWarps);    // 384
+constexpr int kFirstEpiWarp = 2 + kConvWarps;                       // 4: lane quarter = warp % 4 still holds
+
+struct CfgP {
+  static constexpr int kTmaStages = 4, kAbsStages = 3;
+  // TMA stage: L, R (contiguous, so that the converters copy one flat 24 KB run), codes of L, codes of R
+  static constexpr uint32_t kOffL = 0, kOffR = kABf16, kOffCl = kABf16 + kBBf16, kOffCr = kOffCl + kALp;
+  static constexpr uint32_t kTmaStageBytes = kOffCr + kBLp;          // 36 KB
+  static constexpr uint32_t kOffLa = 0, kOffRa = kABf16;
+  static constexpr uint32_t kAbsStageBytes = kABf16 + kBBf16;        // 24 KB
+  static constexpr uint32_t kTileBytes = kTmaStages * kTmaStageBytes + kAbsStages * kAbsStageBytes;   // 216 KB
+};
+
+struct SharedP {
+  uint64_t full[CfgP::kTmaStages];    // per CTA: this CTA's loads of a stage have landed
+  uint64_t empty[CfgP::kTmaStages];   // per CTA: the pair's MMAs have finished reading the k-block of the stage
+  uint64_t ready[CfgP::kAbsStages];   // leader: both CTAs' converters have finished a k-block
+  uint64_t tmem_full;                 // per CTA: the tile's accumulators are complete
+  uint64_t tmem_empty;                // leader: both CTAs' epilogues have copied out reference and denominator
+  uint64_t lp_done;                   // leader: both CTAs' epilogues have finished a tile
+  uint64_t drain;                     // leader, give-up path only: every MMA issued so far has completed
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+  uint32_t is_last;
+  uint32_t issued;                    // k-blocks whose loads the producer has issued (read on the give-up path)
+  float delta_r[2][kBlockN];
+  double red[5][kEpiWarps];
+};
 
 struct GroupProblem {
-  CUtensorMap maps[6];        // L, R, |L|, |R|, codes L, codes R
+  CUtensorMap maps[4];        // L, R, codes L, codes R
   KernelArgs a;               // num_tiles, tiles_m, tiles_n: of this probe
   int32_t tile_begin;         // position of its first tile in the sequence
   int32_t kind;               // kKindF8 or kKindI8
@@ -1097,7 +1068,10 @@ struct GroupProblem {
 };
 struct GroupTable {
   int32_t n, total_tiles;
-  int32_t pad[14];
+  uint32_t stop_after_kb;     // test hook: the producer issues no k-block beyond this many (0xffffffff: off)
+  uint32_t pad0;
+  uint64_t wait_limit_ns;     // bound of every barrier wait
+  int32_t pad[10];
   GroupProblem p[kMaxGroup];
 };
 
@@ -1112,93 +1086,148 @@ __device__ __forceinline__ int group_find(const GroupTable& tab, int pos) {
   return pi;
 }
 
-// The MMAs of one tile of the grouped kernel (leader CTA, converged warp); g counts k-blocks,
-// `it` tiles of this pair.  Returns false when a wait gave up.
+// Bounded wait with the launch's limit; see mbar_wait.
+struct Waiter {
+  volatile uint32_t* abort_flag;
+  uint32_t* err_word;
+  uint64_t limit_ns;
+  __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity) const {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t polls = 0;
+    while (true) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((++polls & 0x3fu) == 0) {
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > limit_ns) {
+          *abort_flag = 1u;
+          if (err_word) atomicOr(err_word, QM_DEVERR_TIMEOUT);
+          return false;
+        }
+      }
+    }
+  }
+  __device__ __forceinline__ bool wait_warp(uint32_t bar, uint32_t parity) const {
+    return __all_sync(0xffffffffu, wait(bar, parity));
+  }
+};
+
+// Tile load into this CTA's shared memory, completing on this CTA's barrier.
+__device__ __forceinline__ void tma_load_3d_local(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                  int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// The MMAs of one tile (leader CTA, converged warp); g counts k-blocks, `it` tiles of this pair.
+// Returns false when a wait gave up.
 template <int LPK>
-__device__ __forceinline__ bool group_mma_tile(Shared* sh, uint8_t* tiles, uint32_t tmem_base, uint32_t& g, uint32_t it,
-                                               int num_kb, uint32_t idesc_lp, bool lead,
-                                               volatile uint32_t* abort_flag, uint32_t* err0) {
-  using C = Cfg<kProbe>;
-  constexpr int kStages = C::kStages;
+__device__ __forceinline__ bool group_mma_tile(SharedP* sh, uint32_t tma_tiles, uint32_t abs_tiles, uint32_t tmem_base,
+                                               uint32_t& g, uint32_t it, int num_kb, uint32_t idesc_lp, bool lead,
+                                               const Waiter& w) {
+  using C = CfgP;
   constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
   const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
   const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
-  auto issue_ref = [&](uint32_t base, int kb) {
+  auto issue_ref = [&](uint32_t gg, int kb) {
+    const uint32_t base = tma_tiles + (gg % C::kTmaStages) * C::kTmaStageBytes;
     const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
 #pragma unroll
-    for (int k = 0; k < kBlockK / 16; ++k)
+    for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
       mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
   };
-  auto issue_rest = [&](uint32_t base, int kb) {
-    const uint64_t dl = smem_desc(base + C::kOffLa, 128), dr = smem_desc(base + C::kOffRa, 128);
+  auto issue_rest = [&](uint32_t gg, int kb) {
+    const uint32_t abase = abs_tiles + (gg % C::kAbsStages) * C::kAbsStageBytes;
+    const uint64_t dl = smem_desc(abase + C::kOffLa, 128), dr = smem_desc(abase + C::kOffRa, 128);
 #pragma unroll
     for (int k = 0; k < kBlockK / 16; ++k)
       mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+    const uint32_t base = tma_tiles + (gg % C::kTmaStages) * C::kTmaStageBytes;
     const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
 #pragma unroll
-    for (int k = 0; k < kBlockK / 32; ++k)
+    for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
       mma_pair<LPK>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
   };
-  // reference MMAs of the first k-blocks go ahead of the hand-back of the previous tile
+  // The reference block of this tile has been free since the epilogue of tile it-2 ended (awaited
+  // before tile it-1 was committed, below), so the reference MMAs of the first k-blocks are issued
+  // at once and keep the tensor pipe busy while both epilogues copy the previous tile's reference
+  // and denominator blocks out and hand them back; the denominator and 8-bit MMAs of those
+  // k-blocks follow that signal.
   int kb = 0;
   const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
   for (int j = 0; j < n_ahead; ++j) {
-    const int s = (g + j) % kStages;
-    if (!mbar_wait_warp(smem_u32(&sh->full[s]), ((g + j) / kStages) & 1, abort_flag, err0)) return false;
+    const uint32_t gg = g + j;
+    if (!w.wait_warp(smem_u32(&sh->ready[gg % C::kAbsStages]), (gg / C::kAbsStages) & 1)) return false;
     tc_fence_after();
-    issue_ref(smem_u32(tiles + (size_t)s * C::kStageBytes), j);
+    issue_ref(gg, j);
   }
-  if (it > 0 && !mbar_wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1, abort_flag, err0)) return false;
+  if (it > 0 && !w.wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1)) return false;
   tc_fence_after();
   for (; kb < n_ahead; ++kb, ++g) {
-    const int s = g % kStages;
-    issue_rest(smem_u32(tiles + (size_t)s * C::kStageBytes), kb);
-    tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+    issue_rest(g, kb);
+    tc_commit_pair(smem_u32(&sh->empty[g % C::kTmaStages]), lead);
   }
   for (; kb < num_kb; ++kb, ++g) {
-    const int s = g % kStages;
-    if (!mbar_wait_warp(smem_u32(&sh->full[s]), (g / kStages) & 1, abort_flag, err0)) return false;
+    if (!w.wait_warp(smem_u32(&sh->ready[g % C::kAbsStages]), (g / C::kAbsStages) & 1)) return false;
     tc_fence_after();
-    const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
-    issue_ref(base, kb);
-    issue_rest(base, kb);
-    tc_commit_pair(smem_u32(&sh->empty[s]), lead);
+    issue_ref(g, kb);
+    issue_rest(g, kb);
+    tc_commit_pair(smem_u32(&sh->empty[g % C::kTmaStages]), lead);        // frees the k-block in both CTAs
   }
-  if (it > 0 && !mbar_wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1, abort_flag, err0)) return false;
-  tc_commit_pair(smem_u32(&sh->tmem_full), lead);
+  // The next tile's reference block is this tile's free one, last read by the epilogue of tile
+  // it-1: wait for that epilogue here, where the barrier cannot yet have moved on to this tile's
+  // phase.
+  if (it > 0 && !w.wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1)) return false;
+  tc_commit_pair(smem_u32(&sh->tmem_full), lead);                          // this tile's accumulators are complete
   return true;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kProbeThreads, 1)
 tc_group_kernel(const __grid_constant__ GroupTable tab) {
-  using C = Cfg<kProbe>;
-  constexpr int kStages = C::kStages;
+  using C = CfgP;
   extern __shared__ uint8_t smem_raw[];
+  // tiles start on a 1024-byte boundary (the 128-byte swizzle atom); the offset is the same in
+  // both CTAs of the pair because their dynamic shared memory starts at the same address
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  Shared* sh = reinterpret_cast<Shared*>(tiles + (size_t)kStages * C::kStageBytes);
+  SharedP* sh = reinterpret_cast<SharedP*>(tiles + C::kTileBytes);
+  const uint32_t tma_tiles = smem_u32(tiles), abs_tiles = tma_tiles + C::kTmaStages * C::kTmaStageBytes;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  volatile uint32_t* abort_flag = &sh->abort_flag;
-  uint32_t* const err0 = tab.p[0].a.err_word;                 // where a timed-out wait is reported
+  const Waiter w{&sh->abort_flag, tab.p[0].a.err_word, tab.wait_limit_ns};   // a timed-out wait is reported in probe 0's word
 
   if (warp == 0) {
     // fetch the tensor maps of this pair's first tile into the descriptor cache
     const int pos = group_position(0, pair, num_pairs);
-    if (pos < tab.total_tiles && lane < 6)
+    if (pos < tab.total_tiles && lane < 4)
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tab.p[group_find(tab, pos)].maps[lane]) : "memory");
   }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < C::kTmaStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
+    for (int s = 0; s < C::kAbsStages; ++s) mbar_init(smem_u32(&sh->ready[s]), 2 * kConvWarps);
     mbar_init(smem_u32(&sh->tmem_full), 1);
     mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
     mbar_init(smem_u32(&sh->lp_done), 2 * kEpiWarps);
+    mbar_init(smem_u32(&sh->drain), 1);
     sh->abort_flag = 0;
     sh->is_last = 0;
+    sh->issued = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -1209,8 +1238,8 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
   tc_fence_before();
   __syncthreads();
   __syncwarp();
-  cluster_sync();
-  pdl_prologue();
+  cluster_sync();          // the peer's barriers and tensor memory exist before anyone uses them
+  pdl_prologue();          // everything above overlapped the tail of the previous kernel
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
@@ -1228,25 +1257,25 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         const GroupProblem& pr = tab.p[group_find(tab, pos)];
         const TileCoord tc = tile_coord(pos - pr.tile_begin, pr.a);
         const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
-        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;
-        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;
+        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
+        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;     // this CTA's half of the right operand
         for (int kb = 0; kb < num_kb; ++kb, ++g) {
-          const int s = g % kStages;
-          const uint32_t use = g / kStages;
-          if (use > 0 && !mbar_wait(smem_u32(&sh->empty[s]), (use - 1) & 1, abort_flag, err0)) {
+          const int s = g % C::kTmaStages;
+          const uint32_t use = g / C::kTmaStages;
+          if (g >= tab.stop_after_kb) { ok = false; break; }    // test hook: the consumers' waits run out
+          if (use > 0 && !w.wait(smem_u32(&sh->empty[s]), (use - 1) & 1)) {
             ok = false;
             break;
           }
-          if (rank == 0) mbar_expect_tx(smem_u32(&sh->full[s]), 2 * C::kStageBytes);
-          const uint32_t bar = map_to_cta(smem_u32(&sh->full[s]), 0);
-          const uint32_t base = smem_u32(tiles + (size_t)s * C::kStageBytes);
+          const uint32_t bar = smem_u32(&sh->full[s]);
+          mbar_expect_tx(bar, C::kTmaStageBytes);
+          const uint32_t base = tma_tiles + s * C::kTmaStageBytes;
           const int k0 = kb * kBlockK;
-          tma_load_3d(base + C::kOffL, &pr.maps[0], bar, k0, r0, tc.b);
-          tma_load_3d(base + C::kOffR, &pr.maps[1], bar, k0, c0, tc.b);
-          tma_load_3d(base + C::kOffLa, &pr.maps[2], bar, k0, r0, tc.b);
-          tma_load_3d(base + C::kOffRa, &pr.maps[3], bar, k0, c0, tc.b);
-          tma_load_3d(base + C::kOffCl, &pr.maps[4], bar, k0, r0, tc.b);
-          tma_load_3d(base + C::kOffCr, &pr.maps[5], bar, k0, c0, tc.b);
+          tma_load_3d_local(base + C::kOffL, &pr.maps[0], bar, k0, r0, tc.b);
+          tma_load_3d_local(base + C::kOffCl, &pr.maps[2], bar, k0, r0, tc.b);
+          tma_load_3d_local(base + C::kOffR, &pr.maps[1], bar, k0, c0, tc.b);
+          tma_load_3d_local(base + C::kOffCr, &pr.maps[3], bar, k0, c0, tc.b);
+          sh->issued = g + 1;
         }
       }
     }
@@ -1265,17 +1294,63 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         const GroupProblem& pr = tab.p[group_find(tab, pos)];
         const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
         ok = pr.kind == kKindI8
-                 ? group_mma_tile<kKindI8>(sh, tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, abort_flag, err0)
-                 : group_mma_tile<kKindF8>(sh, tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, abort_flag, err0);
+                 ? group_mma_tile<kKindI8>(sh, tma_tiles, abs_tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, w)
+                 : group_mma_tile<kKindF8>(sh, tma_tiles, abs_tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, w);
         if (!ok) break;
         ++it;
       }
     }
+  } else if (warp < kFirstEpiWarp) {
+    // ------------------------------------------------------------ converters (both CTAs)
+    // |L| and |R| tiles of every k-block: L and R follow each other in the stage, so the job is one
+    // flat run of 1536 16-byte vectors; thread t takes vectors t, t + 64, ...
+    constexpr int kVec = (int)(C::kAbsStageBytes / 16);                 // 1536
+    constexpr int kPer = kVec / (32 * kConvWarps);                      // 24
+    const uint32_t t16 = (uint32_t)(threadIdx.x - 64) * 16u;
+    const uint32_t ready_leader = map_to_cta(smem_u32(&sh->ready[0]), 0);
+    uint32_t g = 0;
+    bool ok = true;
+    for (int r = 0; ok; ++r) {
+      const int pos = group_position(r, pair, num_pairs);
+      if (pos >= tab.total_tiles) {
+        if (r * num_pairs >= tab.total_tiles) break;
+        continue;
+      }
+      const GroupProblem& pr = tab.p[group_find(tab, pos)];
+      const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+      for (int kb = 0; kb < num_kb; ++kb, ++g) {
+        // the slot of the |x| ring was last read by the MMAs of k-block g - kAbsStages
+        if (g >= (uint32_t)C::kAbsStages) {
+          const uint32_t gp = g - C::kAbsStages;
+          if (!w.wait_warp(smem_u32(&sh->empty[gp % C::kTmaStages]), (gp / C::kTmaStages) & 1)) { ok = false; break; }
+        }
+        if (!w.wait_warp(smem_u32(&sh->full[g % C::kTmaStages]), (g / C::kTmaStages) & 1)) { ok = false; break; }
+        const uint32_t src = tma_tiles + (g % C::kTmaStages) * C::kTmaStageBytes + t16;
+        const uint32_t dst = abs_tiles + (g % C::kAbsStages) * C::kAbsStageBytes + t16;
+        uint4 v[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) v[i] = lds128(src + (uint32_t)i * (32u * kConvWarps * 16u));
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const uint32_t m = 0x7fff7fffu;
+          sts128(dst + (uint32_t)i * (32u * kConvWarps * 16u), make_uint4(v[i].x & m, v[i].y & m, v[i].z & m, v[i].w & m));
+        }
+        // generic-proxy writes -> visible to the tensor core's (async proxy) reads, then signal
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(ready_leader + (g % C::kAbsStages) * 8u);
+      }
+    }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+    // ------------------------------------------------------------ epilogue (warps 4..11, both CTAs)
+    // A warp may touch the tensor-memory lane quarter warp % 4; the two warps of a quarter split
+    // the columns.  Copy this warp's 64 columns of the reference and denominator blocks into
+    // registers, hand those two blocks back to the MMA lane, then walk the 8-bit block in chunks
+    // of 16 columns; the statistics arithmetic runs under the next tile's main loop.
     const int q = warp & 3;
-    const int h = (warp - 2) >> 2;
-    const int et = (warp - 2) * 32 + lane;
+    const int ew = warp - kFirstEpiWarp;           // 0..7
+    const int h = ew >> 2;                         // which 64-column half of the tile
+    const int et = ew * 32 + lane;                 // 0..255
     const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
     double acc[5] = {0, 0, 0, 0, 0};               // of the probe in hand: sum BE, max BE, sum diff^2, C^2, D^2
     int cur = -1;                                  // the probe in hand
@@ -1289,13 +1364,13 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
           const double y = __shfl_xor_sync(0xffffffffu, x, o);
           x = i == 1 ? fmax(x, y) : x + y;
         }
-        if (lane == 0) sh->red[i][warp - 2] = x;
+        if (lane == 0) sh->red[i][ew] = x;
         acc[i] = 0.0;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (et < 5) {
         double x = 0.0;
-        for (int w = 0; w < kEpiWarps; ++w) x = et == 1 ? fmax(x, sh->red[et][w]) : x + sh->red[et][w];
+        for (int k = 0; k < kEpiWarps; ++k) x = et == 1 ? fmax(x, sh->red[et][k]) : x + sh->red[et][k];
         __stcg(tab.p[pi].a.partials + (int64_t)blockIdx.x * kPartialDoubles + et, x);
         __threadfence();
       }
@@ -1332,13 +1407,14 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       if (a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
       else dlv = __ldg(a.dl);
 
-      const bool ok = mbar_wait(smem_u32(&sh->tmem_full), it & 1, abort_flag, err0);
+      const bool ok = w.wait(smem_u32(&sh->tmem_full), it & 1);
+      // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
       if (epi_barrier_any(!ok)) { live = false; break; }
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
       const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
       const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
-      const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;
+      const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;      // first column of this warp
       uint32_t rc[64], rd[64], rq[16];
       tmem_ld32(lane_addr + col_ref + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
       tmem_ld32(lane_addr + col_ref + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
@@ -1355,7 +1431,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       for (int c = 0; c < 4; ++c) {
         const int cc0 = h * 64 + c * 16;
         const int64_t col0 = colw + c * 16;
-        if (col0 < a.N) {
+        if (col0 < a.N) {                         // uniform across the warp
           tmem_ld16(lane_addr + col_lp + cc0, rq);
           tmem_ld_wait();
           const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
@@ -1377,7 +1453,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         acc[1] = fmax(acc[1], (double)st.mx);
         if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
       }
-      tc_fence_before();
+      tc_fence_before();                          // the 8-bit block's loads are complete as well
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
       ++it;
@@ -1400,10 +1476,11 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (sh->is_last) {
       // last CTA: every record of every probe is visible; each epilogue warp takes probes
-      // warp-2, warp-2+8, ...; fixed-order sum (lane l takes records l, l+32, ...)
+      // ew, ew + 8, ...; fixed-order sum (lane l takes records l, l+32, ...)
       __threadfence();
+      uint32_t* const err0 = tab.p[0].a.err_word;
       const uint32_t timed_out = err0 ? (*reinterpret_cast<volatile uint32_t*>(err0) & QM_DEVERR_TIMEOUT) : 0u;
-      for (int pi = warp - 2; pi < tab.n; pi += kEpiWarps) {
+      for (int pi = ew; pi < tab.n; pi += kEpiWarps) {
         const KernelArgs& a = tab.p[pi].a;
         double s5[5] = {0, 0, 0, 0, 0};
         for (int i = lane; i < (int)gridDim.x; i += 32) {
@@ -1423,15 +1500,42 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
           a.result->sum_be = s5[0]; a.result->max_be = s5[1]; a.result->sum_diff2 = s5[2];
           a.result->sum_ref2 = s5[3]; a.result->sum_den2 = s5[4];
           a.result->count = a.count;
-          a.result->device_error =
-              (a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u) | timed_out;
+          uint32_t flags = (a.err_word ? *reinterpret_cast<volatile uint32_t*>(a.err_word) : 0u) | timed_out;
+          for (int k = 0; k < 2; ++k)
+            if (a.err_also[k]) flags |= *reinterpret_cast<const volatile uint32_t*>(a.err_also[k]);
+          a.result->device_error = flags;
           a.result->reserved = 0;
         }
       }
     }
   }
 
+  // ---------------------------------------------------------------- common exit
+  // Neither CTA may leave while the other can still read its shared memory, signal its barriers
+  // or write its tensor memory, and no bulk load may still be writing into a CTA that retires.
   tc_fence_before();
+  __syncthreads();
+  if (sh->abort_flag && threadIdx.x == 0) {
+    // give-up path: the loads of the last kTmaStages k-blocks this producer issued may not have
+    // been awaited by anyone; wait (bounded) until each has landed
+    const uint32_t n = sh->issued;
+    for (uint32_t j = n > (uint32_t)C::kTmaStages ? n - C::kTmaStages : 0u; j < n; ++j) {
+      const uint32_t bar = smem_u32(&sh->full[j % C::kTmaStages]), parity = (j / C::kTmaStages) & 1;
+      const uint64_t t0 = global_timer_ns();
+      while (!mbar_try_wait(bar, parity) && global_timer_ns() - t0 < tab.wait_limit_ns) {}
+    }
+  }
+  if (sh->abort_flag && warp == 1 && rank == 0) {
+    // ... and the MMAs issued so far may still be running: one more commit, awaited (bounded) here
+    __syncwarp();
+    if (elect_one())
+      asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                       smem_u32(&sh->drain)) : "memory");
+    __syncwarp();
+    const uint64_t t0 = global_timer_ns();
+    while (!mbar_try_wait(smem_u32(&sh->drain), 0) && global_timer_ns() - t0 < tab.wait_limit_ns) {}
+    __syncwarp();
+  }
   __syncthreads();
   __syncwarp();
   cluster_sync();
@@ -1541,23 +1645,6 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   static bool attr_done[kMaxDevices] = {};     // per instantiation
   const qm_status as = allow_smem(kern, smem_bytes<MODE>(), attr_done);
   if (as != QM_OK) return as;
-  const int dev = current_device();
-  if (MODE == kProbe && g_max_pairs[dev] == 0) {
-    // the probe configuration has the largest footprint: its residency bounds the grid of all modes
-    cudaLaunchConfig_t q{};
-    q.gridDim = dim3((unsigned)(2 * (sm_count() / 2))); q.blockDim = dim3(kThreads);
-    q.dynamicSmemBytes = smem_bytes<MODE>();
-    cudaLaunchAttribute qa[1];
-    qa[0].id = cudaLaunchAttributeClusterDimension;
-    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-    q.attrs = qa; q.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kern, &q) == cudaSuccess && n > 0)
-      g_max_pairs[dev] = n < sm_count() / 2 ? n : sm_count() / 2;
-    else
-      g_max_pairs[dev] = sm_count() / 2;
-    (void)cudaGetLastError();
-  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid_size(g));
   cfg.blockDim = dim3(kThreads);
@@ -1571,7 +1658,7 @@ qm_status launch(const CUtensorMap* maps, const KernelArgs& ka, GemmShape g, cud
   cfg.attrs = attr;
   cfg.numAttrs = pdl_enabled() ? 2 : 1;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  if (MODE == kProbe || MODE == kProbe2) profile_events(&ev0, &ev1);
+  if (MODE == kProbe2) profile_events(&ev0, &ev1);
   if (ev0) QM_CUDA_OK(cudaEventRecord(ev0, s));
   QM_CUDA_OK(cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6], maps[7],
                                 ka));
@@ -1617,6 +1704,43 @@ qm_status launch_wide(const CUtensorMap& ma, const CUtensorMap& mb, KernelArgs k
 
 int tc_group_max() { return kMaxGroup; }
 
+namespace {
+constexpr size_t kProbeSmem = (size_t)CfgP::kTileBytes + sizeof(SharedP) + 1024;
+
+// Bound of the fused kernels' barrier waits and the producer's test hook (see qm_debug_* in qm.h).
+std::atomic<uint64_t> g_wait_limit_ns{1000000000ull};
+std::atomic<uint32_t> g_stop_after_kb{0xffffffffu};
+
+// CTA pairs of the fused probe kernel that can be resident at once (its footprint is the largest
+// of all modes, so its residency bounds every grid); queried once per device.
+qm_status probe_residency() {
+  const int dev = current_device();
+  if (dev < 0) return QM_ERR_UNSUPPORTED;
+  static bool attr_done[kMaxDevices] = {};
+  const qm_status as = allow_smem(tc_group_kernel, kProbeSmem, attr_done);
+  if (as != QM_OK) return as;
+  if (g_max_pairs[dev] == 0) {
+    cudaLaunchConfig_t q{};
+    q.gridDim = dim3((unsigned)(2 * (sm_count() / 2))); q.blockDim = dim3(kProbeThreads);
+    q.dynamicSmemBytes = kProbeSmem;
+    cudaLaunchAttribute qa[1];
+    qa[0].id = cudaLaunchAttributeClusterDimension;
+    qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+    q.attrs = qa; q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc_group_kernel, &q) == cudaSuccess && n > 0)
+      g_max_pairs[dev] = n < sm_count() / 2 ? n : sm_count() / 2;
+    else
+      g_max_pairs[dev] = sm_count() / 2;
+    (void)cudaGetLastError();
+  }
+  return QM_OK;
+}
+}  // namespace
+
+void set_wait_limit_ns(uint64_t ns) { g_wait_limit_ns.store(ns ? ns : 1000000000ull); }
+void set_stop_after_kb(uint32_t kb) { g_stop_after_kb.store(kb); }
+
 qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
   if (n < 1 || n > kMaxGroup) return QM_ERR_INVALID_ARG;
   // descending contraction length = descending tile cost
@@ -1626,10 +1750,12 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     for (int j = i; j > 0 && ps[order[j]].g.K > ps[order[j - 1]].g.K; --j) {
       const int t = order[j]; order[j] = order[j - 1]; order[j - 1] = t;
     }
-  static GroupTable tab;               // 15 KB: kept off the stack; guarded by the mutex below
+  static GroupTable tab;               // 11 KB: kept off the stack; guarded by the mutex below
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
   tab.n = n;
+  tab.wait_limit_ns = g_wait_limit_ns.load();
+  tab.stop_after_kb = g_stop_after_kb.load();
   int64_t total = 0;
   for (int k = 0; k < n; ++k) {
     const TcProbeArgs& p = ps[order[k]];
@@ -1639,10 +1765,8 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     GroupProblem& gp = tab.p[k];
     const bool ok = make_map(&gp.maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
                     make_map(&gp.maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
-                    make_map(&gp.maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
-                    make_map(&gp.maps[3], p.r_abs, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K) &&
-                    make_map(&gp.maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-                    make_map(&gp.maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
+                    make_map(&gp.maps[2], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+                    make_map(&gp.maps[3], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
     if (!ok) return QM_ERR_CUDA;
     KernelArgs ka{};
     fill_tiles(&ka, g);
@@ -1651,6 +1775,7 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     ka.count = (uint64_t)(g.M * g.N * g.batch);
     ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
     ka.row_stats = p.row_stats;
+    ka.err_also[0] = p.err_also[0]; ka.err_also[1] = p.err_also[1];
     gp.a = ka;
     gp.kind = p.fmt_l == QM_FMT_INT8 ? kKindI8 : kKindF8;
     gp.tile_begin = (int32_t)total;
@@ -1658,14 +1783,13 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     if (total >= (1ll << 31)) return QM_ERR_UNSUPPORTED;
   }
   tab.total_tiles = (int32_t)total;
-  static bool attr_done[kMaxDevices] = {};
-  const qm_status as = allow_smem(tc_group_kernel, smem_bytes<kProbe>(), attr_done);
-  if (as != QM_OK) return as;
+  const qm_status rs = probe_residency();
+  if (rs != QM_OK) return rs;
   const int pairs = max_pairs();
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(2 * (total < pairs ? total : pairs)));
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = smem_bytes<kProbe>();
+  cfg.blockDim = dim3(kProbeThreads);
+  cfg.dynamicSmemBytes = kProbeSmem;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1683,10 +1807,17 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
   return QM_OK;
 }
 
-int tc_probe_records(GemmShape) { return 2 * max_pairs(); }   // per format; the grouped launch uses the whole grid
+// per format; a launch writes one record per CTA of its grid
+int tc_probe_records(GemmShape) {
+  (void)probe_residency();
+  return 2 * max_pairs();
+}
 
 qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
+  if (!p.cl2) return launch_tc_probe_group(&p, 1, s);       // one format: a group of one
   if (!shape_ok(p.g)) return QM_ERR_UNSUPPORTED;
+  const qm_status rs = probe_residency();
+  if (rs != QM_OK) return rs;
   const GemmShape g = p.g;
   const int64_t ldc = qm_code_ld(g.K);
   CUtensorMap maps[8];
@@ -1695,32 +1826,21 @@ qm_status launch_tc_probe(const TcProbeArgs& p, cudaStream_t s) {
             make_map(&maps[2], p.l_abs, true, kBlockM, g.K, g.M, g.batch, g.K, g.M * g.K) &&
             make_map(&maps[3], p.r_abs, true, kHalfN, g.K, g.N, g.batch, g.K, g.N * g.K) &&
             make_map(&maps[4], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-            make_map(&maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
+            make_map(&maps[5], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc) &&
+            make_map(&maps[6], p.cl2, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
+            make_map(&maps[7], p.cr2, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
   if (!ok) return QM_ERR_CUDA;
-  const bool two = p.cl2 != nullptr;
-  if (two) {
-    ok = make_map(&maps[6], p.cl2, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-         make_map(&maps[7], p.cr2, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
-    if (!ok) return QM_ERR_CUDA;
-  } else {
-    maps[6] = maps[4]; maps[7] = maps[5];
-  }
   KernelArgs ka{};
   fill_tiles(&ka, g);
   ka.dl = p.dl; ka.pc_l = p.gran_l == QM_GRAN_CHANNEL; ka.dr = p.dr; ka.pc_r = p.gran_r == QM_GRAN_CHANNEL;
   ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
   ka.count = (uint64_t)(g.M * g.N * g.batch);
   ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
-  ka.row_stats = two ? nullptr : p.row_stats;
-  if (two) {
-    // the first format is an FP8 one (the caller orders them), the second FP8 or INT8
-    if (p.fmt_l == QM_FMT_INT8) return QM_ERR_UNSUPPORTED;
-    ka.dl2 = p.dl2; ka.dr2 = p.dr2; ka.idesc_lp2 = lp_idesc(p.fmt_l2, p.fmt_r2);
-    return p.fmt_l2 == QM_FMT_INT8 ? launch<kProbe2, kKindF8, kKindI8>(maps, ka, g, s)
-                                   : launch<kProbe2, kKindF8, kKindF8>(maps, ka, g, s);
-  }
-  return p.fmt_l == QM_FMT_INT8 ? launch<kProbe, kKindI8>(maps, ka, g, s)
-                                : launch<kProbe, kKindF8>(maps, ka, g, s);
+  // the first format is an FP8 one (the caller orders them), the second FP8 or INT8
+  if (p.fmt_l == QM_FMT_INT8) return QM_ERR_UNSUPPORTED;
+  ka.dl2 = p.dl2; ka.dr2 = p.dr2; ka.idesc_lp2 = lp_idesc(p.fmt_l2, p.fmt_r2);
+  return p.fmt_l2 == QM_FMT_INT8 ? launch<kProbe2, kKindF8, kKindI8>(maps, ka, g, s)
+                                 : launch<kProbe2, kKindF8, kKindF8>(maps, ka, g, s);
 }
 
 qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,

@@ -111,7 +111,8 @@ struct Workspace {
   bool tc;
 };
 
-Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg) {
+// with_abs: room for the bf16 |x| copies (only the two-format kernel still loads them)
+Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg, bool with_abs = false) {
   Workspace w{};
   w.tc = cfg.ref == QM_REF_BF16_FP32ACC;
   size_t o = 0;
@@ -125,8 +126,10 @@ Workspace plan(const View& L, const View& R, const qm_probe_cfg& cfg) {
   w.off_cl = take((size_t)(L.batch * L.nc * ldc));
   w.off_cr = take((size_t)(R.batch * R.nc * ldc));
   if (w.tc) {
-    w.off_al = take((size_t)(L.batch * L.nc * L.c) * 2);
-    w.off_ar = take((size_t)(R.batch * R.nc * R.c) * 2);
+    if (with_abs) {
+      w.off_al = take((size_t)(L.batch * L.nc * L.c) * 2);
+      w.off_ar = take((size_t)(R.batch * R.nc * R.c) * 2);
+    }
     w.off_kl = L.c_contig() ? 0 : take((size_t)(L.batch * L.nc * L.c) * 2);
     w.off_kr = R.c_contig() ? 0 : take((size_t)(R.batch * R.nc * R.c) * 2);
   }
@@ -310,32 +313,14 @@ size_t qm_workspace_bytes(const qm_operand* Lo, const qm_operand* Ro, const qm_p
   return plan(L, R, *cfg).total;
 }
 
-// The probe in phases that may be issued apart, on different streams (same arguments every time):
-// kClear clears the workspace words, kPrepareL / kPrepareR run scale + quantize of one operand
-// (after kClear), kProducts the products and the Eq. 3 reduction (after both).  With `defer` set and a tensor-core configuration, kProducts only describes the
-// fused kernel's work in *defer (for a grouped launch) instead of launching it.
-// What one prepared operand leaves behind that does not depend on the 8-bit format: the max|x|
-// bit patterns, the |x| copy and (for a strided contraction) the contraction-major copy.  Inside
-// a batch a later probe whose operand is the same tensor under the same scale grouping borrows
-// them and runs only its own quantize kernel.
-struct OperandShare {
-  const uint32_t* amax = nullptr;
-  void* abs_copy = nullptr;
-  void* kmaj_copy = nullptr;
-};
-struct ProbeShare {
-  const OperandShare* from_l = nullptr;   // borrow (inputs)
-  const OperandShare* from_r = nullptr;
-  OperandShare* own_l = nullptr;          // what this probe's own chains produce (outputs)
-  OperandShare* own_r = nullptr;
-};
-
+// The probe in phases that may be issued apart (same arguments every time): kClear clears the
+// workspace words (or only lists them in *clear_later, for one clearing kernel over a batch),
+// kPrepareL / kPrepareR run scale + quantize of one operand (after kClear), kProducts the
+// products and the Eq. 3 reduction (after both).
 enum { kClear = 1, kPrepareL = 2, kPrepareR = 4, kPrepare = kClear | kPrepareL | kPrepareR, kProducts = 8 };
 static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
                               qm_metric_result* out, void* ws, size_t ws_bytes, void* stream, int phases,
-                              TcProbeArgs* defer, bool* deferred, const ProbeShare* share = nullptr,
                               ClearList* clear_later = nullptr) {
-  if (deferred) *deferred = false;
   View L, R;
   qm_status st = check_probe(Lo, Ro, cfg, &L, &R);
   if (st != QM_OK) return st;
@@ -362,31 +347,22 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
     QM_CUDA_OK(cudaMemsetAsync(cfg->row_stats, 0, sizeof(double) * QM_ROW_STATS * (size_t)(L.batch * L.nc), s));
   uint32_t* ml = reinterpret_cast<uint32_t*>(base + w.off_ml);
   uint32_t* mr = reinterpret_cast<uint32_t*>(base + w.off_mr);
-  void* al = w.tc ? base + w.off_al : nullptr;
-  void* ar = w.tc ? base + w.off_ar : nullptr;
+  // the fused kernel forms |L| and |R| tiles in shared memory: no |x| copy is written
+  void* al = nullptr;
+  void* ar = nullptr;
   void* kl = (w.tc && !L.c_contig()) ? base + w.off_kl : nullptr;
   void* kr = (w.tc && !R.c_contig()) ? base + w.off_kr : nullptr;
   const StochasticDraw draw_l{cfg->seed, 0u}, draw_r{cfg->seed, 1u};
   const StochasticDraw* dl_draw = (cfg->round & QM_ROUND_STOCHASTIC_L) ? &draw_l : nullptr;
   const StochasticDraw* dr_draw = (cfg->round & QM_ROUND_STOCHASTIC_R) ? &draw_r : nullptr;
-  const OperandShare* from_l = share ? share->from_l : nullptr;
-  const OperandShare* from_r = share ? share->from_r : nullptr;
-  if (share && share->own_l) *share->own_l = OperandShare{ml, al, kl};
-  if (share && share->own_r) *share->own_r = OperandShare{mr, ar, kr};
   if (phases & kPrepareL) {
-    st = from_l ? launch_quantize(L, cfg->fmt_l, cfg->gran_l, reinterpret_cast<const float*>(from_l->amax), true, dl,
-                                  err, cl, nullptr, nullptr, s, dl_draw)
-                : prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err, dl_draw, cfg->batch_groups_l, s);
+    st = prepare_operand(L, cfg->fmt_l, cfg->gran_l, ml, dl, cl, al, kl, err, dl_draw, cfg->batch_groups_l, s);
     if (st != QM_OK) return st;
   }
   if (phases & kPrepareR) {
-    st = from_r ? launch_quantize(R, cfg->fmt_r, cfg->gran_r, reinterpret_cast<const float*>(from_r->amax), true, dr,
-                                  err, cr, nullptr, nullptr, s, dr_draw)
-                : prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err, dr_draw, cfg->batch_groups_r, s);
+    st = prepare_operand(R, cfg->fmt_r, cfg->gran_r, mr, dr, cr, ar, kr, err, dr_draw, cfg->batch_groups_r, s);
     if (st != QM_OK) return st;
   }
-  if (from_l) { al = from_l->abs_copy; kl = from_l->kmaj_copy; }
-  if (from_r) { ar = from_r->abs_copy; kr = from_r->kmaj_copy; }
   if (!(phases & kProducts)) return QM_OK;
   GemmShape g{L.nc, R.nc, L.c, L.batch};
   if (w.tc) {
@@ -400,11 +376,6 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
     p.done_counter = err + 1;               // second word of the cleared error slot
     p.result = out;
     p.row_stats = cfg->row_stats;
-    if (defer) {
-      *defer = p;
-      *deferred = true;
-      return QM_OK;
-    }
     return launch_tc_probe(p, s);           // the last CTA writes the record
   }
   st = launch_simt_probe(L, R, cl, cfg->fmt_l, dl, cfg->gran_l, cr, cfg->fmt_r, dr, cfg->gran_r, part, s);
@@ -414,7 +385,7 @@ static qm_status probe_phases(const qm_operand* Lo, const qm_operand* Ro, const 
 
 qm_status qm_probe_layer(const qm_operand* Lo, const qm_operand* Ro, const qm_probe_cfg* cfg,
                          qm_metric_result* out, void* ws, size_t ws_bytes, void* stream) {
-  return probe_phases(Lo, Ro, cfg, out, ws, ws_bytes, stream, kPrepare | kProducts, nullptr, nullptr);
+  return probe_phases(Lo, Ro, cfg, out, ws, ws_bytes, stream, kPrepare | kProducts);
 }
 
 // ---- two formats in one pass -------------------------------------------------------------------
@@ -443,7 +414,7 @@ bool order2(const qm_probe_cfg* ca, const qm_probe_cfg* cb, const qm_probe_cfg**
 }
 Workspace2 plan2(const View& L, const View& R, const qm_probe_cfg& first) {
   Workspace2 w{};
-  w.a = plan(L, R, first);
+  w.a = plan(L, R, first, true);
   size_t o = w.a.total;
   auto take = [&](size_t bytes) { size_t at = o; o += align256(bytes); return at; };
   w.off_dl2 = take(sizeof(float) * delta_count(L, first.gran_l));
@@ -641,26 +612,65 @@ qm_status batch_streams(BatchStreams** out) {
   return QM_OK;
 }
 
-// The earlier probe (j < i) of a batch whose operand on side `side` (0 = L, 1 = R) is the very
-// tensor of probe i's, scaled in the same groups, and that has prepared it itself through the
-// absmax -> quantize route (so that its max|x| array exists); -1 if there is none.
-int find_lender(const qm_operand* ops, const qm_probe_cfg* cfg, int i, int side, const std::vector<int>& lender) {
-  const qm_operand& x = ops[i];
-  const int gran = side ? cfg[i].gran_r : cfg[i].gran_l;
-  const int groups = side ? cfg[i].batch_groups_r : cfg[i].batch_groups_l;
-  const bool grouped = gran == QM_GRAN_CHANNEL && groups > 0 && groups < x.batch;
-  // per-channel scales of a contiguous contraction take the single-pass kernel, which keeps no maxima
-  if (gran == QM_GRAN_CHANNEL && !grouped && (x.stride_c == 1 || x.contract == 1)) return -1;
-  for (int j = 0; j < i; ++j) {
-    if (cfg[j].ref != QM_REF_BF16_FP32ACC || lender[2 * j + side] >= 0) continue;
-    const qm_operand& y = ops[j];
-    const int gj = side ? cfg[j].gran_r : cfg[j].gran_l, pj = side ? cfg[j].batch_groups_r : cfg[j].batch_groups_l;
-    if (y.data == x.data && y.dtype == x.dtype && y.noncontract == x.noncontract && y.contract == x.contract &&
-        y.stride_nc == x.stride_nc && y.stride_c == x.stride_c && y.batch == x.batch &&
-        y.stride_batch == x.stride_batch && gj == gran && pj == groups)
-      return j;
+// One operand of one tensor-core probe of a batch: what has to be prepared, where this probe's own
+// buffers for it are, and whose results it uses.  Preparing an operand leaves four things behind:
+// the max|x| bit patterns, the contraction-major bf16 copy (strided contraction only), the
+// scales and the codes.  A sweep of formats over a layer, and a layer whose activations feed
+// several products, ask for the same things many times over; inside a batch each is made once:
+//   code_root: the earlier operand with the same view, scale grouping, format and rounding: its
+//              scales, codes and copy are used as they are and nothing is launched;
+//   copy_root: the earlier operand with the same view and scale grouping under another format:
+//              its max|x| and contraction-major copy are borrowed, only the codes are made;
+//   amax_root: per-tensor scales only: the earlier operand over the same elements in either
+//              orientation (max|x| does not depend on which dimension contracts).
+// A root index equal to the slot's own index means "makes it itself".
+struct Slot {
+  View v;
+  int fmt, gran, groups;
+  bool stochastic;
+  StochasticDraw draw;
+  uint32_t* amax; float* delta; uint8_t* codes; void* kmaj; uint32_t* err;
+  bool keeps_amax;                 // false when the single-pass per-row kernel prepares it (no maxima are stored)
+  int code_root, copy_root, amax_root;
+  int stream;                      // index of the library stream its kernels go to
+};
+
+bool same_view(const View& a, const View& b) {
+  return a.data == b.data && a.dtype == b.dtype && a.nc == b.nc && a.c == b.c && a.s_nc == b.s_nc && a.s_c == b.s_c &&
+         a.batch == b.batch && a.s_b == b.s_b;
+}
+// the same elements with the two matrix dimensions exchanged
+bool transposed_view(const View& a, const View& b) {
+  return a.data == b.data && a.dtype == b.dtype && a.nc == b.c && a.c == b.nc && a.s_nc == b.s_c && a.s_c == b.s_nc &&
+         a.batch == b.batch && a.s_b == b.s_b;
+}
+bool grouped_scales(const Slot& x) { return x.gran == QM_GRAN_CHANNEL && x.groups > 0 && x.groups < x.v.batch; }
+
+void find_roots(std::vector<Slot>& slots, int t) {
+  Slot& x = slots[t];
+  x.code_root = x.copy_root = x.amax_root = t;
+  const int gx = grouped_scales(x) ? x.groups : 0;
+  for (int u = 0; u < t; ++u) {
+    const Slot& y = slots[u];
+    if (y.code_root != u || !same_view(x.v, y.v) || y.gran != x.gran || (grouped_scales(y) ? y.groups : 0) != gx) continue;
+    const bool same_round = x.stochastic == y.stochastic &&
+                            (!x.stochastic || (x.draw.seed == y.draw.seed && x.draw.stream == y.draw.stream));
+    if (y.fmt == x.fmt && same_round) { x.code_root = u; x.copy_root = y.copy_root; x.amax_root = y.amax_root; return; }
   }
-  return -1;
+  for (int u = 0; u < t; ++u) {
+    const Slot& y = slots[u];
+    if (y.code_root != u || y.copy_root != u || !y.keeps_amax) continue;
+    if (same_view(x.v, y.v) && y.gran == x.gran && (grouped_scales(y) ? y.groups : 0) == gx) {
+      x.copy_root = u; x.amax_root = y.amax_root;
+      return;
+    }
+  }
+  if (x.gran != QM_GRAN_TENSOR) return;
+  for (int u = 0; u < t; ++u) {
+    const Slot& y = slots[u];
+    if (y.code_root != u || y.copy_root != u || y.amax_root != u || y.gran != QM_GRAN_TENSOR) continue;
+    if (same_view(x.v, y.v) || transposed_view(x.v, y.v)) { x.amax_root = u; return; }
+  }
 }
 
 // Runs issue(i, stream_i) for i < n round-robin over the library's streams, between a fork from
@@ -698,88 +708,144 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
   qm_status st = batch_streams(&b);
   if (st != QM_OK) return st;
   std::lock_guard<std::mutex> lock(b->issue);
-  // Scale + quantize of every OPERAND is a chain of two or three short, latency-bound kernels, and
-  // all 2n chains are independent: the workspace words of every probe are cleared on the caller's
-  // stream, then the chains are spread over the library's streams so that they run beside one
-  // another.  Probes that do not take the fused tensor-core kernel (fp32 reference) run whole on
-  // one of those streams.  A refused probe ends the issue there; the ones before it complete.
-  std::vector<int32_t> fused;
-  int32_t good = 0;
+  // Pass 1 (host only): check every probe, lay out its workspace, list the control words to clear
+  // and describe the two operands of every tensor-core probe.  A refused probe ends the batch
+  // there; the ones before it complete.
+  struct Planned { View Lv, Rv; Workspace w; bool tc; };
+  std::vector<Planned> plans;
+  std::vector<Slot> slots;
+  std::vector<int> slot_of((size_t)n, -1);            // probe -> index of its left operand's slot
   ClearList clears{};
-  for (; good < n && st == QM_OK; ++good)
-    if (cfg[good].ref == QM_REF_BF16_FP32ACC)
-      st = probe_phases(&L[good], &R[good], &cfg[good], out + good, ws[good], ws_bytes[good], user, kClear, nullptr,
-                        nullptr, nullptr, &clears);
-  if (st != QM_OK) --good;
+  int32_t good = 0;
+  qm_status refused = QM_OK;                          // why probe `good` was not taken, if one was not
+  for (; good < n; ++good) {
+    const int32_t i = good;
+    Planned pl{};
+    refused = check_probe(&L[i], &R[i], &cfg[i], &pl.Lv, &pl.Rv);
+    if (refused == QM_OK && (!ws[i] || (reinterpret_cast<uintptr_t>(ws[i]) & 255)))
+      refused = ws[i] ? QM_ERR_ALIGNMENT : QM_ERR_INVALID_ARG;
+    if (refused != QM_OK) break;
+    pl.w = plan(pl.Lv, pl.Rv, cfg[i]);
+    pl.tc = pl.w.tc;
+    if (ws_bytes[i] < pl.w.total) { refused = QM_ERR_WORKSPACE_TOO_SMALL; break; }
+    plans.push_back(pl);
+    if (!pl.tc) continue;
+    uint8_t* base = static_cast<uint8_t*>(ws[i]);
+    if (clears.n == kClearMax) {
+      const qm_status e = launch_clear_many(clears, user);
+      if (e != QM_OK) return e;
+      clears.n = 0;
+    }
+    clears.ptr[clears.n] = base;                       // error word, CTA counter and both max|x| buffers are adjacent
+    clears.words[clears.n++] = (uint32_t)(pl.w.off_dl / 4);
+    if (cfg[i].row_stats)
+      QM_CUDA_OK(cudaMemsetAsync(cfg[i].row_stats, 0, sizeof(double) * QM_ROW_STATS * (size_t)(pl.Lv.batch * pl.Lv.nc), user));
+    slot_of[i] = (int)slots.size();
+    for (int side = 0; side < 2; ++side) {
+      const View& v = side ? pl.Rv : pl.Lv;
+      Slot x{};
+      x.v = v;
+      x.fmt = side ? cfg[i].fmt_r : cfg[i].fmt_l;
+      x.gran = side ? cfg[i].gran_r : cfg[i].gran_l;
+      x.groups = side ? cfg[i].batch_groups_r : cfg[i].batch_groups_l;
+      x.stochastic = (cfg[i].round & (side ? QM_ROUND_STOCHASTIC_R : QM_ROUND_STOCHASTIC_L)) != 0;
+      x.draw = StochasticDraw{cfg[i].seed, (uint32_t)side};
+      x.amax = reinterpret_cast<uint32_t*>(base + (side ? pl.w.off_mr : pl.w.off_ml));
+      x.delta = reinterpret_cast<float*>(base + (side ? pl.w.off_dr : pl.w.off_dl));
+      x.codes = base + (side ? pl.w.off_cr : pl.w.off_cl);
+      x.kmaj = v.c_contig() ? nullptr : base + (side ? pl.w.off_kr : pl.w.off_kl);
+      x.err = reinterpret_cast<uint32_t*>(base + pl.w.off_err);
+      x.keeps_amax = !(!x.stochastic && !grouped_scales(x) && x.gran == QM_GRAN_CHANNEL && v.c_contig());
+      slots.push_back(x);
+      find_roots(slots, (int)slots.size() - 1);
+    }
+  }
   if (clears.n > 0) {
     const qm_status e = launch_clear_many(clears, user);
     if (e != QM_OK) return e;
   }
+  // Pass 2: the scale / quantize chains.  Each chain is two or three short kernels and the chains
+  // of different tensors are independent, so they are spread over the library's streams and run
+  // beside one another; whatever borrows from an earlier operand goes to that operand's stream,
+  // behind the kernels that make what it borrows.  Probes that do not take the fused tensor-core
+  // kernel (fp32 reference) run whole on one of those streams.
   QM_CUDA_OK(cudaEventRecord(b->fork, user));
-  const int used = 2 * good < kBatchStreams ? 2 * good : kBatchStreams;
-  for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
-  // One chunk: all chains, then the caller's stream waits for the library's streams and takes the
-  // fused kernels as one persistent launch.  (Two chunks, the second one's chains running under
-  // the first one's launch, measured slower: the chains wait for the SMs the launch holds.)
-  const int32_t chunk = good;
-  std::vector<OperandShare> own(2 * (size_t)n);
-  std::vector<int> lender(2 * (size_t)n, -1);     // per operand: the probe it borrows from, or -1
-  std::vector<ProbeShare> shares((size_t)n);
-  std::vector<TcProbeArgs> args;
-  for (int32_t c0 = 0; c0 < good; c0 += chunk) {
-    const int32_t c1 = c0 + chunk < good ? c0 + chunk : good;
-    fused.clear();
-    for (int32_t i = c0; i < c1; ++i) {
-      cudaStream_t sl = b->s[(2 * i) % kBatchStreams], sr = b->s[(2 * i + 1) % kBatchStreams];
-      qm_status e;
-      if (cfg[i].ref == QM_REF_BF16_FP32ACC) {
-        // An operand that an earlier probe of the batch has already prepared (the same tensor under
-        // the same scale grouping: a sweep of formats over one layer) borrows that probe's max|x|,
-        // |x| copy and contraction-major copy and only quantizes, on the lender's stream.
-        ProbeShare sh;
-        sh.own_l = &own[2 * i]; sh.own_r = &own[2 * i + 1];
-        const int dl_i = find_lender(L, cfg, i, 0, lender), dr_i = find_lender(R, cfg, i, 1, lender);
-        lender[2 * i] = dl_i; lender[2 * i + 1] = dr_i;
-        if (dl_i >= 0) { sh.from_l = &own[2 * dl_i]; sl = b->s[(2 * dl_i) % kBatchStreams]; }
-        if (dr_i >= 0) { sh.from_r = &own[2 * dr_i + 1]; sr = b->s[(2 * dr_i + 1) % kBatchStreams]; }
-        shares[i] = sh;
-        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepareL, nullptr, nullptr, &sh);
-        if (e == QM_OK)
-          e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sr, kPrepareR, nullptr, nullptr, &sh);
-        if (e == QM_OK) fused.push_back(i);
-      } else {
-        e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], sl, kPrepare | kProducts, nullptr, nullptr);
-      }
-      if (e != QM_OK && st == QM_OK) st = e;
+  for (int j = 0; j < kBatchStreams; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
+  int next_stream = 0;
+  for (size_t t = 0; t < slots.size(); ++t) {
+    Slot& x = slots[t];
+    if (x.code_root != (int)t) { x.stream = slots[x.code_root].stream; continue; }     // nothing to launch
+    cudaStream_t s;
+    qm_status e;
+    const StochasticDraw* draw = x.stochastic ? &x.draw : nullptr;
+    if (x.copy_root != (int)t) {
+      x.stream = slots[x.copy_root].stream; s = b->s[x.stream];
+      e = launch_quantize(x.v, x.fmt, x.gran, reinterpret_cast<const float*>(slots[x.amax_root].amax), true, x.delta, x.err,
+                          x.codes, nullptr, nullptr, s, draw);
+    } else if (x.amax_root != (int)t) {
+      x.stream = slots[x.amax_root].stream; s = b->s[x.stream];
+      e = launch_quantize(x.v, x.fmt, x.gran, reinterpret_cast<const float*>(slots[x.amax_root].amax), true, x.delta, x.err,
+                          x.codes, nullptr, x.kmaj, s, draw);
+    } else {
+      x.stream = next_stream; next_stream = (next_stream + 1) % kBatchStreams; s = b->s[x.stream];
+      e = prepare_operand(x.v, x.fmt, x.gran, x.amax, x.delta, x.codes, nullptr, x.kmaj, x.err, draw, x.groups, s);
     }
-    for (int j = 0; j < used; ++j) {
-      QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
-      QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
-    }
-    // up to tc_group_max() probes per persistent launch
-    auto flush_group = [&]() -> qm_status {
-      if (args.empty()) return QM_OK;
-      const qm_status e = args.size() == 1 ? launch_tc_probe(args[0], user)
-                                           : launch_tc_probe_group(args.data(), (int)args.size(), user);
-      args.clear();
-      return e;
-    };
-    for (int32_t i : fused) {
-      TcProbeArgs p{};
-      bool deferred = false;
-      const qm_status e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], user, kProducts, &p, &deferred,
-                                       &shares[i]);
-      if (e != QM_OK) { if (st == QM_OK) st = e; continue; }
-      if (deferred) args.push_back(p);
-      if ((int)args.size() == tc_group_max()) {
-        const qm_status g = flush_group();
-        if (g != QM_OK && st == QM_OK) st = g;
-      }
-    }
-    const qm_status g = flush_group();
-    if (g != QM_OK && st == QM_OK) st = g;
+    if (e != QM_OK && st == QM_OK) st = e;
   }
-  return st;
+  for (int32_t i = 0; i < good; ++i) {
+    if (plans[i].tc) continue;
+    cudaStream_t s = b->s[next_stream]; next_stream = (next_stream + 1) % kBatchStreams;
+    const qm_status e = probe_phases(&L[i], &R[i], &cfg[i], out + i, ws[i], ws_bytes[i], s, kPrepare | kProducts);
+    if (e != QM_OK && st == QM_OK) st = e;
+  }
+  for (int j = 0; j < kBatchStreams; ++j) {
+    QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
+    QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
+  }
+  // Pass 3: the caller's stream has waited for every chain; the fused kernels go to it as
+  // persistent launches of up to tc_group_max() probes.  (Running a second chunk's chains under
+  // the first chunk's launch measured slower: the chains wait for the SMs the launch holds.)
+  std::vector<TcProbeArgs> args;
+  auto flush_group = [&]() -> qm_status {
+    if (args.empty()) return QM_OK;
+    const qm_status e = launch_tc_probe_group(args.data(), (int)args.size(), user);
+    args.clear();
+    return e;
+  };
+  for (int32_t i = 0; i < good && st == QM_OK; ++i) {
+    if (!plans[i].tc) continue;
+    const Planned& pl = plans[i];
+    uint8_t* base = static_cast<uint8_t*>(ws[i]);
+    const Slot& xl = slots[slot_of[i]];
+    const Slot& xr = slots[slot_of[i] + 1];
+    const Slot& cl = slots[xl.code_root];
+    const Slot& cr = slots[xr.code_root];
+    void* kl = slots[cl.copy_root].kmaj;
+    void* kr = slots[cr.copy_root].kmaj;
+    TcProbeArgs p{};
+    p.l = kl ? kl : pl.Lv.data; p.l_ld = kl ? pl.Lv.c : pl.Lv.s_nc; p.l_sb = kl ? pl.Lv.nc * pl.Lv.c : pl.Lv.s_b;
+    p.r = kr ? kr : pl.Rv.data; p.r_ld = kr ? pl.Rv.c : pl.Rv.s_nc; p.r_sb = kr ? pl.Rv.nc * pl.Rv.c : pl.Rv.s_b;
+    p.cl = cl.codes; p.cr = cr.codes;
+    p.fmt_l = cfg[i].fmt_l; p.fmt_r = cfg[i].fmt_r;
+    p.dl = cl.delta; p.gran_l = cfg[i].gran_l; p.dr = cr.delta; p.gran_r = cfg[i].gran_r;
+    p.g = GemmShape{pl.Lv.nc, pl.Rv.nc, pl.Lv.c, pl.Lv.batch};
+    p.partials = reinterpret_cast<double*>(base + pl.w.off_part);
+    p.err_word = xl.err;
+    p.done_counter = xl.err + 1;            // second word of the cleared error slot
+    // a non-finite operand is flagged in the error word of the probe whose kernel made the codes
+    p.err_also[0] = cl.err != xl.err ? cl.err : nullptr;
+    p.err_also[1] = cr.err != xl.err ? cr.err : nullptr;
+    p.result = out + i;
+    p.row_stats = cfg[i].row_stats;
+    args.push_back(p);
+    if ((int)args.size() == tc_group_max()) {
+      const qm_status g = flush_group();
+      if (g != QM_OK && st == QM_OK) st = g;
+    }
+  }
+  const qm_status g = flush_group();
+  if (g != QM_OK && st == QM_OK) st = g;
+  return st != QM_OK ? st : refused;
 }
 
 qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_operand* R_host,
@@ -847,6 +913,9 @@ qm_status qm_profile_samples(double* start_ms, double* dur_ms, int32_t cap, int3
   *launches = n;
   return QM_OK;
 }
+
+void qm_debug_set_wait_limit_ns(uint64_t ns) { qm::set_wait_limit_ns(ns); }
+void qm_debug_stop_producer_after(uint32_t k_blocks) { qm::set_stop_after_kb(k_blocks); }
 
 qm_status qm_profile_read(double* ms, int32_t* launches) {
   if (!ms || !launches) return QM_ERR_INVALID_ARG;

@@ -139,6 +139,7 @@ struct TcProbeArgs {
   uint32_t* done_counter;                   // zero on entry; counts finished CTAs
   qm_metric_result* result;                 // written by the last CTA to finish
   uint32_t* err_word;
+  const uint32_t* err_also[2] = {nullptr, nullptr};   // error words of other probes whose kernels made this probe's codes
   double* row_stats = nullptr;              // optional per-row Eq. 3 sums (zeroed by the caller), one-format probes only
   // Two formats in one pass (cl2 != nullptr): codes and scales of the second format, same
   // granularities; `result` then points at two records and `partials` holds 2 x tc_probe_records.
@@ -153,6 +154,11 @@ qm_status launch_tc_probe(const TcProbeArgs& a, cudaStream_t s);
 // prepared already; each writes its own record; the first probe's done_counter counts the CTAs).
 int tc_group_max();
 qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s);
+// Bound of every barrier wait of the fused probe kernel (0 restores the default of one second), and
+// a hook for testing the give-up path: the producer issues no more than this many k-blocks
+// per CTA (0xffffffff: off), so that the consumers' waits run out.
+void set_wait_limit_ns(uint64_t ns);
+void set_stop_after_kb(uint32_t kb);
 qm_status launch_tc_gemm_lp(const uint8_t* cl, int fmt_l, const float* dl, int gran_l,
                             const uint8_t* cr, int fmt_r, const float* dr, int gran_r,
                             GemmShape g, float* out_descaled, void* out_raw, uint32_t* err_word,
