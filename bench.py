@@ -32,10 +32,10 @@ sys.path.insert(0, ROOT)
 
 from paper_2408_02897_b200 import workloads  # noqa: E402
 
-# DRAM bytes (read + write) of the grouped fused kernel per byte of distinct operand data it reads
-# (bf16 L, R, their |x| copies and both code tensors), from a profiler capture of the BERT-base
-# workload's launch; every operand byte is read from DRAM once, so a launch of another workload is
-# scaled by its distinct operand bytes.  None: the kernel has changed since the counters were taken.
+# DRAM bytes (read + write) of the fused probe kernel per byte of distinct operand data it reads
+# (bf16 L and R and both code tensors), from a profiler capture of one launch of a smaller workload;
+# a launch of another workload is scaled by its distinct operand bytes.  None: the kernel has
+# changed since the counters were taken.
 TC_DRAM_BYTES_PER_OPERAND_BYTE = None
 
 
@@ -72,15 +72,15 @@ def build_workload(name):
 
 
 def distinct_operand_bytes(ops):
-    """Bytes the fused kernels of a step read when every distinct tensor is counted once: bf16 x and
-    |x| of each distinct (tensor, orientation) and one code tensor per distinct (tensor, orientation,
-    format)."""
+    """Bytes the fused kernels of a step read when every distinct tensor is counted once: the bf16
+    values of each distinct (tensor, orientation) and one code tensor per distinct (tensor,
+    orientation, format)."""
     seen_x, seen_c, total = set(), set(), 0
     for o in ops:
         for t, cd, fmt in ((o["L"], o["cl"], o["fmt_l"]), (o["R"], o["cr"], o["fmt_r"])):
             if (id(t), cd) not in seen_x:
                 seen_x.add((id(t), cd))
-                total += 4 * t.numel()
+                total += 2 * t.numel()
             if (id(t), cd, fmt) not in seen_c:
                 seen_c.add((id(t), cd, fmt))
                 total += t.numel()
@@ -598,11 +598,13 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "fp8/int8 x bf16 (fp32/int32 accumulate)",
             "data": "synthetic", "config": config_of(args, desc),
             "run": {"probes_per_pass": len(ops), "passes_per_step": m["repeat"], "timed_region_s": m["wall_s"],
-                    "issue": "qm_probe_batch: one call per pass; scale/quantize chains on the library's 8 streams, "
-                             "then grouped fused launches of up to 16 probes on the caller's stream"},
+                    "issue": "qm_probe_batch: one call per pass; every distinct operand is scaled and quantized once "
+                             "(all its formats in one pass over it) on the library's 8 streams, then fused launches of "
+                             "up to 16 probes on the caller's stream"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "note": "one pass per step through qm_probe_batch_host (pinned host operands in, records out)"},
+                    "note": "one pass per step through qm_probe_batch_host: every distinct pinned host operand copied in "
+                            "once, records copied out, inside the timed region"},
             "gpu_launches": m["launches"], "roofline": roofline,
             "mean_be": {o["name"]: r.derived()["mean_be"] for o, r in zip(ops, results)}}
     if not args.no_extras:

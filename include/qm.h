@@ -228,6 +228,24 @@ qm_status qm_quantize_stochastic(const qm_operand* x, int32_t fmt, int32_t gran,
                                  uint8_t* codes, void* abs_copy, void* kmaj_copy, void* stream);
 
 /*
+ * The codes of several formats of one operand (Eq. 1 once per format): the
+ * measurement sweeps the 8-bit formats over the same tensors (Table 1), and
+ * max|x| and the pass over the tensor do not depend on the format.  fmts holds
+ * n_fmt (1..3) distinct formats; delta_out[k] (device, 1 value or one per batch
+ * element and non-contracting index) and codes[k] (device, laid out as for
+ * qm_quantize) receive format k's scales and codes, round-to-nearest-even;
+ * kmaj_copy as for qm_quantize.  amax_scratch is device scratch of as many
+ * 32-bit words as one delta_out array has values; the call clears it.  Every
+ * result equals what qm_quantize gives for that format alone.  Per-tensor
+ * scales of a bf16 operand are produced by one kernel that reads the operand
+ * once; other cases by one quantize launch per format after a common max|x|.
+ * A non-finite operand yields NaN scales, as in qm_scale.
+ */
+qm_status qm_quantize_formats(const qm_operand* x, int32_t n_fmt, const int32_t* fmts, int32_t gran,
+                              float* const* delta_out, uint8_t* const* codes, void* kmaj_copy,
+                              uint32_t* amax_scratch, void* stream);
+
+/*
  * The 8-bit product and its descaling (Methodology, 3rd bullet):
  *   A = Lbar . Rbar^T accumulated in int32 (INT8, exact) or fp32 (FP8, any mix
  *   of E4M3 and E5M2), Q_ij = A_ij * delta_l[i] * delta_r[j].
@@ -341,19 +359,31 @@ qm_status qm_quantize_error(const qm_operand* x, int32_t fmt, int32_t gran, cons
  * scale/quantize kernels of all operands beside one another on a few streams of
  * its own (created on the first call on each device, kept until the process
  * exits) and then the fused kernels of all tensor-core probes as one persistent
- * launch over the tiles of all of them (the sums of a record are then taken
- * over another tile-to-CTA assignment than in qm_probe_layer and may differ in
- * the last bits).  All of it is ordered after the work already in `stream`,
- * and work put into `stream` after the call waits for every probe.  `out` is a
- * device array of n records; the n workspaces must be distinct and sized per
- * probe.  With qm_probe_batch_host the operands live in host memory as for
- * qm_probe_layer_host (l_stage[i], r_stage[i]: distinct device staging buffers),
- * whole probes are spread over the library's streams so that the copies of one
- * overlap the kernels of another, out_host receives the n records and the call
- * waits for them; the first device-detected condition is returned.  n == 0 is a
- * no-op.  On an argument error of probe i the probes before it are completed
- * as described; the rest are not issued.  Make the first call on a device
- * outside any stream capture.
+ * launches of up to 16 probes over the tiles of all of them (the sums of a
+ * record are then taken over another tile-to-CTA assignment than in
+ * qm_probe_layer and may differ in the last bits).  A measurement pass asks
+ * for the same preparation many times over (a sweep of formats over one layer,
+ * an activation that feeds several products, a gradient that appears in dgrad
+ * and wgrad): inside a batch, operands that describe the same memory (same
+ * address, extents and strides) under the same scale grouping are prepared
+ * once.  Their max|x| is reduced once (for per-tensor scales also across the
+ * two orientations of a tensor), the contraction-major copy is made once, the
+ * codes of up to three formats come from one pass over the tensor, and equal
+ * (format, rounding) requests share scales and codes outright; a probe then
+ * reads those results from the workspace of the probe that made them, and a
+ * non-finite operand is reported in the record of every probe that uses it.
+ * All of it is ordered after the work already in `stream`, and work put into
+ * `stream` after the call waits for every probe.  `out` is a device array of n
+ * records; the n workspaces must be distinct and sized per probe.  With
+ * qm_probe_batch_host the operands live in host memory as for
+ * qm_probe_layer_host (l_stage[i], r_stage[i]: distinct device staging buffers,
+ * each as large as its operand): every distinct host operand (same address and
+ * extent) is copied to the device once, into the staging buffer of the first
+ * probe that names it, the probes then run as a device batch, out_host
+ * receives the n records and the call waits for them; the first
+ * device-detected condition is returned.  n == 0 is a no-op.  On an argument
+ * error of probe i the probes before it are completed as described; the rest
+ * are not issued.  Make the first call on a device outside any stream capture.
  */
 qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, const qm_probe_cfg* cfg,
                          qm_metric_result* out, void* const* ws, const size_t* ws_bytes, void* stream);
@@ -361,6 +391,10 @@ qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_oper
                               const qm_probe_cfg* cfg, void* const* l_stage, void* const* r_stage,
                               qm_metric_result* out_host, qm_metric_result* out_dev, void* const* ws,
                               const size_t* ws_bytes, void* stream);
+/* The bytes one qm_probe_batch_host call copies to the device (every distinct host operand once:
+ * operands with the same host address and extent share one copy) and back (n records). */
+qm_status qm_probe_batch_host_bytes(int32_t n, const qm_operand* L_host, const qm_operand* R_host, size_t* h2d_bytes,
+                                    size_t* d2h_bytes);
 
 const char* qm_status_string(int32_t status);
 int32_t qm_version(void);
@@ -410,6 +444,19 @@ qm_status qm_profile_read(double* tc_probe_ms, int32_t* tc_probe_launches);
  * `cap`) its start relative to the first recorded launch's start and its duration, both in
  * milliseconds; *launches receives the number recorded so far. */
 qm_status qm_profile_samples(double* start_ms, double* dur_ms, int32_t cap, int32_t* launches);
+
+/*
+ * Read-bandwidth calibration (measurement aid, no counterpart in the paper): one
+ * read-only pass over `bytes` of device memory at `data` (16-byte aligned) and
+ * nothing else, so that the library's read-mostly kernels (max|x|, tensor
+ * statistics) can be compared with what a pure read stream reaches on the same
+ * buffer.  variant: 0 = 8 plain 128-bit loads in flight per thread, 3 = 16 of
+ * them; 1 and 2 = 4 and 8 256-bit loads in flight with streaming cache hints
+ * (data 32-byte aligned); blocks_per_sm (1..32) blocks of 256 threads per SM.
+ * sink may be NULL.  Time it with events.
+ */
+qm_status qm_debug_read_pass(const void* data, size_t bytes, int32_t variant, int32_t blocks_per_sm, uint32_t* sink,
+                             void* stream);
 
 /*
  * Testing aids for the bounded device waits (no counterpart in the paper).

@@ -100,6 +100,7 @@ def lib():
             "qm_scale_shared": (I32, [OP, I32, I32, P, P]),
             "qm_quantize": (I32, [OP, I32, I32, I32, P, P, P, P, P, P]),
             "qm_quantize_stochastic": (I32, [OP, I32, I32, C.c_uint64, C.c_uint32, P, P, P, P, P, P]),
+            "qm_quantize_formats": (I32, [OP, I32, C.POINTER(I32), I32, C.POINTER(P), C.POINTER(P), P, P, P]),
             "qm_gemm": (I32, [P, I32, P, I32, P, I32, P, I32, I64, I64, I64, I64, P, P, I32, P]),
             "qm_gemm_ref": (I32, [P, P, I64, I64, I64, I64, P, P]),
             "qm_metric_workspace_bytes": (SZ, [I64]),
@@ -118,12 +119,14 @@ def lib():
             "qm_probe_batch": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), P, C.POINTER(P), C.POINTER(SZ), P]),
             "qm_probe_batch_host": (I32, [I32, OP, OP, C.POINTER(ProbeCfg), C.POINTER(P), C.POINTER(P),
                                           C.POINTER(MetricResult), P, C.POINTER(P), C.POINTER(SZ), P]),
+            "qm_probe_batch_host_bytes": (I32, [I32, OP, OP, C.POINTER(SZ), C.POINTER(SZ)]),
             "qm_status_string": (C.c_char_p, [I32]),
             "qm_version": (I32, []),
             "qm_last_cuda_error": (C.c_char_p, []),
             "qm_metric_noalloc": (I32, [P, P, P, I64, P, P]),
             "qm_metric_noalloc_max_count": (I64, []),
             "qm_kernel_launches": (I64, []),
+            "qm_debug_read_pass": (I32, [P, SZ, I32, I32, P, P]),
             "qm_debug_set_wait_limit_ns": (None, [C.c_uint64]),
             "qm_debug_stop_producer_after": (None, [C.c_uint32]),
             "qm_profile_enable": (I32, [I32]),
@@ -216,6 +219,22 @@ def qm_quantize(op, fmt, gran, delta=None, want_abs=False, want_kmaj=False, stre
         _check(lib().qm_quantize(C.byref(op), FMT[fmt], GRAN[gran], 0, _ptr(delta), _ptr(dout), _ptr(codes),
                                  _ptr(ab), _ptr(km), _stream(stream)), "qm_quantize")
     return codes, (delta if delta is not None else dout), ab, km
+
+
+def qm_quantize_formats(op, fmts, gran, want_kmaj=False, stream=None):
+    """Codes of several formats of one operand from one pass (qm_quantize_formats).
+    Returns ([codes per format], [delta per format], kmaj or None)."""
+    n = len(fmts)
+    ldc = qm_code_ld(op.contract)
+    codes = [torch.empty((op.batch, op.noncontract, ldc), dtype=torch.uint8, device="cuda") for _ in fmts]
+    deltas = [torch.empty(_n_delta(op, gran), dtype=torch.float32, device="cuda") for _ in fmts]
+    km = torch.empty((op.batch, op.noncontract, op.contract), dtype=torch.bfloat16, device="cuda") if want_kmaj else None
+    scratch = torch.empty(_n_delta(op, gran), dtype=torch.int32, device="cuda")
+    _check(lib().qm_quantize_formats(C.byref(op), n, (C.c_int32 * n)(*[FMT[f] for f in fmts]), GRAN[gran],
+                                     (C.c_void_p * n)(*[t.data_ptr() for t in deltas]),
+                                     (C.c_void_p * n)(*[t.data_ptr() for t in codes]), _ptr(km), _ptr(scratch),
+                                     _stream(stream)), "qm_quantize_formats")
+    return codes, deltas, km
 
 
 def qm_gemm(codes_l, fmt_l, delta_l, gran_l, codes_r, fmt_r, delta_r, gran_r, K, want_raw=False,
@@ -477,8 +496,9 @@ class HostProbeBatch:
         self.ws_bytes = (C.c_size_t * n)(*sizes)
         self.out_dev = torch.zeros(n * C.sizeof(MetricResult), dtype=torch.uint8, device="cuda")
         self._out_host = torch.zeros(n * C.sizeof(MetricResult), dtype=torch.uint8).pin_memory()
-        self.h2d_bytes = sum(t.numel() for t in self._ls) + sum(t.numel() for t in self._rs)
-        self.d2h_bytes = n * C.sizeof(MetricResult)
+        h2d, d2h = C.c_size_t(0), C.c_size_t(0)
+        _check(lib().qm_probe_batch_host_bytes(n, self.L, self.R, C.byref(h2d), C.byref(d2h)), "qm_probe_batch_host_bytes")
+        self.h2d_bytes, self.d2h_bytes = h2d.value, d2h.value      # what one run() copies
 
     def run(self, stream=None):
         out = C.cast(C.c_void_p(self._out_host.data_ptr()), C.POINTER(MetricResult))

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqm.so")
-SOURCES = ["qm_api.cu", "scale_quantize.cu", "tensor_stats.cu", "metric.cu", "gemm_simt.cu", "gemm_tc.cu", "derived.cu"]
+SOURCES = ["qm_api.cu", "scale_quantize.cu", "tensor_stats.cu", "metric.cu", "gemm_simt.cu", "gemm_tc.cu", "derived.cu", "calibrate.cu"]
 
 
 def _nvcc():

@@ -261,6 +261,30 @@ qm_status qm_quantize_stochastic(const qm_operand* x, int32_t fmt, int32_t gran,
   return quantize_entry(x, fmt, gran, &draw, delta, delta_out, codes, abs_copy, kmaj_copy, stream);
 }
 
+qm_status qm_quantize_formats(const qm_operand* x, int32_t n_fmt, const int32_t* fmts, int32_t gran,
+                              float* const* delta_out, uint8_t* const* codes, void* kmaj_copy,
+                              uint32_t* amax_scratch, void* stream) {
+  View v;
+  qm_status st = to_view(x, &v);
+  if (st != QM_OK) return st;
+  if (n_fmt < 1 || n_fmt > 3 || !fmts || !valid_gran(gran) || !delta_out || !codes || !amax_scratch) return QM_ERR_INVALID_ARG;
+  int f[3]; float* d[3]; uint8_t* c[3]; uint32_t* e[3] = {nullptr, nullptr, nullptr};
+  for (int k = 0; k < n_fmt; ++k) {
+    if (!valid_fmt(fmts[k]) || !delta_out[k] || !codes[k]) return QM_ERR_INVALID_ARG;
+    for (int j = 0; j < k; ++j)
+      if (fmts[j] == fmts[k]) return QM_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(codes[k]) & 15) return QM_ERR_ALIGNMENT;
+    f[k] = fmts[k]; d[k] = delta_out[k]; c[k] = codes[k];
+  }
+  if (reinterpret_cast<uintptr_t>(kmaj_copy) & 15) return QM_ERR_ALIGNMENT;
+  if (kmaj_copy && v.dtype != QM_DT_BF16) return QM_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  QM_CUDA_OK(cudaMemsetAsync(amax_scratch, 0, sizeof(uint32_t) * delta_count(v, gran), s));
+  st = launch_absmax(v, gran, amax_scratch, s);
+  if (st != QM_OK) return st;
+  return launch_quantize_multi(v, gran, amax_scratch, n_fmt, f, d, e, c, kmaj_copy, s);
+}
+
 qm_status qm_gemm(const uint8_t* codes_l, int32_t fmt_l, const float* delta_l, int32_t gran_l,
                   const uint8_t* codes_r, int32_t fmt_r, const float* delta_r, int32_t gran_r, int64_t M,
                   int64_t N, int64_t K, int64_t batch, float* out_descaled, void* out_raw, int32_t use_simt,
@@ -585,7 +609,6 @@ qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host
 // ---- batches of probes over the library's own streams ------------------------------------------
 namespace {
 constexpr int kBatchStreams = 8;      // streams of the pool
-constexpr int kHostBatchStreams = 3;  // of which the host-operand batches use this many
 struct BatchStreams {
   std::mutex issue;            // one batch at a time is put into the streams (host side only)
   bool ready = false;
@@ -673,27 +696,6 @@ void find_roots(std::vector<Slot>& slots, int t) {
   }
 }
 
-// Runs issue(i, stream_i) for i < n round-robin over the library's streams, between a fork from
-// and a join back into the caller's stream.  The join happens even when a probe was refused.
-template <typename F>
-qm_status run_batch(int32_t n, cudaStream_t user, F issue) {
-  if (n < 0) return QM_ERR_INVALID_ARG;
-  if (n == 0) return QM_OK;
-  BatchStreams* b = nullptr;
-  qm_status st = batch_streams(&b);
-  if (st != QM_OK) return st;
-  const int used = n < kHostBatchStreams ? n : kHostBatchStreams;
-  // the fork and join events are reused by every call: calls from several host threads take turns
-  std::lock_guard<std::mutex> lock(b->issue);
-  QM_CUDA_OK(cudaEventRecord(b->fork, user));
-  for (int j = 0; j < used; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
-  for (int32_t i = 0; i < n && st == QM_OK; ++i) st = issue(i, b->s[i % kHostBatchStreams]);
-  for (int j = 0; j < used; ++j) {
-    QM_CUDA_OK(cudaEventRecord(b->join[j], b->s[j]));
-    QM_CUDA_OK(cudaStreamWaitEvent(user, b->join[j], 0));
-  }
-  return st;
-}
 }  // namespace
 
 extern "C" {
@@ -754,7 +756,8 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
       x.delta = reinterpret_cast<float*>(base + (side ? pl.w.off_dr : pl.w.off_dl));
       x.codes = base + (side ? pl.w.off_cr : pl.w.off_cl);
       x.kmaj = v.c_contig() ? nullptr : base + (side ? pl.w.off_kr : pl.w.off_kl);
-      x.err = reinterpret_cast<uint32_t*>(base + pl.w.off_err);
+      // words 2 and 3 of the control block: "this operand is not finite", raised by the kernel that scales it
+      x.err = reinterpret_cast<uint32_t*>(base + pl.w.off_err) + 2 + side;
       x.keeps_amax = !(!x.stochastic && !grouped_scales(x) && x.gran == QM_GRAN_CHANNEL && v.c_contig());
       slots.push_back(x);
       find_roots(slots, (int)slots.size() - 1);
@@ -772,24 +775,55 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
   QM_CUDA_OK(cudaEventRecord(b->fork, user));
   for (int j = 0; j < kBatchStreams; ++j) QM_CUDA_OK(cudaStreamWaitEvent(b->s[j], b->fork, 0));
   int next_stream = 0;
+  std::vector<char> done(slots.size(), 0);
   for (size_t t = 0; t < slots.size(); ++t) {
     Slot& x = slots[t];
     if (x.code_root != (int)t) { x.stream = slots[x.code_root].stream; continue; }     // nothing to launch
-    cudaStream_t s;
-    qm_status e;
+    if (done[t]) continue;
+    qm_status e = QM_OK;
     const StochasticDraw* draw = x.stochastic ? &x.draw : nullptr;
     if (x.copy_root != (int)t) {
-      x.stream = slots[x.copy_root].stream; s = b->s[x.stream];
+      // borrows max|x| and the contraction-major copy, and was not served with its lender's formats
+      x.stream = slots[x.copy_root].stream;
       e = launch_quantize(x.v, x.fmt, x.gran, reinterpret_cast<const float*>(slots[x.amax_root].amax), true, x.delta, x.err,
-                          x.codes, nullptr, nullptr, s, draw);
-    } else if (x.amax_root != (int)t) {
-      x.stream = slots[x.amax_root].stream; s = b->s[x.stream];
-      e = launch_quantize(x.v, x.fmt, x.gran, reinterpret_cast<const float*>(slots[x.amax_root].amax), true, x.delta, x.err,
-                          x.codes, nullptr, x.kmaj, s, draw);
+                          x.codes, nullptr, nullptr, b->s[x.stream], draw);
+    } else if (!x.keeps_amax) {
+      x.stream = next_stream; next_stream = (next_stream + 1) % kBatchStreams;
+      e = prepare_operand(x.v, x.fmt, x.gran, x.amax, x.delta, x.codes, nullptr, x.kmaj, x.err, draw, x.groups, b->s[x.stream]);
     } else {
-      x.stream = next_stream; next_stream = (next_stream + 1) % kBatchStreams; s = b->s[x.stream];
-      e = prepare_operand(x.v, x.fmt, x.gran, x.amax, x.delta, x.codes, nullptr, x.kmaj, x.err, draw, x.groups, s);
+      if (x.amax_root == (int)t) {
+        x.stream = next_stream; next_stream = (next_stream + 1) % kBatchStreams;
+        e = launch_absmax(x.v, x.gran, x.amax, b->s[x.stream]);
+        if (e == QM_OK && grouped_scales(x)) e = launch_share_amax(x.amax, x.v.batch, x.groups, x.v.nc, b->s[x.stream]);
+      } else {
+        x.stream = slots[x.amax_root].stream;
+      }
+      cudaStream_t s = b->s[x.stream];
+      const uint32_t* amax = slots[x.amax_root].amax;
+      // this operand's format and those of the later operands that borrow its copy: one pass over
+      // the tensor writes all their codes (round-to-nearest-even ones; stochastic ones go singly)
+      int fmts[3]; float* deltas[3]; uint32_t* errs[3]; uint8_t* codes[3];
+      int nf = 0;
+      bool kmaj_written = false;
+      if (!x.stochastic) { fmts[nf] = x.fmt; deltas[nf] = x.delta; errs[nf] = x.err; codes[nf] = x.codes; ++nf; }
+      for (size_t u = t + 1; u < slots.size() && nf < 3; ++u) {
+        Slot& y = slots[u];
+        if (y.code_root != (int)u || y.copy_root != (int)t || y.stochastic || done[u]) continue;
+        bool dup = false;
+        for (int k = 0; k < nf; ++k) dup |= fmts[k] == y.fmt;
+        if (dup) continue;
+        fmts[nf] = y.fmt; deltas[nf] = y.delta; errs[nf] = y.err; codes[nf] = y.codes; ++nf;
+        y.stream = x.stream; done[u] = 1;
+      }
+      if (e == QM_OK && x.stochastic) {
+        e = launch_quantize(x.v, x.fmt, x.gran, reinterpret_cast<const float*>(amax), true, x.delta, x.err, x.codes, nullptr,
+                            x.kmaj, s, draw);
+        kmaj_written = true;
+      }
+      if (e == QM_OK && nf > 0)
+        e = launch_quantize_multi(x.v, x.gran, amax, nf, fmts, deltas, errs, codes, kmaj_written ? nullptr : x.kmaj, s);
     }
+    done[t] = 1;
     if (e != QM_OK && st == QM_OK) st = e;
   }
   for (int32_t i = 0; i < good; ++i) {
@@ -830,11 +864,11 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
     p.dl = cl.delta; p.gran_l = cfg[i].gran_l; p.dr = cr.delta; p.gran_r = cfg[i].gran_r;
     p.g = GemmShape{pl.Lv.nc, pl.Rv.nc, pl.Lv.c, pl.Lv.batch};
     p.partials = reinterpret_cast<double*>(base + pl.w.off_part);
-    p.err_word = xl.err;
-    p.done_counter = xl.err + 1;            // second word of the cleared error slot
-    // a non-finite operand is flagged in the error word of the probe whose kernel made the codes
-    p.err_also[0] = cl.err != xl.err ? cl.err : nullptr;
-    p.err_also[1] = cr.err != xl.err ? cr.err : nullptr;
+    p.err_word = reinterpret_cast<uint32_t*>(base + pl.w.off_err);
+    p.done_counter = p.err_word + 1;        // second word of the cleared control block
+    // a non-finite operand is flagged in the control block of the probe whose kernel scaled it
+    p.err_also[0] = cl.err;
+    p.err_also[1] = cr.err;
     p.result = out + i;
     p.row_stats = cfg[i].row_stats;
     args.push_back(p);
@@ -848,23 +882,76 @@ qm_status qm_probe_batch(int32_t n, const qm_operand* L, const qm_operand* R, co
   return st != QM_OK ? st : refused;
 }
 
+// Which host operands of a host batch are copied: an operand whose host bytes an earlier operand of
+// the batch has already brought to the device (same address, same extent) uses that copy.
+namespace {
+struct HostCopy { const void* host; size_t bytes; void* dev; };
+void* find_copy(const std::vector<HostCopy>& seen, const void* host, size_t bytes) {
+  for (const HostCopy& c : seen)
+    if (c.host == host && c.bytes == bytes) return c.dev;
+  return nullptr;
+}
+}  // namespace
+
+qm_status qm_probe_batch_host_bytes(int32_t n, const qm_operand* L_host, const qm_operand* R_host, size_t* h2d_bytes,
+                                    size_t* d2h_bytes) {
+  if (n < 0 || (n > 0 && (!L_host || !R_host)) || !h2d_bytes || !d2h_bytes) return QM_ERR_INVALID_ARG;
+  std::vector<HostCopy> seen;
+  size_t total = 0;
+  for (int32_t i = 0; i < n; ++i)
+    for (int side = 0; side < 2; ++side) {
+      const qm_operand& x = side ? R_host[i] : L_host[i];
+      const size_t bytes = qm_operand_span_bytes(&x);
+      if (bytes == 0) return QM_ERR_INVALID_ARG;
+      if (find_copy(seen, x.data, bytes)) continue;
+      seen.push_back(HostCopy{x.data, bytes, const_cast<void*>(x.data)});
+      total += bytes;
+    }
+  *h2d_bytes = total;
+  *d2h_bytes = sizeof(qm_metric_result) * (size_t)n;
+  return QM_OK;
+}
+
 qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_operand* R_host,
                               const qm_probe_cfg* cfg, void* const* l_stage, void* const* r_stage,
                               qm_metric_result* out_host, qm_metric_result* out_dev, void* const* ws,
                               const size_t* ws_bytes, void* stream) {
   if (n > 0 && (!L_host || !R_host || !cfg || !l_stage || !r_stage || !out_host || !out_dev || !ws || !ws_bytes))
     return QM_ERR_INVALID_ARG;
+  if (n < 0) return QM_ERR_INVALID_ARG;
   if (n == 0) return QM_OK;
   cudaStream_t user = static_cast<cudaStream_t>(stream);
-  int32_t issued = 0;
-  qm_status st = run_batch(n, user, [&](int32_t i, cudaStream_t s) {
-    qm_status e = enqueue_host_probe(&L_host[i], &R_host[i], &cfg[i], l_stage[i], r_stage[i], out_host + i,
-                                     out_dev + i, ws[i], ws_bytes[i], s);
-    if (e == QM_OK) ++issued;
-    return e;
-  });
+  // every distinct host operand is copied once; the probes then run as a device batch, which in
+  // turn prepares every distinct operand once
+  std::vector<qm_operand> Ld((size_t)n), Rd((size_t)n);
+  std::vector<HostCopy> seen;
+  qm_status refused = QM_OK;
+  int32_t good = 0;
+  for (; good < n; ++good) {
+    for (int side = 0; side < 2 && refused == QM_OK; ++side) {
+      const qm_operand& x = side ? R_host[good] : L_host[good];
+      void* stage = side ? r_stage[good] : l_stage[good];
+      const size_t bytes = qm_operand_span_bytes(&x);
+      if (bytes == 0 || !stage) { refused = QM_ERR_INVALID_ARG; break; }
+      void* dev = find_copy(seen, x.data, bytes);
+      if (!dev) {
+        QM_CUDA_OK(cudaMemcpyAsync(stage, x.data, bytes, cudaMemcpyHostToDevice, user));
+        seen.push_back(HostCopy{x.data, bytes, stage});
+        dev = stage;
+      }
+      qm_operand& d = side ? Rd[good] : Ld[good];
+      d = x;
+      d.data = dev;
+    }
+    if (refused != QM_OK) break;
+  }
+  qm_status st = qm_probe_batch(good, Ld.data(), Rd.data(), cfg, out_dev, ws, ws_bytes, user);
+  int32_t issued = st == QM_OK ? good : 0;
+  if (issued > 0)
+    QM_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, sizeof(qm_metric_result) * (size_t)issued, cudaMemcpyDeviceToHost, user));
   QM_CUDA_OK(cudaStreamSynchronize(user));
   if (st != QM_OK) return st;
+  if (refused != QM_OK) return refused;
   for (int32_t i = 0; i < issued; ++i) {
     st = host_record_status(out_host + i);
     if (st != QM_OK) return st;

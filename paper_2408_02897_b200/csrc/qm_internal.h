@@ -86,6 +86,14 @@ struct StochasticDraw { uint64_t seed; uint32_t stream; };
 qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, bool from_amax,
                           float* delta_out, uint32_t* err_word, uint8_t* codes, void* abs_copy,
                           void* kmaj_copy, cudaStream_t s, const StochasticDraw* draw = nullptr);
+// The codes of nf (1..3) distinct formats of one operand from the max|x| bit patterns of
+// launch_absmax, round-to-nearest-even; per format k its scales go to delta_out[k], its codes to
+// codes[k] and a non-finite maximum is flagged in err_word[k] (optional).  Per-tensor scales of a
+// bf16 operand are served by one kernel that reads the operand once; everything else by one
+// launch per format.  kmaj_copy as in launch_quantize.
+qm_status launch_quantize_multi(const View& x, int gran, const uint32_t* amax, int nf, const int* fmts,
+                                float* const* delta_out, uint32_t* const* err_word, uint8_t* const* codes,
+                                void* kmaj_copy, cudaStream_t s);
 // Single pass per row: absmax, delta, codes (contiguous contraction, per-channel).
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,
                                      void* abs_copy, uint32_t* err_word, cudaStream_t s);

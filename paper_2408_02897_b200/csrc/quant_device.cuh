@@ -109,6 +109,60 @@ struct Quotient {
   }
 };
 
+// The same correctly rounded quotient for two elements at once with the two-wide fp32
+// instructions (one mul and four fma for a pair), for scales taken from the operand's own max|x|:
+// |x / delta| then never exceeds the format's largest value by more than a rounding, so nothing
+// overflows and the guard of Quotient is not needed.  Only the fast range of delta is served;
+// callers fall back to Quotient otherwise.
+struct QuotientPair {
+  uint64_t recip2, ndelta2;
+  __device__ __forceinline__ explicit QuotientPair(float d) {
+    const float r = __frcp_rn(d), nd = -d;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(recip2) : "f"(r));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(ndelta2) : "f"(nd));
+  }
+  static __device__ __forceinline__ bool serves(float d) { return d >= 8.6736174e-19f && d <= 1.1529215e18f; }
+  // x2 = {x0, x1} packed; returns {RN(x0 / delta), RN(x1 / delta)} packed (a zero comes out as +0)
+  __device__ __forceinline__ uint64_t operator()(uint64_t x2) const {
+    uint64_t q0, t, q1, q;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(q0) : "l"(x2), "l"(recip2));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t) : "l"(q0), "l"(ndelta2), "l"(x2));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q1) : "l"(t), "l"(recip2), "l"(q0));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t) : "l"(q1), "l"(ndelta2), "l"(x2));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(q) : "l"(t), "l"(recip2), "l"(q1));
+    return q;
+  }
+};
+
+// Two codes (bits 0..7 and 8..15) of the bf16 pair held in word w (low half = first element).
+template <int FMT>
+__device__ __forceinline__ uint32_t quant_bf16_pair(uint32_t w, const QuotientPair& quot) {
+  uint64_t x2;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(x2) : "r"(w << 16), "r"(w & 0xffff0000u));
+  const uint64_t q2 = quot(x2);
+  uint32_t q0, q1;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(q0), "=r"(q1) : "l"(q2));
+  if (FMT == QM_FMT_INT8) {
+    return quant2<FMT>(__uint_as_float(q0), __uint_as_float(q1));
+  } else {
+    // a negative input that rounds to zero is -0 in the FP8 formats: give the quotient its sign back
+    q0 |= (w << 16) & 0x80000000u;
+    q1 |= w & 0x80000000u;
+    return quant2<FMT>(__uint_as_float(q0), __uint_as_float(q1));
+  }
+}
+
+// Sixteen codes of sixteen consecutive bf16 values (two 128-bit words).
+template <int FMT>
+__device__ __forceinline__ uint4 quant_bf16x16(const uint4& a, const uint4& b, const QuotientPair& quot) {
+  uint4 r;
+  r.x = quant_bf16_pair<FMT>(a.x, quot) | (quant_bf16_pair<FMT>(a.y, quot) << 16);
+  r.y = quant_bf16_pair<FMT>(a.z, quot) | (quant_bf16_pair<FMT>(a.w, quot) << 16);
+  r.z = quant_bf16_pair<FMT>(b.x, quot) | (quant_bf16_pair<FMT>(b.y, quot) << 16);
+  r.w = quant_bf16_pair<FMT>(b.z, quot) | (quant_bf16_pair<FMT>(b.w, quot) << 16);
+  return r;
+}
+
 template <int FMT>
 __device__ __forceinline__ uint2 quant8(const Vec8& x, const Quotient& quot) {
   float t[8];

@@ -290,6 +290,151 @@ quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const 
   }
 }
 
+// ---------------------------------------------------------------- several formats in one pass
+// A sweep of formats quantizes the same tensor two or three times (Table 1).  These kernels read
+// it once and write the codes of every format in MASK (bit f = qm_format f), with per-tensor
+// scales taken from the tensor's max|x| bit pattern: delta_f = max|x| / qmax_f.  Thread 0 of
+// block 0 stores the scales and raises the non-finite flag for each format's probe.
+struct MultiOut {
+  uint8_t* codes[3];      // indexed by qm_format; null where MASK has no bit
+  float* delta_out[3];
+  uint32_t* err_word[3];
+};
+
+template <int MASK>
+__device__ __forceinline__ void multi_scales(const uint32_t* amax, const MultiOut& o, bool writer, float (&d)[3]) {
+  const uint32_t bits = __ldg(amax);
+#pragma unroll
+  for (int f = 0; f < 3; ++f) {
+    if (!(MASK & (1 << f))) { d[f] = 1.f; continue; }
+    d[f] = bits == 0 ? 1.0f : __fdiv_rn(__uint_as_float(bits), fmt_qmax(f));
+    if (writer) {
+      o.delta_out[f][0] = d[f];
+      if (bits >= 0x7f800000u && o.err_word[f]) atomicOr(o.err_word[f], QM_DEVERR_NONFINITE);
+    }
+  }
+}
+
+// Dense bf16 tensor, rows a multiple of 16 long: one flat run of 16-element chunks.
+template <int MASK, int CHUNKS>
+__global__ void __launch_bounds__(kThreads)
+quantize_dense_multi_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const uint32_t* __restrict__ amax,
+                            const MultiOut o) {
+  pdl_prologue();
+  const uint32_t base = blockIdx.x * (kThreads * CHUNKS) + threadIdx.x;
+  uint4 w[CHUNKS][2];
+#pragma unroll
+  for (int u = 0; u < CHUNKS; ++u) {
+    const uint32_t i = base + u * kThreads;
+    const uint32_t j = i < total_chunks ? i : total_chunks - 1;     // clamp: results of dead lanes are dropped
+    w[u][0] = __ldg(x + 2 * (size_t)j);
+    w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+  }
+  float d[3];
+  multi_scales<MASK>(amax, o, blockIdx.x == 0 && threadIdx.x == 0, d);
+  const bool pair_ok = QuotientPair::serves(d[0]) && QuotientPair::serves(d[1]) && QuotientPair::serves(d[2]);
+#pragma unroll
+  for (int f = 0; f < 3; ++f) {
+    if (!(MASK & (1 << f))) continue;
+    uint4* codes = reinterpret_cast<uint4*>(o.codes[f]);
+    if (pair_ok) {
+      const QuotientPair quot(d[f]);
+#pragma unroll
+      for (int u = 0; u < CHUNKS; ++u) {
+        const uint32_t i = base + u * kThreads;
+        if (i < total_chunks) {
+          codes[i] = f == 0   ? quant_bf16x16<0>(w[u][0], w[u][1], quot)
+                     : f == 1 ? quant_bf16x16<1>(w[u][0], w[u][1], quot)
+                              : quant_bf16x16<2>(w[u][0], w[u][1], quot);
+        }
+      }
+    } else {
+      const Quotient quot(d[f]);
+#pragma unroll 1
+      for (int u = 0; u < CHUNKS; ++u) {
+        const uint32_t i = base + u * kThreads;
+        if (i >= total_chunks) break;
+        uint4 out;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint4 v = w[u][h];
+          Vec8 t;
+          t.v[0] = bf16_lo(v.x); t.v[1] = bf16_hi(v.x); t.v[2] = bf16_lo(v.y); t.v[3] = bf16_hi(v.y);
+          t.v[4] = bf16_lo(v.z); t.v[5] = bf16_hi(v.z); t.v[6] = bf16_lo(v.w); t.v[7] = bf16_hi(v.w);
+          const uint2 q = f == 0 ? quant8<0>(t, quot) : f == 1 ? quant8<1>(t, quot) : quant8<2>(t, quot);
+          if (h == 0) { out.x = q.x; out.y = q.y; } else { out.z = q.x; out.w = q.y; }
+        }
+        codes[i] = out;
+      }
+    }
+  }
+}
+
+// Strided contraction, bf16: the layout of quantize_transpose_bf16_kernel (a thread owns two
+// adjacent columns and 32 consecutive contraction rows), codes of every format in MASK and the
+// contraction-major copy from one read.
+template <int MASK>
+__global__ void __launch_bounds__(kThreads)
+quantize_transpose_bf16_multi_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
+                                     int64_t s_b, const uint32_t* __restrict__ amax, const MultiOut o, int64_t ldc,
+                                     __nv_bfloat16* __restrict__ kmaj_copy) {
+  pdl_prologue();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t b = blockIdx.z;
+  const int64_t n = ((int64_t)blockIdx.x * 32 + lane) * 2;
+  const int64_t k0 = ((int64_t)blockIdx.y * 8 + warp) * 32;
+  float d[3];
+  multi_scales<MASK>(amax, o, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0, d);
+  if (n >= nc || k0 >= c) return;
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(x + b * s_b + k0 * s_c + n);
+  const int64_t step = s_c >> 1;
+  uint32_t w[32];
+#pragma unroll
+  for (int r = 0; r < 32; ++r) w[r] = __ldg(src + r * step);
+  const bool pair_ok = QuotientPair::serves(d[0]) && QuotientPair::serves(d[1]) && QuotientPair::serves(d[2]);
+#pragma unroll
+  for (int col = 0; col < 2; ++col) {
+    const int64_t orow = b * nc + n + col;
+    // this column's 32 values as 16 words of two bf16 each
+    uint32_t pw[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      pw[j] = col == 0 ? __byte_perm(w[2 * j], w[2 * j + 1], 0x5410) : __byte_perm(w[2 * j], w[2 * j + 1], 0x7632);
+    if (kmaj_copy) {
+      uint4* dst = reinterpret_cast<uint4*>(kmaj_copy + orow * c + k0);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dst[j] = make_uint4(pw[4 * j], pw[4 * j + 1], pw[4 * j + 2], pw[4 * j + 3]);
+    }
+#pragma unroll
+    for (int f = 0; f < 3; ++f) {
+      if (!(MASK & (1 << f))) continue;
+      uint4* cdst = reinterpret_cast<uint4*>(o.codes[f] + orow * ldc + k0);
+      if (pair_ok) {
+        const QuotientPair quot(d[f]);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const uint4 a = make_uint4(pw[8 * h], pw[8 * h + 1], pw[8 * h + 2], pw[8 * h + 3]);
+          const uint4 bb = make_uint4(pw[8 * h + 4], pw[8 * h + 5], pw[8 * h + 6], pw[8 * h + 7]);
+          cdst[h] = f == 0 ? quant_bf16x16<0>(a, bb, quot) : f == 1 ? quant_bf16x16<1>(a, bb, quot) : quant_bf16x16<2>(a, bb, quot);
+        }
+      } else {
+        const Quotient quot(d[f]);
+        uint32_t cw[8];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          Vec8 t;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { t.v[2 * j] = bf16_lo(pw[4 * g + j]); t.v[2 * j + 1] = bf16_hi(pw[4 * g + j]); }
+          const uint2 q = f == 0 ? quant8<0>(t, quot) : f == 1 ? quant8<1>(t, quot) : quant8<2>(t, quot);
+          cw[2 * g] = q.x; cw[2 * g + 1] = q.y;
+        }
+        cdst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+        cdst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------- fused per-row scale + quantize
 // G lanes own one row: pass 1 reduces max|x| over the row, pass 2 re-reads it (from L1/L2: the
 // same lanes touched it a moment ago) and writes codes.  HBM sees each element once.
@@ -559,10 +704,21 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
     }
   } else {
     if (gran == QM_GRAN_TENSOR) {
-      // storage rows are the contracting index: walk them as rows of nc contiguous elements
-      for (int64_t b = 0; b < x.batch; ++b)
-        launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.c / 8 + 1, 8)), dim3(kThreads), 0, s, 
-            p + b * x.s_b, x.c, x.nc, x.s_c, amax);
+      // storage rows are the contracting index: walk them as rows of nc contiguous elements; the
+      // rows of all batch elements form one run when the batch stride continues the row stride
+      if (x.batch == 1 || x.s_b == x.c * x.s_c) {
+        const bool dense = x.s_c == x.nc;
+        const int64_t n = x.nc * x.c * x.batch;
+        if (dense)
+          launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s, p, 1, n, n, amax);
+        else
+          launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s,
+              p, x.c * x.batch, x.nc, x.s_c, amax);
+      } else {
+        for (int64_t b = 0; b < x.batch; ++b)
+          launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.c / 8 + 1, 8)), dim3(kThreads), 0, s,
+              p + b * x.s_b, x.c, x.nc, x.s_c, amax);
+      }
     } else {
       const int64_t col_blocks = (x.nc + 255) / 256;
       int64_t want_y = ((int64_t)sm_count() * 8 + col_blocks * x.batch - 1) / (col_blocks * x.batch);
@@ -717,6 +873,72 @@ qm_status launch_quantize(const View& x, int fmt, int gran, const float* delta, 
   return x.dtype == QM_DT_BF16 ? QM_Q(__nv_bfloat16) : QM_Q(float);
 #undef QM_Q
 #undef QM_ARGS
+}
+
+qm_status launch_quantize_multi(const View& x, int gran, const uint32_t* amax, int nf, const int* fmts,
+                                float* const* delta_out, uint32_t* const* err_word, uint8_t* const* codes,
+                                void* kmaj_copy, cudaStream_t s) {
+  if (nf < 1 || nf > 3) return QM_ERR_INVALID_ARG;
+  const int64_t ldc = qm_code_ld(x.c);
+  int mask = 0;
+  MultiOut o{};
+  for (int k = 0; k < nf; ++k) {
+    const int f = fmts[k];
+    if (f < 0 || f > 2 || (mask & (1 << f))) return QM_ERR_INVALID_ARG;
+    mask |= 1 << f;
+    o.codes[f] = codes[k]; o.delta_out[f] = delta_out[k]; o.err_word[f] = err_word[k];
+  }
+  bool one_pass = nf > 1 && gran == QM_GRAN_TENSOR && x.dtype == QM_DT_BF16;
+  const int64_t total = x.nc * x.batch * (ldc >> 4);
+  bool dense = false, transposing = false;
+  if (one_pass && x.c_contig()) {
+    dense = x.s_nc == x.c && (x.c & 15) == 0 && (x.batch == 1 || x.s_b == x.nc * x.c) && total < (1ll << 32);
+    one_pass = dense && !kmaj_copy;
+  } else if (one_pass) {
+    transposing = (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
+                  ((x.nc + 63) / 64) * ((x.c + 255) / 256) * x.batch >= 4 * (int64_t)sm_count();
+    one_pass = transposing;
+  }
+  if (!one_pass) {
+    // one launch per format; the first one also writes the contraction-major copy
+    for (int k = 0; k < nf; ++k) {
+      const qm_status st = launch_quantize(x, fmts[k], gran, reinterpret_cast<const float*>(amax), true, delta_out[k],
+                                           err_word[k], codes[k], nullptr, k == 0 ? kmaj_copy : nullptr, s);
+      if (st != QM_OK) return st;
+    }
+    return QM_OK;
+  }
+  if (dense) {
+    const uint4* src = reinterpret_cast<const uint4*>(x.data);
+    const bool big = total >= (int64_t)sm_count() * 8 * kThreads * 4;
+    const int64_t per_block = (int64_t)kThreads * (big ? 4 : 1);
+    const dim3 grid((unsigned)((total + per_block - 1) / per_block));
+#define QM_DM(M)                                                                                                   \
+  (big ? launch_pdl(quantize_dense_multi_kernel<M, 4>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o) \
+       : launch_pdl(quantize_dense_multi_kernel<M, 1>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o))
+    switch (mask) {
+      case 3: QM_DM(3); break;
+      case 5: QM_DM(5); break;
+      case 6: QM_DM(6); break;
+      default: QM_DM(7); break;
+    }
+#undef QM_DM
+  } else {
+    dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
+    const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(x.data);
+    __nv_bfloat16* km = static_cast<__nv_bfloat16*>(kmaj_copy);
+#define QM_TM(M) launch_pdl(quantize_transpose_bf16_multi_kernel<M>, grid, dim3(kThreads), 0, s, src, x.nc, x.c, x.s_c, x.s_b, amax, o, ldc, km)
+    switch (mask) {
+      case 3: QM_TM(3); break;
+      case 5: QM_TM(5); break;
+      case 6: QM_TM(6); break;
+      default: QM_TM(7); break;
+    }
+#undef QM_TM
+  }
+  count_launch();
+  QM_CUDA_OK(cudaGetLastError());
+  return QM_OK;
 }
 
 qm_status launch_scale_quantize_rows(const View& x, int fmt, float* delta_out, uint8_t* codes,

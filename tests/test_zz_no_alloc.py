@@ -1,4 +1,4 @@
-"""The allocation-free variant of the Eq. 3 reduction against the regular one.
+"""The allocation-free variant of the Eq. 3 reduction against the regular one and the oracle.
 
 qm_metric_noalloc exists for callers that cannot call cudaMalloc (plug-ins that only get
 input/output pointers, code confined to someone else's memory pool, allocator-free loops):
@@ -13,6 +13,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2408_02897_b200 as qm
 from paper_2408_02897_b200 import binding
 
@@ -38,6 +39,12 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
         for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
             assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k]), (k, got[k], want[k])
         assert abs(got["max_be"] - want["max_be"]) <= 1e-6 * want["max_be"]
+        # and against the definition itself (fp64 on the same arrays; the kernel divides in fp32)
+        ref = oracle.metric(c.cpu().numpy(), q.cpu().numpy(), d.cpu().numpy())
+        assert got["count"] == ref["count"]
+        for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
+            assert abs(got[k] - ref[k]) <= 1e-5 * abs(ref[k]), (k, got[k], ref[k])
+        assert abs(got["max_be"] - ref["max_be"]) <= 1e-5 * ref["max_be"]
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
