@@ -49,7 +49,6 @@ constexpr uint32_t kALp = kBlockM * kBlockK;                      //  8 KB,  64-
 constexpr uint32_t kBBf16 = kHalfN * kBlockK * 2;                 //  8 KB
 constexpr uint32_t kBLp = kHalfN * kBlockK;                       //  4 KB
 constexpr int kMaxStages = 8;
-constexpr int kRefAhead = 2;               // k-blocks of reference MMAs issued before the hand-back wait
 
 enum Mode { kLpOnly = 1, kRefOnly = 2, kProbe2 = 3 };
 
@@ -1008,53 +1007,65 @@ tc_gemm_wide_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 // pair's positions increase, so it meets each probe in one run: when the probe changes, the
 // epilogue warps reduce their statistics and write the CTA's record of the probe they leave.
 //
-// Roles in each CTA (384 threads):
-//   warp 0       TMA producer: per 64-deep k-block the bf16 tiles of L and R and both code tiles
-//                (36 KB per CTA) into a ring of kTmaStages stages; a CTA's loads complete on its
-//                own `full` barrier.
-//   warps 2, 3   converters: the denominator product of Eq. 3 multiplies |L| by |R|.  Its operand
-//                tiles are not loaded: once a stage has landed these warps copy its L and R tiles
-//                with the sign bits cleared (the swizzled layout is elementwise-transparent) into
-//                a second ring of kAbsStages stages (24 KB per CTA), make the copies visible to
-//                the tensor core's reads (fence.proxy.async) and arrive on the leader's `ready`
-//                barrier.  The tensor cores are bound by the bytes an SM pulls from L2 per flop;
-//                this takes 24 of 60 KB per k-block off that path, and no |x| copy exists in HBM.
-//   warp 1       allocates tensor memory; in the leader CTA it runs the MMA loop converged and one
-//                elected lane issues the pair's MMAs once `ready` says that both CTAs' tiles and
-//                their sign-cleared copies are in place; tcgen05.commit frees the stage in both
-//                CTAs (`empty`), which the producer (TMA ring) and the converters (|x| ring) await.
-//   warps 4..11  epilogue (see below).
-// Three accumulators live side by side in tensor memory: the reference L.R (bf16, kind::f16), the
-// denominator |L|.|R| (bf16, kind::f16) and the 8-bit product (kind::f8f6f4 or kind::i8), 128
-// columns each, rotating from tile to tile through the four 128-column blocks so that the next
-// tile's MMAs overlap this tile's epilogue; no M x N matrix ever goes to HBM.
+// What bounds this kernel is shared-memory bandwidth: per 64-deep k-block the tensor cores need
+// 640 cycles, and with all six operand tiles (L, |L|, codes, R, |R|, codes) staged in shared
+// memory an SM writes 60 KB and reads 60 KB per k-block, which takes it 940.  So the left operand
+// of the denominator product |L|.|R| is not staged in shared memory: converter warps read this
+// CTA's 128 rows of the L tile, clear the sign bits and store the result into TENSOR memory, from
+// where the denominator MMAs take their A operand; the same warps write the |R| half-tile into
+// the stage.  No |x| copy exists in HBM, TMA brings 36 KB per k-block, the MMAs read 44 KB and the
+// converters move 32 KB.
+//
+// Roles in each CTA (512 threads = 4 warpgroups; registers are re-divided with setmaxnreg):
+//   warp 0        TMA producer: per k-block the bf16 tiles of L and R and both code tiles into a
+//                 ring of kStages stages; a CTA's loads complete on its own `full` barrier.
+//   warp 1        allocates tensor memory; in the leader CTA it runs the MMA loop converged and
+//                 one elected lane issues the pair's MMAs; tcgen05.commit frees a stage (shared
+//                 and tensor memory) in both CTAs (`empty`).
+//   warps 2, 3    idle (they fill the first warpgroup).
+//   warps 4..7    converters, one per tensor-memory lane quarter: thread = one of the CTA's 128
+//                 left-operand rows.
+//   warps 8..15   epilogue.
+// Tensor memory: columns 0..127 reference L.R, 128..255 denominator |L|.|R|, 256..383 the 8-bit
+// product, 384..511 four stages of |L| (32 columns of two bf16 each per stage; the shared-memory
+// ring has five stages, so TMA runs a k-block further ahead than the converters can).  The epilogue
+// copies its reference and denominator columns into registers and hands those two blocks back
+// at once (`tmem_empty`), after which the MMA warp issues the next tile's reference and
+// denominator MMAs for as many k-blocks as there are stages; the 8-bit MMAs of those k-blocks
+// follow when the epilogue has finished the 8-bit block (`lp_done`).  No M x N matrix ever goes
+// to HBM.
 constexpr int kMaxGroup = 16;
-constexpr int kConvWarps = 2;
-constexpr int kProbeThreads = 32 * (2 + kConvWarps + kEpiWarps);    // 384
-constexpr int kFirstEpiWarp = 2 + kConvWarps;                       // 4: lane quarter = warp % 4 still holds
+constexpr int kProbeThreads = 512;
+constexpr int kFirstEpiWarp = 8;               // warps 8..15: lane quarter = warp % 4 holds for both groups
+// registers per thread after the split (launch: 128 each): 56 + 104 + 176 + 176 = 4 x 128
+constexpr int kRegsCtl = 56, kRegsConv = 104, kRegsEpi = 176;
+static_assert(kRegsCtl + kRegsConv + 2 * kRegsEpi <= 4 * 128, "the split must fit what the block was launched with");
 
 struct CfgP {
-  static constexpr int kTmaStages = 4, kAbsStages = 3;
-  // TMA stage: L, R (contiguous, so that the converters copy one flat 24 KB run), codes of L, codes of R
-  static constexpr uint32_t kOffL = 0, kOffR = kABf16, kOffCl = kABf16 + kBBf16, kOffCr = kOffCl + kALp;
-  static constexpr uint32_t kTmaStageBytes = kOffCr + kBLp;          // 36 KB
-  static constexpr uint32_t kOffLa = 0, kOffRa = kABf16;
-  static constexpr uint32_t kAbsStageBytes = kABf16 + kBBf16;        // 24 KB
-  static constexpr uint32_t kTileBytes = kTmaStages * kTmaStageBytes + kAbsStages * kAbsStageBytes;   // 216 KB
+  static constexpr int kStages = 5;          // stages of shared memory (TMA ring)
+  static constexpr int kAbsStages = 4;       // stages of |L| in tensor memory (128 columns / 32)
+  // stage: L, R, |R| (written by the converters), codes of L, codes of R
+  static constexpr uint32_t kOffL = 0, kOffR = kABf16, kOffRa = kOffR + kBBf16, kOffCl = kOffRa + kBBf16;
+  static constexpr uint32_t kOffCr = kOffCl + kALp;
+  static constexpr uint32_t kStageBytes = kOffCr + kBLp;             // 44 KB
+  static constexpr uint32_t kTmaBytes = kABf16 + kBBf16 + kALp + kBLp;   // 36 KB per CTA and k-block
+  static constexpr uint32_t kTileBytes = kStages * kStageBytes;      // 220 KB
+  static constexpr uint32_t kColRef = 0, kColDen = 128, kColLp = 256, kColAbsL = 384;   // tensor-memory columns
 };
 
 struct SharedP {
-  uint64_t full[CfgP::kTmaStages];    // per CTA: this CTA's loads of a stage have landed
-  uint64_t empty[CfgP::kTmaStages];   // per CTA: the pair's MMAs have finished reading the k-block of the stage
-  uint64_t ready[CfgP::kAbsStages];   // leader: both CTAs' converters have finished a k-block
-  uint64_t tmem_full;                 // per CTA: the tile's accumulators are complete
-  uint64_t tmem_empty;                // leader: both CTAs' epilogues have copied out reference and denominator
-  uint64_t lp_done;                   // leader: both CTAs' epilogues have finished a tile
-  uint64_t drain;                     // leader, give-up path only: every MMA issued so far has completed
+  uint64_t full[CfgP::kStages];     // per CTA: this CTA's loads of a stage have landed
+  uint64_t ready[CfgP::kAbsStages]; // leader: both CTAs' converters have seen their loads land and have written
+                                    //         |L| (tensor memory) and |R| (stage)
+  uint64_t empty[CfgP::kStages];    // per CTA: the pair's MMAs have finished with the k-block of the stage
+  uint64_t tmem_full;               // per CTA: the tile's accumulators are complete
+  uint64_t tmem_empty;              // leader: both CTAs' epilogues have copied out reference and denominator
+  uint64_t lp_done;                 // leader: both CTAs' epilogues have finished a tile
+  uint64_t drain;                   // leader, give-up path only: every MMA issued so far has completed
   uint32_t tmem_base;
   uint32_t abort_flag;
   uint32_t is_last;
-  uint32_t issued;                    // k-blocks whose loads the producer has issued (read on the give-up path)
+  uint32_t issued;                  // k-blocks whose loads the producer has issued (read on the give-up path)
   float delta_r[2][kBlockN];
   double red[5][kEpiWarps];
 };
@@ -1085,6 +1096,39 @@ __device__ __forceinline__ int group_find(const GroupTable& tab, int pos) {
   while (pi + 1 < tab.n && pos >= tab.p[pi + 1].tile_begin) ++pi;
   return pi;
 }
+
+// The tiles of one CTA pair in order, k-block by k-block: every role walks the same sequence.
+struct TileWalk {
+  int r, pair, num_pairs;
+  int pi, num_kb, kb;
+  TileCoord tc;
+  bool valid;
+  __device__ __forceinline__ void start(const GroupTable& tab, int pair_, int num_pairs_) {
+    r = -1; pair = pair_; num_pairs = num_pairs_; kb = 0; num_kb = 0; valid = true;
+    next_tile(tab);
+  }
+  // moves to the pair's next tile; valid = false when there is none
+  __device__ __forceinline__ void next_tile(const GroupTable& tab) {
+    while (true) {
+      ++r;
+      const int pos = group_position(r, pair, num_pairs);
+      if (pos >= tab.total_tiles) {
+        if (r * num_pairs >= tab.total_tiles) { valid = false; return; }   // no round reaches further
+        continue;
+      }
+      pi = group_find(tab, pos);
+      const GroupProblem& pr = tab.p[pi];
+      tc = tile_coord(pos - pr.tile_begin, pr.a);
+      num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+      kb = 0;
+      return;
+    }
+  }
+  // moves to the next k-block of the sequence
+  __device__ __forceinline__ void next_kb(const GroupTable& tab) {
+    if (++kb >= num_kb) next_tile(tab);
+  }
+};
 
 // Bounded wait with the launch's limit; see mbar_wait.
 struct Waiter {
@@ -1121,88 +1165,48 @@ __device__ __forceinline__ void tma_load_3d_local(uint32_t dst, const CUtensorMa
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns of tensor memory from registers: lane (base + t) <- thread t.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+// D[256 x N] (+)= A[256 x 16] . B[N x 16]^T across the CTA pair, A (bf16) taken from tensor memory:
+// each CTA's 128 rows at the same column address, two values per 32-bit column.
+__device__ __forceinline__ void mma_pair_a_tmem(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc,
+                                                uint32_t accumulate, bool lead) {
+  if (!lead) return;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
-  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-// The MMAs of one tile (leader CTA, converged warp); g counts k-blocks, `it` tiles of this pair.
-// Returns false when a wait gave up.
-template <int LPK>
-__device__ __forceinline__ bool group_mma_tile(SharedP* sh, uint32_t tma_tiles, uint32_t abs_tiles, uint32_t tmem_base,
-                                               uint32_t& g, uint32_t it, int num_kb, uint32_t idesc_lp, bool lead,
-                                               const Waiter& w) {
-  using C = CfgP;
-  constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
-  const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
-  const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
-  auto issue_ref = [&](uint32_t gg, int kb) {
-    const uint32_t base = tma_tiles + (gg % C::kTmaStages) * C::kTmaStageBytes;
-    const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
-#pragma unroll
-    for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
-      mma_pair<kKindF16>(tmem_base + col_ref, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
-  };
-  auto issue_rest = [&](uint32_t gg, int kb) {
-    const uint32_t abase = abs_tiles + (gg % C::kAbsStages) * C::kAbsStageBytes;
-    const uint64_t dl = smem_desc(abase + C::kOffLa, 128), dr = smem_desc(abase + C::kOffRa, 128);
-#pragma unroll
-    for (int k = 0; k < kBlockK / 16; ++k)
-      mma_pair<kKindF16>(tmem_base + col_den, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
-    const uint32_t base = tma_tiles + (gg % C::kTmaStages) * C::kTmaStageBytes;
-    const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
-#pragma unroll
-    for (int k = 0; k < kBlockK / 32; ++k)   // 32 codes = 32 bytes per step
-      mma_pair<LPK>(tmem_base + col_lp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
-  };
-  // The reference block of this tile has been free since the epilogue of tile it-2 ended (awaited
-  // before tile it-1 was committed, below), so the reference MMAs of the first k-blocks are issued
-  // at once and keep the tensor pipe busy while both epilogues copy the previous tile's reference
-  // and denominator blocks out and hand them back; the denominator and 8-bit MMAs of those
-  // k-blocks follow that signal.
-  int kb = 0;
-  const int n_ahead = num_kb < kRefAhead ? num_kb : kRefAhead;
-  for (int j = 0; j < n_ahead; ++j) {
-    const uint32_t gg = g + j;
-    if (!w.wait_warp(smem_u32(&sh->ready[gg % C::kAbsStages]), (gg / C::kAbsStages) & 1)) return false;
-    tc_fence_after();
-    issue_ref(gg, j);
-  }
-  if (it > 0 && !w.wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1)) return false;
-  tc_fence_after();
-  for (; kb < n_ahead; ++kb, ++g) {
-    issue_rest(g, kb);
-    tc_commit_pair(smem_u32(&sh->empty[g % C::kTmaStages]), lead);
-  }
-  for (; kb < num_kb; ++kb, ++g) {
-    if (!w.wait_warp(smem_u32(&sh->ready[g % C::kAbsStages]), (g / C::kAbsStages) & 1)) return false;
-    tc_fence_after();
-    issue_ref(g, kb);
-    issue_rest(g, kb);
-    tc_commit_pair(smem_u32(&sh->empty[g % C::kTmaStages]), lead);        // frees the k-block in both CTAs
-  }
-  // The next tile's reference block is this tile's free one, last read by the epilogue of tile
-  // it-1: wait for that epilogue here, where the barrier cannot yet have moved on to this tile's
-  // phase.
-  if (it > 0 && !w.wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1)) return false;
-  tc_commit_pair(smem_u32(&sh->tmem_full), lead);                          // this tile's accumulators are complete
-  return true;
-}
 
 __global__ void __launch_bounds__(kProbeThreads, 1)
 tc_group_kernel(const __grid_constant__ GroupTable tab) {
   using C = CfgP;
+  constexpr int kStages = C::kStages, kAbs = C::kAbsStages;
   extern __shared__ uint8_t smem_raw[];
   // tiles start on a 1024-byte boundary (the 128-byte swizzle atom); the offset is the same in
   // both CTAs of the pair because their dynamic shared memory starts at the same address
   uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   SharedP* sh = reinterpret_cast<SharedP*>(tiles + C::kTileBytes);
-  const uint32_t tma_tiles = smem_u32(tiles), abs_tiles = tma_tiles + C::kTmaStages * C::kTmaStageBytes;
+  const uint32_t tile_base = smem_u32(tiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
@@ -1216,11 +1220,11 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(&tab.p[group_find(tab, pos)].maps[lane]) : "memory");
   }
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kTmaStages; ++s) {
+    for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
       mbar_init(smem_u32(&sh->empty[s]), 1);
     }
-    for (int s = 0; s < C::kAbsStages; ++s) mbar_init(smem_u32(&sh->ready[s]), 2 * kConvWarps);
+    for (int s = 0; s < kAbs; ++s) mbar_init(smem_u32(&sh->ready[s]), 2 * 4);   // four converter warps in each CTA
     mbar_init(smem_u32(&sh->tmem_full), 1);
     mbar_init(smem_u32(&sh->tmem_empty), 2 * kEpiWarps);
     mbar_init(smem_u32(&sh->lp_done), 2 * kEpiWarps);
@@ -1243,106 +1247,151 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      uint32_t g = 0;
-      bool ok = true;
-      for (int r = 0; ok; ++r) {
-        const int pos = group_position(r, pair, num_pairs);
-        if (pos >= tab.total_tiles) {
-          if (r * num_pairs >= tab.total_tiles) break;          // no round reaches further
-          continue;
-        }
-        const GroupProblem& pr = tab.p[group_find(tab, pos)];
-        const TileCoord tc = tile_coord(pos - pr.tile_begin, pr.a);
-        const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
-        const int r0 = tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
-        const int c0 = tc.n_tile * kBlockN + (int)rank * kHalfN;     // this CTA's half of the right operand
-        for (int kb = 0; kb < num_kb; ++kb, ++g) {
-          const int s = g % C::kTmaStages;
-          const uint32_t use = g / C::kTmaStages;
-          if (g >= tab.stop_after_kb) { ok = false; break; }    // test hook: the consumers' waits run out
-          if (use > 0 && !w.wait(smem_u32(&sh->empty[s]), (use - 1) & 1)) {
-            ok = false;
-            break;
-          }
+  if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsCtl));
+    if (warp == 0) {
+      // ---------------------------------------------------------- TMA producer (both CTAs)
+      if (lane == 0) {
+        TileWalk tw;
+        tw.start(tab, pair, num_pairs);
+        for (uint32_t g = 0; tw.valid; ++g, tw.next_kb(tab)) {
+          const int s = g % kStages;
+          const uint32_t use = g / kStages;
+          if (g >= tab.stop_after_kb) break;                  // test hook: the consumers' waits run out
+          if (use > 0 && !w.wait(smem_u32(&sh->empty[s]), (use - 1) & 1)) break;
+          const GroupProblem& pr = tab.p[tw.pi];
+          const int r0 = tw.tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
+          const int c0 = tw.tc.n_tile * kBlockN + (int)rank * kHalfN;     // this CTA's half of the right operand
           const uint32_t bar = smem_u32(&sh->full[s]);
-          mbar_expect_tx(bar, C::kTmaStageBytes);
-          const uint32_t base = tma_tiles + s * C::kTmaStageBytes;
-          const int k0 = kb * kBlockK;
-          tma_load_3d_local(base + C::kOffL, &pr.maps[0], bar, k0, r0, tc.b);
-          tma_load_3d_local(base + C::kOffCl, &pr.maps[2], bar, k0, r0, tc.b);
-          tma_load_3d_local(base + C::kOffR, &pr.maps[1], bar, k0, c0, tc.b);
-          tma_load_3d_local(base + C::kOffCr, &pr.maps[3], bar, k0, c0, tc.b);
+          mbar_expect_tx(bar, C::kTmaBytes);
+          const uint32_t base = tile_base + s * C::kStageBytes;
+          const int k0 = tw.kb * kBlockK;
+          tma_load_3d_local(base + C::kOffR, &pr.maps[1], bar, k0, c0, tw.tc.b);     // the converters read this one
+          tma_load_3d_local(base + C::kOffL, &pr.maps[0], bar, k0, r0, tw.tc.b);
+          tma_load_3d_local(base + C::kOffCl, &pr.maps[2], bar, k0, r0, tw.tc.b);
+          tma_load_3d_local(base + C::kOffCr, &pr.maps[3], bar, k0, c0, tw.tc.b);
           sh->issued = g + 1;
         }
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------ MMA issuer (leader CTA, converged warp)
-    if (rank == 0) {
+    } else if (warp == 1 && rank == 0) {
+      // ---------------------------------------------------------- MMA issuer (leader CTA, converged warp)
       const bool lead = elect_one();
-      uint32_t g = 0, it = 0;
-      bool ok = true;
-      for (int r = 0; ok; ++r) {
-        const int pos = group_position(r, pair, num_pairs);
-        if (pos >= tab.total_tiles) {
-          if (r * num_pairs >= tab.total_tiles) break;
-          continue;
+      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
+      auto issue_ref_den = [&](uint32_t gg, int kb) {
+        const uint32_t s = gg % kStages, base = tile_base + s * C::kStageBytes;
+        const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 32 bytes = 2 descriptor units per step
+          mma_pair<kKindF16>(tmem_base + C::kColRef, dl + 2 * k, dr + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+        const uint64_t da = smem_desc(base + C::kOffRa, 128);
+        const uint32_t ta = tmem_base + C::kColAbsL + 32u * (gg % kAbs);
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k)   // 16 bf16 = 8 columns of tensor memory per step
+          mma_pair_a_tmem(tmem_base + C::kColDen, ta + 8u * k, da + 2 * k, idesc_bf16, (kb | k) != 0, lead);
+      };
+      auto issue_lp = [&](uint32_t gg, int kb, int kind, uint32_t idesc_lp) {
+        const uint32_t base = tile_base + (gg % kStages) * C::kStageBytes;
+        const uint64_t cl = smem_desc(base + C::kOffCl, 64), cr = smem_desc(base + C::kOffCr, 64);
+#pragma unroll
+        for (int k = 0; k < kBlockK / 32; ++k) {  // 32 codes = 32 bytes per step
+          if (kind == kKindI8) mma_pair<kKindI8>(tmem_base + C::kColLp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
+          else mma_pair<kKindF8>(tmem_base + C::kColLp, cl + 2 * k, cr + 2 * k, idesc_lp, (kb | k) != 0, lead);
         }
-        const GroupProblem& pr = tab.p[group_find(tab, pos)];
-        const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
-        ok = pr.kind == kKindI8
-                 ? group_mma_tile<kKindI8>(sh, tma_tiles, abs_tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, w)
-                 : group_mma_tile<kKindF8>(sh, tma_tiles, abs_tiles, tmem_base, g, it, num_kb, pr.a.idesc_lp, lead, w);
+      };
+      auto wait_stage = [&](uint32_t gg) {
+        if (!w.wait_warp(smem_u32(&sh->ready[gg % kAbs]), (gg / kAbs) & 1)) return false;
+        tc_fence_after();
+        return true;
+      };
+      TileWalk tw;
+      tw.start(tab, pair, num_pairs);
+      uint32_t g = 0;
+      bool ok = true;
+      for (uint32_t it = 0; tw.valid && ok; ++it, tw.next_tile(tab)) {
+        const GroupProblem& pr = tab.p[tw.pi];
+        const int num_kb = tw.num_kb, kind = pr.kind;
+        const uint32_t idesc_lp = pr.a.idesc_lp;
+        // the reference and denominator blocks come back when both epilogues have copied the
+        // previous tile's values out; the 8-bit block when they have finished that tile
+        if (it > 0 && !w.wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1)) break;
+        tc_fence_after();
+        const int n_ahead = num_kb < kAbs ? num_kb : kAbs;
+        for (int j = 0; j < n_ahead && ok; ++j) {
+          ok = wait_stage(g + j);
+          if (ok) issue_ref_den(g + j, j);
+        }
         if (!ok) break;
-        ++it;
+        if (it > 0 && !w.wait_warp(smem_u32(&sh->lp_done), (it - 1) & 1)) break;
+        tc_fence_after();
+        int kb = 0;
+        for (; kb < n_ahead; ++kb, ++g) {
+          issue_lp(g, kb, kind, idesc_lp);
+          tc_commit_pair(smem_u32(&sh->empty[g % kStages]), lead);
+        }
+        for (; kb < num_kb && ok; ++kb, ++g) {
+          ok = wait_stage(g);
+          if (!ok) break;
+          issue_ref_den(g, kb);
+          issue_lp(g, kb, kind, idesc_lp);
+          tc_commit_pair(smem_u32(&sh->empty[g % kStages]), lead);        // frees the k-block in both CTAs
+        }
+        if (ok) tc_commit_pair(smem_u32(&sh->tmem_full), lead);           // this tile's accumulators are complete
       }
     }
   } else if (warp < kFirstEpiWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsConv));
     // ------------------------------------------------------------ converters (both CTAs)
-    // |L| and |R| tiles of every k-block: L and R follow each other in the stage, so the job is one
-    // flat run of 1536 16-byte vectors; thread t takes vectors t, t + 64, ...
-    constexpr int kVec = (int)(C::kAbsStageBytes / 16);                 // 1536
-    constexpr int kPer = kVec / (32 * kConvWarps);                      // 24
-    const uint32_t t16 = (uint32_t)(threadIdx.x - 64) * 16u;
+    // Thread t of the four warps owns row t of this CTA's 128 left-operand rows (its warp's
+    // tensor-memory lane quarter holds that row): once the stage has landed it reads its row of the
+    // L tile from shared memory (128-byte swizzle: 16-byte chunk c of row r sits at c ^ (r & 7),
+    // which makes these row-per-thread reads conflict-free), clears the sign bits and stores the
+    // 32 words into the stage's tensor-memory columns.  (Loading the rows with plain global loads
+    // instead, to spare shared memory the 16 KB, was tried: a warp then touches 32 lines per
+    // instruction and the converters became the bottleneck, 1.6 x slower overall.)  The |R|
+    // half-tile is a flat sign-cleared copy of the R half-tile (8 KB: four vectors per thread).
+    const int q = warp & 3;
+    const int t = q * 32 + lane;                   // 0..127
     const uint32_t ready_leader = map_to_cta(smem_u32(&sh->ready[0]), 0);
-    uint32_t g = 0;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + C::kColAbsL;
+    const uint32_t row_off = (uint32_t)t * 128u, sw = (uint32_t)t & 7u;
+    TileWalk tw;
+    tw.start(tab, pair, num_pairs);
     bool ok = true;
-    for (int r = 0; ok; ++r) {
-      const int pos = group_position(r, pair, num_pairs);
-      if (pos >= tab.total_tiles) {
-        if (r * num_pairs >= tab.total_tiles) break;
-        continue;
+    for (uint32_t g = 0; ok && tw.valid; ++g, tw.next_kb(tab)) {
+      const uint32_t s = g % kStages, sa = g % kAbs, m = 0x7fff7fffu;
+      // the tensor-memory columns were last read by the MMAs of k-block g - kAbs (its commit also
+      // covers every earlier k-block, so the |R| slot of the stage is free as well)
+      if (g >= (uint32_t)kAbs) {
+        const uint32_t gp = g - kAbs;
+        if (!w.wait_warp(smem_u32(&sh->empty[gp % kStages]), (gp / kStages) & 1)) { ok = false; break; }
       }
-      const GroupProblem& pr = tab.p[group_find(tab, pos)];
-      const int num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
-      for (int kb = 0; kb < num_kb; ++kb, ++g) {
-        // the slot of the |x| ring was last read by the MMAs of k-block g - kAbsStages
-        if (g >= (uint32_t)C::kAbsStages) {
-          const uint32_t gp = g - C::kAbsStages;
-          if (!w.wait_warp(smem_u32(&sh->empty[gp % C::kTmaStages]), (gp / C::kTmaStages) & 1)) { ok = false; break; }
-        }
-        if (!w.wait_warp(smem_u32(&sh->full[g % C::kTmaStages]), (g / C::kTmaStages) & 1)) { ok = false; break; }
-        const uint32_t src = tma_tiles + (g % C::kTmaStages) * C::kTmaStageBytes + t16;
-        const uint32_t dst = abs_tiles + (g % C::kAbsStages) * C::kAbsStageBytes + t16;
-        uint4 v[kPer];
+      if (!w.wait_warp(smem_u32(&sh->full[s]), (g / kStages) & 1)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t base = tile_base + s * C::kStageBytes;
+      uint4 v[8], u[4];
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) v[i] = lds128(src + (uint32_t)i * (32u * kConvWarps * 16u));
+      for (int j = 0; j < 8; ++j) v[j] = lds128(base + C::kOffL + row_off + (((uint32_t)j ^ sw) << 4));
+      const uint32_t rsrc = base + C::kOffR + (uint32_t)t * 16u;
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-          const uint32_t m = 0x7fff7fffu;
-          sts128(dst + (uint32_t)i * (32u * kConvWarps * 16u), make_uint4(v[i].x & m, v[i].y & m, v[i].z & m, v[i].w & m));
-        }
-        // generic-proxy writes -> visible to the tensor core's (async proxy) reads, then signal
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(ready_leader + (g % C::kAbsStages) * 8u);
+      for (int j = 0; j < 4; ++j) u[j] = lds128(rsrc + (uint32_t)j * 2048u);
+      uint32_t a[32];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        a[4 * j] = v[j].x & m; a[4 * j + 1] = v[j].y & m; a[4 * j + 2] = v[j].z & m; a[4 * j + 3] = v[j].w & m;
       }
+      tmem_st32(taddr + 32u * sa, a);
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        sts128(rsrc + (C::kOffRa - C::kOffR) + (uint32_t)j * 2048u, make_uint4(u[j].x & m, u[j].y & m, u[j].z & m, u[j].w & m));
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> the tensor core's reads
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(ready_leader + sa * 8u);
     }
   } else {
-    // ------------------------------------------------------------ epilogue (warps 4..11, both CTAs)
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsEpi));
+    // ------------------------------------------------------------ epilogue (warps 8..15, both CTAs)
     // A warp may touch the tensor-memory lane quarter warp % 4; the two warps of a quarter split
     // the columns.  Copy this warp's 64 columns of the reference and denominator blocks into
     // registers, hand those two blocks back to the MMA lane, then walk the 8-bit block in chunks
@@ -1376,16 +1425,11 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");       // red[] may be reused
     };
-    uint32_t it = 0;
     uint32_t met = 0;                              // bit pi: this CTA has had tiles of probe pi
-    bool live = true;
-    for (int r = 0; live; ++r) {
-      const int pos = group_position(r, pair, num_pairs);
-      if (pos >= tab.total_tiles) {
-        if (r * num_pairs >= tab.total_tiles) break;
-        continue;
-      }
-      const int pi = group_find(tab, pos);
+    TileWalk tw;
+    tw.start(tab, pair, num_pairs);
+    for (uint32_t it = 0; tw.valid; ++it, tw.next_tile(tab)) {
+      const int pi = tw.pi;
       if (pi != cur) {
         if (cur >= 0) flush(cur);
         cur = pi;
@@ -1393,7 +1437,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       }
       const GroupProblem& pr = tab.p[pi];
       const KernelArgs& a = pr.a;
-      const TileCoord tc = tile_coord(pos - pr.tile_begin, a);
+      const TileCoord tc = tw.tc;
       const bool per_col = a.pc_r != 0;
       const float dr_tensor = per_col ? 1.f : __ldg(a.dr);
       float* dr_s = sh->delta_r[it & 1];
@@ -1409,17 +1453,15 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
 
       const bool ok = w.wait(smem_u32(&sh->tmem_full), it & 1);
       // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
-      if (epi_barrier_any(!ok)) { live = false; break; }
+      if (epi_barrier_any(!ok)) break;
       tc_fence_after();
       const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      const uint32_t col_ref = ((3 * it) & 3) * 128u, col_den = ((3 * it + 1) & 3) * 128u;
-      const uint32_t col_lp = ((3 * it + 2) & 3) * 128u;
       const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;      // first column of this warp
       uint32_t rc[64], rd[64], rq[16];
-      tmem_ld32(lane_addr + col_ref + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
-      tmem_ld32(lane_addr + col_ref + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
-      tmem_ld32(lane_addr + col_den + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
-      tmem_ld32(lane_addr + col_den + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+      tmem_ld32(lane_addr + C::kColRef + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
+      tmem_ld32(lane_addr + C::kColRef + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
+      tmem_ld32(lane_addr + C::kColDen + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
+      tmem_ld32(lane_addr + C::kColDen + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
@@ -1432,7 +1474,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         const int cc0 = h * 64 + c * 16;
         const int64_t col0 = colw + c * 16;
         if (col0 < a.N) {                         // uniform across the warp
-          tmem_ld16(lane_addr + col_lp + cc0, rq);
+          tmem_ld16(lane_addr + C::kColLp + cc0, rq);
           tmem_ld_wait();
           const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
           if (is_i8) {
@@ -1444,6 +1486,10 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
           }
         }
       }
+      // the 8-bit block has been read: the MMA lane may start the next tile's 8-bit MMAs
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
       if (row_ok) {
         float x0, x1;
         unpack2(st.be, x0, x1); acc[0] += (double)x0 + (double)x1;
@@ -1453,10 +1499,6 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         acc[1] = fmax(acc[1], (double)st.mx);
         if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
       }
-      tc_fence_before();                          // the 8-bit block's loads are complete as well
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
-      ++it;
     }
     if (cur >= 0) flush(cur);
     // the records of the probes this CTA never met are zero
@@ -1516,11 +1558,11 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
   tc_fence_before();
   __syncthreads();
   if (sh->abort_flag && threadIdx.x == 0) {
-    // give-up path: the loads of the last kTmaStages k-blocks this producer issued may not have
-    // been awaited by anyone; wait (bounded) until each has landed
+    // give-up path: the loads of the last kStages k-blocks this producer issued may not have been
+    // awaited by anyone; wait (bounded) until each has landed
     const uint32_t n = sh->issued;
-    for (uint32_t j = n > (uint32_t)C::kTmaStages ? n - C::kTmaStages : 0u; j < n; ++j) {
-      const uint32_t bar = smem_u32(&sh->full[j % C::kTmaStages]), parity = (j / C::kTmaStages) & 1;
+    for (uint32_t j = n > (uint32_t)kStages ? n - kStages : 0u; j < n; ++j) {
+      const uint32_t bar = smem_u32(&sh->full[j % kStages]), parity = (j / kStages) & 1;
       const uint64_t t0 = global_timer_ns();
       while (!mbar_try_wait(bar, parity) && global_timer_ns() - t0 < tab.wait_limit_ns) {}
     }
@@ -1720,6 +1762,12 @@ qm_status probe_residency() {
   const qm_status as = allow_smem(tc_group_kernel, kProbeSmem, attr_done);
   if (as != QM_OK) return as;
   if (g_max_pairs[dev] == 0) {
+    // the kernel re-divides the registers its block was launched with (setmaxnreg): refuse to
+    // launch if the compiler gave it fewer than the split adds up to, because an increase that
+    // cannot be served waits forever
+    cudaFuncAttributes fa{};
+    QM_CUDA_OK(cudaFuncGetAttributes(&fa, tc_group_kernel));
+    if (fa.numRegs * 4 < kRegsCtl + kRegsConv + 2 * kRegsEpi) return QM_ERR_UNSUPPORTED;
     cudaLaunchConfig_t q{};
     q.gridDim = dim3((unsigned)(2 * (sm_count() / 2))); q.blockDim = dim3(kProbeThreads);
     q.dynamicSmemBytes = kProbeSmem;
