@@ -22,6 +22,23 @@ __device__ __forceinline__ uint32_t absbits_f32(uint32_t w) { return w & 0x7ffff
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// 32 bytes in one load (sm_100 has 256-bit global loads), read-only path, no L1 allocation.
+// STREAM adds evict-first in L2: for tensors much larger than L2 that are read once per pass.
+struct Vec256 { uint4 lo, hi; };
+template <bool STREAM>
+__device__ __forceinline__ Vec256 ld256(const void* p) {
+  Vec256 v;
+  if (STREAM)
+    asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v.lo.x), "=r"(v.lo.y), "=r"(v.lo.z), "=r"(v.lo.w), "=r"(v.hi.x), "=r"(v.hi.y), "=r"(v.hi.z), "=r"(v.hi.w)
+                 : "l"(p));
+  else
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v.lo.x), "=r"(v.lo.y), "=r"(v.lo.z), "=r"(v.lo.w), "=r"(v.hi.x), "=r"(v.hi.y), "=r"(v.hi.z), "=r"(v.hi.w)
+                 : "l"(p));
+  return v;
+}
+
 // Two quantized bytes from t = x / delta: t0 in bits 0..7, t1 in bits 8..15.
 // RTNE, saturating at the largest finite magnitude.
 template <int FMT>
@@ -135,13 +152,21 @@ struct QuotientPair {
 };
 
 // Two codes (bits 0..7 and 8..15) of the bf16 pair held in word w (low half = first element).
-template <int FMT>
+// GUARD: the scale may come from elsewhere, so x r can overflow and the corrections then evaluate
+// inf - inf; fminf returns its non-NaN operand, which turns that case into the largest float and
+// lets the conversion saturate, as the division would.
+template <int FMT, bool GUARD = false>
 __device__ __forceinline__ uint32_t quant_bf16_pair(uint32_t w, const QuotientPair& quot) {
   uint64_t x2;
   asm("mov.b64 %0, {%1, %2};" : "=l"(x2) : "r"(w << 16), "r"(w & 0xffff0000u));
   const uint64_t q2 = quot(x2);
   uint32_t q0, q1;
   asm("mov.b64 {%0, %1}, %2;" : "=r"(q0), "=r"(q1) : "l"(q2));
+  if (GUARD) {
+    q0 = __float_as_uint(fminf(fabsf(__uint_as_float(q0)), 3.402823466e38f)) | ((w << 16) & 0x80000000u);
+    q1 = __float_as_uint(fminf(fabsf(__uint_as_float(q1)), 3.402823466e38f)) | (w & 0x80000000u);
+    return quant2<FMT>(__uint_as_float(q0), __uint_as_float(q1));
+  }
   if (FMT == QM_FMT_INT8) {
     return quant2<FMT>(__uint_as_float(q0), __uint_as_float(q1));
   } else {
@@ -153,13 +178,22 @@ __device__ __forceinline__ uint32_t quant_bf16_pair(uint32_t w, const QuotientPa
 }
 
 // Sixteen codes of sixteen consecutive bf16 values (two 128-bit words).
-template <int FMT>
+template <int FMT, bool GUARD = false>
 __device__ __forceinline__ uint4 quant_bf16x16(const uint4& a, const uint4& b, const QuotientPair& quot) {
   uint4 r;
-  r.x = quant_bf16_pair<FMT>(a.x, quot) | (quant_bf16_pair<FMT>(a.y, quot) << 16);
-  r.y = quant_bf16_pair<FMT>(a.z, quot) | (quant_bf16_pair<FMT>(a.w, quot) << 16);
-  r.z = quant_bf16_pair<FMT>(b.x, quot) | (quant_bf16_pair<FMT>(b.y, quot) << 16);
-  r.w = quant_bf16_pair<FMT>(b.z, quot) | (quant_bf16_pair<FMT>(b.w, quot) << 16);
+  r.x = quant_bf16_pair<FMT, GUARD>(a.x, quot) | (quant_bf16_pair<FMT, GUARD>(a.y, quot) << 16);
+  r.y = quant_bf16_pair<FMT, GUARD>(a.z, quot) | (quant_bf16_pair<FMT, GUARD>(a.w, quot) << 16);
+  r.z = quant_bf16_pair<FMT, GUARD>(b.x, quot) | (quant_bf16_pair<FMT, GUARD>(b.y, quot) << 16);
+  r.w = quant_bf16_pair<FMT, GUARD>(b.z, quot) | (quant_bf16_pair<FMT, GUARD>(b.w, quot) << 16);
+  return r;
+}
+
+// Eight codes of eight consecutive bf16 values (one 128-bit word).
+template <int FMT, bool GUARD = false>
+__device__ __forceinline__ uint2 quant_bf16x8(const uint4& a, const QuotientPair& quot) {
+  uint2 r;
+  r.x = quant_bf16_pair<FMT, GUARD>(a.x, quot) | (quant_bf16_pair<FMT, GUARD>(a.y, quot) << 16);
+  r.y = quant_bf16_pair<FMT, GUARD>(a.z, quot) | (quant_bf16_pair<FMT, GUARD>(a.w, quot) << 16);
   return r;
 }
 

@@ -72,6 +72,43 @@ absmax_tensor_kernel(const T* __restrict__ x, int64_t rows, int64_t c, int64_t r
   if (threadIdx.x == 0 && acc) atomicMax(amax, acc);
 }
 
+// ---------------------------------------------------------------- absmax, dense tensor
+// One flat run of 32-byte vectors (base 32-byte aligned): 256-bit loads, IN_FLIGHT of them
+// outstanding per thread, and the maximum taken on packed words: for bf16 two sign-cleared 16-bit
+// patterns per word (unsigned 16-bit maxima order like the magnitudes), for fp32 one 31-bit pattern.
+template <typename T, int IN_FLIGHT, bool STREAM>
+__global__ void __launch_bounds__(kThreads)
+absmax_dense_kernel(const uint8_t* __restrict__ x, uint64_t n_vec, uint32_t* __restrict__ amax) {
+  pdl_prologue();
+  constexpr bool kBf16 = sizeof(T) == 2;
+  const uint32_t mask = kBf16 ? 0x7fff7fffu : 0x7fffffffu;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t m = 0;
+  auto fold = [&](const Vec256& v) {
+    if (kBf16) {
+      const uint32_t a = __vmaxu2(__vmaxu2(v.lo.x & mask, v.lo.y & mask), __vmaxu2(v.lo.z & mask, v.lo.w & mask));
+      const uint32_t b = __vmaxu2(__vmaxu2(v.hi.x & mask, v.hi.y & mask), __vmaxu2(v.hi.z & mask, v.hi.w & mask));
+      m = __vmaxu2(m, __vmaxu2(a, b));
+    } else {
+      const uint32_t a = max(max(v.lo.x & mask, v.lo.y & mask), max(v.lo.z & mask, v.lo.w & mask));
+      const uint32_t b = max(max(v.hi.x & mask, v.hi.y & mask), max(v.hi.z & mask, v.hi.w & mask));
+      m = max(m, max(a, b));
+    }
+  };
+  for (; i + (IN_FLIGHT - 1) * stride < n_vec; i += IN_FLIGHT * stride) {
+    Vec256 v[IN_FLIGHT];
+#pragma unroll
+    for (int u = 0; u < IN_FLIGHT; ++u) v[u] = ld256<STREAM>(x + (i + u * stride) * 32);
+#pragma unroll
+    for (int u = 0; u < IN_FLIGHT; ++u) fold(v[u]);
+  }
+  for (; i < n_vec; i += stride) fold(ld256<STREAM>(x + i * 32));
+  uint32_t acc = kBf16 ? (max(m & 0xffffu, m >> 16) << 16) : m;      // as an fp32 bit pattern
+  acc = block_max(acc);
+  if (threadIdx.x == 0 && acc) atomicMax(amax, acc);
+}
+
 // ---------------------------------------------------------------- absmax per row (contiguous rows)
 // G lanes share a row; rows are (batch, nc) pairs.
 template <typename T, int G>
@@ -246,7 +283,9 @@ quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64_t s_n
 // any of them (2 x CHUNKS loads in flight per thread; 4 for tensors that fill the GPU several
 // times over, 1 for small ones, which need the parallelism more); |x| copies are the raw
 // bit patterns with the sign bits cleared.
-template <int FMT, int CHUNKS>
+// WIDE: the tensor starts on a 32-byte boundary and a chunk is fetched with one 256-bit load (the
+// four-chunk variant, used for tensors far larger than L2, also asks for evict-first).
+template <int FMT, int CHUNKS, bool WIDE>
 __global__ void __launch_bounds__(kThreads)
 quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const DeltaSrc ds,
                       const FastDiv by_chunks, uint32_t chunks_per_row, uint4* __restrict__ codes,
@@ -258,10 +297,27 @@ quantize_dense_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const 
   for (int u = 0; u < CHUNKS; ++u) {
     const uint32_t i = base + u * kThreads;
     const uint32_t j = i < total_chunks ? i : total_chunks - 1;     // clamp: results of dead lanes are dropped
-    w[u][0] = __ldg(x + 2 * (size_t)j);
-    w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+    if (WIDE) {
+      const Vec256 v = ld256<CHUNKS == 4>(x + 2 * (size_t)j);
+      w[u][0] = v.lo; w[u][1] = v.hi;
+    } else {
+      w[u][0] = __ldg(x + 2 * (size_t)j);
+      w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+    }
   }
   const float d_tensor = ds.per_channel ? 0.f : ds.get(0, blockIdx.x == 0 && threadIdx.x == 0);
+  if (!ds.per_channel && !abs_copy && QuotientPair::serves(d_tensor)) {
+    // one scale for the whole tensor: the two-wide exact quotient (guarded against overflow
+    // when the scale was handed in rather than taken from the tensor's own max|x|)
+    const QuotientPair qp(d_tensor);
+#pragma unroll
+    for (int u = 0; u < CHUNKS; ++u) {
+      const uint32_t i = base + u * kThreads;
+      if (i < total_chunks)
+        codes[i] = ds.from_amax ? quant_bf16x16<FMT, false>(w[u][0], w[u][1], qp) : quant_bf16x16<FMT, true>(w[u][0], w[u][1], qp);
+    }
+    return;
+  }
   const Quotient quot_tensor(d_tensor);
 #pragma unroll
   for (int u = 0; u < CHUNKS; ++u) {
@@ -316,7 +372,7 @@ __device__ __forceinline__ void multi_scales(const uint32_t* amax, const MultiOu
 }
 
 // Dense bf16 tensor, rows a multiple of 16 long: one flat run of 16-element chunks.
-template <int MASK, int CHUNKS>
+template <int MASK, int CHUNKS, bool WIDE>
 __global__ void __launch_bounds__(kThreads)
 quantize_dense_multi_kernel(const uint4* __restrict__ x, uint32_t total_chunks, const uint32_t* __restrict__ amax,
                             const MultiOut o) {
@@ -327,8 +383,13 @@ quantize_dense_multi_kernel(const uint4* __restrict__ x, uint32_t total_chunks, 
   for (int u = 0; u < CHUNKS; ++u) {
     const uint32_t i = base + u * kThreads;
     const uint32_t j = i < total_chunks ? i : total_chunks - 1;     // clamp: results of dead lanes are dropped
-    w[u][0] = __ldg(x + 2 * (size_t)j);
-    w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+    if (WIDE) {
+      const Vec256 v = ld256<CHUNKS == 4>(x + 2 * (size_t)j);
+      w[u][0] = v.lo; w[u][1] = v.hi;
+    } else {
+      w[u][0] = __ldg(x + 2 * (size_t)j);
+      w[u][1] = __ldg(x + 2 * (size_t)j + 1);
+    }
   }
   float d[3];
   multi_scales<MASK>(amax, o, blockIdx.x == 0 && threadIdx.x == 0, d);
@@ -523,6 +584,15 @@ scale_quantize_rows_reg_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, 
     delta_out[row] = d;
     if (acc >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
   }
+  if (!abs_copy && QuotientPair::serves(d)) {
+    const QuotientPair qp(d);                                // the row's own scale: nothing can overflow
+#pragma unroll
+    for (int u = 0; u < VPL; ++u) {
+      const int k = lane + 32 * u;
+      if (k < nvec) codes[row * nvec + k] = quant_bf16x8<FMT>(w[u], qp);
+    }
+    return;
+  }
   const Quotient quot(d);
 #pragma unroll
   for (int u = 0; u < VPL; ++u) {
@@ -631,25 +701,36 @@ quantize_transpose_bf16_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, 
 #pragma unroll
   for (int col = 0; col < 2; ++col) {
     const int64_t orow = b * nc + n + col;
-    const Quotient quot(ds.per_channel ? ds.get(orow, k0 == 0) : d_tensor);
-    uint32_t cw[8];
+    const float dv = ds.per_channel ? ds.get(orow, k0 == 0) : d_tensor;
+    // this column's 32 values as 16 words of two bf16 each
+    uint32_t pw[16];
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {
-      Vec8 f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) f.v[j] = col == 0 ? bf16_lo(w[g * 8 + j]) : bf16_hi(w[g * 8 + j]);
-      const uint2 q = quant8<FMT>(f, quot);
-      cw[2 * g] = q.x; cw[2 * g + 1] = q.y;
-    }
+    for (int j = 0; j < 16; ++j)
+      pw[j] = col == 0 ? __byte_perm(w[2 * j], w[2 * j + 1], 0x5410) : __byte_perm(w[2 * j], w[2 * j + 1], 0x7632);
     uint4* cdst = reinterpret_cast<uint4*>(codes + orow * ldc + k0);
-    cdst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-    cdst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
-    if (abs_copy || kmaj_copy) {
-      // gather this column's 32 values as 16 words of two bf16 each
-      uint32_t pw[16];
+    if (QuotientPair::serves(dv)) {
+      const QuotientPair qp(dv);
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        pw[j] = col == 0 ? __byte_perm(w[2 * j], w[2 * j + 1], 0x5410) : __byte_perm(w[2 * j], w[2 * j + 1], 0x7632);
+      for (int h = 0; h < 2; ++h) {
+        const uint4 a = make_uint4(pw[8 * h], pw[8 * h + 1], pw[8 * h + 2], pw[8 * h + 3]);
+        const uint4 bb = make_uint4(pw[8 * h + 4], pw[8 * h + 5], pw[8 * h + 6], pw[8 * h + 7]);
+        cdst[h] = ds.from_amax ? quant_bf16x16<FMT, false>(a, bb, qp) : quant_bf16x16<FMT, true>(a, bb, qp);
+      }
+    } else {
+      const Quotient quot(dv);
+      uint32_t cw[8];
+#pragma unroll
+      for (int g = 0; g < 4; ++g) {
+        Vec8 f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { f.v[2 * j] = bf16_lo(pw[4 * g + j]); f.v[2 * j + 1] = bf16_hi(pw[4 * g + j]); }
+        const uint2 q = quant8<FMT>(f, quot);
+        cw[2 * g] = q.x; cw[2 * g + 1] = q.y;
+      }
+      cdst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      cdst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+    }
+    if (abs_copy || kmaj_copy) {
       if (kmaj_copy) {
         uint4* d = reinterpret_cast<uint4*>(kmaj_copy + orow * c + k0);
 #pragma unroll
@@ -672,6 +753,28 @@ int grid_for(int64_t work_items, int per_sm) {
   return (int)(want < 1 ? 1 : (want < cap ? want : cap));
 }
 
+// max|x| over n dense elements: the 32-byte aligned middle by the 256-bit kernel, what is left at
+// either end (less than 32 bytes each) by the general one.
+template <typename T>
+void absmax_dense(const T* p, int64_t n, uint32_t* amax, cudaStream_t s) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(p), a1 = a0 + (uintptr_t)n * sizeof(T);
+  const uintptr_t m0 = (a0 + 31) & ~(uintptr_t)31, m1 = a1 & ~(uintptr_t)31;
+  if (m1 <= m0) {
+    launch_pdl(absmax_tensor_kernel<T>, dim3(1), dim3(kThreads), 0, s, p, 1, n, n, amax);
+    return;
+  }
+  const uint64_t n_vec = (m1 - m0) / 32;
+  const dim3 grid((unsigned)grid_for((int64_t)n_vec, 8));
+  const uint8_t* mid = reinterpret_cast<const uint8_t*>(m0);
+  if (m1 - m0 > (64u << 20))        // read once and far larger than what stays in L2: evict first
+    launch_pdl(absmax_dense_kernel<T, 4, true>, grid, dim3(kThreads), 0, s, mid, n_vec, amax);
+  else
+    launch_pdl(absmax_dense_kernel<T, 4, false>, grid, dim3(kThreads), 0, s, mid, n_vec, amax);
+  const int64_t head = (int64_t)((m0 - a0) / sizeof(T)), tail = (int64_t)((a1 - m1) / sizeof(T));
+  if (head > 0) launch_pdl(absmax_tensor_kernel<T>, dim3(1), dim3(32), 0, s, p, 1, head, head, amax);
+  if (tail > 0) launch_pdl(absmax_tensor_kernel<T>, dim3(1), dim3(32), 0, s, p + (n - tail), 1, tail, tail, amax);
+}
+
 template <typename T>
 qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
   const T* p = static_cast<const T*>(x.data);
@@ -681,7 +784,7 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
       const bool even = x.batch == 1 || x.s_b == x.nc * x.s_nc;
       if (dense) {
         const int64_t n = x.nc * x.batch * x.c;
-        launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s, p, 1, n, n, amax);
+        absmax_dense<T>(p, n, amax, s);
       } else if (even) {
         launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(x.nc * x.batch * x.c / 8 + 1, 8)), dim3(kThreads), 0, s, 
             p, x.nc * x.batch, x.c, x.s_nc, amax);
@@ -710,7 +813,7 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
         const bool dense = x.s_c == x.nc;
         const int64_t n = x.nc * x.c * x.batch;
         if (dense)
-          launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s, p, 1, n, n, amax);
+          absmax_dense<T>(p, n, amax, s);
         else
           launch_pdl(absmax_tensor_kernel<T>, dim3(grid_for(n / 8 + 1, 8)), dim3(kThreads), 0, s,
               p, x.c * x.batch, x.nc, x.s_c, amax);
@@ -753,16 +856,16 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
     if (dense) {
       const uint4* src = reinterpret_cast<const uint4*>(x.data);
       const FastDiv by_chunks((uint32_t)(ldc >> 4));
-      if (total >= (int64_t)sm_count() * 8 * kThreads * 4) {
-        const int64_t per_block = (int64_t)kThreads * 4;
-        launch_pdl(quantize_dense_kernel<FMT, 4>, dim3((unsigned)((total + per_block - 1) / per_block)), dim3(kThreads),
-                   0, s, src, (uint32_t)total, ds, by_chunks, (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes),
-                   reinterpret_cast<uint4*>(abs_copy));
-      } else {
-        launch_pdl(quantize_dense_kernel<FMT, 1>, dim3((unsigned)((total + kThreads - 1) / kThreads)), dim3(kThreads),
-                   0, s, src, (uint32_t)total, ds, by_chunks, (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes),
-                   reinterpret_cast<uint4*>(abs_copy));
-      }
+      const bool big = total >= (int64_t)sm_count() * 8 * kThreads * 4;
+      const bool wide = (reinterpret_cast<uintptr_t>(x.data) & 31) == 0;
+      const int64_t per_block = (int64_t)kThreads * (big ? 4 : 1);
+      const dim3 grid((unsigned)((total + per_block - 1) / per_block));
+#define QM_QD(C, W)                                                                                                 \
+  launch_pdl(quantize_dense_kernel<FMT, C, W>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, ds, by_chunks, \
+             (uint32_t)(ldc >> 4), reinterpret_cast<uint4*>(codes), reinterpret_cast<uint4*>(abs_copy))
+      if (big) { if (wide) QM_QD(4, true); else QM_QD(4, false); }
+      else { if (wide) QM_QD(1, true); else QM_QD(1, false); }
+#undef QM_QD
     } else
     launch_pdl(quantize_rows_kernel<T, FMT>, dim3(grid_for(total, 16)), dim3(kThreads), 0, s, 
         p, x.nc, x.c, x.s_nc, x.batch, x.s_b, ds, FastDiv((uint32_t)(ldc >> 4)), FastDiv((uint32_t)x.nc),
@@ -913,9 +1016,12 @@ qm_status launch_quantize_multi(const View& x, int gran, const uint32_t* amax, i
     const bool big = total >= (int64_t)sm_count() * 8 * kThreads * 4;
     const int64_t per_block = (int64_t)kThreads * (big ? 4 : 1);
     const dim3 grid((unsigned)((total + per_block - 1) / per_block));
-#define QM_DM(M)                                                                                                   \
-  (big ? launch_pdl(quantize_dense_multi_kernel<M, 4>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o) \
-       : launch_pdl(quantize_dense_multi_kernel<M, 1>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o))
+    const bool wide = (reinterpret_cast<uintptr_t>(x.data) & 31) == 0;
+#define QM_DM(M)                                                                                                           \
+  (big ? (wide ? launch_pdl(quantize_dense_multi_kernel<M, 4, true>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o)    \
+               : launch_pdl(quantize_dense_multi_kernel<M, 4, false>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o))  \
+       : (wide ? launch_pdl(quantize_dense_multi_kernel<M, 1, true>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o)    \
+               : launch_pdl(quantize_dense_multi_kernel<M, 1, false>, grid, dim3(kThreads), 0, s, src, (uint32_t)total, amax, o)))
     switch (mask) {
       case 3: QM_DM(3); break;
       case 5: QM_DM(5); break;

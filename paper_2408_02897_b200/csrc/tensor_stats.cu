@@ -142,6 +142,133 @@ struct Batch {
   }
 };
 
+// The block's record from its threads' sums, and, in the last block to finish, the fixed-order
+// sum of all records into the result.
+template <int KIND>
+__device__ __forceinline__ void finish_pass(Acc& acc, double* __restrict__ partials, uint32_t* __restrict__ counter,
+                                            void* __restrict__ result, uint64_t count) {
+  // block record
+  __shared__ double red[kRec][kThreads / 32];
+  __shared__ uint32_t is_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < kRec; ++i) {
+    double x = acc.d[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double y = __shfl_xor_sync(0xffffffffu, x, o);
+      x = is_max<KIND>(i) ? fmax(x, y) : x + y;
+    }
+    if (lane == 0) red[i][warp] = x;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double* rec = partials + (int64_t)blockIdx.x * kRec;
+    for (int i = 0; i < kRec; ++i) {
+      double x = red[i][0];
+      for (int w = 1; w < kThreads / 32; ++w) x = is_max<KIND>(i) ? fmax(x, red[i][w]) : x + red[i][w];
+      __stcg(rec + i, x);
+    }
+    __threadfence();
+    is_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  // last block: every record is visible.  Thread t adds records t, t + 256, ... (all 256 threads, so
+  // that the loads of this last step run side by side), then warps and block combine in a fixed order.
+  __threadfence();
+  double tot[kRec];
+#pragma unroll
+  for (int i = 0; i < kRec; ++i) tot[i] = 0.0;
+  for (int b = threadIdx.x; b < (int)gridDim.x; b += kThreads) {
+    const double* rec = partials + (int64_t)b * kRec;
+#pragma unroll
+    for (int i = 0; i < kRec; ++i) {
+      const double y = __ldcg(rec + i);
+      tot[i] = is_max<KIND>(i) ? fmax(tot[i], y) : tot[i] + y;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kRec; ++i) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double y = __shfl_xor_sync(0xffffffffu, tot[i], o);
+      tot[i] = is_max<KIND>(i) ? fmax(tot[i], y) : tot[i] + y;
+    }
+    if (lane == 0) red[i][warp] = tot[i];
+  }
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+#pragma unroll
+  for (int i = 0; i < kRec; ++i) {
+    double x = red[i][0];
+    for (int w = 1; w < kThreads / 32; ++w) x = is_max<KIND>(i) ? fmax(x, red[i][w]) : x + red[i][w];
+    tot[i] = x;
+  }
+  if (KIND == kStats) {
+    qm_tensor_stats_result* r = static_cast<qm_tensor_stats_result*>(result);
+    r->sum1 = tot[0]; r->sum2 = tot[1]; r->sum3 = tot[2]; r->sum4 = tot[3];
+    r->max_abs = tot[4];
+    r->count = count;
+    // a NaN or Inf element (or a power that left the fp32 range) makes sum x^4 NaN or Inf
+    r->device_error = (tot[3] != tot[3] || tot[3] > 1.7e308 || tot[4] > 3.5e38) ? QM_DEVERR_NONFINITE : 0u;
+    r->reserved = 0;
+  } else {
+    qm_quant_error_result* r = static_cast<qm_quant_error_result*>(result);
+    r->sum_re = tot[0]; r->sum_re_round = tot[1]; r->max_re_round = tot[9];
+    r->err2_round = tot[2]; r->err2_overflow = tot[3]; r->err2_underflow = tot[4]; r->sum_x2 = tot[5];
+    r->count = count;
+    r->n_nonzero = (uint64_t)tot[6]; r->n_overflow = (uint64_t)tot[7]; r->n_underflow = (uint64_t)tot[8];
+    r->device_error = (tot[5] != tot[5] || tot[5] > 1.7e308) ? QM_DEVERR_NONFINITE : 0u;   // NaN / Inf seen
+    r->reserved = 0;
+  }
+}
+
+// Statistics of a dense tensor that starts on a 32-byte boundary and is a whole number of 32-byte
+// vectors long: 256-bit loads, four in flight per thread, the same arithmetic (fp32 inside the 64
+// or 32 elements of a batch of loads, fp64 above).
+template <typename T, bool STREAM>
+__global__ void __launch_bounds__(kThreads)
+tensor_stats_dense_kernel(const uint8_t* __restrict__ x, uint64_t n_vec, double* __restrict__ partials,
+                          uint32_t* __restrict__ counter, void* __restrict__ result, uint64_t count) {
+  pdl_prologue();
+  Acc acc;
+#pragma unroll
+  for (int i = 0; i < kRec; ++i) acc.d[i] = 0.0;
+  constexpr int U = 4;
+  const uint64_t stride = (uint64_t)gridDim.x * kThreads;
+  auto eat = [&](Batch<kStats, 0>& bt, const Vec256& v) {
+    Vec8 a, b;
+    if (sizeof(T) == 2) {
+      a.v[0] = bf16_lo(v.lo.x); a.v[1] = bf16_hi(v.lo.x); a.v[2] = bf16_lo(v.lo.y); a.v[3] = bf16_hi(v.lo.y);
+      a.v[4] = bf16_lo(v.lo.z); a.v[5] = bf16_hi(v.lo.z); a.v[6] = bf16_lo(v.lo.w); a.v[7] = bf16_hi(v.lo.w);
+      b.v[0] = bf16_lo(v.hi.x); b.v[1] = bf16_hi(v.hi.x); b.v[2] = bf16_lo(v.hi.y); b.v[3] = bf16_hi(v.hi.y);
+      b.v[4] = bf16_lo(v.hi.z); b.v[5] = bf16_hi(v.hi.z); b.v[6] = bf16_lo(v.hi.w); b.v[7] = bf16_hi(v.hi.w);
+      bt.stats(a); bt.stats(b);
+    } else {
+      a.v[0] = __uint_as_float(v.lo.x); a.v[1] = __uint_as_float(v.lo.y); a.v[2] = __uint_as_float(v.lo.z); a.v[3] = __uint_as_float(v.lo.w);
+      a.v[4] = __uint_as_float(v.hi.x); a.v[5] = __uint_as_float(v.hi.y); a.v[6] = __uint_as_float(v.hi.z); a.v[7] = __uint_as_float(v.hi.w);
+      bt.stats(a);
+    }
+  };
+  uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  for (; i + (U - 1) * stride < n_vec; i += U * stride) {
+    Vec256 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) v[u] = ld256<STREAM>(x + (i + u * stride) * 32);
+    Batch<kStats, 0> bt;
+#pragma unroll
+    for (int u = 0; u < U; ++u) eat(bt, v[u]);
+    bt.flush(acc);
+  }
+  for (; i < n_vec; i += stride) {
+    Batch<kStats, 0> bt;
+    eat(bt, ld256<STREAM>(x + i * 32));
+    bt.flush(acc);
+  }
+  finish_pass<kStats>(acc, partials, counter, result, count);
+}
+
 template <typename T, int KIND, int FMT>
 __global__ void __launch_bounds__(kThreads, KIND == kError ? 3 : 1)
 tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __restrict__ counter,
@@ -220,71 +347,7 @@ tensor_pass_kernel(const Lines p, double* __restrict__ partials, uint32_t* __res
     bt.flush(acc);
   }
 
-  // block record
-  __shared__ double red[kRec][kThreads / 32];
-  __shared__ uint32_t is_last;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int i = 0; i < kRec; ++i) {
-    double x = acc.d[i];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const double y = __shfl_xor_sync(0xffffffffu, x, o);
-      x = is_max<KIND>(i) ? fmax(x, y) : x + y;
-    }
-    if (lane == 0) red[i][warp] = x;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double* rec = partials + (int64_t)blockIdx.x * kRec;
-    for (int i = 0; i < kRec; ++i) {
-      double x = red[i][0];
-      for (int w = 1; w < kThreads / 32; ++w) x = is_max<KIND>(i) ? fmax(x, red[i][w]) : x + red[i][w];
-      __stcg(rec + i, x);
-    }
-    __threadfence();
-    is_last = atomicAdd(counter, 1u) == gridDim.x - 1 ? 1u : 0u;
-  }
-  __syncthreads();
-  if (!is_last || warp != 0) return;
-  __threadfence();
-  double tot[kRec];
-#pragma unroll
-  for (int i = 0; i < kRec; ++i) tot[i] = 0.0;
-  for (int b = lane; b < (int)gridDim.x; b += 32) {            // fixed order: deterministic
-    const double* rec = partials + (int64_t)b * kRec;
-#pragma unroll
-    for (int i = 0; i < kRec; ++i) {
-      const double y = __ldcg(rec + i);
-      tot[i] = is_max<KIND>(i) ? fmax(tot[i], y) : tot[i] + y;
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < kRec; ++i) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const double y = __shfl_xor_sync(0xffffffffu, tot[i], o);
-      tot[i] = is_max<KIND>(i) ? fmax(tot[i], y) : tot[i] + y;
-    }
-  }
-  if (lane != 0) return;
-  if (KIND == kStats) {
-    qm_tensor_stats_result* r = static_cast<qm_tensor_stats_result*>(result);
-    r->sum1 = tot[0]; r->sum2 = tot[1]; r->sum3 = tot[2]; r->sum4 = tot[3];
-    r->max_abs = tot[4];
-    r->count = count;
-    // a NaN or Inf element (or a power that left the fp32 range) makes sum x^4 NaN or Inf
-    r->device_error = (tot[3] != tot[3] || tot[3] > 1.7e308 || tot[4] > 3.5e38) ? QM_DEVERR_NONFINITE : 0u;
-    r->reserved = 0;
-  } else {
-    qm_quant_error_result* r = static_cast<qm_quant_error_result*>(result);
-    r->sum_re = tot[0]; r->sum_re_round = tot[1]; r->max_re_round = tot[9];
-    r->err2_round = tot[2]; r->err2_overflow = tot[3]; r->err2_underflow = tot[4]; r->sum_x2 = tot[5];
-    r->count = count;
-    r->n_nonzero = (uint64_t)tot[6]; r->n_overflow = (uint64_t)tot[7]; r->n_underflow = (uint64_t)tot[8];
-    r->device_error = (tot[5] != tot[5] || tot[5] > 1.7e308) ? QM_DEVERR_NONFINITE : 0u;   // NaN / Inf seen
-    r->reserved = 0;
-  }
+  finish_pass<KIND>(acc, partials, counter, result, count);
 }
 
 // Describes the view as contiguous lines.  channel_delta: deltas follow the non-contracting index.
@@ -349,6 +412,26 @@ qm_status launch_tensor_stats(const View& x, qm_tensor_stats_result* out, void* 
   qm_status st = make_lines(x, false, nullptr, &p);
   if (st != QM_OK) return st;
   const uint64_t n = (uint64_t)(x.nc * x.c * x.batch);
+  const uint64_t bytes = n * (x.dtype == QM_DT_BF16 ? 2 : 4);
+  if (p.outer == 1 && p.groups_per_line == p.total_groups && (reinterpret_cast<uintptr_t>(x.data) & 31) == 0 &&
+      (bytes & 31) == 0 && bytes >= (1u << 20)) {
+    // dense, aligned and large enough to be worth it: the 256-bit kernel
+    uint32_t* counter = static_cast<uint32_t*>(ws);
+    double* partials = reinterpret_cast<double*>(static_cast<char*>(ws) + kCounterBytes);
+    QM_CUDA_OK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), s));
+    const uint64_t n_vec = bytes / 32;
+    int64_t blocks = (int64_t)((n_vec + kThreads - 1) / kThreads);
+    const int64_t cap = (int64_t)sm_count() * 8 < kMaxBlocks ? (int64_t)sm_count() * 8 : kMaxBlocks;
+    if (blocks > cap) blocks = cap;
+    const uint8_t* src = static_cast<const uint8_t*>(x.data);
+    const bool stream = bytes > (64u << 20);
+#define QM_TS(T, S) launch_pdl(tensor_stats_dense_kernel<T, S>, dim3((unsigned)blocks), dim3(kThreads), 0, s, src, n_vec, partials, counter, static_cast<void*>(out), n)
+    if (x.dtype == QM_DT_BF16) { if (stream) QM_CUDA_OK(QM_TS(__nv_bfloat16, true)); else QM_CUDA_OK(QM_TS(__nv_bfloat16, false)); }
+    else { if (stream) QM_CUDA_OK(QM_TS(float, true)); else QM_CUDA_OK(QM_TS(float, false)); }
+#undef QM_TS
+    count_launch();
+    return QM_OK;
+  }
   return x.dtype == QM_DT_BF16 ? launch_pass<__nv_bfloat16, kStats, 0>(p, out, n, ws, s)
                                : launch_pass<float, kStats, 0>(p, out, n, ws, s);
 }
