@@ -392,6 +392,8 @@ def run_case(a):
             qm.qm_quantize(Lop, a.fmt, "tensor", None)
             qm.qm_quantize(Lop, a.fmt, "channel", None)
             qm.qm_quantize(Lt, a.fmt, "tensor", None)
+            qm.qm_quantize_formats(Lop, ["e4m3", "e5m2", "int8"], "tensor")
+            qm.qm_quantize_formats(Lt, ["e4m3", "e5m2", "int8"], "tensor", want_kmaj=True)
         torch.cuda.synchronize()
         print("done")
     else:

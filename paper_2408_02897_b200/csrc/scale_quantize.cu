@@ -528,9 +528,16 @@ scale_quantize_rows_kernel(const T* __restrict__ x, int64_t nc, int64_t c, int64
     if (acc >= 0x7f800000u && err_word) atomicOr(err_word, QM_DEVERR_NONFINITE);
   }
   const Quotient quot(d);
+  const bool pair_ok = sizeof(T) == 2 && !abs_copy && QuotientPair::serves(d);
+  const QuotientPair qp(pair_ok ? d : 1.f);                 // the row's own scale: nothing can overflow
   const int64_t nchunk = ldc >> 3;                          // 8 codes per step, padding included
   for (int64_t k = sub; k < nchunk; k += G) {
     const int64_t k0 = k * 8;
+    if (pair_ok && k0 + 8 <= c) {
+      const uint4 raw = __ldg(reinterpret_cast<const uint4*>(p + k0));
+      *reinterpret_cast<uint2*>(codes + row * ldc + k0) = quant_bf16x8<FMT>(raw, qp);
+      continue;
+    }
     Vec8 v;
     if (k0 + 8 <= c) v = Loader<T>::load8(p + k0);
     else {
