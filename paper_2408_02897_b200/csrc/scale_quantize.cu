@@ -431,69 +431,136 @@ quantize_dense_multi_kernel(const uint4* __restrict__ x, uint32_t total_chunks, 
   }
 }
 
-// Strided contraction, bf16: the layout of quantize_transpose_bf16_kernel (a thread owns two
-// adjacent columns and 32 consecutive contraction rows), codes of every format in MASK and the
-// contraction-major copy from one read.
-template <int MASK>
-__global__ void __launch_bounds__(kThreads)
-quantize_transpose_bf16_multi_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
-                                     int64_t s_b, const uint32_t* __restrict__ amax, const MultiOut o, int64_t ldc,
-                                     __nv_bfloat16* __restrict__ kmaj_copy) {
-  pdl_prologue();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t b = blockIdx.z;
-  const int64_t n = ((int64_t)blockIdx.x * 32 + lane) * 2;
-  const int64_t k0 = ((int64_t)blockIdx.y * 8 + warp) * 32;
-  float d[3];
-  multi_scales<MASK>(amax, o, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0, d);
-  if (n >= nc || k0 >= c) return;
-  const uint32_t* src = reinterpret_cast<const uint32_t*>(x + b * s_b + k0 * s_c + n);
-  const int64_t step = s_c >> 1;
-  uint32_t w[32];
+// ---------------------------------------------------------------- quantize + transpose through shared memory
+// Storage [c][nc] (nc contiguous, bf16), c a multiple of 128 and nc a multiple of 64.  A block
+// takes a tile of 128 contraction rows x 64 columns: it loads the tile with whole-line reads (8
+// threads per 128-byte row), reads it back column-wise (a thread takes 16 contraction entries of two
+// adjacent columns; consecutive lanes read consecutive words: conflict-free), quantizes, and hands
+// the codes (128 bytes per output row and format) and the contraction-major copy (256 bytes per
+// output row) to global memory through a second shared-memory tile so that every store instruction
+// writes whole lines: 16-byte chunk ch of output row n sits at ch ^ ((n >> 1) & 7), which keeps
+// both the column-wise writes and the row-wise reads of that tile conflict-free.
+// d_lo / d_hi: the scales of the thread's two columns, per format in MASK (bit f = qm_format f).
+template <int MASK, bool GUARD>
+__device__ __forceinline__ void transpose_tile(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
+                                               int64_t s_b, const float (&d_lo)[3], const float (&d_hi)[3],
+                                               uint8_t* const (&codes)[3], int64_t ldc,
+                                               __nv_bfloat16* __restrict__ kmaj_copy, uint4* smem) {
+  const int t = threadIdx.x;
+  const int64_t b = blockIdx.z, n0 = (int64_t)blockIdx.x * 64, k0 = (int64_t)blockIdx.y * 128;
+  // phase 1: 128 rows x 128 bytes, four 16-byte loads per thread in flight
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(x + b * s_b + k0 * s_c + n0);
+    const int64_t pitch = s_c >> 3;                                   // row stride in 16-byte units
+    uint4 v[4];
 #pragma unroll
-  for (int r = 0; r < 32; ++r) w[r] = __ldg(src + r * step);
-  const bool pair_ok = QuotientPair::serves(d[0]) && QuotientPair::serves(d[1]) && QuotientPair::serves(d[2]);
+    for (int i = 0; i < 4; ++i) v[i] = __ldg(src + (int64_t)((t >> 3) + 32 * i) * pitch + (t & 7));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) smem[((t >> 3) + 32 * i) * 8 + (t & 7)] = v[i];
+  }
+  __syncthreads();
+  // phase 2: columns 2p, 2p + 1, contraction entries 16g .. 16g + 15
+  const int pcol = t & 31, g = t >> 5;
+  uint32_t w[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) w[j] = reinterpret_cast<const uint32_t*>(smem)[(16 * g + j) * 32 + pcol];
+  __syncthreads();                                                     // the output tiles reuse the input tile's memory
+  uint4* const s_codes = smem;                                         // [3][64 rows][8 chunks]
+  uint4* const s_kmaj = smem + 3 * 64 * 8;                             // [64 rows][16 chunks]
+  const uint32_t sw = (uint32_t)pcol & 7u;
 #pragma unroll
   for (int col = 0; col < 2; ++col) {
-    const int64_t orow = b * nc + n + col;
-    // this column's 32 values as 16 words of two bf16 each
-    uint32_t pw[16];
+    const int n = 2 * pcol + col;
+    uint32_t pw[8];                                                    // this column's 16 values, two bf16 per word
 #pragma unroll
-    for (int j = 0; j < 16; ++j)
+    for (int j = 0; j < 8; ++j)
       pw[j] = col == 0 ? __byte_perm(w[2 * j], w[2 * j + 1], 0x5410) : __byte_perm(w[2 * j], w[2 * j + 1], 0x7632);
+    const uint4 a = make_uint4(pw[0], pw[1], pw[2], pw[3]), bb = make_uint4(pw[4], pw[5], pw[6], pw[7]);
     if (kmaj_copy) {
-      uint4* dst = reinterpret_cast<uint4*>(kmaj_copy + orow * c + k0);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) dst[j] = make_uint4(pw[4 * j], pw[4 * j + 1], pw[4 * j + 2], pw[4 * j + 3]);
+      s_kmaj[n * 16 + ((2 * g) ^ sw)] = a;
+      s_kmaj[n * 16 + ((2 * g + 1) ^ sw)] = bb;
     }
 #pragma unroll
     for (int f = 0; f < 3; ++f) {
       if (!(MASK & (1 << f))) continue;
-      uint4* cdst = reinterpret_cast<uint4*>(o.codes[f] + orow * ldc + k0);
-      if (pair_ok) {
-        const QuotientPair quot(d[f]);
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint4 a = make_uint4(pw[8 * h], pw[8 * h + 1], pw[8 * h + 2], pw[8 * h + 3]);
-          const uint4 bb = make_uint4(pw[8 * h + 4], pw[8 * h + 5], pw[8 * h + 6], pw[8 * h + 7]);
-          cdst[h] = f == 0 ? quant_bf16x16<0>(a, bb, quot) : f == 1 ? quant_bf16x16<1>(a, bb, quot) : quant_bf16x16<2>(a, bb, quot);
-        }
+      const float d = col == 0 ? d_lo[f] : d_hi[f];
+      uint4 cw;
+      if (QuotientPair::serves(d)) {
+        const QuotientPair qp(d);
+        cw = f == 0 ? quant_bf16x16<0, GUARD>(a, bb, qp) : f == 1 ? quant_bf16x16<1, GUARD>(a, bb, qp) : quant_bf16x16<2, GUARD>(a, bb, qp);
       } else {
-        const Quotient quot(d[f]);
-        uint32_t cw[8];
+        const Quotient quot(d);
+        Vec8 lo, hi;
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          Vec8 t;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) { t.v[2 * j] = bf16_lo(pw[4 * g + j]); t.v[2 * j + 1] = bf16_hi(pw[4 * g + j]); }
-          const uint2 q = f == 0 ? quant8<0>(t, quot) : f == 1 ? quant8<1>(t, quot) : quant8<2>(t, quot);
-          cw[2 * g] = q.x; cw[2 * g + 1] = q.y;
+        for (int j = 0; j < 4; ++j) {
+          lo.v[2 * j] = bf16_lo(pw[j]); lo.v[2 * j + 1] = bf16_hi(pw[j]);
+          hi.v[2 * j] = bf16_lo(pw[4 + j]); hi.v[2 * j + 1] = bf16_hi(pw[4 + j]);
         }
-        cdst[0] = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-        cdst[1] = make_uint4(cw[4], cw[5], cw[6], cw[7]);
+        const uint2 q0 = f == 0 ? quant8<0>(lo, quot) : f == 1 ? quant8<1>(lo, quot) : quant8<2>(lo, quot);
+        const uint2 q1 = f == 0 ? quant8<0>(hi, quot) : f == 1 ? quant8<1>(hi, quot) : quant8<2>(hi, quot);
+        cw = make_uint4(q0.x, q0.y, q1.x, q1.y);
       }
+      s_codes[(f * 64 + n) * 8 + ((uint32_t)g ^ sw)] = cw;
     }
   }
+  __syncthreads();
+  // phase 3: whole output rows
+#pragma unroll
+  for (int f = 0; f < 3; ++f) {
+    if (!(MASK & (1 << f))) continue;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int row = (t >> 3) + 32 * i, ch = t & 7;
+      const uint4 v = s_codes[(f * 64 + row) * 8 + (ch ^ ((row >> 1) & 7))];
+      *reinterpret_cast<uint4*>(codes[f] + (b * nc + n0 + row) * ldc + k0 + ch * 16) = v;
+    }
+  }
+  if (kmaj_copy) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = (t >> 4) + 16 * i, ch = t & 15;
+      const uint4 v = s_kmaj[row * 16 + (ch ^ ((row >> 1) & 7))];
+      *reinterpret_cast<uint4*>(kmaj_copy + (b * nc + n0 + row) * c + k0 + ch * 8) = v;
+    }
+  }
+}
+
+constexpr int kTileSmemVec = 3 * 64 * 8 + 64 * 16;                    // 40 KB in 16-byte units
+
+// One format, scales from a DeltaSrc (per tensor or per output row, finished or from max|x|).
+template <int FMT>
+__global__ void __launch_bounds__(kThreads)
+quantize_transpose_tile_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c, int64_t s_b,
+                               const DeltaSrc ds, uint8_t* __restrict__ codes, int64_t ldc,
+                               __nv_bfloat16* __restrict__ kmaj_copy) {
+  pdl_prologue();
+  __shared__ uint4 smem[kTileSmemVec];
+  const int pcol = threadIdx.x & 31, g = threadIdx.x >> 5;
+  const int64_t orow = (int64_t)blockIdx.z * nc + (int64_t)blockIdx.x * 64 + 2 * pcol;
+  float d_lo[3] = {1.f, 1.f, 1.f}, d_hi[3] = {1.f, 1.f, 1.f};
+  if (ds.per_channel) {
+    d_lo[FMT] = ds.get(orow, blockIdx.y == 0 && g == 0);
+    d_hi[FMT] = ds.get(orow + 1, blockIdx.y == 0 && g == 0);
+  } else {
+    d_lo[FMT] = d_hi[FMT] = ds.get(0, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0);
+  }
+  uint8_t* const cd[3] = {codes, codes, codes};
+  if (ds.from_amax) transpose_tile<1 << FMT, false>(x, nc, c, s_c, s_b, d_lo, d_hi, cd, ldc, kmaj_copy, smem);
+  else transpose_tile<1 << FMT, true>(x, nc, c, s_c, s_b, d_lo, d_hi, cd, ldc, kmaj_copy, smem);
+}
+
+// Every format in MASK from one read, per-tensor scales from the tensor's max|x|.
+template <int MASK>
+__global__ void __launch_bounds__(kThreads)
+quantize_transpose_tile_multi_kernel(const __nv_bfloat16* __restrict__ x, int64_t nc, int64_t c, int64_t s_c,
+                                     int64_t s_b, const uint32_t* __restrict__ amax, const MultiOut o, int64_t ldc,
+                                     __nv_bfloat16* __restrict__ kmaj_copy) {
+  pdl_prologue();
+  __shared__ uint4 smem[kTileSmemVec];
+  float d[3];
+  multi_scales<MASK>(amax, o, blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0, d);
+  uint8_t* const cd[3] = {o.codes[0], o.codes[1], o.codes[2]};
+  transpose_tile<MASK, false>(x, nc, c, s_c, s_b, d, d, cd, ldc, kmaj_copy, smem);
 }
 
 // ---------------------------------------------------------------- fused per-row scale + quantize
@@ -845,6 +912,13 @@ qm_status absmax_t(const View& x, int gran, uint32_t* amax, cudaStream_t s) {
   return QM_OK;
 }
 
+// The shared-memory transposing kernels serve bf16 views whose contraction is strided, in whole
+// tiles of 128 contraction entries x 64 columns.
+bool tile_transposable(const View& x) {
+  return x.dtype == QM_DT_BF16 && !x.c_contig() && (x.c & 127) == 0 && (x.nc & 63) == 0 && x.c / 128 <= 65535 &&
+         x.batch <= 65535;
+}
+
 template <typename T, int FMT>
 qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax, float* delta_out,
                      uint32_t* err_word, uint8_t* codes, void* abs_copy, void* kmaj_copy, const Rounding& rnd,
@@ -886,6 +960,15 @@ qm_status quantize_t(const View& x, int gran, const float* delta, bool from_amax
                                      x.c * 2, x.nc, cudaMemcpyDeviceToDevice, s));
     }
   } else {
+    if (!rnd.stochastic && !abs_copy && tile_transposable(x)) {
+      dim3 grid((unsigned)(x.nc / 64), (unsigned)(x.c / 128), (unsigned)x.batch);
+      launch_pdl(quantize_transpose_tile_kernel<FMT>, dim3(grid), dim3(kThreads), 0, s,
+                 static_cast<const __nv_bfloat16*>(x.data), x.nc, x.c, x.s_c, x.s_b, ds, codes, ldc,
+                 static_cast<__nv_bfloat16*>(kmaj_copy));
+      count_launch();
+      QM_CUDA_OK(cudaGetLastError());
+      return QM_OK;
+    }
     if (!rnd.stochastic && x.dtype == QM_DT_BF16 && (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
         ((x.nc + 63) / 64) * ((x.c + 255) / 256) * x.batch >= 4 * (int64_t)sm_count()) {
       dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
@@ -912,7 +995,7 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
   const T* p = static_cast<const T*>(x.data);
   const int64_t rows = x.nc * x.batch, ldc = qm_code_ld(x.c), nvec = x.c / 8;
   const float qmax = fmt_qmax(FMT);
-  if (x.dtype == QM_DT_BF16 && (x.c & 15) == 0 && x.c <= 4 * 256) {
+  if (x.dtype == QM_DT_BF16 && (x.c & 15) == 0 && x.c <= 16 * 256) {
     // the row fits in one warp's registers
     const unsigned blocks = (unsigned)((rows * 32 + kThreads - 1) / kThreads);
     const __nv_bfloat16* pb = static_cast<const __nv_bfloat16*>(x.data);
@@ -1005,8 +1088,7 @@ qm_status launch_quantize_multi(const View& x, int gran, const uint32_t* amax, i
     dense = x.s_nc == x.c && (x.c & 15) == 0 && (x.batch == 1 || x.s_b == x.nc * x.c) && total < (1ll << 32);
     one_pass = dense && !kmaj_copy;
   } else if (one_pass) {
-    transposing = (x.c & 31) == 0 && (x.nc & 1) == 0 && (x.c + 255) / 256 <= 65535 &&
-                  ((x.nc + 63) / 64) * ((x.c + 255) / 256) * x.batch >= 4 * (int64_t)sm_count();
+    transposing = tile_transposable(x);
     one_pass = transposing;
   }
   if (!one_pass) {
@@ -1037,10 +1119,10 @@ qm_status launch_quantize_multi(const View& x, int gran, const uint32_t* amax, i
     }
 #undef QM_DM
   } else {
-    dim3 grid((unsigned)((x.nc + 63) / 64), (unsigned)((x.c + 255) / 256), (unsigned)x.batch);
+    dim3 grid((unsigned)(x.nc / 64), (unsigned)(x.c / 128), (unsigned)x.batch);
     const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(x.data);
     __nv_bfloat16* km = static_cast<__nv_bfloat16*>(kmaj_copy);
-#define QM_TM(M) launch_pdl(quantize_transpose_bf16_multi_kernel<M>, grid, dim3(kThreads), 0, s, src, x.nc, x.c, x.s_c, x.s_b, amax, o, ldc, km)
+#define QM_TM(M) launch_pdl(quantize_transpose_tile_multi_kernel<M>, grid, dim3(kThreads), 0, s, src, x.nc, x.c, x.s_c, x.s_b, amax, o, ldc, km)
     switch (mask) {
       case 3: QM_TM(3); break;
       case 5: QM_TM(5); break;
