@@ -995,7 +995,7 @@ qm_status scale_quantize_rows_t(const View& x, float* delta_out, uint8_t* codes,
   const T* p = static_cast<const T*>(x.data);
   const int64_t rows = x.nc * x.batch, ldc = qm_code_ld(x.c), nvec = x.c / 8;
   const float qmax = fmt_qmax(FMT);
-  if (x.dtype == QM_DT_BF16 && (x.c & 15) == 0 && x.c <= 16 * 256) {
+  if (x.dtype == QM_DT_BF16 && (x.c & 15) == 0 && x.c <= 4 * 256) {
     // the row fits in one warp's registers
     const unsigned blocks = (unsigned)((rows * 32 + kThreads - 1) / kThreads);
     const __nv_bfloat16* pb = static_cast<const __nv_bfloat16*>(x.data);
