@@ -231,3 +231,41 @@ def test_supplied_scale_that_overflows_the_quotient_saturates(fmt, dtype):
         assert np.array_equal(codes.cpu().numpy()[..., :64], want)
         v = oracle.dequantize(want, fmt)
         assert v[0, 0, 0] == oracle.qmax(fmt) and v[0, 1, 5] == -oracle.qmax(fmt)
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("gran", ["tensor", "channel"])
+@pytest.mark.parametrize("fused", [False, True])
+def test_codes_bf16_strided_in_whole_tiles(fmt, gran, fused):
+    """Strided contraction in whole 128 x 64 tiles: the shared-memory transposing kernel (several
+    tiles in both directions, batched, scales per tensor and per output row, finished or fused)."""
+    t = make((3, 256, 192), torch.bfloat16, 5)             # [b][c = 256][nc = 192], contraction strided
+    td = t.cuda()
+    op = qm.operand_of(td, -2)
+    x = as3(oriented(t, -2))
+    want_d = oracle.scale(x, fmt, gran)
+    want_c = oracle.quantize(x, fmt, want_d)
+    if fused:
+        codes, d, _, km = qm.qm_quantize(op, fmt, gran, None, want_kmaj=True)
+    else:
+        d = qm.qm_scale(op, fmt, gran)
+        codes, _, _, km = qm.qm_quantize(op, fmt, gran, d, want_kmaj=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(d.cpu().numpy().view(np.uint32), want_d.ravel().view(np.uint32))
+    assert np.array_equal(codes.cpu().numpy(), want_c)
+    assert torch.equal(km.cpu(), torch.from_numpy(x).to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_strided_tiles_with_a_scale_from_elsewhere_saturate(fmt):
+    """A supplied scale far below the operand's own drives x / delta past the float range: the codes
+    saturate at the format's largest magnitude (Methodology, saturation rule), as the oracle's do."""
+    t = make((256, 128), torch.bfloat16, 6) * 1e30
+    op = qm.operand_of(t.cuda(), -2)
+    x = as3(oriented(t, -2))
+    tiny = np.array([1e-12], dtype=np.float32)
+    want = oracle.quantize(x, fmt, tiny)
+    codes, _, _, _ = qm.qm_quantize(op, fmt, "tensor", torch.from_numpy(tiny).cuda())
+    assert np.array_equal(codes.cpu().numpy(), want)
+    dense, _, _, _ = qm.qm_quantize(qm.operand_of(t.cuda(), -1), fmt, "tensor", torch.from_numpy(tiny).cuda())
+    assert np.array_equal(dense.cpu().numpy(), oracle.quantize(as3(oriented(t, -1)), fmt, tiny))
