@@ -59,7 +59,8 @@ def load_peaks():
 def build_workload(name):
     if name == "bert_large_sweep_layer":
         t = workloads.config5_layer_tensors(0)
-        ops = [o for fmt in ("e4m3", "e5m2", "int8") for o in workloads.config5_layer(0, fmt, tensors=t)]
+        per_fmt = [workloads.config5_layer(0, fmt, tensors=t) for fmt in ("e4m3", "e5m2", "int8")]
+        ops = [o for triple in zip(*per_fmt) for o in triple]        # the three formats of a product side by side
         return ops, ("one layer of the BERT-large 24-layer sweep (batch 32 x seq 512): projections fwd+dgrad+wgrad and "
                      "batched attention products fwd+bwd, each in E4M3, E5M2 and INT8, per-tensor scales")
     if name == "bert_base_fwd":

@@ -379,9 +379,13 @@ qm_status qm_quantize_error(const qm_operand* x, int32_t fmt, int32_t gran, cons
  * qm_probe_layer_host (l_stage[i], r_stage[i]: distinct device staging buffers,
  * each as large as its operand): every distinct host operand (same address and
  * extent) is copied to the device once, into the staging buffer of the first
- * probe that names it, the probes then run as a device batch, out_host
- * receives the n records and the call waits for them; the first
- * device-detected condition is returned.  n == 0 is a no-op.  On an argument
+ * probe that names it, on a stream of the library's own and in the order in
+ * which the probes first name them; the probes run as device batches of 16
+ * consecutive probes, each waiting only for the copies it needs, so that the
+ * copies of later probes run under the kernels of earlier ones (keep the
+ * probes of one product next to each other: operands are shared within such a
+ * batch of 16); out_host receives the n records and the call waits for them;
+ * the first device-detected condition is returned.  n == 0 is a no-op.  On an argument
  * error of probe i the probes before it are completed as described; the rest
  * are not issued.  Make the first call on a device outside any stream capture.
  */

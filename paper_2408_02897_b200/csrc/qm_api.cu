@@ -609,11 +609,15 @@ qm_status qm_probe_layer_host(const qm_operand* L_host, const qm_operand* R_host
 // ---- batches of probes over the library's own streams ------------------------------------------
 namespace {
 constexpr int kBatchStreams = 8;      // streams of the pool
+constexpr int kCopyEvents = 64;       // chunks of a host batch that can wait for their own copies
 struct BatchStreams {
   std::mutex issue;            // one batch at a time is put into the streams (host side only)
   bool ready = false;
   cudaStream_t s[kBatchStreams];
   cudaEvent_t fork, join[kBatchStreams];
+  std::mutex host_issue;       // one host batch at a time uses the copy stream and its events
+  cudaStream_t copy;           // host batches: the host-to-device copies, beside the probes of earlier chunks
+  cudaEvent_t copy_fork, copied[kCopyEvents];
 };
 // One set per device, created on first use (never inside a stream capture) and kept.
 qm_status batch_streams(BatchStreams** out) {
@@ -629,6 +633,9 @@ qm_status batch_streams(BatchStreams** out) {
       QM_CUDA_OK(cudaEventCreateWithFlags(&b.join[i], cudaEventDisableTiming));
     }
     QM_CUDA_OK(cudaEventCreateWithFlags(&b.fork, cudaEventDisableTiming));
+    QM_CUDA_OK(cudaStreamCreateWithFlags(&b.copy, cudaStreamNonBlocking));
+    QM_CUDA_OK(cudaEventCreateWithFlags(&b.copy_fork, cudaEventDisableTiming));
+    for (int i = 0; i < kCopyEvents; ++i) QM_CUDA_OK(cudaEventCreateWithFlags(&b.copied[i], cudaEventDisableTiming));
     b.ready = true;
   }
   *out = &b;
@@ -921,32 +928,54 @@ qm_status qm_probe_batch_host(int32_t n, const qm_operand* L_host, const qm_oper
   if (n < 0) return QM_ERR_INVALID_ARG;
   if (n == 0) return QM_OK;
   cudaStream_t user = static_cast<cudaStream_t>(stream);
-  // every distinct host operand is copied once; the probes then run as a device batch, which in
-  // turn prepares every distinct operand once
+  BatchStreams* bs = nullptr;
+  qm_status st = batch_streams(&bs);
+  if (st != QM_OK) return st;
+  // Every distinct host operand is copied once, on a stream of the library's own and in the order
+  // in which the probes first name them.  The probes go to the device in chunks of one fused
+  // launch's worth, each chunk as a device batch (which prepares every distinct operand of the
+  // chunk once) that waits only for the copies it needs: the copies of later chunks run under the
+  // kernels of earlier ones.  Order the probes so that those of one product are neighbours and the
+  // first chunks need only the first tensors.
   std::vector<qm_operand> Ld((size_t)n), Rd((size_t)n);
   std::vector<HostCopy> seen;
+  const int32_t chunk = tc_group_max();
+  const bool pipelined = (n + chunk - 1) / chunk <= kCopyEvents;
+  std::lock_guard<std::mutex> lock(bs->host_issue);
+  QM_CUDA_OK(cudaEventRecord(bs->copy_fork, user));               // the copies follow the work already in the stream
+  QM_CUDA_OK(cudaStreamWaitEvent(bs->copy, bs->copy_fork, 0));
   qm_status refused = QM_OK;
-  int32_t good = 0;
-  for (; good < n; ++good) {
-    for (int side = 0; side < 2 && refused == QM_OK; ++side) {
-      const qm_operand& x = side ? R_host[good] : L_host[good];
-      void* stage = side ? r_stage[good] : l_stage[good];
-      const size_t bytes = qm_operand_span_bytes(&x);
-      if (bytes == 0 || !stage) { refused = QM_ERR_INVALID_ARG; break; }
-      void* dev = find_copy(seen, x.data, bytes);
-      if (!dev) {
-        QM_CUDA_OK(cudaMemcpyAsync(stage, x.data, bytes, cudaMemcpyHostToDevice, user));
-        seen.push_back(HostCopy{x.data, bytes, stage});
-        dev = stage;
+  int32_t good = 0, issued = 0;
+  for (int32_t c0 = 0; c0 < n && st == QM_OK && refused == QM_OK; c0 += chunk) {
+    const int32_t c1 = c0 + chunk < n ? c0 + chunk : n;
+    for (good = c0; good < c1; ++good) {
+      for (int side = 0; side < 2 && refused == QM_OK; ++side) {
+        const qm_operand& x = side ? R_host[good] : L_host[good];
+        void* stage = side ? r_stage[good] : l_stage[good];
+        const size_t bytes = qm_operand_span_bytes(&x);
+        if (bytes == 0 || !stage) { refused = QM_ERR_INVALID_ARG; break; }
+        void* dev = find_copy(seen, x.data, bytes);
+        if (!dev) {
+          QM_CUDA_OK(cudaMemcpyAsync(stage, x.data, bytes, cudaMemcpyHostToDevice, bs->copy));
+          seen.push_back(HostCopy{x.data, bytes, stage});
+          dev = stage;
+        }
+        qm_operand& d = side ? Rd[good] : Ld[good];
+        d = x;
+        d.data = dev;
       }
-      qm_operand& d = side ? Rd[good] : Ld[good];
-      d = x;
-      d.data = dev;
+      if (refused != QM_OK) break;
     }
-    if (refused != QM_OK) break;
+    // this chunk's copies (and all earlier ones) are in the copy stream: the caller's stream waits for them
+    cudaEvent_t ev = bs->copied[pipelined ? c0 / chunk : 0];
+    QM_CUDA_OK(cudaEventRecord(ev, bs->copy));
+    QM_CUDA_OK(cudaStreamWaitEvent(user, ev, 0));
+    if (good > c0) {
+      st = qm_probe_batch(good - c0, Ld.data() + c0, Rd.data() + c0, cfg + c0, out_dev + c0, ws + c0, ws_bytes + c0, user);
+      if (st == QM_OK) issued = good;
+    }
+    if (!pipelined) QM_CUDA_OK(cudaStreamSynchronize(user));       // the one event is about to be recorded again
   }
-  qm_status st = qm_probe_batch(good, Ld.data(), Rd.data(), cfg, out_dev, ws, ws_bytes, user);
-  int32_t issued = st == QM_OK ? good : 0;
   if (issued > 0)
     QM_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, sizeof(qm_metric_result) * (size_t)issued, cudaMemcpyDeviceToHost, user));
   QM_CUDA_OK(cudaStreamSynchronize(user));
