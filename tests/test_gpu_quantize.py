@@ -269,3 +269,24 @@ def test_strided_tiles_with_a_scale_from_elsewhere_saturate(fmt):
     assert np.array_equal(codes.cpu().numpy(), want)
     dense, _, _, _ = qm.qm_quantize(qm.operand_of(t.cuda(), -1), fmt, "tensor", torch.from_numpy(tiny).cuda())
     assert np.array_equal(dense.cpu().numpy(), oracle.quantize(as3(oriented(t, -1)), fmt, tiny))
+
+
+@pytest.mark.parametrize("fmt", ["e4m3", "int8"])
+def test_dense_tensors_off_the_32_byte_grid(fmt):
+    """The dense kernels use 256-bit loads on the 32-byte aligned middle of a tensor: a tensor that
+    starts 16 bytes past such a boundary, and one whose size leaves a 16-byte tail, still give the
+    oracle's scale and codes (the ends go through the general kernels or the 128-bit variant)."""
+    base = make((1 << 20) + 64, torch.bfloat16, 7).reshape(-1)
+    dev = base.cuda()
+    for off, rows, cols in ((8, 512, 1024), (0, 33, 72), (8, 129, 4088), (24, 1024, 512)):
+        t = base[off:off + rows * cols].reshape(rows, cols)
+        td = dev[off:off + rows * cols].view(rows, cols)
+        assert td.data_ptr() % 16 == 0
+        op = qm.operand_of(td, -1)
+        x = as3(oriented(t, -1))
+        want_d = oracle.scale(x, fmt, "tensor")
+        d = qm.qm_scale(op, fmt, "tensor")
+        assert np.array_equal(d.cpu().numpy().view(np.uint32), want_d.ravel().view(np.uint32)), (off, rows, cols)
+        if cols % 16 == 0:
+            codes, _, _, _ = qm.qm_quantize(op, fmt, "tensor", d)
+            assert np.array_equal(codes.cpu().numpy()[..., :cols], oracle.quantize(x, fmt, want_d)), (off, rows, cols)

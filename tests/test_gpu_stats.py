@@ -171,3 +171,19 @@ def test_error_argument_checks():
     bad[0, 0] = float("nan")
     r = qm.qm_quantize_error(qm.operand_of(bad, -1), "int8", "tensor", delta=torch.ones(1, device="cuda"))
     assert r.device_error == 1
+
+
+def test_stats_dense_kernel_and_its_fallbacks_agree_with_the_oracle():
+    """Large dense tensors take the 256-bit kernel; the same data 16 bytes off the 32-byte grid takes
+    the general one: both against the oracle."""
+    big = tensor((2048, 1024), torch.bfloat16, 16, scale=0.5)
+    check_stats(big)                                           # 4 MB, aligned: the 256-bit kernel
+    flat = torch.cat([big.reshape(-1), big.reshape(-1)[:8]])
+    dev = flat.cuda()
+    shifted = dev[8:].view(2048, 1024)
+    got = qm.qm_tensor_stats(qm.operand_of(shifted, -1))
+    want = oracle.tensor_stats(flat[8:].float().numpy().reshape(2048, 1024))
+    assert got.count == want["count"] and got.max_abs == want["max_abs"]
+    assert abs(got.sum2 - want["sum2"]) <= 2e-6 * want["sum2"] and abs(got.sum4 - want["sum4"]) <= 2e-6 * want["sum4"]
+    f32 = tensor((1024, 1024), torch.float32, 17)
+    check_stats(f32)                                           # fp32 through the same kernel
