@@ -1,26 +1,24 @@
 // Tensor-core products of the probe for sm_100a: tcgen05.mma with accumulators in tensor
 // memory, operands staged in shared memory by TMA, warp-specialised persistent CTA pairs.
 //
-// Two CTAs on the two SMs of a TPC form a cluster and work on one 256 x 128 output tile with
-// cta_group::2 MMAs: each CTA stages its own 128 rows of the left operand and HALF (64 rows) of
-// the right operand's tile, so every byte of the right operand enters and leaves shared memory
-// once per pair instead of once per SM.
-//
-// Roles in each CTA (320 threads):
-//   warp 0      TMA producer: per 64-wide k-block, bulk-tensor loads of its operand tiles into a
-//               ring of stages; completion is signalled on the LEADER CTA's barrier.  It runs
-//               ahead across tile boundaries, so loads overlap the epilogue.
-//   warp 1      allocates tensor memory; in the leader CTA it runs the MMA loop converged and one
-//               elected lane issues the pair's MMAs
-//   warps 2..9  epilogue: read the CTA's 128 x 128 accumulators with tcgen05.ld (a warp may touch
-//               the lane quarter warp_id % 4; the two warps of a quarter split the columns) and
-//               either reduce the Eq. 3 statistics (probe) or store the product.
-// In probe mode three accumulators live side by side in tensor memory: the reference L.R
-// (bf16 operands, kind::f16), the denominator |L|.|R| (bf16, kind::f16) and the 8-bit product
-// (kind::f8f6f4 or kind::i8), 128 columns each, rotating from tile to tile through the four
-// 128-column blocks so that the next tile's MMAs overlap this tile's epilogue; no M x N matrix
-// ever goes to HBM.  A CTA keeps its Eq. 3 statistics in registers across tiles and
-// writes one record; the last CTA to finish adds the records up in a fixed order.
+// Two CTAs on the two SMs of a TPC form a cluster and work on one output tile with cta_group::2
+// MMAs: each CTA stages its own 128 rows of the left operand and HALF of the right operand's
+// tile, so every byte of the right operand enters and leaves shared memory once per pair instead
+// of once per SM.  Three kernels, in this order in the file:
+//   tc_kernel            256 x 128 tiles, 320 threads (TMA warp, MMA warp, 8 epilogue warps): the
+//                        stand-alone 8-bit and reference products on narrow outputs, and the
+//                        two-formats-in-one-pass probe (four accumulators fill tensor memory);
+//   tc_gemm_wide_kernel  256 x 256 tiles, two accumulator buffers: stand-alone products on outputs at
+//                        least 256 wide;
+//   tc_group_kernel      the fused probe (Eq. 3 record of one probe, or of up to 16 probes, per
+//                        persistent launch): reference L.R, denominator |L|.|R| and 8-bit product side
+//                        by side in tensor memory, |L| fed to the MMAs from tensor memory by converter
+//                        warps, the Eq. 3 statistics reduced in the epilogue; no M x N matrix ever
+//                        goes to HBM.  Its own comment describes roles and barriers.
+// Common to all: the MMA warp runs its loop converged and one elected lane issues; the epilogue
+// warps read the accumulators with tcgen05.ld (a warp may touch the lane quarter warp_id % 4; the
+// two warps of a quarter split the columns); a CTA keeps Eq. 3 statistics in registers across tiles
+// and writes one record, and the last CTA to finish adds the records up in a fixed order.
 //
 // Every mbarrier wait is bounded: when one gives up it raises QM_DEVERR_TIMEOUT in the caller's
 // error word and flags the CTA, after which every role falls through to the common exit, tensor
