@@ -1073,7 +1073,8 @@ struct GroupProblem {
   KernelArgs a;               // num_tiles, tiles_m, tiles_n: of this probe
   int32_t tile_begin;         // position of its first tile in the sequence
   int32_t kind;               // kKindF8 or kKindI8
-  int32_t pad[2];
+  int32_t half_n;             // right-operand rows each CTA stages: 64, or 32 for outputs at most 64 wide
+  uint32_t idesc_ref;         // instruction descriptor of the bf16 MMAs (N = 2 * half_n)
 };
 struct GroupTable {
   int32_t n, total_tiles;
@@ -1259,9 +1260,9 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
           if (use > 0 && !w.wait(smem_u32(&sh->empty[s]), (use - 1) & 1)) break;
           const GroupProblem& pr = tab.p[tw.pi];
           const int r0 = tw.tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
-          const int c0 = tw.tc.n_tile * kBlockN + (int)rank * kHalfN;     // this CTA's half of the right operand
+          const int c0 = tw.tc.n_tile * kBlockN + (int)rank * pr.half_n;  // this CTA's half of the right operand
           const uint32_t bar = smem_u32(&sh->full[s]);
-          mbar_expect_tx(bar, C::kTmaBytes);
+          mbar_expect_tx(bar, kABf16 + kALp + (uint32_t)pr.half_n * (kBlockK * 2 + kBlockK));
           const uint32_t base = tile_base + s * C::kStageBytes;
           const int k0 = tw.kb * kBlockK;
           tma_load_3d_local(base + C::kOffR, &pr.maps[1], bar, k0, c0, tw.tc.b);     // the converters read this one
@@ -1274,7 +1275,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     } else if (warp == 1 && rank == 0) {
       // ---------------------------------------------------------- MMA issuer (leader CTA, converged warp)
       const bool lead = elect_one();
-      constexpr uint32_t idesc_bf16 = make_idesc(1, 1, 1, kPairM, kBlockN);
+      uint32_t idesc_bf16 = 0;                 // of the tile in hand
       auto issue_ref_den = [&](uint32_t gg, int kb) {
         const uint32_t s = gg % kStages, base = tile_base + s * C::kStageBytes;
         const uint64_t dl = smem_desc(base + C::kOffL, 128), dr = smem_desc(base + C::kOffR, 128);
@@ -1309,6 +1310,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         const GroupProblem& pr = tab.p[tw.pi];
         const int num_kb = tw.num_kb, kind = pr.kind;
         const uint32_t idesc_lp = pr.a.idesc_lp;
+        idesc_bf16 = pr.idesc_ref;
         // the reference and denominator blocks come back when both epilogues have copied the
         // previous tile's values out; the 8-bit block when they have finished that tile
         if (it > 0 && !w.wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1)) break;
@@ -1370,8 +1372,9 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) v[j] = lds128(base + C::kOffL + row_off + (((uint32_t)j ^ sw) << 4));
       const uint32_t rsrc = base + C::kOffR + (uint32_t)t * 16u;
+      const int r_vec = tab.p[tw.pi].half_n * 8;                 // 16-byte vectors of the R half-tile that are in use
 #pragma unroll
-      for (int j = 0; j < 4; ++j) u[j] = lds128(rsrc + (uint32_t)j * 2048u);
+      for (int j = 0; j < 4; ++j) u[j] = t + 128 * j < r_vec ? lds128(rsrc + (uint32_t)j * 2048u) : make_uint4(0u, 0u, 0u, 0u);
       uint32_t a[32];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
@@ -1380,7 +1383,8 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       tmem_st32(taddr + 32u * sa, a);
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        sts128(rsrc + (C::kOffRa - C::kOffR) + (uint32_t)j * 2048u, make_uint4(u[j].x & m, u[j].y & m, u[j].z & m, u[j].w & m));
+        if (t + 128 * j < r_vec)
+          sts128(rsrc + (C::kOffRa - C::kOffR) + (uint32_t)j * 2048u, make_uint4(u[j].x & m, u[j].y & m, u[j].z & m, u[j].w & m));
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // generic-proxy writes -> the tensor core's reads
       tc_fence_before();
@@ -1624,10 +1628,10 @@ bool make_map(CUtensorMap* m, const void* base, bool bf16, int box_rows, int64_t
   return r == CUDA_SUCCESS;
 }
 
-uint32_t lp_idesc(int fmt_l, int fmt_r) {
-  if (fmt_l == QM_FMT_INT8) return make_idesc(2, 1, 1, kPairM, kBlockN);           // s8 x s8 -> s32
+uint32_t lp_idesc(int fmt_l, int fmt_r, int n = kBlockN) {
+  if (fmt_l == QM_FMT_INT8) return make_idesc(2, 1, 1, kPairM, n);                 // s8 x s8 -> s32
   const uint32_t fa = fmt_l == QM_FMT_E4M3 ? 0u : 1u, fb = fmt_r == QM_FMT_E4M3 ? 0u : 1u;
-  return make_idesc(1, fa, fb, kPairM, kBlockN);                                   // fp8 x fp8 -> f32
+  return make_idesc(1, fa, fb, kPairM, n);                                         // fp8 x fp8 -> f32
 }
 
 template <int MODE>
@@ -1809,20 +1813,25 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     const GemmShape g = p.g;
     const int64_t ldc = qm_code_ld(g.K);
     GroupProblem& gp = tab.p[k];
+    // outputs at most 64 wide (the context and score-gradient products of attention): MMAs of N = 64,
+    // half as many right-operand rows staged
+    const int half_n = g.N <= 64 ? 32 : kHalfN;
     const bool ok = make_map(&gp.maps[0], p.l, true, kBlockM, g.K, g.M, g.batch, p.l_ld, p.l_sb) &&
-                    make_map(&gp.maps[1], p.r, true, kHalfN, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
+                    make_map(&gp.maps[1], p.r, true, half_n, g.K, g.N, g.batch, p.r_ld, p.r_sb) &&
                     make_map(&gp.maps[2], p.cl, false, kBlockM, g.K, g.M, g.batch, ldc, g.M * ldc) &&
-                    make_map(&gp.maps[3], p.cr, false, kHalfN, g.K, g.N, g.batch, ldc, g.N * ldc);
+                    make_map(&gp.maps[3], p.cr, false, half_n, g.K, g.N, g.batch, ldc, g.N * ldc);
     if (!ok) return QM_ERR_CUDA;
     KernelArgs ka{};
     fill_tiles(&ka, g);
     ka.dl = p.dl; ka.pc_l = p.gran_l == QM_GRAN_CHANNEL; ka.dr = p.dr; ka.pc_r = p.gran_r == QM_GRAN_CHANNEL;
     ka.partials = p.partials; ka.done_counter = p.done_counter; ka.result = p.result;
     ka.count = (uint64_t)(g.M * g.N * g.batch);
-    ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r);
+    ka.err_word = p.err_word; ka.idesc_lp = lp_idesc(p.fmt_l, p.fmt_r, 2 * half_n);
     ka.row_stats = p.row_stats;
     ka.err_also[0] = p.err_also[0]; ka.err_also[1] = p.err_also[1];
     gp.a = ka;
+    gp.half_n = half_n;
+    gp.idesc_ref = make_idesc(1, 1, 1, kPairM, 2 * half_n);
     gp.kind = p.fmt_l == QM_FMT_INT8 ? kKindI8 : kKindF8;
     gp.tile_begin = (int32_t)total;
     total += ka.num_tiles;
