@@ -392,11 +392,60 @@ __device__ __forceinline__ void stats16(const uint32_t* rc, const uint32_t* rd, 
   }
 }
 
+// The same statistics for the grouped kernel, which first brings a chunk into one form (the
+// 8-bit accumulator as fp32, dead columns zeroed) so that one instantiation per scale layout
+// serves every format and the ragged edge.  PER_COL: the right operand has a scale per column
+// (dr_s), otherwise kd2 holds (-delta_l delta_r) twice.
+struct StatsG {
+  float be0, be1;
+  uint64_t d2, r2, n2;
+  float mx;
+};
+template <bool PER_COL>
+__device__ __forceinline__ void stats16g(const uint32_t* rc, const uint32_t* rd, const uint32_t* rq, uint64_t kd2,
+                                         const float* dr_s, StatsG& s) {
+#pragma unroll
+  for (int j = 0; j < 16; j += 2) {
+    const uint64_t a2 = pack2(__uint_as_float(rq[j]), __uint_as_float(rq[j + 1]));
+    const uint64_t cv2 = pack2(__uint_as_float(rc[j]), __uint_as_float(rc[j + 1]));
+    const float d0 = __uint_as_float(rd[j]), d1 = __uint_as_float(rd[j + 1]);
+    const uint64_t dd2 = pack2(d0, d1);
+    uint64_t diff2;                                              // C - A dl dr
+    if (PER_COL) diff2 = fma2(mul2(a2, kd2), *reinterpret_cast<const uint64_t*>(dr_s + j), cv2);
+    else diff2 = fma2(a2, kd2, cv2);
+    // D == 0 implies C == Q == 0, so clamping the divisor keeps BE = 0 there without a branch
+    const uint64_t be2 = mul2(diff2, pack2(rcp_approx(fmaxf(d0, 1e-37f)), rcp_approx(fmaxf(d1, 1e-37f))));
+    float b0, b1;
+    unpack2(be2, b0, b1);
+    s.be0 += fabsf(b0);
+    s.be1 += fabsf(b1);
+    s.mx = fmaxf(s.mx, fmaxf(fabsf(b0), fabsf(b1)));
+    s.d2 = fma2(diff2, diff2, s.d2);
+    s.r2 = fma2(cv2, cv2, s.r2);
+    s.n2 = fma2(dd2, dd2, s.n2);
+  }
+}
+// Chunk CH (16 columns) of a warp's share of a tile: rq holds its 8-bit accumulators as read from
+// tensor memory; n_live < 16 only at the ragged edge of the matrix, whose dead columns count as zeros.
+template <int CH>
+__device__ __forceinline__ void stats_chunk(uint32_t (&rc)[64], uint32_t (&rd)[64], uint32_t (&rq)[16], int n_live,
+                                            bool is_i8, bool per_col, uint64_t kd2, const float* dr_s, StatsG& st) {
+  if (is_i8) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k) rq[k] = __float_as_uint((float)(int)rq[k]);
+  }
+  if (n_live < 16) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+      if (k >= n_live) { rc[CH * 16 + k] = 0u; rd[CH * 16 + k] = 0u; rq[k] = 0u; }
+  }
+  if (per_col) stats16g<true>(&rc[CH * 16], &rd[CH * 16], rq, kd2, dr_s + CH * 16, st);
+  else stats16g<false>(&rc[CH * 16], &rd[CH * 16], rq, kd2, nullptr, st);
+}
 // Adds one tile's share of a row's Eq. 3 sums to the optional per-row check output.
-__device__ __forceinline__ void row_stats_add(double* rs, const Stats2& st) {
+__device__ __forceinline__ void row_stats_add(double* rs, const StatsG& st) {
   float x0, x1;
-  unpack2(st.be, x0, x1); atomicAdd(rs + 0, (double)x0 + (double)x1);
-  // BE >= 0: the bit patterns of non-negative doubles order like the values
+  atomicAdd(rs + 0, (double)st.be0 + (double)st.be1);
   atomicMax(reinterpret_cast<unsigned long long*>(rs + 1), (unsigned long long)__double_as_longlong((double)st.mx));
   unpack2(st.d2, x0, x1); atomicAdd(rs + 2, (double)x0 + (double)x1);
   unpack2(st.r2, x0, x1); atomicAdd(rs + 3, (double)x0 + (double)x1);
@@ -1046,9 +1095,17 @@ struct CfgP {
   static constexpr uint32_t kOffL = 0, kOffR = kABf16, kOffRa = kOffR + kBBf16, kOffCl = kOffRa + kBBf16;
   static constexpr uint32_t kOffCr = kOffCl + kALp;
   static constexpr uint32_t kStageBytes = kOffCr + kBLp;             // 44 KB
-  static constexpr uint32_t kTmaBytes = kABf16 + kBBf16 + kALp + kBLp;   // 36 KB per CTA and k-block
   static constexpr uint32_t kTileBytes = kStages * kStageBytes;      // 220 KB
   static constexpr uint32_t kColRef = 0, kColDen = 128, kColLp = 256, kColAbsL = 384;   // tensor-memory columns
+};
+
+// What the roles need of a probe for every tile, copied to shared memory once per CTA: the
+// launch's table sits in the kernel's parameter space, and reads of it with an index known only
+// at run time go through the small constant cache, which eleven kilobytes of table thrash.
+struct WalkInfo {
+  int32_t tile_begin, per_b, tiles_n, num_kb;       // per_b = tiles_m * tiles_n (tiles per batch element)
+  int32_t half_n, kind;
+  uint32_t idesc_ref, idesc_lp;
 };
 
 struct SharedP {
@@ -1066,6 +1123,7 @@ struct SharedP {
   uint32_t issued;                  // k-blocks whose loads the producer has issued (read on the give-up path)
   float delta_r[2][kBlockN];
   double red[5][kEpiWarps];
+  WalkInfo walk[kMaxGroup];
 };
 
 struct GroupProblem {
@@ -1089,43 +1147,46 @@ struct GroupTable {
 __device__ __forceinline__ int group_position(int r, int pair, int num_pairs) {
   return r * num_pairs + ((r & 1) ? num_pairs - 1 - pair : pair);
 }
-// which probe a position belongs to (tile_begin is ascending)
-__device__ __forceinline__ int group_find(const GroupTable& tab, int pos) {
-  int pi = 0;
-  while (pi + 1 < tab.n && pos >= tab.p[pi + 1].tile_begin) ++pi;
-  return pi;
-}
 
 // The tiles of one CTA pair in order, k-block by k-block: every role walks the same sequence.
+// A pair's positions ascend, so the search for a position's probe continues from the probe in hand.
 struct TileWalk {
+  const WalkInfo* wk;
+  int n, total_tiles;
   int r, pair, num_pairs;
-  int pi, num_kb, kb;
+  int pi, num_kb, kb, half_n;
   TileCoord tc;
   bool valid;
-  __device__ __forceinline__ void start(const GroupTable& tab, int pair_, int num_pairs_) {
-    r = -1; pair = pair_; num_pairs = num_pairs_; kb = 0; num_kb = 0; valid = true;
-    next_tile(tab);
+  __device__ __forceinline__ void start(const WalkInfo* wk_, int n_, int total_tiles_, int pair_, int num_pairs_) {
+    wk = wk_; n = n_; total_tiles = total_tiles_;
+    r = -1; pair = pair_; num_pairs = num_pairs_; kb = 0; num_kb = 0; pi = 0; half_n = 0; valid = true;
+    next_tile();
   }
   // moves to the pair's next tile; valid = false when there is none
-  __device__ __forceinline__ void next_tile(const GroupTable& tab) {
+  __device__ __forceinline__ void next_tile() {
     while (true) {
       ++r;
       const int pos = group_position(r, pair, num_pairs);
-      if (pos >= tab.total_tiles) {
-        if (r * num_pairs >= tab.total_tiles) { valid = false; return; }   // no round reaches further
+      if (pos >= total_tiles) {
+        if (r * num_pairs >= total_tiles) { valid = false; return; }   // no round reaches further
         continue;
       }
-      pi = group_find(tab, pos);
-      const GroupProblem& pr = tab.p[pi];
-      tc = tile_coord(pos - pr.tile_begin, pr.a);
-      num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+      while (pi + 1 < n && pos >= wk[pi + 1].tile_begin) ++pi;
+      const int4 w4 = *reinterpret_cast<const int4*>(&wk[pi]);          // tile_begin, per_b, tiles_n, num_kb
+      const int t = pos - w4.x;
+      tc.b = t / w4.y;
+      const int rem = t - tc.b * w4.y;
+      tc.m_tile = rem / w4.z;
+      tc.n_tile = rem - tc.m_tile * w4.z;
+      num_kb = w4.w;
+      half_n = wk[pi].half_n;
       kb = 0;
       return;
     }
   }
   // moves to the next k-block of the sequence
-  __device__ __forceinline__ void next_kb(const GroupTable& tab) {
-    if (++kb >= num_kb) next_tile(tab);
+  __device__ __forceinline__ void next_kb() {
+    if (++kb >= num_kb) next_tile();
   }
 };
 
@@ -1215,8 +1276,11 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
   if (warp == 0) {
     // fetch the tensor maps of this pair's first tile into the descriptor cache
     const int pos = group_position(0, pair, num_pairs);
-    if (pos < tab.total_tiles && lane < 4)
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tab.p[group_find(tab, pos)].maps[lane]) : "memory");
+    if (pos < tab.total_tiles && lane < 4) {
+      int pi = 0;
+      while (pi + 1 < tab.n && pos >= tab.p[pi + 1].tile_begin) ++pi;
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tab.p[pi].maps[lane]) : "memory");
+    }
   }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -1238,6 +1302,14 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
                      smem_u32(&sh->tmem_base)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  if (warp == 2 && lane < tab.n) {
+    const GroupProblem& pr = tab.p[lane];
+    WalkInfo wi;
+    wi.tile_begin = pr.tile_begin; wi.per_b = pr.a.tiles_m * pr.a.tiles_n; wi.tiles_n = pr.a.tiles_n;
+    wi.num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
+    wi.half_n = pr.half_n; wi.kind = pr.kind; wi.idesc_ref = pr.idesc_ref; wi.idesc_lp = pr.a.idesc_lp;
+    sh->walk[lane] = wi;
+  }
   tc_fence_before();
   __syncthreads();
   __syncwarp();
@@ -1252,17 +1324,17 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       // ---------------------------------------------------------- TMA producer (both CTAs)
       if (lane == 0) {
         TileWalk tw;
-        tw.start(tab, pair, num_pairs);
-        for (uint32_t g = 0; tw.valid; ++g, tw.next_kb(tab)) {
+        tw.start(sh->walk, tab.n, tab.total_tiles, pair, num_pairs);
+        for (uint32_t g = 0; tw.valid; ++g, tw.next_kb()) {
           const int s = g % kStages;
           const uint32_t use = g / kStages;
           if (g >= tab.stop_after_kb) break;                  // test hook: the consumers' waits run out
           if (use > 0 && !w.wait(smem_u32(&sh->empty[s]), (use - 1) & 1)) break;
           const GroupProblem& pr = tab.p[tw.pi];
           const int r0 = tw.tc.m_tile * kPairM + (int)rank * kBlockM;     // this CTA's left-operand rows
-          const int c0 = tw.tc.n_tile * kBlockN + (int)rank * pr.half_n;  // this CTA's half of the right operand
+          const int c0 = tw.tc.n_tile * kBlockN + (int)rank * tw.half_n;  // this CTA's half of the right operand
           const uint32_t bar = smem_u32(&sh->full[s]);
-          mbar_expect_tx(bar, kABf16 + kALp + (uint32_t)pr.half_n * (kBlockK * 2 + kBlockK));
+          mbar_expect_tx(bar, kABf16 + kALp + (uint32_t)tw.half_n * (kBlockK * 2 + kBlockK));
           const uint32_t base = tile_base + s * C::kStageBytes;
           const int k0 = tw.kb * kBlockK;
           tma_load_3d_local(base + C::kOffR, &pr.maps[1], bar, k0, c0, tw.tc.b);     // the converters read this one
@@ -1303,14 +1375,14 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         return true;
       };
       TileWalk tw;
-      tw.start(tab, pair, num_pairs);
+      tw.start(sh->walk, tab.n, tab.total_tiles, pair, num_pairs);
       uint32_t g = 0;
       bool ok = true;
-      for (uint32_t it = 0; tw.valid && ok; ++it, tw.next_tile(tab)) {
-        const GroupProblem& pr = tab.p[tw.pi];
-        const int num_kb = tw.num_kb, kind = pr.kind;
-        const uint32_t idesc_lp = pr.a.idesc_lp;
-        idesc_bf16 = pr.idesc_ref;
+      for (uint32_t it = 0; tw.valid && ok; ++it, tw.next_tile()) {
+        const WalkInfo& wi = sh->walk[tw.pi];
+        const int num_kb = tw.num_kb, kind = wi.kind;
+        const uint32_t idesc_lp = wi.idesc_lp;
+        idesc_bf16 = wi.idesc_ref;
         // the reference and denominator blocks come back when both epilogues have copied the
         // previous tile's values out; the 8-bit block when they have finished that tile
         if (it > 0 && !w.wait_warp(smem_u32(&sh->tmem_empty), (it - 1) & 1)) break;
@@ -1355,9 +1427,9 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + C::kColAbsL;
     const uint32_t row_off = (uint32_t)t * 128u, sw = (uint32_t)t & 7u;
     TileWalk tw;
-    tw.start(tab, pair, num_pairs);
+    tw.start(sh->walk, tab.n, tab.total_tiles, pair, num_pairs);
     bool ok = true;
-    for (uint32_t g = 0; ok && tw.valid; ++g, tw.next_kb(tab)) {
+    for (uint32_t g = 0; ok && tw.valid; ++g, tw.next_kb()) {
       const uint32_t s = g % kStages, sa = g % kAbs, m = 0x7fff7fffu;
       // the tensor-memory columns were last read by the MMAs of k-block g - kAbs (its commit also
       // covers every earlier k-block, so the |R| slot of the stage is free as well)
@@ -1372,7 +1444,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) v[j] = lds128(base + C::kOffL + row_off + (((uint32_t)j ^ sw) << 4));
       const uint32_t rsrc = base + C::kOffR + (uint32_t)t * 16u;
-      const int r_vec = tab.p[tw.pi].half_n * 8;                 // 16-byte vectors of the R half-tile that are in use
+      const int r_vec = tw.half_n * 8;                           // 16-byte vectors of the R half-tile that are in use
 #pragma unroll
       for (int j = 0; j < 4; ++j) u[j] = t + 128 * j < r_vec ? lds128(rsrc + (uint32_t)j * 2048u) : make_uint4(0u, 0u, 0u, 0u);
       uint32_t a[32];
@@ -1400,7 +1472,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     // of 16 columns; the statistics arithmetic runs under the next tile's main loop.
     const int q = warp & 3;
     const int ew = warp - kFirstEpiWarp;           // 0..7
-    const int h = ew >> 2;                         // which 64-column half of the tile
+    const int h = ew >> 2;                         // which half of the tile's columns
     const int et = ew * 32 + lane;                 // 0..255
     const uint32_t tmem_empty_leader = map_to_cta(smem_u32(&sh->tmem_empty), 0);
     double acc[5] = {0, 0, 0, 0, 0};               // of the probe in hand: sum BE, max BE, sum diff^2, C^2, D^2
@@ -1428,78 +1500,107 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       asm volatile("bar.sync 1, 256;" ::: "memory");       // red[] may be reused
     };
     uint32_t met = 0;                              // bit pi: this CTA has had tiles of probe pi
+    // of the probe in hand (reloaded when the probe changes, not per tile)
+    bool per_col = false, pc_l = false, is_i8 = false, narrow = false;
+    float dr_tensor = 1.f, dl_tensor = 0.f;
+    int pM = 0, pN = 0;                            // a probe's M and N are below 2^31 (its tensor maps require it)
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     TileWalk tw;
-    tw.start(tab, pair, num_pairs);
-    for (uint32_t it = 0; tw.valid; ++it, tw.next_tile(tab)) {
+    tw.start(sh->walk, tab.n, tab.total_tiles, pair, num_pairs);
+    for (uint32_t it = 0; tw.valid; ++it, tw.next_tile()) {
       const int pi = tw.pi;
       if (pi != cur) {
         if (cur >= 0) flush(cur);
         cur = pi;
         met |= 1u << pi;
+        const GroupProblem& pr = tab.p[pi];
+        per_col = pr.a.pc_r != 0; pc_l = pr.a.pc_l != 0; is_i8 = pr.kind == kKindI8; narrow = pr.half_n < 64;
+        pM = (int)pr.a.M; pN = (int)pr.a.N;
+        dr_tensor = per_col ? 1.f : __ldg(pr.a.dr);
+        dl_tensor = pc_l ? 0.f : __ldg(pr.a.dl);
       }
-      const GroupProblem& pr = tab.p[pi];
-      const KernelArgs& a = pr.a;
       const TileCoord tc = tw.tc;
-      const bool per_col = a.pc_r != 0;
-      const float dr_tensor = per_col ? 1.f : __ldg(a.dr);
       float* dr_s = sh->delta_r[it & 1];
       if (per_col && et < kBlockN) {
-        const int64_t col = (int64_t)tc.n_tile * kBlockN + et;
-        dr_s[et] = col < a.N ? __ldg(a.dr + (int64_t)tc.b * a.N + col) : 0.f;
+        const int col = tc.n_tile * kBlockN + et;
+        dr_s[et] = col < pN ? __ldg(tab.p[pi].a.dr + (int64_t)tc.b * pN + col) : 0.f;
       }
-      const int64_t row = (int64_t)tc.m_tile * kPairM + rank * kBlockM + q * 32 + lane;
-      const bool row_ok = row < a.M;
-      float dlv;
-      if (a.pc_l) dlv = row_ok ? __ldg(a.dl + (int64_t)tc.b * a.M + row) : 0.f;
-      else dlv = __ldg(a.dl);
+      const int row = tc.m_tile * kPairM + (int)rank * kBlockM + q * 32 + lane;
+      const bool row_ok = row < pM;
+      float dlv = dl_tensor;
+      if (pc_l) dlv = row_ok ? __ldg(tab.p[pi].a.dl + (int64_t)tc.b * pM + row) : 0.f;
+      // the two warps of a lane quarter split the tile's columns: 64 each, or 32 each where the
+      // tile is 64 wide (outputs at most 64 wide)
+      const int cw = narrow ? 32 : 64, cbase = h * cw;
+      const int colw = tc.n_tile * kBlockN + cbase;                  // first column of this warp
 
       const bool ok = w.wait(smem_u32(&sh->tmem_full), it & 1);
       // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
       if (epi_barrier_any(!ok)) break;
       tc_fence_after();
-      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-      const int64_t colw = (int64_t)tc.n_tile * kBlockN + h * 64;      // first column of this warp
-      uint32_t rc[64], rd[64], rq[16];
-      tmem_ld32(lane_addr + C::kColRef + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
-      tmem_ld32(lane_addr + C::kColRef + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
-      tmem_ld32(lane_addr + C::kColDen + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
-      tmem_ld32(lane_addr + C::kColDen + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+      uint32_t rc[64], rd[64];
+      tmem_ld32(lane_addr + C::kColRef + cbase, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
+      tmem_ld32(lane_addr + C::kColDen + cbase, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
+      if (!narrow) {
+        tmem_ld32(lane_addr + C::kColRef + cbase + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
+        tmem_ld32(lane_addr + C::kColDen + cbase + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
+      }
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
-      Stats2 st{0ull, 0ull, 0ull, 0ull, 0.f};
-      const uint64_t ndl2 = pack2(-dlv, -dlv), drt2 = pack2(dr_tensor, dr_tensor);
-      const bool is_i8 = pr.kind == kKindI8;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int cc0 = h * 64 + c * 16;
-        const int64_t col0 = colw + c * 16;
-        if (col0 < a.N) {                         // uniform across the warp
-          tmem_ld16(lane_addr + C::kColLp + cc0, rq);
-          tmem_ld_wait();
-          const int n_live = (int)(a.N - col0 < 16 ? a.N - col0 : 16);
-          if (is_i8) {
-            if (n_live == 16) stats16<kKindI8, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
-            else stats16<kKindI8, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
-          } else {
-            if (n_live == 16) stats16<kKindF8, false>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, 16, st);
-            else stats16<kKindF8, true>(&rc[c * 16], &rd[c * 16], rq, ndl2, dr_s + cc0, per_col, drt2, n_live, st);
-          }
-        }
+      StatsG st{0.f, 0.f, 0ull, 0ull, 0ull, 0.f};
+      const float kd = -dlv * dr_tensor;
+      const uint64_t kd2 = per_col ? pack2(-dlv, -dlv) : pack2(kd, kd);
+      // The 8-bit block: the first half of the warp's columns chunk by chunk, the second half in
+      // one go (the registers of the first half's reference and denominator values are free by
+      // then); as soon as the last of it is in registers the MMA lane may start the next tile's
+      // 8-bit MMAs, while the remaining chunks are still being evaluated.  Every warp arrives on
+      // lp_done exactly once per tile.  live = columns of this warp that exist in the matrix.
+      const int live = pN - colw < cw ? pN - colw : cw;          // <= 0: none
+      const uint32_t lp_addr = lane_addr + C::kColLp + cbase;
+      const uint32_t lp_done_leader = map_to_cta(smem_u32(&sh->lp_done), 0);
+      const float* const drc = dr_s + cbase;
+      uint32_t rqa[16], rqb[16];
+      if (live > 0) {
+        tmem_ld16(lp_addr, rqa);
+        tmem_ld_wait();
       }
-      // the 8-bit block has been read: the MMA lane may start the next tile's 8-bit MMAs
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&sh->lp_done), 0));
+      if (live <= 16) {                               // nothing further to read
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(lp_done_leader);
+      }
+      if (live > 0) stats_chunk<0>(rc, rd, rqa, live, is_i8, per_col, kd2, drc, st);
+      if (live > 16) {
+        tmem_ld16(lp_addr + 16, rqb);
+        tmem_ld_wait();
+        if (live <= 32) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(lp_done_leader);
+        }
+        stats_chunk<1>(rc, rd, rqb, live - 16, is_i8, per_col, kd2, drc, st);
+      }
+      if (live > 32) {
+        tmem_ld16(lp_addr + 32, rqa);
+        if (live > 48) tmem_ld16(lp_addr + 48, rqb);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(lp_done_leader);
+        stats_chunk<2>(rc, rd, rqa, live - 32, is_i8, per_col, kd2, drc, st);
+        if (live > 48) stats_chunk<3>(rc, rd, rqb, live - 48, is_i8, per_col, kd2, drc, st);
+      }
       if (row_ok) {
         float x0, x1;
-        unpack2(st.be, x0, x1); acc[0] += (double)x0 + (double)x1;
+        acc[0] += (double)st.be0 + (double)st.be1;
         unpack2(st.d2, x0, x1); acc[2] += (double)x0 + (double)x1;
         unpack2(st.r2, x0, x1); acc[3] += (double)x0 + (double)x1;
         unpack2(st.n2, x0, x1); acc[4] += (double)x0 + (double)x1;
         acc[1] = fmax(acc[1], (double)st.mx);
-        if (a.row_stats) row_stats_add(a.row_stats + ((int64_t)tc.b * a.M + row) * 5, st);
+        double* const rows = tab.p[pi].a.row_stats;
+        if (rows) row_stats_add(rows + ((int64_t)tc.b * pM + row) * 5, st);
       }
     }
     if (cur >= 0) flush(cur);
