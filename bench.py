@@ -526,7 +526,7 @@ def main():
     ap.add_argument("--workload", default="bert_large_sweep_layer")
     ap.add_argument("--step-ms", type=float, default=50.0,
                     help="the workload is repeated inside a step until the step lasts about this long")
-    ap.add_argument("--oracle-rows", type=int, default=1536)
+    ap.add_argument("--oracle-rows", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the other workloads, the scale/quantize and the stand-alone GEMM rate blocks")

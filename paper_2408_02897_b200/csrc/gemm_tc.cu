@@ -1507,7 +1507,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     TileWalk tw;
     tw.start(sh->walk, tab.n, tab.total_tiles, pair, num_pairs);
-    for (uint32_t it = 0; tw.valid; ++it, tw.next_tile()) {
+    for (uint32_t it = 0; tw.valid; ++it) {
       const int pi = tw.pi;
       if (pi != cur) {
         if (cur >= 0) flush(cur);
@@ -1538,59 +1538,51 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
       // one barrier publishes delta_r and makes the give-up decision uniform over the epilogue
       if (epi_barrier_any(!ok)) break;
       tc_fence_after();
-      uint32_t rc[64], rd[64];
+      // live = columns of this warp that exist in the matrix
+      const int live = pN - colw < cw ? pN - colw : cw;          // <= 0: none
+      const uint32_t lp_addr = lane_addr + C::kColLp + cbase;
+      const uint32_t lp_done_leader = map_to_cta(smem_u32(&sh->lp_done), 0);
+      const float* const drc = dr_s + cbase;
+      uint32_t rc[64], rd[64], rq0[16];
       tmem_ld32(lane_addr + C::kColRef + cbase, *reinterpret_cast<uint32_t(*)[32]>(&rc[0]));
       tmem_ld32(lane_addr + C::kColDen + cbase, *reinterpret_cast<uint32_t(*)[32]>(&rd[0]));
       if (!narrow) {
         tmem_ld32(lane_addr + C::kColRef + cbase + 32, *reinterpret_cast<uint32_t(*)[32]>(&rc[32]));
         tmem_ld32(lane_addr + C::kColDen + cbase + 32, *reinterpret_cast<uint32_t(*)[32]>(&rd[32]));
       }
+      if (live > 0) tmem_ld16(lp_addr, rq0);
       tmem_ld_wait();
+      // The reference and denominator blocks are in registers: the MMA lane may start the next
+      // tile's bf16 MMAs.  The 8-bit block follows in two steps, its first 16 columns with the
+      // loads above and the rest once the first chunk has been evaluated (which frees the
+      // registers the rest is read into); then the MMA lane may start the next tile's 8-bit MMAs as well, while the
+      // remaining chunks are still being evaluated.  Every warp arrives on each barrier exactly
+      // once per tile.
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+      if (lane == 0) {
+        mbar_arrive_cluster(tmem_empty_leader);
+        if (live <= 16) mbar_arrive_cluster(lp_done_leader);      // nothing further to read
+      }
       StatsG st{0.f, 0.f, 0ull, 0ull, 0ull, 0.f};
       const float kd = -dlv * dr_tensor;
       const uint64_t kd2 = per_col ? pack2(-dlv, -dlv) : pack2(kd, kd);
-      // The 8-bit block: the first half of the warp's columns chunk by chunk, the second half in
-      // one go (the registers of the first half's reference and denominator values are free by
-      // then); as soon as the last of it is in registers the MMA lane may start the next tile's
-      // 8-bit MMAs, while the remaining chunks are still being evaluated.  Every warp arrives on
-      // lp_done exactly once per tile.  live = columns of this warp that exist in the matrix.
-      const int live = pN - colw < cw ? pN - colw : cw;          // <= 0: none
-      const uint32_t lp_addr = lane_addr + C::kColLp + cbase;
-      const uint32_t lp_done_leader = map_to_cta(smem_u32(&sh->lp_done), 0);
-      const float* const drc = dr_s + cbase;
-      uint32_t rqa[16], rqb[16];
-      if (live > 0) {
-        tmem_ld16(lp_addr, rqa);
-        tmem_ld_wait();
-      }
-      if (live <= 16) {                               // nothing further to read
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(lp_done_leader);
-      }
-      if (live > 0) stats_chunk<0>(rc, rd, rqa, live, is_i8, per_col, kd2, drc, st);
+      if (live > 0) stats_chunk<0>(rc, rd, rq0, live, is_i8, per_col, kd2, drc, st);
       if (live > 16) {
-        tmem_ld16(lp_addr + 16, rqb);
-        tmem_ld_wait();
-        if (live <= 32) {
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(lp_done_leader);
-        }
-        stats_chunk<1>(rc, rd, rqb, live - 16, is_i8, per_col, kd2, drc, st);
-      }
-      if (live > 32) {
-        tmem_ld16(lp_addr + 32, rqa);
-        if (live > 48) tmem_ld16(lp_addr + 48, rqb);
+        // chunk 1 into the first chunk's registers, chunks 2 and 3 into those of the first
+        // chunk's reference and denominator values
+        uint32_t(&rq2)[16] = *reinterpret_cast<uint32_t(*)[16]>(&rc[0]);
+        uint32_t(&rq3)[16] = *reinterpret_cast<uint32_t(*)[16]>(&rd[0]);
+        tmem_ld16(lp_addr + 16, rq0);
+        if (live > 32) tmem_ld16(lp_addr + 32, rq2);
+        if (live > 48) tmem_ld16(lp_addr + 48, rq3);
         tmem_ld_wait();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(lp_done_leader);
-        stats_chunk<2>(rc, rd, rqa, live - 32, is_i8, per_col, kd2, drc, st);
-        if (live > 48) stats_chunk<3>(rc, rd, rqb, live - 48, is_i8, per_col, kd2, drc, st);
+        stats_chunk<1>(rc, rd, rq0, live - 16, is_i8, per_col, kd2, drc, st);
+        if (live > 32) stats_chunk<2>(rc, rd, rq2, live - 32, is_i8, per_col, kd2, drc, st);
+        if (live > 48) stats_chunk<3>(rc, rd, rq3, live - 48, is_i8, per_col, kd2, drc, st);
       }
       if (row_ok) {
         float x0, x1;
@@ -1602,6 +1594,7 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
         double* const rows = tab.p[pi].a.row_stats;
         if (rows) row_stats_add(rows + ((int64_t)tc.b * pM + row) * 5, st);
       }
+      tw.next_tile();
     }
     if (cur >= 0) flush(cur);
     // the records of the probes this CTA never met are zero

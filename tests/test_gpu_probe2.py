@@ -20,6 +20,18 @@ def both(o, fa, fb, **kw):
     return two, one
 
 
+def agree(a, b):
+    """The two-format kernel and the one-format kernel evaluate Eq. 3 in fp32 per row of a tile with
+    the operations in a different order (the one-format kernel folds the two scales into one factor
+    and splits narrow tiles 32 columns per warp), so their records agree to fp32 rounding of those
+    row sums, not bit for bit: 1e-6 on the sums, 1e-5 on the maximum (one element's quotient)."""
+    assert a["count"] == b["count"]
+    for k in ("sum_be", "sum_diff2", "sum_ref2", "sum_den2"):
+        assert abs(a[k] - b[k]) <= 1e-6 * abs(b[k]), (k, a[k], b[k])
+    assert abs(a["max_be"] - b["max_be"]) <= 1e-5 * abs(b["max_be"]), (a["max_be"], b["max_be"])
+    return True
+
+
 PAIRS = [(("e4m3", "e4m3"), ("int8", "int8")), (("int8", "int8"), ("e5m2", "e5m2")),
          (("e4m3", "e4m3"), ("e5m2", "e5m2")), (("e5m2", "e4m3"), ("e4m3", "e5m2"))]
 
@@ -36,7 +48,7 @@ def test_two_formats_small_ragged(fa, fb, gran, layout):
     two, one = both(o, fa, fb)
     for got, single, f in zip(two, one, (fa, fb)):
         assert got.device_error == 0
-        assert got.record() == single.record(), (f, got.record(), single.record())
+        assert agree(got.record(), single.record()), f
         oo = dict(o, fmt_l=f[0], fmt_r=f[1])
         assert_record_close(got.record(), oracle_probe(oo), what=str((f, gran, layout)))
 
@@ -47,19 +59,19 @@ def test_two_formats_many_tiles_and_batches():
     o = workloads.op("big", workloads.normal(rng, (2000, 2560)), -1, workloads.normal(rng, (2560, 1096), 0.02), -2,
                      "e4m3", "e4m3")
     two, one = both(o, ("e4m3", "e4m3"), ("int8", "int8"))
-    assert two[0].record() == one[0].record() and two[1].record() == one[1].record()
+    assert agree(two[0].record(), one[0].record()) and agree(two[1].record(), one[1].record())
     # batched attention-like product, channel scales shared per head
     Q = workloads.normal(rng, (12, 136, 64))
     Kt = workloads.normal(rng, (12, 200, 64))
     o = workloads.op("attn", Q, -1, Kt, -1, "e5m2", "e5m2", "channel", "channel")
     two, one = both(o, ("e5m2", "e5m2"), ("int8", "int8"), groups=(4, 4))
-    assert two[0].record() == one[0].record() and two[1].record() == one[1].record()
+    assert agree(two[0].record(), one[0].record()) and agree(two[1].record(), one[1].record())
     # a stochastically rounded gradient operand
     dY = workloads.lognormal_signed(rng, (256, 64), -8.0, 2.0)
     X = workloads.normal(rng, (256, 96))
     o = workloads.op("wgrad", X, -2, dY, -2, "e4m3", "e5m2")
     two, one = both(o, ("e4m3", "e5m2"), ("int8", "int8"), rounding="stochastic_r", seed=5)
-    assert two[0].record() == one[0].record() and two[1].record() == one[1].record()
+    assert agree(two[0].record(), one[0].record()) and agree(two[1].record(), one[1].record())
 
 
 def test_two_formats_k64_and_repeat():
@@ -74,7 +86,7 @@ def test_two_formats_k64_and_repeat():
         torch.cuda.synchronize()
         recs.append([r.record() for r in plan.results()])
     assert recs[0] == recs[1] == recs[2]
-    assert recs[0][0] == qm.qm_probe_layer(Lop, Rop, "e4m3", "e4m3", "tensor", "tensor").record()
+    assert agree(recs[0][0], qm.qm_probe_layer(Lop, Rop, "e4m3", "e4m3", "tensor", "tensor").record())
 
 
 def test_two_formats_refusals():
