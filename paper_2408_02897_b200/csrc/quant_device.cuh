@@ -261,37 +261,43 @@ __device__ __forceinline__ float sr_value(float t, uint32_t word) {
   return copysignf(r, t);
 }
 
-// Eight consecutive elements whose first has number idx0 in the operand.
-template <int FMT>
+// Eight consecutive elements whose first has number idx0 in the operand.  ALIGNED: idx0 is a
+// multiple of 4 (rows whose length is one, the common case), so the eight draws are exactly the
+// words of two counter blocks; otherwise they straddle three.
+template <int FMT, bool ALIGNED>
 __device__ __forceinline__ uint2 quant8_sr(const Vec8& x, const Quotient& quot, const Rounding& rnd,
                                            uint64_t idx0) {
   uint32_t w[12];
   const uint64_t blk = idx0 >> 2;
-  const int first = (int)(idx0 & 3);
+  const int first = ALIGNED ? 0 : (int)(idx0 & 3);
 #pragma unroll
-  for (int b = 0; b < 3; ++b) {
-    if (b < 2 || first != 0) {
-      const uint64_t c = blk + b;
-      philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), rnd.stream, 0u, rnd.k0, rnd.k1,
-                    *reinterpret_cast<uint32_t(*)[4]>(&w[4 * b]));
-    } else {
-      w[8] = w[9] = w[10] = w[11] = 0u;
-    }
+  for (int b = 0; b < (ALIGNED ? 2 : 3); ++b) {
+    const uint64_t c = blk + b;
+    philox4x32_10((uint32_t)c, (uint32_t)(c >> 32), rnd.stream, 0u, rnd.k0, rnd.k1,
+                  *reinterpret_cast<uint32_t(*)[4]>(&w[4 * b]));
   }
   float t[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    // word first + i without dynamic indexing of the register array
-    uint32_t word = 0;
+    uint32_t word = w[i];
+    if (!ALIGNED) {
+      // word first + i without dynamic indexing of the register array
 #pragma unroll
-    for (int f = 0; f < 4; ++f)
-      if (first == f) word = w[f + i];
+      for (int f = 1; f < 4; ++f)
+        if (first == f) word = w[f + i];
+    }
     t[i] = sr_value<FMT>(quot(x.v[i]), word);
   }
   uint2 r;
   r.x = quant2<FMT>(t[0], t[1]) | (quant2<FMT>(t[2], t[3]) << 16);
   r.y = quant2<FMT>(t[4], t[5]) | (quant2<FMT>(t[6], t[7]) << 16);
   return r;
+}
+// The same, choosing the variant from idx0 (uniform over a launch whenever rows are a multiple of 4 long).
+template <int FMT>
+__device__ __forceinline__ uint2 quant8_sr(const Vec8& x, const Quotient& quot, const Rounding& rnd,
+                                           uint64_t idx0) {
+  return (idx0 & 3) == 0 ? quant8_sr<FMT, true>(x, quot, rnd, idx0) : quant8_sr<FMT, false>(x, quot, rnd, idx0);
 }
 
 __device__ __forceinline__ uint4 abs_bf16x8(const Vec8& x) {
