@@ -34,12 +34,12 @@ from paper_2408_02897_b200 import workloads  # noqa: E402
 
 # DRAM bytes (read + write) of the fused probe kernel per byte of distinct operand data it reads
 # (bf16 L and R and both code tensors), from a profiler capture of one launch over the 12 probes of
-# the BERT-large layer workload (3.00 GB moved for 1.485 GB of distinct operand bytes: activations
-# larger than L2 are re-read for part of the column tiles, and an earlier capture of the same
-# launch moved 2.38 GB, so the figure varies by a fifth; 1.07 on the BERT-base workload, which
+# the BERT-large layer workload (2.56 GB moved for 1.485 GB of distinct operand bytes: activations
+# larger than L2 are re-read for part of the column tiles; other captures of the same launch
+# moved 2.38 and 3.00 GB, so the figure varies by a fifth; 1.07 on the BERT-base workload, which
 # fits in L2).  A launch of the default workload has the same projection shapes and is scaled by its
 # distinct operand bytes.  None: the kernel has changed since the counters were taken.
-TC_DRAM_BYTES_PER_OPERAND_BYTE = 2.02
+TC_DRAM_BYTES_PER_OPERAND_BYTE = 1.72
 
 
 METRIC = "probe TFLOPS"

@@ -1103,7 +1103,8 @@ struct CfgP {
 // launch's table sits in the kernel's parameter space, and reads of it with an index known only
 // at run time go through the small constant cache, which eleven kilobytes of table thrash.
 struct WalkInfo {
-  int32_t tile_begin, per_b, tiles_n, num_kb;       // per_b = tiles_m * tiles_n (tiles per batch element)
+  int32_t tile_begin, per_b, inner, num_kb;         // per_b = tiles_m * tiles_n (tiles per batch element);
+                                                    // inner = tiles_n: column tiles run fastest, -tiles_m: row tiles do
   int32_t half_n, kind;
   uint32_t idesc_ref, idesc_lp;
 };
@@ -1132,6 +1133,7 @@ struct GroupProblem {
   int32_t tile_begin;         // position of its first tile in the sequence
   int32_t kind;               // kKindF8 or kKindI8
   int32_t half_n;             // right-operand rows each CTA stages: 64, or 32 for outputs at most 64 wide
+  int32_t m_fastest;          // the tiles of a batch element are walked down the rows first (below)
   uint32_t idesc_ref;         // instruction descriptor of the bf16 MMAs (N = 2 * half_n)
 };
 struct GroupTable {
@@ -1172,12 +1174,14 @@ struct TileWalk {
         continue;
       }
       while (pi + 1 < n && pos >= wk[pi + 1].tile_begin) ++pi;
-      const int4 w4 = *reinterpret_cast<const int4*>(&wk[pi]);          // tile_begin, per_b, tiles_n, num_kb
+      const int4 w4 = *reinterpret_cast<const int4*>(&wk[pi]);          // tile_begin, per_b, inner, num_kb
       const int t = pos - w4.x;
       tc.b = t / w4.y;
       const int rem = t - tc.b * w4.y;
-      tc.m_tile = rem / w4.z;
-      tc.n_tile = rem - tc.m_tile * w4.z;
+      const int inner = w4.z < 0 ? -w4.z : w4.z;
+      const int outer_i = rem / inner, inner_i = rem - outer_i * inner;
+      tc.m_tile = w4.z < 0 ? inner_i : outer_i;
+      tc.n_tile = w4.z < 0 ? outer_i : inner_i;
       num_kb = w4.w;
       half_n = wk[pi].half_n;
       kb = 0;
@@ -1305,7 +1309,8 @@ tc_group_kernel(const __grid_constant__ GroupTable tab) {
   if (warp == 2 && lane < tab.n) {
     const GroupProblem& pr = tab.p[lane];
     WalkInfo wi;
-    wi.tile_begin = pr.tile_begin; wi.per_b = pr.a.tiles_m * pr.a.tiles_n; wi.tiles_n = pr.a.tiles_n;
+    wi.tile_begin = pr.tile_begin; wi.per_b = pr.a.tiles_m * pr.a.tiles_n;
+    wi.inner = pr.m_fastest ? -pr.a.tiles_m : pr.a.tiles_n;
     wi.num_kb = (int)((pr.a.K + kBlockK - 1) / kBlockK);
     wi.half_n = pr.half_n; wi.kind = pr.kind; wi.idesc_ref = pr.idesc_ref; wi.idesc_lp = pr.a.idesc_lp;
     sh->walk[lane] = wi;
@@ -1925,6 +1930,10 @@ qm_status launch_tc_probe_group(const TcProbeArgs* ps, int n, cudaStream_t s) {
     ka.err_also[0] = p.err_also[0]; ka.err_also[1] = p.err_also[1];
     gp.a = ka;
     gp.half_n = half_n;
+    // Tiles that run at the same time should share the LARGER operand's blocks, so that it is
+    // streamed from HBM once and the smaller one is what gets fetched again (from L2, if it fits):
+    // the tiles of a batch element are walked along the shorter side first.
+    gp.m_fastest = g.M < g.N ? 1 : 0;
     gp.idesc_ref = make_idesc(1, 1, 1, kPairM, 2 * half_n);
     gp.kind = p.fmt_l == QM_FMT_INT8 ? kKindI8 : kKindF8;
     gp.tile_begin = (int32_t)total;
