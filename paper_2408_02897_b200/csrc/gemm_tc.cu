@@ -1744,7 +1744,9 @@ int64_t tile_count(GemmShape g) {
 
 bool shape_ok(GemmShape g) {
   if (!(g.M > 0 && g.N > 0 && g.K > 0 && g.batch > 0 && (g.K % 16) == 0)) return false;
-  if (g.M >= (1ll << 31) || g.N >= (1ll << 31) || g.K >= (1ll << 31) || g.batch >= (1ll << 31)) return false;
+  // row, column and contraction indices of a tile's far edge are formed in 32-bit integers
+  constexpr int64_t kLimit = (1ll << 31) - 1024;
+  if (g.M >= kLimit || g.N >= kLimit || g.K >= kLimit || g.batch >= (1ll << 31)) return false;
   return tile_count(g) < (1ll << 31);
 }
 
